@@ -1,0 +1,594 @@
+"""fp64 CPU oracle of pdADMM-G and pdADMM-G-Q (test infrastructure, not product code).
+
+Everything here is written in the paper's own orientation and notation:
+matrices are ``width x |V|`` (one column per node), ``W_l`` is ``n_l x n_{l-1}``,
+``p_l`` is the input of layer l (``p_1 = X``), ``z_l, q_l, u_l`` are ``n_l x |V|``.
+Python lists are 0-based, so ``p[l-1]`` holds ``p_l`` and ``q[l-1], u[l-1]`` hold
+``q_l, u_l`` (l = 1..L-1).  All arithmetic is float64 numpy; the only library
+primitives are dense/sparse matrix products.
+
+Steps follow Algorithm 1 and the appendix "Solutions to Subproblems" in the
+paper's order: p (l = 2..L), W, b, z, q, residual, u.  Where the paper leaves a
+choice open the reading is stated in the function's docstring.
+
+Parity status: every function below is pinned by the CPU tests (grid search,
+closed forms, invariants); nothing is "parity unpinned".
+"""
+
+from __future__ import annotations
+
+import copy
+import dataclasses
+from typing import List, Optional
+
+import numpy as np
+import scipy.sparse as sp
+
+
+# ----------------------------------------------------------------------------
+# Graph pre-processing and feature augmentation
+# ----------------------------------------------------------------------------
+
+def renormalized_adjacency(n_nodes: int, edge_src, edge_dst) -> sp.csr_matrix:
+    """A~ = (D+I)^{-1/2} (A+I) (D+I)^{-1/2}, D_ii = sum_j A_ij  (Experiments, "Datasets and Settings").
+
+    ``A`` is the symmetric 0/1 adjacency of the undirected simple graph given
+    by the edge list (each edge once; self-loops and repeats are ignored).
+    """
+    src = np.asarray(edge_src, dtype=np.int64)
+    dst = np.asarray(edge_dst, dtype=np.int64)
+    keep = src != dst
+    src, dst = src[keep], dst[keep]
+    rows = np.concatenate([src, dst])
+    cols = np.concatenate([dst, src])
+    A = sp.coo_matrix((np.ones(rows.size), (rows, cols)), shape=(n_nodes, n_nodes)).tocsr()
+    A.data[:] = 1.0                      # repeated pairs collapse to a single 1
+    deg = np.asarray(A.sum(axis=1)).ravel()
+    d_inv_sqrt = 1.0 / np.sqrt(deg + 1.0)
+    A_hat = (A + sp.identity(n_nodes, format="csr")).tocsr()
+    S = sp.diags(d_inv_sqrt)
+    out = (S @ A_hat @ S).tocsr()
+    out.sort_indices()
+    return out
+
+
+def augment(H: np.ndarray, A_tilde: sp.csr_matrix, n_blocks: int) -> np.ndarray:
+    """X = [X_1; ...; X_K], X_k = H psi_k(A), psi = {I, A~, A~^2, ...}  (Problem Formulation).
+
+    ``H`` is ``d x |V|``; the result is ``(n_blocks d) x |V|``.
+    """
+    H = np.asarray(H, dtype=np.float64)
+    blocks = [H]
+    for _ in range(n_blocks - 1):
+        # X_{k+1} = X_k A~ ;  (X A~) = (A~^T X^T)^T and the sparse product wants the sparse factor first
+        blocks.append(np.asarray((A_tilde.T @ blocks[-1].T).T))
+    return np.concatenate(blocks, axis=0)
+
+
+# ----------------------------------------------------------------------------
+# State
+# ----------------------------------------------------------------------------
+
+@dataclasses.dataclass
+class Params:
+    rho: float
+    nu: float
+    quant_levels: int = 0                 # 0: pdADMM-G ; m >= 2: pdADMM-G-Q with m levels per layer
+    max_trials: int = 30                  # cap of the tau search in the quantised p-update
+    accept_slack: float = 1e-6
+
+
+@dataclasses.dataclass
+class State:
+    p: List[np.ndarray]                   # p_1..p_L ; p_1 = X is never updated
+    W: List[np.ndarray]
+    b: List[np.ndarray]                   # each n_l (a vector, broadcast over nodes)
+    z: List[np.ndarray]
+    q: List[np.ndarray]                   # q_1..q_{L-1}
+    u: List[np.ndarray]                   # u_1..u_{L-1}
+    y: np.ndarray                         # labels, |V| ints
+    mask: np.ndarray                      # |V| bools: node contributes to R
+    scale: List[float]                    # quantisation step s_l of p_l (index l-1; entry 0 unused)
+    tau: List[float] = dataclasses.field(default_factory=list)     # last tau_l (index l-1; entry 0 unused)
+    theta: List[float] = dataclasses.field(default_factory=list)   # last theta_l
+    trials: List[int] = dataclasses.field(default_factory=list)    # trials the quantised p-update took
+
+    @property
+    def L(self) -> int:
+        return len(self.W)
+
+    def copy(self) -> "State":
+        return copy.deepcopy(self)
+
+
+def relu(x):
+    return np.maximum(x, 0.0)
+
+
+# ----------------------------------------------------------------------------
+# phi, its gradients, and the quadratic models U_l, V_l
+# ----------------------------------------------------------------------------
+
+def phi(p, W, b, z, nu, q_prev=None, u_prev=None, rho=0.0) -> float:
+    """phi(p_l,W_l,b_l,z_l[,q_{l-1},u_{l-1}])  (definition below the augmented Lagrangian).
+
+    (nu/2)||z - W p - b||^2  [+ <u_{l-1}, p - q_{l-1}> + (rho/2)||p - q_{l-1}||^2 for l > 1].
+    """
+    lin = z - W @ p - b[:, None]
+    val = 0.5 * nu * np.sum(lin * lin)
+    if q_prev is not None:
+        diff = p - q_prev
+        val += np.sum(u_prev * diff) + 0.5 * rho * np.sum(diff * diff)
+    return float(val)
+
+
+def grad_p_phi(p, W, b, z, nu, q_prev, u_prev, rho):
+    """nabla_p phi = nu W^T (W p + b - z) + u_{l-1} + rho (p - q_{l-1})."""
+    return nu * (W.T @ (W @ p + b[:, None] - z)) + u_prev + rho * (p - q_prev)
+
+
+def grad_W_phi(p, W, b, z, nu):
+    """nabla_W phi = nu (W p + b - z) p^T."""
+    return nu * ((W @ p + b[:, None] - z) @ p.T)
+
+
+def grad_b_phi(p, W, b, z, nu):
+    """nabla_b phi = nu sum_j (W p + b - z)_{:,j}  (b is broadcast over the |V| columns)."""
+    return nu * np.sum(W @ p + b[:, None] - z, axis=1)
+
+
+def U_model(p_new, p_old, W, b, z, nu, q_prev, u_prev, rho, tau) -> float:
+    """U_l(p; tau) = phi(p^k) + <nabla_p phi(p^k), p - p^k> + (tau/2)||p - p^k||^2  (Eq. update p)."""
+    g = grad_p_phi(p_old, W, b, z, nu, q_prev, u_prev, rho)
+    d = p_new - p_old
+    return phi(p_old, W, b, z, nu, q_prev, u_prev, rho) + float(np.sum(g * d)) + 0.5 * tau * float(np.sum(d * d))
+
+
+def V_model(W_new, W_old, p, b, z, nu, theta) -> float:
+    """V_l(W; theta) = phi(W^k) + <nabla_W phi(W^k), W - W^k> + (theta/2)||W - W^k||^2  (Eq. update W).
+
+    The q/u terms of phi do not depend on W and cancel on both sides, so they are left out.
+    """
+    G = grad_W_phi(p, W_old, b, z, nu)
+    D = W_new - W_old
+    return phi(p, W_old, b, z, nu) + float(np.sum(G * D)) + 0.5 * theta * float(np.sum(D * D))
+
+
+# ----------------------------------------------------------------------------
+# p-update (Eq. update p) and its step parameter tau
+# ----------------------------------------------------------------------------
+
+def tau_smallest_admissible(g, W, nu, rho) -> float:
+    """Smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
+
+    The paper only states the condition.  phi is quadratic in p with Hessian
+    nu W^T W + rho I, so for a step d the condition reads
+    nu||W d||^2 + rho||d||^2 <= tau||d||^2; with d parallel to g the trial
+    value of tau drops out and the smallest admissible value is
+    rho + nu||W g||^2 / ||g||^2.  If g = 0 any tau works; rho is returned.
+    """
+    gg = float(np.sum(g * g))
+    if gg == 0.0:
+        return float(rho)
+    Wg = W @ g
+    return float(rho + nu * float(np.sum(Wg * Wg)) / gg)
+
+
+def tau_by_backtracking(p, W, b, z, nu, q_prev, u_prev, rho, tau0=None, factor=2.0, max_trials=200):
+    """Generic search by definition: grow tau geometrically until phi(p+) <= U_l(p+; tau).
+
+    Used by the tests to bracket ``tau_smallest_admissible``; not used by ``iterate``.
+    """
+    g = grad_p_phi(p, W, b, z, nu, q_prev, u_prev, rho)
+    tau = float(rho if tau0 is None else tau0)
+    for _ in range(max_trials):
+        p_new = p - g / tau
+        lhs = phi(p_new, W, b, z, nu, q_prev, u_prev, rho)
+        rhs = U_model(p_new, p, W, b, z, nu, q_prev, u_prev, rho, tau)
+        if lhs <= rhs:
+            return tau
+        tau *= factor
+    raise RuntimeError("tau search did not terminate")
+
+
+def update_p(p, W, b, z, nu, q_prev, u_prev, rho):
+    """p^{k+1} = p^k - nabla_p phi / tau^{k+1}, tau the smallest admissible value.  Returns (p+, tau)."""
+    g = grad_p_phi(p, W, b, z, nu, q_prev, u_prev, rho)
+    tau = tau_smallest_admissible(g, W, nu, rho)
+    return p - g / tau, tau
+
+
+# ----------------------------------------------------------------------------
+# Quantisation set and the quantised p-update (Eq. update p quantized)
+# ----------------------------------------------------------------------------
+
+def level_set(scale: float, m: int) -> np.ndarray:
+    """Delta = {delta_0..delta_{m-1}}, delta_c = fl32(c * s): m uniform levels starting at 0.
+
+    The levels are single-precision numbers (one rounded multiply), so that a
+    quantised p is exactly representable in the fp32 state of the CUDA path.
+    """
+    return (np.arange(m, dtype=np.float32) * np.float32(scale)).astype(np.float64)
+
+
+def quantize(x, scale: float, m: int):
+    """Nearest element of Delta, element by element: argmin_delta |delta - x|.
+
+    Since ||delta - x||^2 is separable the argmin of Eq. (update p quantized)
+    is taken per element.  For uniform levels it is a rounding:
+    code = clamp(floor(x/s + 1/2), 0, m-1) (ties at half-levels go up).  The
+    rounding decision is taken in single precision, the precision of the
+    kernel that takes the same decision.  Returns (codes uint8, p in Delta).
+    """
+    x32 = np.asarray(x, dtype=np.float32)
+    t = x32 / np.float32(scale)
+    c = np.floor(t + np.float32(0.5))
+    c = np.clip(c, np.float32(0.0), np.float32(m - 1))
+    codes = c.astype(np.uint8)
+    vals = (c * np.float32(scale)).astype(np.float64)
+    return codes, vals
+
+
+def quantization_scale(x, m: int) -> float:
+    """s = max(x) / (m - 1) as a single-precision number; s = 1 if max(x) <= 0."""
+    mx = np.float32(np.max(x)) if np.size(x) else np.float32(0.0)
+    if not mx > 0:
+        return 1.0
+    return float(np.float32(mx) / np.float32(m - 1))
+
+
+def update_p_quantized(p, W, b, z, nu, q_prev, u_prev, rho, scale, m, max_trials=30, slack=1e-6):
+    """p^{k+1} = argmin_{delta in Delta} ||delta - (p^k - nabla_p phi / tau)||.
+
+    tau starts at the smallest value admissible for the unprojected step and
+    is doubled until phi(p+) <= U_l(p+; tau) (up to a relative slack on the
+    quadratic term, which only matters at exact ties).  Returns
+    (p+, codes, tau, trials); trials = -1 if the cap was hit (last p+ is kept).
+    """
+    g = grad_p_phi(p, W, b, z, nu, q_prev, u_prev, rho)
+    tau = tau_smallest_admissible(g, W, nu, rho)
+    phi_old = phi(p, W, b, z, nu, q_prev, u_prev, rho)
+    for trial in range(1, max_trials + 1):
+        codes, p_new = quantize(p - g / tau, scale, m)
+        d = p_new - p
+        dd = float(np.sum(d * d))
+        lhs = phi(p_new, W, b, z, nu, q_prev, u_prev, rho)
+        rhs = phi_old + float(np.sum(g * d)) + 0.5 * tau * dd
+        if lhs <= rhs + 0.5 * slack * tau * dd:
+            return p_new, codes, tau, trial
+        tau *= 2.0
+    return p_new, codes, tau, -1
+
+
+# ----------------------------------------------------------------------------
+# W-update (Eq. update W), b-update (Eq. update b)
+# ----------------------------------------------------------------------------
+
+def theta_smallest_admissible(G, p, nu) -> float:
+    """Smallest theta with phi(W - G/theta) <= V_l(W - G/theta; theta): nu||G p||^2 / ||G||^2.
+
+    phi is quadratic in W: phi(W + D) = phi(W) + <G, D> + (nu/2)||D p||^2.  G = 0 returns 0
+    (the caller leaves W unchanged).
+    """
+    GG = float(np.sum(G * G))
+    if GG == 0.0:
+        return 0.0
+    Gp = G @ p
+    return float(nu * float(np.sum(Gp * Gp)) / GG)
+
+
+def theta_by_backtracking(p, W, b, z, nu, theta0, factor=2.0, max_trials=400):
+    """Generic search by definition on V_l (tests only)."""
+    G = grad_W_phi(p, W, b, z, nu)
+    theta = float(theta0)
+    for _ in range(max_trials):
+        W_new = W - G / theta
+        if phi(p, W_new, b, z, nu) <= V_model(W_new, W, p, b, z, nu, theta):
+            return theta
+        theta *= factor
+    raise RuntimeError("theta search did not terminate")
+
+
+def update_W(p, W, b, z, nu):
+    """W^{k+1} = W^k - nabla_W phi(p^{k+1}, W^k, b^k, z^k) / theta^{k+1}.  Returns (W+, theta)."""
+    G = grad_W_phi(p, W, b, z, nu)
+    theta = theta_smallest_admissible(G, p, nu)
+    if theta == 0.0:
+        return W.copy(), 0.0
+    return W - G / theta, theta
+
+
+def update_b(p, W, b, z, nu):
+    """b^{k+1} = b^k - nabla_b phi / (nu |V|).
+
+    The paper divides by nu, stating that nabla_b phi is nu-Lipschitz.  With b
+    broadcast over |V| columns the gradient is nu sum_j(...) and its Lipschitz
+    constant is nu|V|; dividing by that constant gives the exact minimiser
+    mean_j (z - W p)_{:,j}, and the descent inequality of Lemma (optimality 1)
+    still holds.  ``update_b_literal`` keeps the printed constant for the test
+    that shows it diverges.
+    """
+    n_nodes = p.shape[1]
+    return b - grad_b_phi(p, W, b, z, nu) / (nu * n_nodes)
+
+
+def update_b_literal(p, W, b, z, nu):
+    """The step exactly as printed (division by nu); tests only."""
+    return b - grad_b_phi(p, W, b, z, nu) / nu
+
+
+# ----------------------------------------------------------------------------
+# z-update (Eq. update z, Eq. update zl)
+# ----------------------------------------------------------------------------
+
+def z_objective_hidden(c, a, q, z_old):
+    """(c - a)^2 + (q - relu(c))^2 + (c - z^k)^2: Eq. (update z) per element, without the common nu/2."""
+    return (c - a) ** 2 + (q - relu(c)) ** 2 + (c - z_old) ** 2
+
+
+def update_z_hidden(a, q, z_old):
+    """ReLU closed form of Eq. (update z), a = W^{k+1} p^{k+1} + b^{k+1}.
+
+    The printed case distinction refers to the sign of the unknown; it is
+    resolved by minimising on each half-line and keeping the better of the two:
+    z- = min((a + z^k)/2, 0) on z <= 0, z+ = max((a + q^k + z^k)/3, 0) on z >= 0.
+    An exact tie keeps z-.
+    """
+    z_neg = np.minimum(0.5 * (a + z_old), 0.0)
+    z_pos = np.maximum((a + q + z_old) / 3.0, 0.0)
+    f_neg = z_objective_hidden(z_neg, a, q, z_old)
+    f_pos = z_objective_hidden(z_pos, a, q, z_old)
+    return np.where(f_pos < f_neg, z_pos, z_neg)
+
+
+def cross_entropy(z_col, y: int) -> float:
+    """CE(z; y) = -z_y + log sum_c exp(z_c) for one node."""
+    m = np.max(z_col)
+    return float(-z_col[y] + m + np.log(np.sum(np.exp(z_col - m))))
+
+
+def risk(zL, y, mask) -> float:
+    """R(z_L; y) = sum over labelled nodes of the cross-entropy (an unnormalised sum,
+    like the unnormalised squared norms it is added to)."""
+    m = np.max(zL, axis=0)
+    lse = m + np.log(np.sum(np.exp(zL - m[None, :]), axis=0))
+    ce = lse - zL[y, np.arange(zL.shape[1])]
+    return float(np.sum(ce[np.asarray(mask, dtype=bool)]))
+
+
+def softmax_col(z_col):
+    e = np.exp(z_col - np.max(z_col))
+    return e / np.sum(e)
+
+
+def prox_ce_newton(a_col, y: int, nu: float, tol=1e-12, max_iter=200):
+    """argmin_z CE(z; y) + (nu/2)||z - a||^2 for one node, damped Newton.
+
+    The objective is nu-strongly convex, so the minimiser is unique and is the
+    solution of softmax(z) - e_y + nu (z - a) = 0.  The Hessian is
+    diag(s) + nu I - s s^T, inverted with the rank-one update formula.
+    """
+    z = np.array(a_col, dtype=np.float64)
+    C = z.size
+    e_y = np.zeros(C)
+    e_y[y] = 1.0
+
+    def f(zz):
+        return cross_entropy(zz, y) + 0.5 * nu * float(np.sum((zz - a_col) ** 2))
+
+    fz = f(z)
+    for _ in range(max_iter):
+        s = softmax_col(z)
+        grad = s - e_y + nu * (z - a_col)
+        if np.max(np.abs(grad)) <= tol:
+            break
+        m_inv = 1.0 / (s + nu)
+        mg = m_inv * grad
+        ms = m_inv * s
+        step = -(mg + ms * (np.dot(s, mg) / (1.0 - np.dot(s, ms))))
+        t = 1.0
+        slope = float(np.dot(grad, step))
+        # once the predicted decrease is below what f can resolve in double precision the
+        # iteration is in Newton's quadratic regime: full steps, no sufficient-decrease test
+        resolvable = -slope > 1e-9 * (1.0 + abs(fz))
+        while True:
+            z_try = z + t * step
+            f_try = f(z_try)
+            if not resolvable or f_try <= fz + 1e-4 * t * slope or t < 1e-12:
+                break
+            t *= 0.5
+        z, fz = z_try, f_try
+    return z
+
+
+def prox_ce_fista(a_col, y: int, nu: float, n_iter=20000, tol=1e-13):
+    """The same minimiser by FISTA (the solver the paper names for Eq. update zl).
+
+    Smooth part CE (gradient 1-Lipschitz, step 1), proximable part
+    (nu/2)||z - a||^2 with prox(v) = (v + nu a) / (1 + nu).  Cross-check only.
+    """
+    C = a_col.size
+    e_y = np.zeros(C)
+    e_y[y] = 1.0
+    x = np.array(a_col, dtype=np.float64)
+    v = x.copy()
+    t = 1.0
+    for _ in range(n_iter):
+        x_new = ((v - (softmax_col(v) - e_y)) + nu * a_col) / (1.0 + nu)
+        t_new = 0.5 * (1.0 + np.sqrt(1.0 + 4.0 * t * t))
+        v = x_new + ((t - 1.0) / t_new) * (x_new - x)
+        done = np.max(np.abs(x_new - x)) <= tol
+        x, t = x_new, t_new
+        if done:
+            break
+    return x
+
+
+def prox_ce_newton_batched(A, y, nu: float, tol=1e-12, max_iter=200):
+    """``prox_ce_newton`` for many nodes at once (columns of ``A``), same steps per column.
+
+    Each column runs its own damped Newton iteration with its own step length;
+    a column stops moving once its gradient is below ``tol``.
+    """
+    A = np.asarray(A, dtype=np.float64)
+    C, n = A.shape
+    cols = np.arange(n)
+    E = np.zeros((C, n))
+    E[np.asarray(y, dtype=np.int64), cols] = 1.0
+
+    def f(Z):
+        m = np.max(Z, axis=0)
+        lse = m + np.log(np.sum(np.exp(Z - m[None, :]), axis=0))
+        return lse - np.sum(E * Z, axis=0) + 0.5 * nu * np.sum((Z - A) ** 2, axis=0)
+
+    Z = A.copy()
+    fz = f(Z)
+    for _ in range(max_iter):
+        Ex = np.exp(Z - np.max(Z, axis=0)[None, :])
+        S = Ex / np.sum(Ex, axis=0)[None, :]
+        grad = S - E + nu * (Z - A)
+        active = np.max(np.abs(grad), axis=0) > tol
+        if not active.any():
+            break
+        m_inv = 1.0 / (S + nu)
+        mg = m_inv * grad
+        ms = m_inv * S
+        step = -(mg + ms * (np.sum(S * mg, axis=0) / (1.0 - np.sum(S * ms, axis=0)))[None, :])
+        step[:, ~active] = 0.0
+        slope = np.sum(grad * step, axis=0)
+        t = np.ones(n)
+        resolvable = -slope > 1e-9 * (1.0 + np.abs(fz))
+        searching = active.copy()
+        Z_try, f_try = Z.copy(), fz.copy()
+        while searching.any():
+            Zc = Z[:, searching] + t[searching][None, :] * step[:, searching]
+            fc = f_cols(Zc, A[:, searching], E[:, searching], nu)
+            ok = (~resolvable[searching]) | (fc <= fz[searching] + 1e-4 * t[searching] * slope[searching]) \
+                | (t[searching] < 1e-12)
+            idx = np.flatnonzero(searching)
+            Z_try[:, idx[ok]] = Zc[:, ok]
+            f_try[idx[ok]] = fc[ok]
+            t[idx[~ok]] *= 0.5
+            searching[idx[ok]] = False
+        Z, fz = Z_try, f_try
+    return Z
+
+
+def f_cols(Z, A, E, nu):
+    """CE(z; y) + (nu/2)||z - a||^2 for each column."""
+    m = np.max(Z, axis=0)
+    lse = m + np.log(np.sum(np.exp(Z - m[None, :]), axis=0))
+    return lse - np.sum(E * Z, axis=0) + 0.5 * nu * np.sum((Z - A) ** 2, axis=0)
+
+
+def update_z_last(a, y, mask, nu):
+    """Eq. (update zl): labelled nodes take the proximal point of the cross-entropy,
+    unlabelled nodes (no risk term) take z = a.  No proximal ||z - z^k||^2 term for l = L."""
+    z = np.array(a, dtype=np.float64)
+    lab = np.flatnonzero(np.asarray(mask, dtype=bool))
+    if lab.size:
+        z[:, lab] = prox_ce_newton_batched(a[:, lab], np.asarray(y)[lab], nu)
+    return z
+
+
+# ----------------------------------------------------------------------------
+# q-update (Eq. update q), dual update (Eq. update u)
+# ----------------------------------------------------------------------------
+
+def update_q(p_next, u, z, rho, nu):
+    """q_l^{k+1} = (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)."""
+    return (rho * p_next + u + nu * relu(z)) / (rho + nu)
+
+
+def update_u(u, p_next, q, rho):
+    """u_l^{k+1} = u_l^k + rho (p_{l+1}^{k+1} - q_l^{k+1})."""
+    return u + rho * (p_next - q)
+
+
+# ----------------------------------------------------------------------------
+# Initial state, one iteration (Algorithm 1), objective and residuals
+# ----------------------------------------------------------------------------
+
+def init_state(X, W0, y, mask, prm: Params) -> State:
+    """Feasible start (the paper only says "k = 0"; its theorems allow any start).
+
+    b = 0 and a forward pass: z_l = W_l p_l, q_l = relu(z_l), p_{l+1} = q_l, u = 0.
+    pdADMM-G-Q: the pass is sequential in l; the step s_{l+1} of p_{l+1} is
+    max(q_l) / (m - 1) and p_{l+1} = Proj_Delta(q_l), so the residual starts non-zero.
+    """
+    L = len(W0)
+    p = [np.asarray(X, dtype=np.float64)]
+    W = [np.asarray(w, dtype=np.float64).copy() for w in W0]
+    b = [np.zeros(w.shape[0]) for w in W]
+    z, q, u = [], [], []
+    scale = [1.0] * L
+    for l in range(L):
+        z.append(W[l] @ p[l])
+        if l < L - 1:
+            q.append(relu(z[l]))
+            u.append(np.zeros_like(q[l]))
+            if prm.quant_levels:
+                scale[l + 1] = quantization_scale(q[l], prm.quant_levels)
+                p.append(quantize(q[l], scale[l + 1], prm.quant_levels)[1])
+            else:
+                p.append(q[l].copy())
+    return State(p, W, b, z, q, u, np.asarray(y), np.asarray(mask, dtype=bool), scale,
+                 [0.0] * L, [0.0] * L, [0] * L)
+
+
+def iterate(s: State, prm: Params) -> State:
+    """One pass of Algorithm 1: p (l=2..L), W, b, z (l=1..L), q, residual, u (l=1..L-1).
+
+    Each family is finished for all layers before the next one starts.
+    """
+    rho, nu, L = prm.rho, prm.nu, s.L
+    n = s.copy()
+    # p_l^{k+1}, l = 2..L, from (W^k, b^k, z^k, q^k, u^k)
+    for l in range(1, L):
+        if prm.quant_levels:
+            n.p[l], _, n.tau[l], n.trials[l] = update_p_quantized(
+                s.p[l], s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho,
+                s.scale[l], prm.quant_levels, prm.max_trials, prm.accept_slack)
+        else:
+            n.p[l], n.tau[l] = update_p(s.p[l], s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho)
+    # W_l^{k+1} from (p^{k+1}, b^k, z^k)
+    for l in range(L):
+        n.W[l], n.theta[l] = update_W(n.p[l], s.W[l], s.b[l], s.z[l], nu)
+    # b_l^{k+1} from (p^{k+1}, W^{k+1}, z^k)
+    for l in range(L):
+        n.b[l] = update_b(n.p[l], n.W[l], s.b[l], s.z[l], nu)
+    # z_l^{k+1} from (p^{k+1}, W^{k+1}, b^{k+1}, q^k)
+    for l in range(L):
+        a = n.W[l] @ n.p[l] + n.b[l][:, None]
+        if l < L - 1:
+            n.z[l] = update_z_hidden(a, s.q[l], s.z[l])
+        else:
+            n.z[l] = update_z_last(a, s.y, s.mask, nu)
+    # q_l^{k+1}, then u_l^{k+1}
+    for l in range(L - 1):
+        n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu)
+    for l in range(L - 1):
+        n.u[l] = update_u(s.u[l], n.p[l + 1], n.q[l], rho)
+    return n
+
+
+def residuals_sq(s: State) -> np.ndarray:
+    """||r_l||^2 = ||p_{l+1} - q_l||^2, l = 1..L-1 (the residual line of Algorithm 1)."""
+    return np.array([float(np.sum((s.p[l + 1] - s.q[l]) ** 2)) for l in range(s.L - 1)])
+
+
+def objective(s: State, prm: Params) -> np.ndarray:
+    """Components of the augmented Lagrangian L_rho and their sum:
+    [R, (nu/2) sum||z - W p - b||^2, (nu/2) sum||q - f(z)||^2, sum<u, p+ - q>, (rho/2) sum||p+ - q||^2, L_rho]."""
+    rho, nu, L = prm.rho, prm.nu, s.L
+    R = risk(s.z[L - 1], s.y, s.mask)
+    lin = sum(float(np.sum((s.z[l] - s.W[l] @ s.p[l] - s.b[l][:, None]) ** 2)) for l in range(L))
+    act = sum(float(np.sum((s.q[l] - relu(s.z[l])) ** 2)) for l in range(L - 1))
+    dual = sum(float(np.sum(s.u[l] * (s.p[l + 1] - s.q[l]))) for l in range(L - 1))
+    pen = float(np.sum(residuals_sq(s)))
+    comps = [R, 0.5 * nu * lin, 0.5 * nu * act, dual, 0.5 * rho * pen]
+    return np.array(comps + [sum(comps)])
+
+
+def lagrangian(s: State, prm: Params) -> float:
+    return float(objective(s, prm)[5])
