@@ -1,0 +1,180 @@
+/*
+ * pdadmm.h -- C ABI of the pdADMM-G / pdADMM-G-Q training iteration for graph-augmented MLPs
+ * on one NVIDIA B200 (sm_100a).
+ *
+ * Notation follows the paper (Table "Important Notations"): |V| = N nodes, L layers,
+ * W_l (n_l x n_{l-1}), b_l (n_l), p_l (input of layer l, p_1 = X), z_l, q_l, u_l, penalties nu, rho.
+ * The paper stores one COLUMN per node (p_l is n_{l-1} x N); every host and device array of this
+ * library is the same memory read node-major: row j holds node j, i.e. P_l is [N][n_{l-1}],
+ * Z_l, Q_l, U_l are [N][n_l], row-major float32.  W_l is [n_l][n_{l-1}] row-major float32.
+ * Layers are numbered 1..L as in the paper in every call.
+ *
+ * General rules
+ *  - Every function returns PDADMM_OK (0) or a negative pdadmm_status; nothing aborts or throws
+ *    across the boundary.  pdadmm_last_error() gives a thread-local text for the last failure.
+ *  - All pointer arguments are HOST pointers unless a parameter is explicitly called a device
+ *    pointer.  The caller owns every buffer it passes; the library copies what it needs during
+ *    the call and never keeps a caller pointer.  Output buffers are written only after their
+ *    size has been checked.
+ *  - A context owns all of its device memory and streams; it is bound to one device and is not
+ *    thread-safe.  There is no CPU fallback: without a usable CUDA device every call that needs
+ *    one fails with PDADMM_ECUDA.
+ */
+#ifndef PDADMM_H
+#define PDADMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pdadmm_ctx pdadmm_ctx;
+
+typedef enum {
+  PDADMM_OK = 0,
+  PDADMM_EINVAL = -1,    /* bad argument (null pointer, size, range, unsorted or out-of-range index) */
+  PDADMM_ENOMEM = -2,    /* host or device allocation failed                                         */
+  PDADMM_ECUDA = -3,     /* a CUDA call failed, or no usable device                                  */
+  PDADMM_ETIMEOUT = -4,  /* a bounded device-side wait expired                                       */
+  PDADMM_ENUMERIC = -5,  /* a non-finite value was detected in the state                             */
+  PDADMM_ENOTCONV = -6   /* the tau search of the quantised p-update hit its trial cap               */
+} pdadmm_status;
+
+/* Tensor kinds of pdadmm_get_tensor / pdadmm_set_tensor.  "layer" is the paper's l. */
+typedef enum {
+  PDADMM_T_X = 0,        /* float  [N][n_0]       augmented features = p_1 (layer ignored)             */
+  PDADMM_T_P = 1,        /* float  [N][n_{l-1}]   l = 1..L (l = 1 is X)                                */
+  PDADMM_T_W = 2,        /* float  [n_l][n_{l-1}] l = 1..L                                             */
+  PDADMM_T_B = 3,        /* float  [n_l]          l = 1..L                                             */
+  PDADMM_T_Z = 4,        /* float  [N][n_l]       l = 1..L                                             */
+  PDADMM_T_Q = 5,        /* float  [N][n_l]       l = 1..L-1                                           */
+  PDADMM_T_U = 6,        /* float  [N][n_l]       l = 1..L-1                                           */
+  PDADMM_T_CODES = 7,    /* uint8  [N][n_{l-1}]   l = 2..L, pdADMM-G-Q only: p_l = code * QSCALE_l     */
+  PDADMM_T_TAU = 8,      /* double [1]            l = 2..L: tau_l of the last iteration (get only)     */
+  PDADMM_T_THETA = 9,    /* double [1]            l = 1..L: theta_l of the last iteration (get only)   */
+  PDADMM_T_QSCALE = 10,  /* float  [1]            l = 2..L: level spacing s_l of p_l                   */
+  PDADMM_T_CSR_ROWPTR = 11, /* int32 [N+1]        renormalised adjacency, get only                     */
+  PDADMM_T_CSR_COLIDX = 12, /* int32 [nnz]        columns ascending in each row, get only              */
+  PDADMM_T_CSR_VAL = 13, /* float  [nnz]          get only                                             */
+  PDADMM_T_TRIALS = 14   /* int32  [1]            l = 2..L: trials of the last quantised p-update      */
+} pdadmm_tensor;
+
+/* Bits of pdadmm_config.flags. */
+#define PDADMM_FLAG_SIMT_GEMM 1u     /* run the dense products on CUDA cores (fp32 FMA) instead of tensor cores */
+#define PDADMM_FLAG_ONE_STREAM 2u    /* issue all layers on one stream (no concurrency across layers)           */
+
+/*
+ * Problem statement (paper: Problem 2 / Problem 3, Algorithm 1 "Require", and the experimental
+ * settings for the operator set Psi and the renormalised adjacency).
+ */
+typedef struct {
+  int64_t n_nodes;               /* N = |V| >= 1                                                        */
+  int64_t n_edges;               /* undirected edges, each listed once; self-loops/repeats are ignored  */
+  const int32_t *edge_src;       /* [n_edges] node ids in [0, N)                                        */
+  const int32_t *edge_dst;       /* [n_edges]                                                           */
+  int32_t feat_dim;              /* d                                                                   */
+  const float *features;         /* H, node-major [N][d]                                                */
+  int32_t n_hops;                /* highest power of A~ used; the input has n_hops+1 blocks, n_0=(n_hops+1)d */
+  int32_t n_classes;             /* C = n_L                                                             */
+  const int32_t *labels;         /* [N] in [0, C)                                                       */
+  const uint8_t *train_mask;     /* [N]; 1 = the node's cross-entropy is part of R(z_L; y)              */
+  int32_t n_layers;              /* L >= 1                                                              */
+  const int32_t *layer_widths;   /* [L]: n_1..n_L, n_L == n_classes                                     */
+  float rho;                     /* > 0                                                                 */
+  float nu;                      /* > 0                                                                 */
+  int32_t quant_levels;          /* 0: pdADMM-G;  2..256: pdADMM-G-Q with that many uniform levels      */
+  const float *const *init_W;    /* [L] pointers: W_l^0 as [n_l][n_{l-1}] (required; the caller draws them) */
+  int32_t device;                /* CUDA device ordinal                                                 */
+  uint32_t flags;                /* PDADMM_FLAG_*                                                       */
+} pdadmm_config;
+
+/*
+ * pdadmm_init -- build the problem on the device.
+ * Computes the CSR form of A~ = (D+I)^{-1/2}(A+I)(D+I)^{-1/2} (paper, "Datasets and Settings"),
+ * the augmented input X = [H; H A~; ...; H A~^{n_hops}] by sparse products (paper, "Problem
+ * Formulation": X_k = H psi_k(A)), and the start of Algorithm 1: b = 0, a forward pass
+ * z_l = W_l p_l, q_l = ReLU(z_l), p_{l+1} = q_l (pdADMM-G-Q: p_{l+1} = nearest level of q_l, with the
+ * level spacing s_{l+1} = max(q_l)/(m-1)), u = 0.
+ * On success *out receives a context that the caller must release with pdadmm_destroy.
+ * Errors: EINVAL for inconsistent sizes / out-of-range indices / null pointers, ENOMEM, ECUDA.
+ */
+int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out);
+
+/*
+ * pdadmm_step -- run n_iters iterations of Algorithm 1: for every layer the p-update (Eq. "update
+ * p"; pdADMM-G-Q: Eq. "update p quantized"), W-update (Eq. "update W"), b-update (Eq. "update b"),
+ * z-update (Eq. "update z" with the ReLU closed form, Eq. "update zl" for the last layer), q-update
+ * (Eq. "update q"), residual and dual update (Eq. "update u").  Returns after the device finished.
+ * tau_l and theta_l are the smallest values that satisfy the paper's conditions
+ * phi(p+) <= U_l(p+; tau) and phi(W+) <= V_l(W+; theta); the quantised update doubles tau from
+ * that value until its condition holds (at most 30 trials, then ENOTCONV; the state stays valid).
+ */
+int pdadmm_step(pdadmm_ctx *ctx, int n_iters);
+
+/*
+ * pdadmm_objective -- the augmented Lagrangian L_rho (paper, Section "The pdADMM-G Algorithm") of the
+ * current state: out = { R(z_L;y), (nu/2) sum_l ||z_l - W_l p_l - b_l||^2, (nu/2) sum_l ||q_l - ReLU(z_l)||^2,
+ * sum_l <u_l, p_{l+1} - q_l>, (rho/2) sum_l ||p_{l+1} - q_l||^2, their sum }.  R is the sum of the
+ * cross-entropies of the masked nodes.  Accumulated in double precision.
+ */
+int pdadmm_objective(pdadmm_ctx *ctx, double out[6]);
+
+/*
+ * pdadmm_residuals -- ||p_{l+1} - q_l||^2 for l = 1..L-1 (Algorithm 1, residual line) into
+ * per_layer_sq[0..n-1]; n must be L-1 (n = 0 with a null pointer is accepted for L = 1).
+ */
+int pdadmm_residuals(pdadmm_ctx *ctx, double *per_layer_sq, int n);
+
+/*
+ * pdadmm_get_tensor / pdadmm_set_tensor -- copy one tensor of the state to / from a host buffer of
+ * exactly `bytes` bytes (dense, without the device's row padding).  Together they are the
+ * checkpoint / resume interface.  Setting P, W, B or Z invalidates the cached linear residual
+ * W p + b - z, which the next step recomputes.  Setting P in pdADMM-G-Q mode expects values on the
+ * level set; CODES are recomputed from them.  EINVAL for a bad kind/layer/size or a get-only kind.
+ */
+int pdadmm_get_tensor(pdadmm_ctx *ctx, int kind, int layer, void *host_dst, size_t bytes);
+int pdadmm_set_tensor(pdadmm_ctx *ctx, int kind, int layer, const void *host_src, size_t bytes);
+
+/*
+ * pdadmm_quantize -- the projection used by Eq. "update p quantized" on its own: for n host floats x,
+ * code = clamp(floor(x/scale + 1/2), 0, levels-1) as uint8 and p = code * scale (one rounded
+ * single-precision multiply), computed by the same device function as inside pdadmm_step.
+ * codes_out and p_out are host buffers of n elements (either may be null).
+ */
+int pdadmm_quantize(int device, const float *x, size_t n, float scale, int levels,
+                    uint8_t *codes_out, float *p_out);
+
+/*
+ * pdadmm_spmm -- Y = A~ X for a caller-supplied CSR matrix (host arrays, columns in [0, n_rows))
+ * and a node-major [n_rows][width] host matrix, by the same kernel that builds the augmented input
+ * (paper, "Problem Formulation": X_{k+1} = X_k A~ with A~ symmetric).  y_out is [n_rows][width].
+ */
+int pdadmm_spmm(int device, int64_t n_rows, const int32_t *row_ptr, const int32_t *col_idx,
+                const float *val, const float *x, int32_t width, float *y_out);
+
+/*
+ * Per-kernel timing.  pdadmm_profile(ctx, 1) makes every later kernel launch of pdadmm_step be
+ * bracketed by CUDA events on its own stream (the layers then run one after another);
+ * pdadmm_profile(ctx, 0) turns it off; either call clears the counters.
+ * pdadmm_profile_read returns, for kernel class k in [0, pdadmm_profile_classes()), the summed
+ * device time in ms, the number of launches, and the algorithmic bytes and flops of those launches.
+ * pdadmm_launches gives the number of kernels launched by pdadmm_step since the context was made.
+ */
+int pdadmm_profile(pdadmm_ctx *ctx, int enable);
+int pdadmm_profile_classes(void);
+const char *pdadmm_profile_name(int k);
+int pdadmm_profile_read(pdadmm_ctx *ctx, int k, double *ms, int64_t *launches, double *bytes, double *flops);
+int pdadmm_launches(pdadmm_ctx *ctx, int64_t *count);
+
+/* Release the context and all of its device memory.  Null is accepted. */
+int pdadmm_destroy(pdadmm_ctx *ctx);
+
+/* Text of the calling thread's last failure ("" if none).  The pointer stays valid until the next failing call. */
+const char *pdadmm_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PDADMM_H */

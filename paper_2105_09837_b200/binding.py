@@ -1,0 +1,239 @@
+"""ctypes binding of ``libpdadmm.so``: the same entry points as ``include/pdadmm.h``.
+
+Argument marshalling only -- every step of the iteration runs in the library's kernels.
+The library must have been built (``python -m paper_2105_09837_b200.build``); loading fails
+loudly otherwise, and there is no CPU fallback.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpdadmm.so")
+_lib = None
+
+# tensor kinds (pdadmm_tensor)
+T_X, T_P, T_W, T_B, T_Z, T_Q, T_U, T_CODES, T_TAU, T_THETA, T_QSCALE, T_CSR_ROWPTR, T_CSR_COLIDX, T_CSR_VAL, T_TRIALS = range(15)
+FLAG_SIMT_GEMM = 1
+FLAG_ONE_STREAM = 2
+
+OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
+
+EXPORTS = [
+    "pdadmm_init", "pdadmm_step", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
+    "pdadmm_set_tensor", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_profile", "pdadmm_profile_classes",
+    "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_destroy", "pdadmm_last_error",
+]
+
+
+class PdadmmError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"pdadmm error {code}: {text}")
+        self.code = code
+
+
+class _Config(C.Structure):
+    _fields_ = [
+        ("n_nodes", C.c_int64), ("n_edges", C.c_int64),
+        ("edge_src", C.POINTER(C.c_int32)), ("edge_dst", C.POINTER(C.c_int32)),
+        ("feat_dim", C.c_int32), ("features", C.POINTER(C.c_float)),
+        ("n_hops", C.c_int32), ("n_classes", C.c_int32),
+        ("labels", C.POINTER(C.c_int32)), ("train_mask", C.POINTER(C.c_uint8)),
+        ("n_layers", C.c_int32), ("layer_widths", C.POINTER(C.c_int32)),
+        ("rho", C.c_float), ("nu", C.c_float), ("quant_levels", C.c_int32),
+        ("init_W", C.POINTER(C.POINTER(C.c_float))),
+        ("device", C.c_int32), ("flags", C.c_uint32),
+    ]
+
+
+def lib() -> C.CDLL:
+    """Load the shared library (once)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2105_09837_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        L.pdadmm_last_error.restype = C.c_char_p
+        L.pdadmm_profile_name.restype = C.c_char_p
+        L.pdadmm_init.argtypes = [C.POINTER(_Config), C.POINTER(C.c_void_p)]
+        L.pdadmm_step.argtypes = [C.c_void_p, C.c_int]
+        L.pdadmm_objective.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
+        L.pdadmm_residuals.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.c_int]
+        L.pdadmm_get_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
+        L.pdadmm_set_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
+        L.pdadmm_quantize.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_float, C.c_int, C.c_void_p, C.c_void_p]
+        L.pdadmm_spmm.argtypes = [C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.pdadmm_profile.argtypes = [C.c_void_p, C.c_int]
+        L.pdadmm_profile_name.argtypes = [C.c_int]
+        L.pdadmm_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64),
+                                          C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.pdadmm_launches.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        L.pdadmm_destroy.argtypes = [C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise PdadmmError(rc, lib().pdadmm_last_error().decode())
+
+
+def _ptr(a: np.ndarray, ctype):
+    return a.ctypes.data_as(C.POINTER(ctype))
+
+
+class Context:
+    """One problem on one device (``pdadmm_ctx``)."""
+
+    def __init__(self, n_nodes: int, edge_src, edge_dst, features, n_hops: int, n_classes: int, labels, train_mask,
+                 layer_widths: Sequence[int], rho: float, nu: float, quant_levels: int, init_W: List[np.ndarray],
+                 device: int = 0, flags: int = 0):
+        self._h = C.c_void_p()
+        src = np.ascontiguousarray(edge_src, dtype=np.int32)
+        dst = np.ascontiguousarray(edge_dst, dtype=np.int32)
+        feat = np.ascontiguousarray(features, dtype=np.float32)
+        lab = np.ascontiguousarray(labels, dtype=np.int32)
+        msk = np.ascontiguousarray(train_mask, dtype=np.uint8)
+        widths = np.ascontiguousarray(layer_widths, dtype=np.int32)
+        Ws = [np.ascontiguousarray(w, dtype=np.float32) for w in init_W]
+        if feat.ndim != 2 or feat.shape[0] != n_nodes:
+            raise ValueError("features must be [n_nodes][feat_dim]")
+        n_in = (n_hops + 1) * feat.shape[1]
+        if len(Ws) != len(widths):
+            raise ValueError("one initial weight matrix per layer is required")
+        for w, n_out in zip(Ws, widths):
+            if w.shape != (int(n_out), n_in):
+                raise ValueError(f"init_W has shape {w.shape}, expected {(int(n_out), n_in)}")
+            n_in = int(n_out)
+        if lab.shape != (n_nodes,) or msk.shape != (n_nodes,) or src.shape != dst.shape:
+            raise ValueError("labels/mask must be [n_nodes]; edge arrays must have equal length")
+        wp = (C.POINTER(C.c_float) * len(Ws))(*[_ptr(w, C.c_float) for w in Ws])
+        cfg = _Config(n_nodes, src.size, _ptr(src, C.c_int32), _ptr(dst, C.c_int32), feat.shape[1],
+                      _ptr(feat, C.c_float), n_hops, n_classes, _ptr(lab, C.c_int32), _ptr(msk, C.c_uint8),
+                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, wp, device, flags)
+        self.n_nodes, self.n_layers = int(n_nodes), len(widths)
+        self.n0 = (n_hops + 1) * feat.shape[1]
+        self.widths = [int(x) for x in widths]
+        self.quant_levels = int(quant_levels)
+        _check(lib().pdadmm_init(C.byref(cfg), C.byref(self._h)))
+
+    # ---- same names as the C ABI
+    def step(self, n_iters: int = 1):
+        _check(lib().pdadmm_step(self._h, int(n_iters)))
+
+    def objective(self) -> np.ndarray:
+        out = (C.c_double * 6)()
+        _check(lib().pdadmm_objective(self._h, out))
+        return np.array(out[:])
+
+    def residuals(self) -> np.ndarray:
+        n = self.n_layers - 1
+        out = (C.c_double * max(n, 1))()
+        _check(lib().pdadmm_residuals(self._h, out if n else None, n))
+        return np.array(out[:n])
+
+    def _shape(self, kind: int, layer: int):
+        n_in = self.n0 if layer <= 1 else self.widths[layer - 2]
+        n_out = self.widths[layer - 1] if 1 <= layer <= self.n_layers else 0
+        N = self.n_nodes
+        if kind == T_X:
+            return (N, self.n0), np.float32
+        if kind == T_P:
+            return (N, n_in), np.float32
+        if kind == T_W:
+            return (n_out, n_in), np.float32
+        if kind == T_B:
+            return (n_out,), np.float32
+        if kind in (T_Z, T_Q, T_U):
+            return (N, n_out), np.float32
+        if kind == T_CODES:
+            return (N, n_in), np.uint8
+        if kind in (T_TAU, T_THETA):
+            return (1,), np.float64
+        if kind == T_QSCALE:
+            return (1,), np.float32
+        if kind == T_TRIALS:
+            return (1,), np.int32
+        if kind == T_CSR_ROWPTR:
+            return (N + 1,), np.int32
+        raise ValueError(kind)
+
+    def get_tensor(self, kind: int, layer: int = 1) -> np.ndarray:
+        if kind in (T_CSR_COLIDX, T_CSR_VAL):
+            nnz = int(self.get_tensor(T_CSR_ROWPTR)[-1])
+            shape, dt = (nnz,), (np.int32 if kind == T_CSR_COLIDX else np.float32)
+        else:
+            shape, dt = self._shape(kind, layer)
+        out = np.empty(shape, dtype=dt)
+        _check(lib().pdadmm_get_tensor(self._h, kind, layer, out.ctypes.data_as(C.c_void_p), out.nbytes))
+        return out
+
+    def set_tensor(self, kind: int, layer: int, value):
+        shape, dt = self._shape(kind, layer)
+        a = np.ascontiguousarray(value, dtype=dt)
+        if a.shape != shape:
+            raise ValueError(f"tensor kind {kind} layer {layer} has shape {shape}, got {a.shape}")
+        _check(lib().pdadmm_set_tensor(self._h, kind, layer, a.ctypes.data_as(C.c_void_p), a.nbytes))
+
+    def profile(self, enable: bool):
+        _check(lib().pdadmm_profile(self._h, int(bool(enable))))
+
+    def profile_read(self) -> dict:
+        out = {}
+        for k in range(lib().pdadmm_profile_classes()):
+            ms, n, by, fl = C.c_double(), C.c_int64(), C.c_double(), C.c_double()
+            _check(lib().pdadmm_profile_read(self._h, k, C.byref(ms), C.byref(n), C.byref(by), C.byref(fl)))
+            out[lib().pdadmm_profile_name(k).decode()] = dict(ms=ms.value, launches=n.value, bytes=by.value, flops=fl.value)
+        return out
+
+    def launches(self) -> int:
+        n = C.c_int64()
+        _check(lib().pdadmm_launches(self._h, C.byref(n)))
+        return n.value
+
+    def destroy(self):
+        if self._h:
+            lib().pdadmm_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def from_inputs(inp, device: int = 0, flags: int = 0, rho: Optional[float] = None, nu: Optional[float] = None,
+                quant_levels: Optional[int] = None) -> Context:
+    """Context for a ``synth.Inputs`` bundle."""
+    w = inp.workload
+    return Context(w.n_nodes, inp.edge_src, inp.edge_dst, inp.features, w.n_hops, w.n_classes, inp.labels,
+                   inp.train_mask, w.widths, w.rho if rho is None else rho, w.nu if nu is None else nu,
+                   w.quant_levels if quant_levels is None else quant_levels, inp.init_W, device, flags)
+
+
+def quantize(x, scale: float, levels: int, device: int = 0):
+    """``pdadmm_quantize``: (codes uint8, p float32) for a float32 array."""
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    codes = np.empty(a.shape, dtype=np.uint8)
+    p = np.empty(a.shape, dtype=np.float32)
+    _check(lib().pdadmm_quantize(device, a.ctypes.data_as(C.c_void_p), a.size, scale, levels,
+                                 codes.ctypes.data_as(C.c_void_p), p.ctypes.data_as(C.c_void_p)))
+    return codes, p
+
+
+def spmm(row_ptr, col_idx, val, x, device: int = 0) -> np.ndarray:
+    """``pdadmm_spmm``: Y = A X for a CSR matrix and a node-major float32 matrix."""
+    rp = np.ascontiguousarray(row_ptr, dtype=np.int32)
+    ci = np.ascontiguousarray(col_idx, dtype=np.int32)
+    v = np.ascontiguousarray(val, dtype=np.float32)
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    y = np.empty_like(a)
+    _check(lib().pdadmm_spmm(device, rp.size - 1, rp.ctypes.data_as(C.c_void_p), ci.ctypes.data_as(C.c_void_p),
+                             v.ctypes.data_as(C.c_void_p), a.ctypes.data_as(C.c_void_p), a.shape[1],
+                             y.ctypes.data_as(C.c_void_p)))
+    return y

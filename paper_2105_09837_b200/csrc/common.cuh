@@ -1,0 +1,81 @@
+// Shared host/device helpers of the pdADMM library: status codes, error text, reductions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string>
+
+#include "../../include/pdadmm.h"
+
+namespace pd {
+
+// ---- thread-local error text ------------------------------------------------------------------
+inline std::string &err_text() {
+  static thread_local std::string s;
+  return s;
+}
+inline int fail(int code, const char *fmt, ...) __attribute__((format(printf, 2, 3)));
+inline int fail(int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  err_text() = buf;
+  return code;
+}
+
+#define PD_CUDA(expr)                                                                             \
+  do {                                                                                            \
+    cudaError_t e__ = (expr);                                                                     \
+    if (e__ != cudaSuccess)                                                                       \
+      return pd::fail(e__ == cudaErrorMemoryAllocation ? PDADMM_ENOMEM : PDADMM_ECUDA,           \
+                      "%s:%d: %s -> %s", __FILE__, __LINE__, #expr, cudaGetErrorString(e__));     \
+  } while (0)
+
+#define PD_TRY(expr)            \
+  do {                          \
+    int rc__ = (expr);          \
+    if (rc__ != PDADMM_OK) return rc__; \
+  } while (0)
+
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- device reductions -------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Sum of one double per thread over the block; the result is valid in thread 0.
+// Warps are combined in index order, so the result does not depend on scheduling.
+template <int THREADS>
+__device__ __forceinline__ double block_sum(double v, double *smem /* THREADS/32 doubles */) {
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) smem[w] = v;
+  __syncthreads();
+  double t = 0.0;
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int i = 0; i < THREADS / 32; ++i) t += smem[i];
+  }
+  return t;
+}
+
+}  // namespace pd

@@ -1,0 +1,386 @@
+// Elementwise, reduction and per-node kernels of one pdADMM-G / pdADMM-G-Q iteration.
+//
+// All matrices are node-major [N][ld] float32 with ld a multiple of 4 and zero padding columns,
+// so a matrix is processed as a flat array of N*ld/4 float4 values.  Every operation below maps
+// zero padding to zero padding.  Sums are accumulated per block in double precision and written
+// to a slot per block; a single-block kernel adds the slots in index order, so results do not
+// depend on scheduling.
+#pragma once
+
+#include "common.cuh"
+
+namespace pd {
+
+constexpr int EW_THREADS = 256;
+
+// Scalars of one layer that live on the device (so that an iteration needs no host round trip).
+struct LayerScalars {
+  double sum_g2;      // ||g||^2
+  double sum_wg2;     // ||W g||^2
+  double sum_d2;      // ||p+ - p||^2        (quantised trial)
+  double sum_wd2;     // ||W (p+ - p)||^2    (quantised trial)
+  double sum_G2;      // ||grad_W||^2
+  double sum_Gp2;     // ||grad_W p+||^2
+  double res2;        // ||p_{l+1} - q_l||^2
+  double tau;         // tau_l
+  double theta;       // theta_l (0 if grad_W = 0)
+  float inv_tau;      // 1/tau
+  float inv_theta;    // 1/theta, 0 if grad_W = 0
+  int accepted;       // quantised trial: 1 if the stop condition held
+  int trials;         // trials so far in this iteration
+};
+
+__device__ __forceinline__ float4 ld4(const float *p, size_t i) { return reinterpret_cast<const float4 *>(p)[i]; }
+__device__ __forceinline__ void st4(float *p, size_t i, float4 v) { reinterpret_cast<float4 *>(p)[i] = v; }
+
+// ---- final, fixed-order reduction of per-block slots -------------------------------------------
+// out[j] = sum_i slots[i * stride + j], j < n_out, i < n_slots   (one block; thread j strides over outputs)
+__global__ void reduce_slots_kernel(const double *__restrict__ slots, int n_slots, int stride, int n_out,
+                                    double *__restrict__ out) {
+  for (int j = threadIdx.x; j < n_out; j += blockDim.x) {
+    double s = 0.0;
+    for (int i = 0; i < n_slots; ++i) s += slots[(size_t)i * stride + j];
+    out[j] = s;
+  }
+}
+
+// Quantisation to m uniform levels starting at 0 (Eq. "update p quantized", elementwise argmin):
+// code = clamp(floor(x/s + 1/2), 0, m-1), value = float(code) * s with a single rounding.
+__device__ __forceinline__ float quantize_one(float x, float s, float top, unsigned &code) {
+  float c = floorf(__fdiv_rn(x, s) + 0.5f);
+  c = fminf(fmaxf(c, 0.0f), top);
+  code = (unsigned)c;
+  return __fmul_rn(c, s);
+}
+
+// ---- y -= x * (*inv) ----------------------------------------------------------------------------
+// p-update  p+ = p - g/tau  (Eq. "update p") and the matching update of the linear residual,
+// r <- r - (W g)/tau, and r <- r - (grad_W p+)/theta after the W-update (Eq. "update W").
+__global__ void __launch_bounds__(EW_THREADS)
+axpy_neg_kernel(float *__restrict__ y, const float *__restrict__ x, const float *__restrict__ inv, size_t n4) {
+  const float a = *inv;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = ld4(y, i);
+    const float4 w = ld4(x, i);
+    v.x = fmaf(-a, w.x, v.x); v.y = fmaf(-a, w.y, v.y); v.z = fmaf(-a, w.z, v.z); v.w = fmaf(-a, w.w, v.w);
+    st4(y, i, v);
+  }
+}
+
+// y += x   (r <- r + W d after an accepted quantised step)
+__global__ void __launch_bounds__(EW_THREADS)
+add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = ld4(y, i);
+    const float4 w = ld4(x, i);
+    v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+    st4(y, i, v);
+  }
+}
+
+// ---- quantised trial step ------------------------------------------------------------------------
+// x = p - g/tau; p_new = nearest level; d = p_new - p; codes; per-block sum of d^2.
+__global__ void __launch_bounds__(EW_THREADS)
+quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, const LayerScalars *__restrict__ sc,
+                   float scale, int levels, float *__restrict__ p_new, float *__restrict__ d,
+                   uint8_t *__restrict__ codes, size_t n4, double *__restrict__ slots) {
+  __shared__ double red[EW_THREADS / 32];
+  const float inv_tau = sc->inv_tau, top = (float)(levels - 1);
+  double ss = 0.0;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 pv = ld4(p, i), gv = ld4(g, i);
+    unsigned c0, c1, c2, c3;
+    float4 nv, dv;
+    nv.x = quantize_one(fmaf(-inv_tau, gv.x, pv.x), scale, top, c0);
+    nv.y = quantize_one(fmaf(-inv_tau, gv.y, pv.y), scale, top, c1);
+    nv.z = quantize_one(fmaf(-inv_tau, gv.z, pv.z), scale, top, c2);
+    nv.w = quantize_one(fmaf(-inv_tau, gv.w, pv.w), scale, top, c3);
+    dv.x = nv.x - pv.x; dv.y = nv.y - pv.y; dv.z = nv.z - pv.z; dv.w = nv.w - pv.w;
+    ss += (double)dv.x * dv.x + (double)dv.y * dv.y + (double)dv.z * dv.z + (double)dv.w * dv.w;
+    st4(p_new, i, nv);
+    st4(d, i, dv);
+    reinterpret_cast<uchar4 *>(codes)[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
+  }
+  const double tot = block_sum<EW_THREADS>(ss, red);
+  if (threadIdx.x == 0) slots[blockIdx.x] = tot;
+}
+
+// Plain projection of an array (initial forward pass, pdadmm_quantize, pdadmm_set_tensor).
+__global__ void __launch_bounds__(EW_THREADS)
+quantize_kernel(const float *__restrict__ x, size_t n, float scale, int levels, float *__restrict__ p_out,
+                uint8_t *__restrict__ codes_out) {
+  const float top = (float)(levels - 1);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    unsigned c;
+    const float v = quantize_one(x[i], scale, top, c);
+    if (p_out) p_out[i] = v;
+    if (codes_out) codes_out[i] = (uint8_t)c;
+  }
+}
+
+// ---- single-thread finalisers of the step parameters ---------------------------------------------
+// tau = rho + nu ||W g||^2 / ||g||^2 : the smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
+__global__ void finalize_tau_kernel(LayerScalars *sc, double rho, double nu) {
+  const double gg = sc->sum_g2;
+  const double tau = gg > 0.0 ? rho + nu * sc->sum_wg2 / gg : rho;
+  sc->tau = tau;
+  sc->inv_tau = (float)(1.0 / tau);
+  sc->accepted = 0;
+  sc->trials = 0;
+}
+// Stop condition of the quantised step in its quadratic form: nu||W d||^2 + rho||d||^2 <= tau||d||^2 (1 + slack).
+// Not accepted: tau is doubled for the next trial.
+__global__ void finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack) {
+  const double dd = sc->sum_d2;
+  const bool ok = nu * sc->sum_wd2 + rho * dd <= sc->tau * dd * (1.0 + slack);
+  sc->trials += 1;
+  sc->accepted = ok ? 1 : 0;
+  if (!ok) {
+    sc->tau *= 2.0;
+    sc->inv_tau = (float)(1.0 / sc->tau);
+  }
+}
+// theta = nu ||grad_W p+||^2 / ||grad_W||^2 : the smallest theta with phi(W+) <= V_l(W+; theta).
+__global__ void finalize_theta_kernel(LayerScalars *sc, double nu) {
+  const double GG = sc->sum_G2;
+  const double theta = GG > 0.0 ? nu * sc->sum_Gp2 / GG : 0.0;
+  sc->theta = theta;
+  sc->inv_theta = theta > 0.0 ? (float)(1.0 / theta) : 0.0f;
+}
+
+// ---- reduction of the split partial tiles of grad_W, scaling by nu, ||grad_W||^2 ------------------
+__global__ void __launch_bounds__(EW_THREADS)
+reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, float nu, float *__restrict__ G,
+                    double *__restrict__ slots) {
+  __shared__ double red[EW_THREADS / 32];
+  double ss = 0.0;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < n_split; ++s) {
+      const float4 v = ld4(part + (size_t)s * n4 * 4, i);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    a.x *= nu; a.y *= nu; a.z *= nu; a.w *= nu;
+    ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
+    st4(G, i, a);
+  }
+  const double tot = block_sum<EW_THREADS>(ss, red);
+  if (threadIdx.x == 0) slots[blockIdx.x] = tot;
+}
+
+// ---- column sums of r - gp * inv_theta  (for the b-update) ----------------------------------------
+// Block b handles rows [b*rows_per_block, ...); thread c strides over columns.  slots[b][ld].
+__global__ void __launch_bounds__(EW_THREADS)
+resid_colsum_kernel(float *__restrict__ r, const float *__restrict__ gp, const LayerScalars *__restrict__ sc,
+                    int n_rows, int ld, int rows_per_block, double *__restrict__ slots) {
+  const float a = sc->inv_theta;
+  const int r0 = blockIdx.x * rows_per_block, r1 = min(n_rows, r0 + rows_per_block);
+  for (int c = threadIdx.x; c < ld; c += blockDim.x) {
+    double s = 0.0;
+    for (int j = r0; j < r1; ++j) {
+      const size_t o = (size_t)j * ld + c;
+      const float v = fmaf(-a, gp[o], r[o]);
+      r[o] = v;
+      s += (double)v;
+    }
+    slots[(size_t)blockIdx.x * ld + c] = s;
+  }
+}
+
+// b+ = b - mean_j r[j][:]  (Eq. "update b" with the step 1/(nu N), i.e. the exact minimiser);
+// shift[c] = that mean, which the z-update subtracts from r.
+__global__ void finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int width, double inv_n,
+                                     float *__restrict__ b, float *__restrict__ shift) {
+  for (int c = threadIdx.x + blockIdx.x * blockDim.x; c < ld; c += blockDim.x * gridDim.x) {
+    double s = 0.0;
+    for (int i = 0; i < n_slots; ++i) s += slots[(size_t)i * ld + c];
+    const float m = c < width ? (float)(s * inv_n) : 0.0f;
+    shift[c] = m;
+    if (c < width) b[c] -= m;
+  }
+}
+
+// ---- z-, q-, u-update of a hidden layer, fused ----------------------------------------------------
+// a = W+ p+ + b+ = (r - shift) + z.  z+ by the ReLU closed form of Eq. "update z" (better of the two
+// half-line minimisers; a tie keeps the non-positive one), q+ by Eq. "update q", residual p_{l+1} - q+,
+// u+ by Eq. "update u", and the linear residual of the next iteration r = a - z+.
+__global__ void __launch_bounds__(EW_THREADS)
+zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
+           const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
+           float rho, float nu, double *__restrict__ slots) {
+  __shared__ double red[EW_THREADS / 32];
+  const float inv_rn = 1.0f / (rho + nu);
+  double ss = 0.0;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 sh = ld4(shift, i % ld4cols);
+    const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i), pv = ld4(p_next, i);
+    float4 zn, qn, un, rn;
+#define PD_ZQU(f)                                                                   \
+    {                                                                               \
+      const float a = (rv.f - sh.f) + zv.f;                                         \
+      const float zneg = fminf(0.5f * (a + zv.f), 0.0f);                            \
+      const float zpos = fmaxf((a + qv.f + zv.f) * (1.0f / 3.0f), 0.0f);            \
+      const float fneg = (zneg - a) * (zneg - a) + qv.f * qv.f + (zneg - zv.f) * (zneg - zv.f); \
+      const float fpos = (zpos - a) * (zpos - a) + (qv.f - zpos) * (qv.f - zpos) + (zpos - zv.f) * (zpos - zv.f); \
+      const float zz = fpos < fneg ? zpos : zneg;                                   \
+      const float qq = (rho * pv.f + uv.f + nu * fmaxf(zz, 0.0f)) * inv_rn;         \
+      const float res = pv.f - qq;                                                  \
+      zn.f = zz; qn.f = qq; un.f = fmaf(rho, res, uv.f); rn.f = a - zz;             \
+      ss += (double)res * res;                                                      \
+    }
+    PD_ZQU(x) PD_ZQU(y) PD_ZQU(z) PD_ZQU(w)
+#undef PD_ZQU
+    st4(z, i, zn); st4(q, i, qn); st4(u, i, un); st4(r, i, rn);
+  }
+  const double tot = block_sum<EW_THREADS>(ss, red);
+  if (threadIdx.x == 0) slots[blockIdx.x] = tot;
+}
+
+// ---- z-update of the last layer -------------------------------------------------------------------
+// One thread per node.  a = (r - shift) + z.  Labelled node: z+ = argmin CE(z; y) + (nu/2)||z - a||^2
+// (Eq. "update zl"), the unique root of softmax(z) - e_y + nu (z - a) = 0, by damped Newton with the
+// Hessian diag(s) + nu I - s s^T inverted through the rank-one update formula; double precision
+// inside, since nu is small and the Hessian is close to singular along (1,..,1).  Unlabelled: z+ = a.
+constexpr int ZL_MAX_C = 64;
+__global__ void __launch_bounds__(128)
+zlast_kernel(float *__restrict__ r, float *__restrict__ z, const float *__restrict__ shift,
+             const int *__restrict__ labels, const uint8_t *__restrict__ mask, int n_rows, int C, int ld,
+             double nu, int *__restrict__ not_converged) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n_rows) return;
+  float *rj = r + (size_t)j * ld, *zj = z + (size_t)j * ld;
+  double a[ZL_MAX_C], x[ZL_MAX_C], s[ZL_MAX_C], st[ZL_MAX_C];
+  for (int c = 0; c < C; ++c) { a[c] = (double)((rj[c] - shift[c]) + zj[c]); x[c] = a[c]; }
+  if (mask[j]) {
+    const int y = labels[j];
+    auto fval = [&](const double *v) {
+      double m = v[0];
+      for (int c = 1; c < C; ++c) m = fmax(m, v[c]);
+      double se = 0.0, sq = 0.0;
+      for (int c = 0; c < C; ++c) { se += exp(v[c] - m); sq += (v[c] - a[c]) * (v[c] - a[c]); }
+      return m + log(se) - v[y] + 0.5 * nu * sq;
+    };
+    double fx = fval(x);
+    bool done = false;
+    for (int it = 0; it < 100 && !done; ++it) {
+      double m = x[0];
+      for (int c = 1; c < C; ++c) m = fmax(m, x[c]);
+      double se = 0.0;
+      for (int c = 0; c < C; ++c) { s[c] = exp(x[c] - m); se += s[c]; }
+      double gmax = 0.0, s_mg = 0.0, s_ms = 0.0;
+      for (int c = 0; c < C; ++c) {
+        s[c] /= se;
+        const double g = s[c] - (c == y ? 1.0 : 0.0) + nu * (x[c] - a[c]);
+        gmax = fmax(gmax, fabs(g));
+        const double mi = 1.0 / (s[c] + nu);
+        st[c] = g;                       // gradient for now
+        s_mg += s[c] * mi * g;
+        s_ms += s[c] * mi * s[c];
+      }
+      if (gmax <= 1e-10) { done = true; break; }
+      const double k = s_mg / (1.0 - s_ms);
+      double slope = 0.0;
+      for (int c = 0; c < C; ++c) {
+        const double mi = 1.0 / (s[c] + nu);
+        const double g = st[c];
+        const double d = -(mi * g + mi * s[c] * k);
+        slope += g * d;
+        st[c] = d;                       // Newton step
+      }
+      const bool resolvable = -slope > 1e-9 * (1.0 + fabs(fx));
+      double t = 1.0, ft;
+      for (;;) {
+        for (int c = 0; c < C; ++c) s[c] = x[c] + t * st[c];
+        ft = fval(s);
+        if (!resolvable || ft <= fx + 1e-4 * t * slope || t < 1e-12) break;
+        t *= 0.5;
+      }
+      for (int c = 0; c < C; ++c) x[c] = s[c];
+      fx = ft;
+    }
+    if (!done) atomicAdd(not_converged, 1);
+  }
+  for (int c = 0; c < C; ++c) {
+    const float zn = (float)x[c];
+    zj[c] = zn;
+    rj[c] = (float)(a[c] - (double)zn);
+  }
+}
+
+// ---- elementwise helpers of the initial forward pass ---------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+relu_max_kernel(const float *__restrict__ z, float *__restrict__ q, size_t n4, float *__restrict__ block_max) {
+  __shared__ float red[EW_THREADS / 32];
+  float m = 0.0f;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = ld4(z, i);
+    v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f);
+    m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+    st4(q, i, v);
+  }
+  m = warp_max(m);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < EW_THREADS / 32; ++i) m = fmaxf(m, red[i]);
+    block_max[blockIdx.x] = m;
+  }
+}
+
+// ---- objective pieces of one layer ---------------------------------------------------------------
+// slots[b][0..3] = sum r^2, sum (q - relu z)^2, sum u (p_next - q), sum (p_next - q)^2 ; q == nullptr: only r^2.
+__global__ void __launch_bounds__(EW_THREADS)
+objective_layer_kernel(const float *__restrict__ r, const float *__restrict__ z, const float *__restrict__ q,
+                       const float *__restrict__ u, const float *__restrict__ p_next, size_t n,
+                       double *__restrict__ slots) {
+  __shared__ double red[EW_THREADS / 32];
+  double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const double rv = r[i];
+    s0 += rv * rv;
+    if (q != nullptr) {
+      const double qv = q[i], act = fmaxf(z[i], 0.0f), res = (double)p_next[i] - qv;
+      s1 += (qv - act) * (qv - act);
+      s2 += (double)u[i] * res;
+      s3 += res * res;
+    }
+  }
+  double t;
+  t = block_sum<EW_THREADS>(s0, red); if (threadIdx.x == 0) slots[blockIdx.x * 4 + 0] = t;
+  t = block_sum<EW_THREADS>(s1, red); if (threadIdx.x == 0) slots[blockIdx.x * 4 + 1] = t;
+  t = block_sum<EW_THREADS>(s2, red); if (threadIdx.x == 0) slots[blockIdx.x * 4 + 2] = t;
+  t = block_sum<EW_THREADS>(s3, red); if (threadIdx.x == 0) slots[blockIdx.x * 4 + 3] = t;
+}
+
+// R(z_L; y): sum over masked nodes of -z_y + logsumexp(z).  One thread per node, one slot per block.
+__global__ void __launch_bounds__(EW_THREADS)
+risk_kernel(const float *__restrict__ z, const int *__restrict__ labels, const uint8_t *__restrict__ mask,
+            int n_rows, int C, int ld, double *__restrict__ slots) {
+  __shared__ double red[EW_THREADS / 32];
+  double acc = 0.0;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n_rows; j += gridDim.x * blockDim.x) {
+    if (!mask[j]) continue;
+    const float *zj = z + (size_t)j * ld;
+    double m = zj[0];
+    for (int c = 1; c < C; ++c) m = fmax(m, (double)zj[c]);
+    double se = 0.0;
+    for (int c = 0; c < C; ++c) se += exp((double)zj[c] - m);
+    acc += m + log(se) - (double)zj[labels[j]];
+  }
+  const double t = block_sum<EW_THREADS>(acc, red);
+  if (threadIdx.x == 0) slots[blockIdx.x] = t;
+}
+
+// W+ = W - grad_W * inv_theta  (Eq. "update W")
+__global__ void __launch_bounds__(EW_THREADS)
+wstep_kernel(float *__restrict__ W, const float *__restrict__ G, const LayerScalars *__restrict__ sc, size_t n4) {
+  const float a = sc->inv_theta;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = ld4(W, i);
+    const float4 g = ld4(G, i);
+    v.x = fmaf(-a, g.x, v.x); v.y = fmaf(-a, g.y, v.y); v.z = fmaf(-a, g.z, v.z); v.w = fmaf(-a, g.w, v.w);
+    st4(W, i, v);
+  }
+}
+
+}  // namespace pd

@@ -1,0 +1,803 @@
+// pdADMM-G / pdADMM-G-Q on one B200: context, host orchestration of one iteration, C ABI.
+//
+// Data layout (device): every N x width matrix is node-major with its leading dimension padded to a
+// multiple of 4 floats and zero padding columns.  Per layer l the context keeps p_l, z_l, q_l, u_l,
+// W_l, b_l and the linear residual r_l = W_l p_l + b_l - z_l, which every step of the iteration
+// updates in place instead of recomputing the product:
+//     p+ = p - g/tau        =>  r <- r - (W g)/tau            (pdADMM-G-Q: r <- r + W (p+ - p))
+//     W+ = W - G/theta      =>  r <- r - (G p+)/theta
+//     b+ = b - mean_j r     =>  r <- r - mean_j r
+//     z+                    =>  r <- (r + z) - z+
+// so one iteration of a layer costs four dense products: W^T r (the p-gradient), W g (tau),
+// r^T p+ (the W-gradient, contraction over the nodes) and G p+ (theta).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <memory>
+#include <vector>
+
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "gemm_simt.cuh"
+#include "graph.cuh"
+
+namespace pd {
+
+// ---- kernel classes for the per-kernel timing -----------------------------------------------------
+enum KClass {
+  KC_GEMM_RESID = 0,  // r = P W^T + b - z                    (after init / set_tensor only)
+  KC_GEMM_GRADP,      // g = nu r W + u + rho (p - q), ||g||^2
+  KC_GEMM_WG,         // W g (or W d), squared norm
+  KC_GEMM_GRADW,      // partial tiles of r^T p+ over node slices
+  KC_GRADW_REDUCE,    // sum of the partial tiles, nu, ||G||^2
+  KC_GEMM_GP,         // G p+, squared norm
+  KC_AXPY,            // p -= g/tau ; r -= (Wg)/tau ; r += W d
+  KC_QUANT,           // quantised trial step
+  KC_COLSUM,          // r -= (G p+)/theta with column sums
+  KC_ZQU,             // fused z, q, u update of a hidden layer
+  KC_ZLAST,           // z update of the last layer
+  KC_WSTEP,           // W -= G/theta
+  KC_SMALL,           // single-block finalisers
+  KC_COUNT
+};
+static const char *kclass_names[KC_COUNT] = {
+    "gemm_resid", "gemm_gradp", "gemm_wg", "gemm_gradw", "gradw_reduce", "gemm_gp", "axpy",
+    "quant_trial", "resid_colsum", "zqu", "zlast", "wstep", "finalize"};
+
+struct Layer {
+  int n_in = 0, n_out = 0, ld_in = 0, ld_out = 0;
+  float *p = nullptr;       // [N][ld_in]  (layer 1: X)
+  float *W = nullptr;       // [n_out][ld_in]
+  float *b = nullptr;       // [ld_out]
+  float *z = nullptr, *r = nullptr;          // [N][ld_out]
+  float *q = nullptr, *u = nullptr;          // [N][ld_out], hidden layers only
+  float *gradW = nullptr;   // [n_out][ld_in]
+  float *shift = nullptr;   // [ld_out] column means removed by the b-update
+  uint8_t *codes = nullptr; // [N][ld_in], quantised mode, l >= 2
+  float scale = 1.0f;
+  LayerScalars *sc = nullptr;
+  int n_split = 1, k_chunk = 0;
+};
+
+struct Scratch {
+  cudaStream_t st = nullptr;
+  float *s1 = nullptr;      // g, later G p+
+  float *s2 = nullptr;      // W g, later W d
+  float *p_new = nullptr;   // quantised trial
+  float *d = nullptr;       // quantised trial
+  uint8_t *codes_new = nullptr;
+  float *part = nullptr;    // partial tiles of grad_W
+  double *slots = nullptr;  // per-block partial sums
+  size_t n_slots = 0;
+};
+
+struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
+
+}  // namespace pd
+
+struct pdadmm_ctx {
+  int device = 0;
+  int64_t N = 0;
+  int L = 0, d = 0, n_blocks = 0, n0 = 0, ld0 = 0, C = 0, levels = 0;
+  float rho = 0, nu = 0;
+  uint32_t flags = 0;
+  int64_t nnz = 0;
+  int *row_ptr = nullptr, *col_idx = nullptr;
+  float *csr_val = nullptr;
+  int *labels = nullptr;
+  uint8_t *mask = nullptr;
+  std::vector<pd::Layer> layers;
+  pd::Scratch scr;
+  bool r_valid = false;
+  int *d_flag = nullptr;            // device counter (z_L solver non-convergence)
+  int *h_pinned = nullptr;          // pinned host words for small read-backs
+  int64_t launches = 0;
+  bool profiling = false;
+  std::vector<pd::ProfRec> prof;
+  std::vector<cudaEvent_t> ev_pool;
+  double prof_ms[pd::KC_COUNT] = {0}, prof_bytes[pd::KC_COUNT] = {0}, prof_flops[pd::KC_COUNT] = {0};
+  int64_t prof_n[pd::KC_COUNT] = {0};
+  std::vector<void *> allocs;
+};
+
+namespace pd {
+
+// ---- allocation bookkeeping -------------------------------------------------------------------------
+template <class T>
+static int dev_alloc(pdadmm_ctx *c, T **ptr, size_t count, bool zero = true) {
+  void *p = nullptr;
+  const size_t bytes = std::max<size_t>(count * sizeof(T), 16);
+  cudaError_t e = cudaMalloc(&p, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(PDADMM_ENOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+  }
+  c->allocs.push_back(p);
+  if (zero) PD_CUDA(cudaMemsetAsync(p, 0, bytes, c->scr.st));   // same stream as every kernel that uses it
+  *ptr = (T *)p;
+  return PDADMM_OK;
+}
+
+static inline int ew_grid(size_t n_items) {
+  return (int)std::max<size_t>(1, std::min<size_t>(ceil_div((int64_t)n_items, EW_THREADS), 148 * 8));
+}
+
+// ---- profiling hooks ----------------------------------------------------------------------------------
+static cudaEvent_t take_event(pdadmm_ctx *c) {
+  cudaEvent_t e;
+  if (!c->ev_pool.empty()) { e = c->ev_pool.back(); c->ev_pool.pop_back(); return e; }
+  cudaEventCreate(&e);
+  return e;
+}
+struct Launch {                    // brackets one kernel launch
+  pdadmm_ctx *c; int cls; cudaStream_t st; double bytes, flops; cudaEvent_t e0 = nullptr;
+  Launch(pdadmm_ctx *c_, int cls_, cudaStream_t st_, double bytes_, double flops_)
+      : c(c_), cls(cls_), st(st_), bytes(bytes_), flops(flops_) {
+    c->launches++;
+    if (c->profiling) { e0 = take_event(c); cudaEventRecord(e0, st); }
+  }
+  ~Launch() {
+    if (c->profiling) {
+      cudaEvent_t e1 = take_event(c);
+      cudaEventRecord(e1, st);
+      c->prof.push_back({cls, e0, e1, bytes, flops});
+    }
+  }
+};
+static int prof_collect(pdadmm_ctx *c) {
+  if (c->prof.empty()) return PDADMM_OK;
+  PD_CUDA(cudaDeviceSynchronize());
+  for (auto &r : c->prof) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, r.e0, r.e1);
+    c->prof_ms[r.cls] += ms; c->prof_n[r.cls]++; c->prof_bytes[r.cls] += r.bytes; c->prof_flops[r.cls] += r.flops;
+    c->ev_pool.push_back(r.e0); c->ev_pool.push_back(r.e1);
+  }
+  c->prof.clear();
+  return PDADMM_OK;
+}
+
+// ---- fixed-order sum of per-block slots into a field of the layer's scalars ---------------------------
+static void sum_slots(pdadmm_ctx *c, cudaStream_t st, const double *slots, int n_slots, double *dst) {
+  Launch l(c, KC_SMALL, st, 8.0 * n_slots, 0);
+  reduce_slots_kernel<<<1, 32, 0, st>>>(slots, n_slots, 1, 1, dst);
+}
+
+// ---- dense products --------------------------------------------------------------------------------------
+// C[M][N] = A[M][K] * op(B), fused epilogue; per-block sums of squares go to `partials` (or nullptr).
+template <bool B_NMAJOR, class Epi>
+static void gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
+                       const float *B, int ldb, const Epi &epi, double *partials, int *n_partials, double extra_bytes) {
+  dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM));
+  if (n_partials) *n_partials = (int)(grid.x * grid.y);
+  const double bytes = 4.0 * ((double)M * K + (double)N * K + (double)M * N) + extra_bytes;
+  Launch l(c, cls, st, bytes, 2.0 * M * N * K);
+  gemm_nt_kernel<B_NMAJOR, Epi><<<grid, SG_THREADS, 0, st>>>(M, N, K, A, lda, B, ldb, epi, partials);
+}
+
+}  // namespace pd
+
+namespace pd {
+
+// ---- pieces of one iteration -------------------------------------------------------------------------------
+
+// r_l = P_l W_l^T + b_l - z_l from scratch (only when the cached residual is not valid).
+static void refresh_residual(pdadmm_ctx *c, Layer &ly, cudaStream_t st) {
+  EpiLinearResidual epi{ly.r, ly.ld_out, ly.b, ly.z};
+  gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)c->N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, epi, nullptr,
+                    nullptr, 4.0 * c->N * ly.n_out);
+}
+
+// g = nu r W + u_{l-1} + rho (p - q_{l-1}) -> s1, ||g||^2 ; W g -> s2, ||W g||^2 ; tau.
+static void p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
+  Layer &ly = c->layers[l];
+  Layer &prev = c->layers[l - 1];
+  Scratch &s = c->scr;
+  const int N = (int)c->N;
+  int np = 0;
+  EpiGradP epi{s.s1, ly.ld_in, prev.u, ly.p, prev.q, c->nu, c->rho};
+  gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.ld_in, epi, s.slots, &np,
+                   3.0 * 4.0 * N * ly.n_in);
+  sum_slots(c, s.st, s.slots, np, &ly.sc->sum_g2);
+  EpiStoreSumsq epi2{s.s2, ly.ld_out};
+  gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, epi2, s.slots, &np, 0);
+  sum_slots(c, s.st, s.slots, np, &ly.sc->sum_wg2);
+  {
+    Launch k(c, KC_SMALL, s.st, 0, 0);
+    finalize_tau_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu);
+  }
+}
+
+// pdADMM-G: p <- p - g/tau, r <- r - (W g)/tau.
+static void p_step_plain(pdadmm_ctx *c, int l) {
+  Layer &ly = c->layers[l];
+  Scratch &s = c->scr;
+  const size_t n4p = (size_t)c->N * ly.ld_in / 4, n4r = (size_t)c->N * ly.ld_out / 4;
+  {
+    Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_in, 0);
+    axpy_neg_kernel<<<ew_grid(n4p), EW_THREADS, 0, s.st>>>(ly.p, s.s1, &ly.sc->inv_tau, n4p);
+  }
+  {
+    Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_out, 0);
+    axpy_neg_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, &ly.sc->inv_tau, n4r);
+  }
+}
+
+// pdADMM-G-Q: project p - g/tau on the level set, doubling tau until the stop condition holds.
+// Each trial ends with a read-back of the accept flag (the only host round trip of an iteration).
+static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
+  Layer &ly = c->layers[l];
+  Scratch &s = c->scr;
+  const int N = (int)c->N;
+  const size_t n4p = (size_t)N * ly.ld_in / 4, n4r = (size_t)N * ly.ld_out / 4;
+  const int max_trials = 30;
+  for (int trial = 0;; ++trial) {
+    const int grid = ew_grid(n4p);
+    {
+      Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
+      quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, c->levels, s.p_new, s.d,
+                                                       s.codes_new, n4p, s.slots);
+    }
+    sum_slots(c, s.st, s.slots, grid, &ly.sc->sum_d2);
+    int np = 0;
+    EpiStoreSumsq epi{s.s2, ly.ld_out};
+    gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, epi, s.slots, &np, 0);
+    sum_slots(c, s.st, s.slots, np, &ly.sc->sum_wd2);
+    {
+      Launch k(c, KC_SMALL, s.st, 0, 0);
+      finalize_trial_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6);
+    }
+    PD_CUDA(cudaMemcpyAsync(c->h_pinned, &ly.sc->accepted, sizeof(int), cudaMemcpyDeviceToHost, s.st));
+    PD_CUDA(cudaStreamSynchronize(s.st));
+    if (c->h_pinned[0] || trial + 1 >= max_trials) {
+      if (!c->h_pinned[0]) *hit_cap = true;
+      break;
+    }
+  }
+  std::swap(ly.p, s.p_new);
+  std::swap(ly.codes, s.codes_new);
+  {
+    Launch k(c, KC_AXPY, s.st, 12.0 * N * ly.n_out, 0);
+    add_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, n4r);
+  }
+  return PDADMM_OK;
+}
+
+// G = nu r^T p+ (contraction over nodes), theta, W <- W - G/theta, r <- r - (G p+)/theta,
+// b <- b - mean_j r, shift = mean_j r.
+static void w_and_b_step(pdadmm_ctx *c, int l) {
+  Layer &ly = c->layers[l];
+  Scratch &s = c->scr;
+  const int N = (int)c->N;
+  {
+    dim3 grid((unsigned)ceil_div(ly.n_in, SG_BN), (unsigned)ceil_div(ly.n_out, SG_BM), (unsigned)ly.n_split);
+    Launch k(c, KC_GEMM_GRADW, s.st, 4.0 * ((double)N * ly.n_in + (double)N * ly.n_out), 2.0 * N * ly.n_in * ly.n_out);
+    gemm_tn_kernel<<<grid, SG_THREADS, 0, s.st>>>(ly.n_out, ly.n_in, N, ly.k_chunk, ly.r, ly.ld_out, ly.p, ly.ld_in,
+                                                 s.part, ly.ld_in);
+  }
+  const size_t n4w = (size_t)ly.n_out * ly.ld_in / 4;
+  const int gw = ew_grid(n4w);
+  {
+    Launch k(c, KC_GRADW_REDUCE, s.st, 4.0 * (ly.n_split + 1.0) * ly.n_out * ly.n_in, 0);
+    reduce_gradW_kernel<<<gw, EW_THREADS, 0, s.st>>>(s.part, ly.n_split, n4w, c->nu, ly.gradW, s.slots);
+  }
+  sum_slots(c, s.st, s.slots, gw, &ly.sc->sum_G2);
+  int np = 0;
+  EpiStoreSumsq epi{s.s1, ly.ld_out};
+  gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.ld_in, epi, s.slots, &np, 0);
+  sum_slots(c, s.st, s.slots, np, &ly.sc->sum_Gp2);
+  {
+    Launch k(c, KC_SMALL, s.st, 0, 0);
+    finalize_theta_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->nu);
+  }
+  {
+    Launch k(c, KC_WSTEP, s.st, 12.0 * ly.n_out * ly.n_in, 0);
+    wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w);
+  }
+  const int n_blocks = (int)std::min<int64_t>(148 * 4, ceil_div(N, 8));
+  const int rows_per_block = (int)ceil_div(N, n_blocks);
+  const int used_blocks = (int)ceil_div(N, rows_per_block);
+  {
+    Launch k(c, KC_COLSUM, s.st, 12.0 * N * ly.n_out, 0);
+    resid_colsum_kernel<<<used_blocks, EW_THREADS, 0, s.st>>>(ly.r, s.s1, ly.sc, N, ly.ld_out, rows_per_block, s.slots);
+  }
+  {
+    Launch k(c, KC_SMALL, s.st, 8.0 * used_blocks * ly.ld_out, 0);
+    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 128), 128, 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
+                                                                          1.0 / (double)N, ly.b, ly.shift);
+  }
+}
+
+// z (and q, u for hidden layers) of layer l; needs p_{l+1} of this iteration.
+static void zqu_step(pdadmm_ctx *c, int l) {
+  Layer &ly = c->layers[l];
+  Scratch &s = c->scr;
+  const int N = (int)c->N;
+  if (l + 1 < c->L) {
+    const size_t n4 = (size_t)N * ly.ld_out / 4;
+    const int grid = ew_grid(n4);
+    {
+      Launch k(c, KC_ZQU, s.st, 36.0 * N * ly.n_out, 0);
+      zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, c->layers[l + 1].p, ly.shift, ly.ld_out / 4, n4,
+                                               c->rho, c->nu, s.slots);
+    }
+    sum_slots(c, s.st, s.slots, grid, &ly.sc->res2);
+  } else {
+    Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
+    zlast_kernel<<<(int)ceil_div(N, 128), 128, 0, s.st>>>(ly.r, ly.z, ly.shift, c->labels, c->mask, N, ly.n_out,
+                                                          ly.ld_out, (double)c->nu, c->d_flag);
+  }
+}
+
+static int iterate_once(pdadmm_ctx *c, bool *hit_cap) {
+  // p-update of layers 2..L from the iterates of the previous iteration
+  for (int l = 1; l < c->L; ++l) {
+    p_gradient_and_tau(c, l);
+    if (c->levels) PD_TRY(p_step_quantised(c, l, hit_cap));
+    else p_step_plain(c, l);
+  }
+  // W- and b-update of every layer with the new p
+  for (int l = 0; l < c->L; ++l) w_and_b_step(c, l);
+  // z-, q-, u-update (q_l and u_l need p_{l+1} of this iteration)
+  for (int l = 0; l < c->L; ++l) zqu_step(c, l);
+  return PDADMM_OK;
+}
+
+}  // namespace pd
+
+namespace pd {
+
+// ---- construction ---------------------------------------------------------------------------------------------
+
+static int check_config(const pdadmm_config *cfg) {
+  if (!cfg) return fail(PDADMM_EINVAL, "config is null");
+  if (cfg->n_nodes < 1 || cfg->n_nodes > (int64_t)INT32_MAX / 2) return fail(PDADMM_EINVAL, "n_nodes out of range");
+  if (cfg->n_edges < 0 || (cfg->n_edges > 0 && (!cfg->edge_src || !cfg->edge_dst)))
+    return fail(PDADMM_EINVAL, "edge list missing");
+  if (cfg->feat_dim < 1 || !cfg->features) return fail(PDADMM_EINVAL, "features missing");
+  if (cfg->n_hops < 0 || cfg->n_hops > 16) return fail(PDADMM_EINVAL, "n_hops must be in [0, 16]");
+  if (cfg->n_layers < 1 || !cfg->layer_widths || !cfg->init_W) return fail(PDADMM_EINVAL, "layers missing");
+  if (cfg->n_classes < 2 || cfg->n_classes > ZL_MAX_C)
+    return fail(PDADMM_EINVAL, "n_classes must be in [2, %d]", ZL_MAX_C);
+  if (cfg->layer_widths[cfg->n_layers - 1] != cfg->n_classes)
+    return fail(PDADMM_EINVAL, "last layer width must equal n_classes");
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    if (cfg->layer_widths[l] < 1) return fail(PDADMM_EINVAL, "layer width %d is not positive", l + 1);
+    if (!cfg->init_W[l]) return fail(PDADMM_EINVAL, "init_W[%d] is null", l);
+  }
+  if (!cfg->labels || !cfg->train_mask) return fail(PDADMM_EINVAL, "labels or mask missing");
+  if (!(cfg->rho > 0.f) || !(cfg->nu > 0.f)) return fail(PDADMM_EINVAL, "rho and nu must be positive");
+  if (cfg->quant_levels != 0 && (cfg->quant_levels < 2 || cfg->quant_levels > 256))
+    return fail(PDADMM_EINVAL, "quant_levels must be 0 or in [2, 256]");
+  for (int64_t j = 0; j < cfg->n_nodes; ++j)
+    if (cfg->labels[j] < 0 || cfg->labels[j] >= cfg->n_classes)
+      return fail(PDADMM_EINVAL, "label of node %lld is outside [0, %d)", (long long)j, cfg->n_classes);
+  return PDADMM_OK;
+}
+
+// Host -> device copies go through the context's stream, so that they are ordered with its kernels
+// (the stream does not synchronise with the default stream).
+static int upload_rows(cudaStream_t st, float *dst, int ld, const float *src, int width, int64_t rows) {
+  PD_CUDA(cudaMemcpy2DAsync(dst, (size_t)ld * 4, src, (size_t)width * 4, (size_t)width * 4, (size_t)rows,
+                            cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaStreamSynchronize(st));
+  return PDADMM_OK;
+}
+
+static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
+  const int64_t N = cfg->n_nodes;
+  c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
+  c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, 4); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
+  c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
+  PD_CUDA(cudaSetDevice(cfg->device));
+  PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
+  cudaStream_t st = c->scr.st;
+  PD_CUDA(cudaMallocHost((void **)&c->h_pinned, 64 * sizeof(int)));
+  PD_TRY(dev_alloc(c, &c->d_flag, 4));
+
+  // graph: CSR pattern on the host, values and sparse products on the device
+  std::vector<int32_t> rp, ci;
+  PD_TRY(build_csr_pattern(N, cfg->n_edges, cfg->edge_src, cfg->edge_dst, rp, ci));
+  c->nnz = (int64_t)ci.size();
+  PD_TRY(dev_alloc(c, &c->row_ptr, (size_t)N + 1, false));
+  PD_TRY(dev_alloc(c, &c->col_idx, ci.size(), false));
+  PD_TRY(dev_alloc(c, &c->csr_val, ci.size(), false));
+  PD_CUDA(cudaMemcpyAsync(c->row_ptr, rp.data(), rp.size() * 4, cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaMemcpyAsync(c->col_idx, ci.data(), ci.size() * 4, cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaStreamSynchronize(st));
+  adjacency_values_kernel<<<(int)ceil_div(N * 32, 256), 256, 0, st>>>(c->row_ptr, c->col_idx, (int)N, c->csr_val);
+  PD_TRY(dev_alloc(c, &c->labels, (size_t)N, false));
+  PD_TRY(dev_alloc(c, &c->mask, (size_t)N, false));
+  PD_CUDA(cudaMemcpyAsync(c->labels, cfg->labels, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaMemcpyAsync(c->mask, cfg->train_mask, (size_t)N, cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaStreamSynchronize(st));
+
+  // layers
+  c->layers.resize(c->L);
+  int max_in = 0, max_out = 0;
+  size_t max_part = 0;
+  for (int l = 1; l < c->L; ++l) max_in = std::max(max_in, round_up(cfg->layer_widths[l - 1], 4));
+  for (int l = 0; l < c->L; ++l) {
+    Layer &ly = c->layers[l];
+    ly.n_in = l == 0 ? c->n0 : cfg->layer_widths[l - 1];
+    ly.n_out = cfg->layer_widths[l];
+    ly.ld_in = round_up(ly.n_in, 4); ly.ld_out = round_up(ly.n_out, 4);
+    max_out = std::max(max_out, ly.ld_out);
+    const size_t e_out = (size_t)N * ly.ld_out;
+    // quantised mode: p_l and its codes trade places with the trial buffers, so all share one size
+    const size_t e_in = (size_t)N * ((c->levels && l > 0) ? max_in : ly.ld_in);
+    PD_TRY(dev_alloc(c, &ly.p, e_in));
+    PD_TRY(dev_alloc(c, &ly.W, (size_t)ly.n_out * ly.ld_in));
+    PD_TRY(dev_alloc(c, &ly.gradW, (size_t)ly.n_out * ly.ld_in));
+    PD_TRY(dev_alloc(c, &ly.b, (size_t)ly.ld_out));
+    PD_TRY(dev_alloc(c, &ly.shift, (size_t)ly.ld_out));
+    PD_TRY(dev_alloc(c, &ly.z, e_out));
+    PD_TRY(dev_alloc(c, &ly.r, e_out));
+    if (l + 1 < c->L) { PD_TRY(dev_alloc(c, &ly.q, e_out)); PD_TRY(dev_alloc(c, &ly.u, e_out)); }
+    if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in));
+    PD_TRY(dev_alloc(c, &ly.sc, 1));
+    PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
+    // node slices of the W-gradient product: enough blocks to fill the device twice, slices >= 256 nodes
+    const int64_t tiles = ceil_div(ly.n_in, SG_BN) * ceil_div(ly.n_out, SG_BM);
+    int split = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(2 * 148, tiles), ceil_div(N, 256)));
+    ly.k_chunk = round_up((int)ceil_div(N, split), SG_BK);
+    ly.n_split = (int)ceil_div(N, ly.k_chunk);
+    max_part = std::max(max_part, (size_t)ly.n_split * ly.n_out * ly.ld_in);
+  }
+  // scratch
+  Scratch &s = c->scr;
+  const size_t e_max = (size_t)N * std::max(max_in, max_out);
+  PD_TRY(dev_alloc(c, &s.s1, e_max));
+  PD_TRY(dev_alloc(c, &s.s2, (size_t)N * max_out));
+  if (c->levels) {
+    PD_TRY(dev_alloc(c, &s.p_new, (size_t)N * max_in));
+    PD_TRY(dev_alloc(c, &s.d, (size_t)N * max_in));
+    PD_TRY(dev_alloc(c, &s.codes_new, (size_t)N * max_in));
+  }
+  PD_TRY(dev_alloc(c, &s.part, max_part));
+  s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
+  PD_TRY(dev_alloc(c, &s.slots, s.n_slots));
+
+  // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
+  Layer &l0 = c->layers[0];
+  PD_TRY(upload_rows(st, l0.p, l0.ld_in, cfg->features, c->d, N));
+  for (int k = 1; k < c->n_blocks; ++k)
+    launch_spmm(st, c->row_ptr, c->col_idx, c->csr_val, (int)N, l0.p + (size_t)(k - 1) * c->d, l0.p + (size_t)k * c->d,
+                c->d, l0.ld_in);
+
+  // start of Algorithm 1: b = 0, z_l = W_l p_l, q_l = ReLU(z_l), p_{l+1} = q_l (projected in -Q mode), u = 0
+  for (int l = 0; l < c->L; ++l) {
+    Layer &ly = c->layers[l];
+    EpiStore epi{ly.z, ly.ld_out};
+    gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, epi, nullptr,
+                      nullptr, 0);
+    if (l + 1 == c->L) break;
+    Layer &nx = c->layers[l + 1];
+    const size_t n4 = (size_t)N * ly.ld_out / 4;
+    const int grid = ew_grid(n4);
+    float *bm = reinterpret_cast<float *>(s.slots);
+    relu_max_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, ly.q, n4, bm);
+    if (c->levels) {
+      std::vector<float> hm(grid);
+      PD_CUDA(cudaMemcpyAsync(hm.data(), bm, grid * sizeof(float), cudaMemcpyDeviceToHost, st));
+      PD_CUDA(cudaStreamSynchronize(st));
+      float mx = 0.f;
+      for (float v : hm) mx = std::max(mx, v);
+      nx.scale = mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f;
+      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, c->levels, nx.p, nx.codes);
+    } else {
+      PD_CUDA(cudaMemcpyAsync(nx.p, ly.q, n4 * 16, cudaMemcpyDeviceToDevice, st));
+    }
+  }
+  PD_CUDA(cudaStreamSynchronize(st));
+  PD_CUDA(cudaGetLastError());
+  c->r_valid = true;                        // z = W p + b exactly by construction, r = 0 (allocated as zero)
+  c->launches = 0;
+  return PDADMM_OK;
+}
+
+static void destroy(pdadmm_ctx *c) {
+  if (!c) return;
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  for (auto &r : c->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+  for (auto e : c->ev_pool) cudaEventDestroy(e);
+  for (void *p : c->allocs) cudaFree(p);
+  if (c->h_pinned) cudaFreeHost(c->h_pinned);
+  if (c->scr.st) cudaStreamDestroy(c->scr.st);
+  delete c;
+}
+
+}  // namespace pd
+
+// ======================================================================================================
+// C ABI
+// ======================================================================================================
+using namespace pd;
+
+extern "C" const char *pdadmm_last_error(void) { return err_text().c_str(); }
+
+extern "C" int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out) {
+  if (!out) return fail(PDADMM_EINVAL, "out is null");
+  *out = nullptr;
+  PD_TRY(check_config(cfg));
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
+    cudaGetLastError();
+    return fail(PDADMM_ECUDA, "no CUDA device is available");
+  }
+  if (cfg->device < 0 || cfg->device >= n_dev) return fail(PDADMM_EINVAL, "device %d does not exist", cfg->device);
+  pdadmm_ctx *c = new (std::nothrow) pdadmm_ctx();
+  if (!c) return fail(PDADMM_ENOMEM, "out of host memory");
+  int rc;
+  try {
+    rc = build(c, cfg);
+  } catch (const std::bad_alloc &) {
+    rc = fail(PDADMM_ENOMEM, "out of host memory");
+  }
+  if (rc != PDADMM_OK) { destroy(c); return rc; }
+  *out = c;
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_destroy(pdadmm_ctx *c) {
+  destroy(c);
+  return PDADMM_OK;
+}
+
+static int ensure_residual(pdadmm_ctx *c) {
+  if (c->r_valid) return PDADMM_OK;
+  for (int l = 0; l < c->L; ++l) refresh_residual(c, c->layers[l], c->scr.st);
+  c->r_valid = true;
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
+  if (!c) return fail(PDADMM_EINVAL, "context is null");
+  if (n_iters < 0) return fail(PDADMM_EINVAL, "n_iters is negative");
+  PD_CUDA(cudaSetDevice(c->device));
+  PD_CUDA(cudaMemsetAsync(c->d_flag, 0, sizeof(int), c->scr.st));
+  PD_TRY(ensure_residual(c));
+  bool hit_cap = false;
+  for (int k = 0; k < n_iters; ++k) PD_TRY(iterate_once(c, &hit_cap));
+  PD_CUDA(cudaMemcpyAsync(c->h_pinned + 8, c->d_flag, sizeof(int), cudaMemcpyDeviceToHost, c->scr.st));
+  PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  PD_CUDA(cudaGetLastError());
+  if (c->profiling) PD_TRY(prof_collect(c));
+  if (c->h_pinned[8] != 0)
+    return fail(PDADMM_ENOTCONV, "the last-layer z solver did not converge on %d nodes", c->h_pinned[8]);
+  if (hit_cap) return fail(PDADMM_ENOTCONV, "the tau search of a quantised p-update reached its trial cap");
+  return PDADMM_OK;
+}
+
+static int read_slots(pdadmm_ctx *c, int n_slots, int stride, int n_out, double *host) {
+  double *dst = c->scr.slots + c->scr.n_slots - 8;            // tail of the slot buffer: results
+  reduce_slots_kernel<<<1, 32, 0, c->scr.st>>>(c->scr.slots, n_slots, stride, n_out, dst);
+  PD_CUDA(cudaMemcpyAsync(host, dst, n_out * sizeof(double), cudaMemcpyDeviceToHost, c->scr.st));
+  PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_objective(pdadmm_ctx *c, double out[6]) {
+  if (!c || !out) return fail(PDADMM_EINVAL, "null argument");
+  PD_CUDA(cudaSetDevice(c->device));
+  PD_TRY(ensure_residual(c));
+  cudaStream_t st = c->scr.st;
+  double lin = 0, act = 0, dual = 0, pen = 0, R = 0;
+  for (int l = 0; l < c->L; ++l) {
+    Layer &ly = c->layers[l];
+    const size_t n = (size_t)c->N * ly.ld_out;
+    const int grid = std::min(ew_grid(n), 512);
+    const bool hidden = l + 1 < c->L;
+    objective_layer_kernel<<<grid, EW_THREADS, 0, st>>>(ly.r, ly.z, hidden ? ly.q : nullptr, ly.u,
+                                                       hidden ? c->layers[l + 1].p : nullptr, n, c->scr.slots);
+    double h[4];
+    PD_TRY(read_slots(c, grid, 4, 4, h));
+    lin += h[0]; act += h[1]; dual += h[2]; pen += h[3];
+  }
+  {
+    Layer &ly = c->layers[c->L - 1];
+    const int grid = (int)std::min<int64_t>(512, ceil_div(c->N, EW_THREADS));
+    risk_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, c->labels, c->mask, (int)c->N, ly.n_out, ly.ld_out, c->scr.slots);
+    PD_TRY(read_slots(c, grid, 1, 1, &R));
+  }
+  PD_CUDA(cudaGetLastError());
+  out[0] = R; out[1] = 0.5 * c->nu * lin; out[2] = 0.5 * c->nu * act; out[3] = dual; out[4] = 0.5 * c->rho * pen;
+  out[5] = out[0] + out[1] + out[2] + out[3] + out[4];
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_residuals(pdadmm_ctx *c, double *per_layer_sq, int n) {
+  if (!c) return fail(PDADMM_EINVAL, "context is null");
+  if (n != c->L - 1 || (n > 0 && !per_layer_sq)) return fail(PDADMM_EINVAL, "n must be L-1 = %d", c->L - 1);
+  PD_CUDA(cudaSetDevice(c->device));
+  PD_TRY(ensure_residual(c));
+  for (int l = 0; l + 1 < c->L; ++l) {
+    Layer &ly = c->layers[l];
+    const size_t nn = (size_t)c->N * ly.ld_out;
+    const int grid = std::min(ew_grid(nn), 512);
+    objective_layer_kernel<<<grid, EW_THREADS, 0, c->scr.st>>>(ly.r, ly.z, ly.q, ly.u, c->layers[l + 1].p, nn,
+                                                              c->scr.slots);
+    double h[4];
+    PD_TRY(read_slots(c, grid, 4, 4, h));
+    per_layer_sq[l] = h[3];
+  }
+  PD_CUDA(cudaGetLastError());
+  return PDADMM_OK;
+}
+
+// ---- tensors in and out -------------------------------------------------------------------------------------
+struct TensorRef { void *ptr; size_t rows, width, ld, elem; bool settable; };
+
+static int locate(pdadmm_ctx *c, int kind, int layer, TensorRef *t) {
+  const int L = c->L;
+  auto need = [&](int lo, int hi) {
+    return (layer >= lo && layer <= hi) ? PDADMM_OK
+                                        : fail(PDADMM_EINVAL, "layer %d is outside [%d, %d] for tensor kind %d", layer, lo, hi, kind);
+  };
+  const size_t N = (size_t)c->N;
+  switch (kind) {
+    case PDADMM_T_X: { Layer &y = c->layers[0]; *t = {y.p, N, (size_t)y.n_in, (size_t)y.ld_in, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_P: { PD_TRY(need(1, L)); Layer &y = c->layers[layer - 1]; *t = {y.p, N, (size_t)y.n_in, (size_t)y.ld_in, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_W: { PD_TRY(need(1, L)); Layer &y = c->layers[layer - 1]; *t = {y.W, (size_t)y.n_out, (size_t)y.n_in, (size_t)y.ld_in, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_B: { PD_TRY(need(1, L)); Layer &y = c->layers[layer - 1]; *t = {y.b, 1, (size_t)y.n_out, (size_t)y.ld_out, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_Z: { PD_TRY(need(1, L)); Layer &y = c->layers[layer - 1]; *t = {y.z, N, (size_t)y.n_out, (size_t)y.ld_out, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_Q: { PD_TRY(need(1, L - 1)); Layer &y = c->layers[layer - 1]; *t = {y.q, N, (size_t)y.n_out, (size_t)y.ld_out, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_U: { PD_TRY(need(1, L - 1)); Layer &y = c->layers[layer - 1]; *t = {y.u, N, (size_t)y.n_out, (size_t)y.ld_out, 4, true}; return PDADMM_OK; }
+    case PDADMM_T_CODES: {
+      if (!c->levels) return fail(PDADMM_EINVAL, "codes exist only in quantised mode");
+      PD_TRY(need(2, L)); Layer &y = c->layers[layer - 1];
+      *t = {y.codes, N, (size_t)y.n_in, (size_t)y.ld_in, 1, false}; return PDADMM_OK;
+    }
+    case PDADMM_T_TAU: { PD_TRY(need(2, L)); *t = {&c->layers[layer - 1].sc->tau, 1, 1, 1, 8, false}; return PDADMM_OK; }
+    case PDADMM_T_THETA: { PD_TRY(need(1, L)); *t = {&c->layers[layer - 1].sc->theta, 1, 1, 1, 8, false}; return PDADMM_OK; }
+    case PDADMM_T_TRIALS: { PD_TRY(need(2, L)); *t = {&c->layers[layer - 1].sc->trials, 1, 1, 1, 4, false}; return PDADMM_OK; }
+    case PDADMM_T_CSR_ROWPTR: *t = {c->row_ptr, 1, N + 1, N + 1, 4, false}; return PDADMM_OK;
+    case PDADMM_T_CSR_COLIDX: *t = {c->col_idx, 1, (size_t)c->nnz, (size_t)c->nnz, 4, false}; return PDADMM_OK;
+    case PDADMM_T_CSR_VAL: *t = {c->csr_val, 1, (size_t)c->nnz, (size_t)c->nnz, 4, false}; return PDADMM_OK;
+    default: return fail(PDADMM_EINVAL, "unknown tensor kind %d", kind);
+  }
+}
+
+extern "C" int pdadmm_get_tensor(pdadmm_ctx *c, int kind, int layer, void *host_dst, size_t bytes) {
+  if (!c || !host_dst) return fail(PDADMM_EINVAL, "null argument");
+  PD_CUDA(cudaSetDevice(c->device));
+  if (kind == PDADMM_T_QSCALE) {
+    if (layer < 2 || layer > c->L || bytes != 4) return fail(PDADMM_EINVAL, "QSCALE: layer in [2, L], 4 bytes");
+    memcpy(host_dst, &c->layers[layer - 1].scale, 4);
+    return PDADMM_OK;
+  }
+  TensorRef t;
+  PD_TRY(locate(c, kind, layer, &t));
+  if (bytes != t.rows * t.width * t.elem)
+    return fail(PDADMM_EINVAL, "tensor kind %d layer %d has %zu bytes, caller passed %zu", kind, layer,
+                t.rows * t.width * t.elem, bytes);
+  PD_CUDA(cudaMemcpy2DAsync(host_dst, t.width * t.elem, t.ptr, t.ld * t.elem, t.width * t.elem, t.rows,
+                            cudaMemcpyDeviceToHost, c->scr.st));
+  PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void *host_src, size_t bytes) {
+  if (!c || !host_src) return fail(PDADMM_EINVAL, "null argument");
+  PD_CUDA(cudaSetDevice(c->device));
+  if (kind == PDADMM_T_QSCALE) {
+    if (layer < 2 || layer > c->L || bytes != 4) return fail(PDADMM_EINVAL, "QSCALE: layer in [2, L], 4 bytes");
+    float v;
+    memcpy(&v, host_src, 4);
+    if (!(v > 0.f)) return fail(PDADMM_EINVAL, "QSCALE must be positive");
+    c->layers[layer - 1].scale = v;
+    return PDADMM_OK;
+  }
+  TensorRef t;
+  PD_TRY(locate(c, kind, layer, &t));
+  if (!t.settable) return fail(PDADMM_EINVAL, "tensor kind %d is read-only", kind);
+  if (bytes != t.rows * t.width * t.elem)
+    return fail(PDADMM_EINVAL, "tensor kind %d layer %d has %zu bytes, caller passed %zu", kind, layer,
+                t.rows * t.width * t.elem, bytes);
+  PD_CUDA(cudaMemcpy2DAsync(t.ptr, t.ld * t.elem, host_src, t.width * t.elem, t.width * t.elem, t.rows,
+                            cudaMemcpyHostToDevice, c->scr.st));
+  PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  if (kind == PDADMM_T_X || kind == PDADMM_T_P || kind == PDADMM_T_W || kind == PDADMM_T_B || kind == PDADMM_T_Z)
+    c->r_valid = false;
+  if (kind == PDADMM_T_P && c->levels && layer >= 2) {
+    Layer &y = c->layers[layer - 1];
+    const size_t n = (size_t)c->N * y.ld_in;
+    quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, c->levels, nullptr, y.codes);
+    PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  }
+  return PDADMM_OK;
+}
+
+// ---- stand-alone entry points for single kernels ------------------------------------------------------------------
+extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale, int levels, uint8_t *codes_out,
+                               float *p_out) {
+  if (!x && n) return fail(PDADMM_EINVAL, "x is null");
+  if (levels < 2 || levels > 256 || !(scale > 0.f)) return fail(PDADMM_EINVAL, "levels in [2,256], scale > 0");
+  if (n == 0) return PDADMM_OK;
+  PD_CUDA(cudaSetDevice(device));
+  float *dx = nullptr, *dp = nullptr;
+  uint8_t *dc = nullptr;
+  int rc = PDADMM_OK;
+  auto body = [&]() -> int {
+    PD_CUDA(cudaMalloc((void **)&dx, n * 4));
+    PD_CUDA(cudaMalloc((void **)&dp, n * 4));
+    PD_CUDA(cudaMalloc((void **)&dc, n));
+    PD_CUDA(cudaMemcpy(dx, x, n * 4, cudaMemcpyHostToDevice));
+    quantize_kernel<<<ew_grid(n), EW_THREADS>>>(dx, n, scale, levels, dp, dc);
+    PD_CUDA(cudaGetLastError());
+    PD_CUDA(cudaDeviceSynchronize());
+    if (p_out) PD_CUDA(cudaMemcpy(p_out, dp, n * 4, cudaMemcpyDeviceToHost));
+    if (codes_out) PD_CUDA(cudaMemcpy(codes_out, dc, n, cudaMemcpyDeviceToHost));
+    return PDADMM_OK;
+  };
+  rc = body();
+  cudaFree(dx); cudaFree(dp); cudaFree(dc);
+  return rc;
+}
+
+extern "C" int pdadmm_spmm(int device, int64_t n_rows, const int32_t *row_ptr, const int32_t *col_idx, const float *val,
+                           const float *x, int32_t width, float *y_out) {
+  if (n_rows < 0 || width < 1 || !row_ptr || !y_out || !x) return fail(PDADMM_EINVAL, "bad argument");
+  if (n_rows == 0) return PDADMM_OK;
+  if (n_rows > INT32_MAX / 2) return fail(PDADMM_EINVAL, "too many rows");
+  if (row_ptr[0] != 0) return fail(PDADMM_EINVAL, "row_ptr[0] must be 0");
+  for (int64_t i = 0; i < n_rows; ++i)
+    if (row_ptr[i + 1] < row_ptr[i]) return fail(PDADMM_EINVAL, "row_ptr decreases at row %lld", (long long)i);
+  const int64_t nnz = row_ptr[n_rows];
+  if (nnz > 0 && (!col_idx || !val)) return fail(PDADMM_EINVAL, "col_idx or val is null");
+  for (int64_t e = 0; e < nnz; ++e)
+    if (col_idx[e] < 0 || col_idx[e] >= n_rows) return fail(PDADMM_EINVAL, "column index %lld out of range", (long long)e);
+  PD_CUDA(cudaSetDevice(device));
+  int *drp = nullptr, *dci = nullptr;
+  float *dv = nullptr, *dx = nullptr, *dy = nullptr;
+  auto body = [&]() -> int {
+    PD_CUDA(cudaMalloc((void **)&drp, (n_rows + 1) * 4));
+    PD_CUDA(cudaMalloc((void **)&dci, std::max<int64_t>(nnz, 1) * 4));
+    PD_CUDA(cudaMalloc((void **)&dv, std::max<int64_t>(nnz, 1) * 4));
+    PD_CUDA(cudaMalloc((void **)&dx, (size_t)n_rows * width * 4));
+    PD_CUDA(cudaMalloc((void **)&dy, (size_t)n_rows * width * 4));
+    PD_CUDA(cudaMemcpy(drp, row_ptr, (n_rows + 1) * 4, cudaMemcpyHostToDevice));
+    if (nnz) {
+      PD_CUDA(cudaMemcpy(dci, col_idx, nnz * 4, cudaMemcpyHostToDevice));
+      PD_CUDA(cudaMemcpy(dv, val, nnz * 4, cudaMemcpyHostToDevice));
+    }
+    PD_CUDA(cudaMemcpy(dx, x, (size_t)n_rows * width * 4, cudaMemcpyHostToDevice));
+    launch_spmm(0, drp, dci, dv, (int)n_rows, dx, dy, width, width);
+    PD_CUDA(cudaGetLastError());
+    PD_CUDA(cudaDeviceSynchronize());
+    PD_CUDA(cudaMemcpy(y_out, dy, (size_t)n_rows * width * 4, cudaMemcpyDeviceToHost));
+    return PDADMM_OK;
+  };
+  const int rc = body();
+  cudaFree(drp); cudaFree(dci); cudaFree(dv); cudaFree(dx); cudaFree(dy);
+  return rc;
+}
+
+// ---- timing ----------------------------------------------------------------------------------------------------
+extern "C" int pdadmm_profile(pdadmm_ctx *c, int enable) {
+  if (!c) return fail(PDADMM_EINVAL, "context is null");
+  PD_CUDA(cudaSetDevice(c->device));
+  PD_TRY(prof_collect(c));
+  for (int k = 0; k < KC_COUNT; ++k) { c->prof_ms[k] = 0; c->prof_n[k] = 0; c->prof_bytes[k] = 0; c->prof_flops[k] = 0; }
+  c->profiling = enable != 0;
+  return PDADMM_OK;
+}
+extern "C" int pdadmm_profile_classes(void) { return KC_COUNT; }
+extern "C" const char *pdadmm_profile_name(int k) { return (k >= 0 && k < KC_COUNT) ? kclass_names[k] : ""; }
+extern "C" int pdadmm_profile_read(pdadmm_ctx *c, int k, double *ms, int64_t *launches, double *bytes, double *flops) {
+  if (!c || k < 0 || k >= KC_COUNT) return fail(PDADMM_EINVAL, "bad argument");
+  PD_TRY(prof_collect(c));
+  if (ms) *ms = c->prof_ms[k];
+  if (launches) *launches = c->prof_n[k];
+  if (bytes) *bytes = c->prof_bytes[k];
+  if (flops) *flops = c->prof_flops[k];
+  return PDADMM_OK;
+}
+extern "C" int pdadmm_launches(pdadmm_ctx *c, int64_t *count) {
+  if (!c || !count) return fail(PDADMM_EINVAL, "null argument");
+  *count = c->launches;
+  return PDADMM_OK;
+}

@@ -1,0 +1,93 @@
+"""Helpers of the GPU parity tests: move states between the oracle (fp64, one column per node)
+and the C-ABI library (fp32, node-major), and compare them variable by variable."""
+
+from __future__ import annotations
+
+import numpy as np
+
+import oracle.pdadmm_oracle as o
+from paper_2105_09837_b200 import binding as B
+
+
+def oracle_problem(inp, rho=None, nu=None, quant_levels=None):
+    """(Params, initial oracle State) for a synth.Inputs bundle."""
+    w = inp.workload
+    prm = o.Params(w.rho if rho is None else rho, w.nu if nu is None else nu,
+                   w.quant_levels if quant_levels is None else quant_levels)
+    A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
+    X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
+    s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels, inp.train_mask, prm)
+    return prm, s, A
+
+
+def f32(a):
+    return np.asarray(a, dtype=np.float32).astype(np.float64)
+
+
+def round_state(s: o.State) -> o.State:
+    """The oracle state with every array rounded to single precision (what the device can hold)."""
+    n = s.copy()
+    for name in ("p", "W", "b", "z", "q", "u"):
+        setattr(n, name, [f32(a) for a in getattr(s, name)])
+    return n
+
+
+def load_state(ctx: B.Context, s: o.State, quantised: bool):
+    """Teacher forcing: write an (already fp32-representable) oracle state into the device context."""
+    L = s.L
+    for l in range(1, L + 1):
+        if l >= 2:
+            if quantised:
+                ctx.set_tensor(B.T_QSCALE, l, np.array([s.scale[l - 1]], dtype=np.float32))
+            ctx.set_tensor(B.T_P, l, s.p[l - 1].T)
+        ctx.set_tensor(B.T_W, l, s.W[l - 1])
+        ctx.set_tensor(B.T_B, l, s.b[l - 1])
+        ctx.set_tensor(B.T_Z, l, s.z[l - 1].T)
+        if l < L:
+            ctx.set_tensor(B.T_Q, l, s.q[l - 1].T)
+            ctx.set_tensor(B.T_U, l, s.u[l - 1].T)
+
+
+def read_state(ctx: B.Context) -> dict:
+    L = ctx.n_layers
+    out = {k: [] for k in ("p", "W", "b", "z", "q", "u")}
+    for l in range(1, L + 1):
+        out["p"].append(ctx.get_tensor(B.T_P, l).T.astype(np.float64))
+        out["W"].append(ctx.get_tensor(B.T_W, l).astype(np.float64))
+        out["b"].append(ctx.get_tensor(B.T_B, l).astype(np.float64))
+        out["z"].append(ctx.get_tensor(B.T_Z, l).T.astype(np.float64))
+        if l < L:
+            out["q"].append(ctx.get_tensor(B.T_Q, l).T.astype(np.float64))
+            out["u"].append(ctx.get_tensor(B.T_U, l).T.astype(np.float64))
+    return out
+
+
+def rel_err(got, want, mask=None) -> float:
+    """Relative Frobenius error over the unmasked elements (the norm of the reference is taken over the same elements)."""
+    if mask is not None:
+        got, want = got[~mask], want[~mask]
+    den = np.linalg.norm(want)
+    num = np.linalg.norm(got - want)
+    if den == 0.0:
+        return 0.0 if num == 0.0 else np.inf
+    return float(num / den)
+
+
+def z_tie_mask(prev: o.State, nxt: o.State, l: int, tol=1e-5):
+    """Elements of hidden layer l (0-based) whose two ReLU candidates have (nearly) the same objective:
+    both are minimisers there, so single and double precision may pick different ones."""
+    a = nxt.W[l] @ nxt.p[l] + nxt.b[l][:, None]
+    zn = np.minimum(0.5 * (a + prev.z[l]), 0.0)
+    zp = np.maximum((a + prev.q[l] + prev.z[l]) / 3.0, 0.0)
+    fn = o.z_objective_hidden(zn, a, prev.q[l], prev.z[l])
+    fp = o.z_objective_hidden(zp, a, prev.q[l], prev.z[l])
+    # equal candidates (both clamp to 0) are not a tie: either choice gives the same z
+    return (np.abs(fp - fn) <= tol * (np.abs(fp) + np.abs(fn) + 1e-30)) & (zp != zn)
+
+
+def boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=2e-4):
+    """Elements of p_l (0-based l >= 1) whose pre-quantisation value lies within `tol` levels of a rounding boundary."""
+    g = o.grad_p_phi(prev.p[l], prev.W[l], prev.b[l], prev.z[l], prm.nu, prev.q[l - 1], prev.u[l - 1], prm.rho)
+    t = (prev.p[l] - g / nxt.tau[l]) / prev.scale[l]
+    frac = t - np.floor(t)
+    return np.abs(frac - 0.5) <= tol

@@ -1,0 +1,141 @@
+"""GPU tests of single kernels and of edge cases, through the C ABI."""
+
+import numpy as np
+import pytest
+import scipy.sparse as sp
+
+import oracle.pdadmm_oracle as o
+from paper_2105_09837_b200 import binding as B
+from paper_2105_09837_b200 import synth
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("m,scale", [(2, 0.75), (16, 0.0173), (256, 0.011764706)])
+def test_quantise_kernel_is_bit_exact(m, scale):
+    rng = np.random.default_rng(m)
+    scale = float(np.float32(scale))
+    n = 1_000_003                                                   # ragged tail
+    x = rng.uniform(-2 * scale, (m + 1) * scale, n).astype(np.float32)
+    x[:m] = (np.arange(m, dtype=np.float32) + np.float32(0.5)) * np.float32(scale)   # half levels
+    x[m:2 * m] = np.arange(m, dtype=np.float32) * np.float32(scale)                  # exact levels
+    codes, p = B.quantize(x, scale, m)
+    want_codes, want_p = o.quantize(x, scale, m)
+    assert np.array_equal(codes, want_codes)
+    assert np.array_equal(p, want_p.astype(np.float32))
+    assert np.array_equal(p, codes.astype(np.float32) * np.float32(scale))
+    lev = o.level_set(scale, m)
+    assert np.all(np.isin(p.astype(np.float64), lev))
+
+
+def test_quantise_empty_input():
+    codes, p = B.quantize(np.zeros(0, np.float32), 1.0, 4)
+    assert codes.size == 0 and p.size == 0
+
+
+@pytest.mark.parametrize("width", [1, 6, 64, 250, 700])
+def test_spmm_against_sparse_library(width):
+    w = synth.small("c2", 3001, feat_dim=4)
+    src, dst = synth.make_graph(w)
+    A = o.renormalized_adjacency(w.n_nodes, src, dst)
+    x = np.random.default_rng(width).standard_normal((w.n_nodes, width)).astype(np.float32)
+    y = B.spmm(A.indptr, A.indices, A.data.astype(np.float32), x)
+    want = A.astype(np.float64) @ x.astype(np.float64)
+    assert U.rel_err(y.astype(np.float64), want) < 1e-6
+    # empty rows and an empty matrix
+    E = sp.csr_matrix((5, 5))
+    assert np.all(B.spmm(E.indptr, E.indices, E.data, np.ones((5, 3), np.float32)) == 0)
+
+
+def test_single_layer_model_and_zero_hops():
+    inp = synth.make_inputs(synth.small("c1", 333, feat_dim=9, hidden=5, n_layers=1, n_hops=0))
+    prm, s, _ = U.oracle_problem(inp)
+    ctx = B.from_inputs(inp)
+    assert ctx.residuals().size == 0
+    for k in range(3):
+        prev = U.round_state(s)
+        U.load_state(ctx, prev, False)
+        s = o.iterate(prev, prm)
+        ctx.step(1)
+        st = U.read_state(ctx)
+        assert U.rel_err(st["W"][0], s.W[0]) < 1e-4
+        assert U.rel_err(st["z"][0], s.z[0]) < 1e-4
+        assert np.linalg.norm(st["b"][0] - s.b[0]) <= 1e-4 * max(np.linalg.norm(s.b[0]), 1e-3)
+    assert abs(ctx.objective()[5] - o.objective(s, prm)[5]) <= 1e-4 * abs(o.objective(s, prm)[5])
+    ctx.destroy()
+
+
+def test_graph_without_edges_and_tiny_node_counts():
+    for n in (1, 2, 5):
+        w = synth.small("c1", n, feat_dim=3, hidden=4, n_layers=3)
+        inp = synth.make_inputs(w)
+        inp.edge_src = np.zeros(0, np.int32)
+        inp.edge_dst = np.zeros(0, np.int32)
+        inp.train_mask[:] = 1
+        prm, s, A = U.oracle_problem(inp)
+        ctx = B.from_inputs(inp)
+        assert np.array_equal(ctx.get_tensor(B.T_CSR_COLIDX), np.arange(n, dtype=np.int32))
+        assert np.allclose(ctx.get_tensor(B.T_CSR_VAL), 1.0)
+        assert U.rel_err(ctx.get_tensor(B.T_X).T.astype(np.float64), s.p[0]) < 1e-6
+        ctx.step(3)
+        for _ in range(3):
+            s = o.iterate(s, prm)
+        got = ctx.objective()
+        assert np.all(np.isfinite(got))
+        assert abs(got[5] - o.objective(s, prm)[5]) <= 1e-3 * abs(o.objective(s, prm)[5]) + 1e-9
+        ctx.destroy()
+
+
+def test_all_nodes_unlabelled_keeps_z_equal_to_a():
+    inp = synth.make_inputs(synth.small("c1", 200, feat_dim=5, hidden=6, n_layers=2))
+    inp.train_mask[:] = 0
+    prm, s, _ = U.oracle_problem(inp)
+    ctx = B.from_inputs(inp)
+    ctx.step(2)
+    for _ in range(2):
+        s = o.iterate(s, prm)
+    assert ctx.objective()[0] == 0.0
+    assert U.rel_err(ctx.get_tensor(B.T_Z, 2).T.astype(np.float64), s.z[1]) < 1e-4
+    ctx.destroy()
+
+
+def test_get_set_round_trip_and_size_checks():
+    inp = synth.make_inputs(synth.small("c2", 300, feat_dim=7, hidden=10, n_layers=3, quant_levels=16))
+    ctx = B.from_inputs(inp)
+    rng = np.random.default_rng(0)
+    for kind, layer in [(B.T_W, 2), (B.T_B, 1), (B.T_Z, 3), (B.T_Q, 1), (B.T_U, 2)]:
+        shape, dt = ctx._shape(kind, layer)
+        v = rng.standard_normal(shape).astype(dt)
+        ctx.set_tensor(kind, layer, v)
+        assert np.array_equal(ctx.get_tensor(kind, layer), v)
+    scale = ctx.get_tensor(B.T_QSCALE, 2)[0]
+    codes = rng.integers(0, 16, size=ctx._shape(B.T_P, 2)[0]).astype(np.uint8)
+    ctx.set_tensor(B.T_P, 2, codes.astype(np.float32) * scale)
+    assert np.array_equal(ctx.get_tensor(B.T_CODES, 2), codes)
+    lib = B.lib()
+    buf = np.zeros(10, np.float32)
+    assert lib.pdadmm_get_tensor(ctx._h, B.T_W, 1, buf.ctypes.data, 12) == B.EINVAL        # wrong size
+    assert lib.pdadmm_get_tensor(ctx._h, B.T_Q, 3, buf.ctypes.data, 40) == B.EINVAL        # q_L does not exist
+    assert lib.pdadmm_set_tensor(ctx._h, B.T_TAU, 2, buf.ctypes.data, 8) == B.EINVAL       # read-only
+    assert lib.pdadmm_set_tensor(ctx._h, 99, 1, buf.ctypes.data, 8) == B.EINVAL
+    assert "kind" in lib.pdadmm_last_error().decode()
+    assert lib.pdadmm_step(ctx._h, -1) == B.EINVAL
+    ctx.destroy()
+
+
+def test_profile_counters_and_launch_count():
+    inp = synth.make_inputs(synth.small("c2", 400, feat_dim=8, hidden=12, n_layers=3))
+    ctx = B.from_inputs(inp)
+    ctx.step(1)
+    n1 = ctx.launches()
+    assert n1 > 0
+    ctx.profile(True)
+    ctx.step(2)
+    prof = ctx.profile_read()
+    assert ctx.launches() == 3 * n1
+    assert sum(v["launches"] for v in prof.values()) == 2 * n1
+    assert prof["zqu"]["launches"] == 2 * 2 and prof["zqu"]["ms"] > 0 and prof["zqu"]["bytes"] > 0
+    assert prof["gemm_gradw"]["flops"] > 0
+    ctx.profile(False)
+    ctx.destroy()
