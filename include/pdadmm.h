@@ -114,6 +114,12 @@ int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out);
 int pdadmm_step(pdadmm_ctx *ctx, int n_iters);
 
 /*
+ * pdadmm_last_step_ms -- device time of the last pdadmm_step call in milliseconds, measured with CUDA
+ * events recorded on the context's own stream before the first and after the last kernel of the call.
+ */
+int pdadmm_last_step_ms(pdadmm_ctx *ctx, double *ms);
+
+/*
  * pdadmm_objective -- the augmented Lagrangian L_rho (paper, Section "The pdADMM-G Algorithm") of the
  * current state: out = { R(z_L;y), (nu/2) sum_l ||z_l - W_l p_l - b_l||^2, (nu/2) sum_l ||q_l - ReLU(z_l)||^2,
  * sum_l <u_l, p_{l+1} - q_l>, (rho/2) sum_l ||p_{l+1} - q_l||^2, their sum }.  R is the sum of the
@@ -153,6 +159,18 @@ int pdadmm_quantize(int device, const float *x, size_t n, float scale, int level
  */
 int pdadmm_spmm(int device, int64_t n_rows, const int32_t *row_ptr, const int32_t *col_idx,
                 const float *val, const float *x, int32_t width, float *y_out);
+
+/*
+ * pdadmm_matmul -- one dense product by the kernels that pdadmm_step uses for the W p, W^T r and r p^T
+ * terms (paper, Section "The pdADMM-G Algorithm": the products inside nabla_p phi and nabla_W phi), on
+ * host matrices, row-major float32 without padding:
+ *   mode 0: C[M][N] = A[M][K] * B[N][K]^T      mode 1: C[M][N] = A[M][K] * B[K][N]
+ *   mode 2: C[M][N] = A[K][M]^T * B[K][N]      (contraction over the leading index, split over node slices)
+ * flags: PDADMM_FLAG_SIMT_GEMM selects the CUDA-core kernels, 0 the tensor-core kernels.
+ * sumsq (may be null) receives sum(C^2) accumulated by the fused epilogue (modes 0 and 1).
+ */
+int pdadmm_matmul(int device, int mode, int M, int N, int K, const float *A, const float *B, float *C,
+                  double *sumsq, uint32_t flags);
 
 /*
  * Per-kernel timing.  pdadmm_profile(ctx, 1) makes every later kernel launch of pdadmm_step be

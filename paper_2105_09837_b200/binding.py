@@ -24,8 +24,8 @@ FLAG_ONE_STREAM = 2
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 
 EXPORTS = [
-    "pdadmm_init", "pdadmm_step", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
-    "pdadmm_set_tensor", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_profile", "pdadmm_profile_classes",
+    "pdadmm_init", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
+    "pdadmm_set_tensor", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_profile", "pdadmm_profile_classes",
     "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_destroy", "pdadmm_last_error",
 ]
 
@@ -61,12 +61,15 @@ def lib() -> C.CDLL:
         L.pdadmm_profile_name.restype = C.c_char_p
         L.pdadmm_init.argtypes = [C.POINTER(_Config), C.POINTER(C.c_void_p)]
         L.pdadmm_step.argtypes = [C.c_void_p, C.c_int]
+        L.pdadmm_last_step_ms.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
         L.pdadmm_objective.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
         L.pdadmm_residuals.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.c_int]
         L.pdadmm_get_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
         L.pdadmm_set_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
         L.pdadmm_quantize.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_float, C.c_int, C.c_void_p, C.c_void_p]
         L.pdadmm_spmm.argtypes = [C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.pdadmm_matmul.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.POINTER(C.c_double), C.c_uint32]
         L.pdadmm_profile.argtypes = [C.c_void_p, C.c_int]
         L.pdadmm_profile_name.argtypes = [C.c_int]
         L.pdadmm_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64),
@@ -124,6 +127,11 @@ class Context:
     # ---- same names as the C ABI
     def step(self, n_iters: int = 1):
         _check(lib().pdadmm_step(self._h, int(n_iters)))
+
+    def last_step_ms(self) -> float:
+        ms = C.c_double()
+        _check(lib().pdadmm_last_step_ms(self._h, C.byref(ms)))
+        return ms.value
 
     def objective(self) -> np.ndarray:
         out = (C.c_double * 6)()
@@ -237,3 +245,22 @@ def spmm(row_ptr, col_idx, val, x, device: int = 0) -> np.ndarray:
                              v.ctypes.data_as(C.c_void_p), a.ctypes.data_as(C.c_void_p), a.shape[1],
                              y.ctypes.data_as(C.c_void_p)))
     return y
+
+
+def matmul(mode: int, A, B, flags: int = 0, device: int = 0):
+    """``pdadmm_matmul``: (C, sum(C^2)).  mode 0: A[M,K] B[N,K]^T; 1: A[M,K] B[K,N]; 2: A[K,M]^T B[K,N]."""
+    a = np.ascontiguousarray(A, dtype=np.float32)
+    b = np.ascontiguousarray(B, dtype=np.float32)
+    if mode == 0:
+        (M, K), (N, K2) = a.shape, b.shape
+    elif mode == 1:
+        (M, K), (K2, N) = a.shape, b.shape
+    else:
+        (K, M), (K2, N) = a.shape, b.shape
+    if K != K2:
+        raise ValueError("contraction lengths differ")
+    c = np.empty((M, N), dtype=np.float32)
+    ss = C.c_double()
+    _check(lib().pdadmm_matmul(device, mode, M, N, K, a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p),
+                               c.ctypes.data_as(C.c_void_p), C.byref(ss), flags))
+    return c, ss.value

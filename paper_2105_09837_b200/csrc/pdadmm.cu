@@ -15,12 +15,15 @@
 
 #include <cmath>
 #include <cstring>
+#include <map>
 #include <memory>
+#include <tuple>
 #include <vector>
 
 #include "common.cuh"
 #include "elementwise.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 #include "graph.cuh"
 
 namespace pd {
@@ -54,6 +57,8 @@ struct Layer {
   float *z = nullptr, *r = nullptr;          // [N][ld_out]
   float *q = nullptr, *u = nullptr;          // [N][ld_out], hidden layers only
   float *gradW = nullptr;   // [n_out][ld_in]
+  float *W_hi = nullptr, *W_lo = nullptr;   // tf32 split planes of W (tensor-core path)
+  float *G_hi = nullptr, *G_lo = nullptr;   // tf32 split planes of grad_W
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in], quantised mode, l >= 2
   float scale = 1.0f;
@@ -94,12 +99,17 @@ struct pdadmm_ctx {
   int *d_flag = nullptr;            // device counter (z_L solver non-convergence)
   int *h_pinned = nullptr;          // pinned host words for small read-backs
   int64_t launches = 0;
+  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+  double last_step_ms = 0.0;
   bool profiling = false;
   std::vector<pd::ProfRec> prof;
   std::vector<cudaEvent_t> ev_pool;
   double prof_ms[pd::KC_COUNT] = {0}, prof_bytes[pd::KC_COUNT] = {0}, prof_flops[pd::KC_COUNT] = {0};
   int64_t prof_n[pd::KC_COUNT] = {0};
   std::vector<void *> allocs;
+  bool use_tc = true;               // dense products on the tensor cores
+  bool w_planes_valid = false;
+  std::map<std::tuple<const void *, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t>, CUtensorMap> tmaps;
 };
 
 namespace pd {
@@ -165,16 +175,98 @@ static void sum_slots(pdadmm_ctx *c, cudaStream_t st, const double *slots, int n
   reduce_slots_kernel<<<1, 32, 0, st>>>(slots, n_slots, 1, 1, dst);
 }
 
+
+// ---- tensor maps -------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return (EncodeTiledFn)p;
+  }();
+  return fn;
+}
+// fp32 matrix with `inner` contiguous elements per row, `outer` rows, row stride `ld` elements; tiles of
+// box_inner x box_outer elements land in shared memory with the 128-byte swizzle; out-of-range elements read 0.
+// mn_major = the rows of the tile are K slices (tensor-core "MN-major" operand): 128-byte swizzle with 32-byte
+// atoms, the only shared-memory layout the tf32 MMA accepts for such operands; otherwise 16-byte atoms.
+static int get_tmap(pdadmm_ctx *c, const float *base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_inner,
+                    uint32_t box_outer, bool mn_major, CUtensorMap *out) {
+  auto key = std::make_tuple((const void *)base, inner, outer, ld, box_inner, box_outer + (mn_major ? 1u << 16 : 0u));
+  auto it = c->tmaps.find(key);
+  if (it != c->tmaps.end()) { *out = it->second; return PDADMM_OK; }
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled is not available in this driver");
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * 4};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap m;
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)base, dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  if (c->tmaps.size() > 4096) c->tmaps.clear();
+  c->tmaps[key] = m;
+  *out = m;
+  return PDADMM_OK;
+}
+
+template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
+static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mbl,
+                     const TcParams &prm, const Epi &epi, double *partials, dim3 grid) {
+  auto kern = gemm_tc_kernel<A_MN, B_MN, B_SPLIT, Epi>;
+  static bool configured = false;
+  if (!configured) {
+    PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
+    configured = true;
+  }
+  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, prm, epi, partials);
+  return PDADMM_OK;
+}
+
 // ---- dense products --------------------------------------------------------------------------------------
 // C[M][N] = A[M][K] * op(B), fused epilogue; per-block sums of squares go to `partials` (or nullptr).
+// B is given by its fp32 matrix (CUDA-core path) and by its two tf32 planes (tensor-core path).
 template <bool B_NMAJOR, class Epi>
-static void gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
-                       const float *B, int ldb, const Epi &epi, double *partials, int *n_partials, double extra_bytes) {
-  dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM));
-  if (n_partials) *n_partials = (int)(grid.x * grid.y);
+static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
+                      const float *B, const float *B_hi, const float *B_lo, int ldb, const Epi &epi, double *partials,
+                      int *n_partials, double extra_bytes) {
   const double bytes = 4.0 * ((double)M * K + (double)N * K + (double)M * N) + extra_bytes;
+  if (!c->use_tc) {
+    dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM));
+    if (n_partials) *n_partials = (int)(grid.x * grid.y);
+    Launch l(c, cls, st, bytes, 2.0 * M * N * K);
+    gemm_nt_kernel<B_NMAJOR, Epi><<<grid, SG_THREADS, 0, st>>>(M, N, K, A, lda, B, ldb, epi, partials);
+    return PDADMM_OK;
+  }
+  dim3 grid((unsigned)ceil_div(N, TC_BN), (unsigned)ceil_div(M, TC_BM), 1);
+  if (n_partials) *n_partials = (int)(grid.x * grid.y);
+  CUtensorMap ma, mb, mbl;
+  PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TC_BK, TC_BM, false, &ma));
+  if (B_NMAJOR) {
+    PD_TRY(get_tmap(c, B_hi, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mb));
+    PD_TRY(get_tmap(c, B_lo, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mbl));
+  } else {
+    PD_TRY(get_tmap(c, B_hi, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mb));
+    PD_TRY(get_tmap(c, B_lo, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mbl));
+  }
+  TcParams prm{M, N, K, round_up(K, TC_BK), 0, c->d_flag + 1};
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
-  gemm_nt_kernel<B_NMAJOR, Epi><<<grid, SG_THREADS, 0, st>>>(M, N, K, A, lda, B, ldb, epi, partials);
+  return launch_tc<false, B_NMAJOR, false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, grid);
+}
+
+// hi/lo planes of a weight-sized matrix for the tensor-core path
+static void split_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, float *hi, float *lo, size_t n) {
+  if (!c->use_tc) return;
+  Launch l(c, KC_SMALL, st, 12.0 * n, 0);
+  split_planes_kernel<<<(int)std::min<size_t>(ceil_div((int64_t)n, 256), 1024), 256, 0, st>>>(x, hi, lo, n);
 }
 
 }  // namespace pd
@@ -184,30 +276,32 @@ namespace pd {
 // ---- pieces of one iteration -------------------------------------------------------------------------------
 
 // r_l = P_l W_l^T + b_l - z_l from scratch (only when the cached residual is not valid).
-static void refresh_residual(pdadmm_ctx *c, Layer &ly, cudaStream_t st) {
+static int refresh_residual(pdadmm_ctx *c, Layer &ly, cudaStream_t st) {
   EpiLinearResidual epi{ly.r, ly.ld_out, ly.b, ly.z};
-  gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)c->N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, epi, nullptr,
-                    nullptr, 4.0 * c->N * ly.n_out);
+  return gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)c->N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.W_hi, ly.W_lo,
+                           ly.ld_in, epi, nullptr, nullptr, 4.0 * c->N * ly.n_out);
 }
 
 // g = nu r W + u_{l-1} + rho (p - q_{l-1}) -> s1, ||g||^2 ; W g -> s2, ||W g||^2 ; tau.
-static void p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
+static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   Layer &ly = c->layers[l];
   Layer &prev = c->layers[l - 1];
   Scratch &s = c->scr;
   const int N = (int)c->N;
   int np = 0;
   EpiGradP epi{s.s1, ly.ld_in, prev.u, ly.p, prev.q, c->nu, c->rho};
-  gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.ld_in, epi, s.slots, &np,
-                   3.0 * 4.0 * N * ly.n_in);
+  PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
+                          epi, s.slots, &np, 3.0 * 4.0 * N * ly.n_in));
   sum_slots(c, s.st, s.slots, np, &ly.sc->sum_g2);
   EpiStoreSumsq epi2{s.s2, ly.ld_out};
-  gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, epi2, s.slots, &np, 0);
+  PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
+                           epi2, s.slots, &np, 0));
   sum_slots(c, s.st, s.slots, np, &ly.sc->sum_wg2);
   {
     Launch k(c, KC_SMALL, s.st, 0, 0);
     finalize_tau_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu);
   }
+  return PDADMM_OK;
 }
 
 // pdADMM-G: p <- p - g/tau, r <- r - (W g)/tau.
@@ -243,7 +337,8 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
     sum_slots(c, s.st, s.slots, grid, &ly.sc->sum_d2);
     int np = 0;
     EpiStoreSumsq epi{s.s2, ly.ld_out};
-    gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, epi, s.slots, &np, 0);
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in, epi,
+                             s.slots, &np, 0));
     sum_slots(c, s.st, s.slots, np, &ly.sc->sum_wd2);
     {
       Launch k(c, KC_SMALL, s.st, 0, 0);
@@ -267,15 +362,25 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
 
 // G = nu r^T p+ (contraction over nodes), theta, W <- W - G/theta, r <- r - (G p+)/theta,
 // b <- b - mean_j r, shift = mean_j r.
-static void w_and_b_step(pdadmm_ctx *c, int l) {
+static int w_and_b_step(pdadmm_ctx *c, int l) {
   Layer &ly = c->layers[l];
   Scratch &s = c->scr;
   const int N = (int)c->N;
-  {
+  if (!c->use_tc) {
     dim3 grid((unsigned)ceil_div(ly.n_in, SG_BN), (unsigned)ceil_div(ly.n_out, SG_BM), (unsigned)ly.n_split);
     Launch k(c, KC_GEMM_GRADW, s.st, 4.0 * ((double)N * ly.n_in + (double)N * ly.n_out), 2.0 * N * ly.n_in * ly.n_out);
     gemm_tn_kernel<<<grid, SG_THREADS, 0, s.st>>>(ly.n_out, ly.n_in, N, ly.k_chunk, ly.r, ly.ld_out, ly.p, ly.ld_in,
                                                  s.part, ly.ld_in);
+  } else {
+    // both operands are node-major, i.e. contiguous along their output index: r is [nodes][n_out], p+ is [nodes][n_in]
+    dim3 grid((unsigned)ceil_div(ly.n_in, TC_BN), (unsigned)ceil_div(ly.n_out, TC_BM), (unsigned)ly.n_split);
+    CUtensorMap ma, mb;
+    PD_TRY(get_tmap(c, ly.r, (uint64_t)ly.n_out, (uint64_t)N, (uint64_t)ly.ld_out, 32, TC_BK, true, &ma));
+    PD_TRY(get_tmap(c, ly.p, (uint64_t)ly.n_in, (uint64_t)N, (uint64_t)ly.ld_in, 32, TC_BK, true, &mb));
+    TcParams prm{ly.n_out, ly.n_in, N, ly.k_chunk, (size_t)ly.n_out * ly.ld_in, c->d_flag + 1};
+    EpiStore epi{s.part, ly.ld_in};
+    Launch k(c, KC_GEMM_GRADW, s.st, 4.0 * ((double)N * ly.n_in + (double)N * ly.n_out), 2.0 * N * ly.n_in * ly.n_out);
+    PD_TRY((launch_tc<true, true, true, EpiStore>(c, s.st, ma, mb, mb, prm, epi, nullptr, grid)));
   }
   const size_t n4w = (size_t)ly.n_out * ly.ld_in / 4;
   const int gw = ew_grid(n4w);
@@ -286,7 +391,9 @@ static void w_and_b_step(pdadmm_ctx *c, int l) {
   sum_slots(c, s.st, s.slots, gw, &ly.sc->sum_G2);
   int np = 0;
   EpiStoreSumsq epi{s.s1, ly.ld_out};
-  gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.ld_in, epi, s.slots, &np, 0);
+  split_planes(c, s.st, ly.gradW, ly.G_hi, ly.G_lo, (size_t)ly.n_out * ly.ld_in);
+  PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.G_hi, ly.G_lo, ly.ld_in,
+                           epi, s.slots, &np, 0));
   sum_slots(c, s.st, s.slots, np, &ly.sc->sum_Gp2);
   {
     Launch k(c, KC_SMALL, s.st, 0, 0);
@@ -296,6 +403,7 @@ static void w_and_b_step(pdadmm_ctx *c, int l) {
     Launch k(c, KC_WSTEP, s.st, 12.0 * ly.n_out * ly.n_in, 0);
     wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w);
   }
+  split_planes(c, s.st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
   const int n_blocks = (int)std::min<int64_t>(148 * 4, ceil_div(N, 8));
   const int rows_per_block = (int)ceil_div(N, n_blocks);
   const int used_blocks = (int)ceil_div(N, rows_per_block);
@@ -308,6 +416,7 @@ static void w_and_b_step(pdadmm_ctx *c, int l) {
     finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 128), 128, 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
                                                                           1.0 / (double)N, ly.b, ly.shift);
   }
+  return PDADMM_OK;
 }
 
 // z (and q, u for hidden layers) of layer l; needs p_{l+1} of this iteration.
@@ -334,12 +443,12 @@ static void zqu_step(pdadmm_ctx *c, int l) {
 static int iterate_once(pdadmm_ctx *c, bool *hit_cap) {
   // p-update of layers 2..L from the iterates of the previous iteration
   for (int l = 1; l < c->L; ++l) {
-    p_gradient_and_tau(c, l);
+    PD_TRY(p_gradient_and_tau(c, l));
     if (c->levels) PD_TRY(p_step_quantised(c, l, hit_cap));
     else p_step_plain(c, l);
   }
   // W- and b-update of every layer with the new p
-  for (int l = 0; l < c->L; ++l) w_and_b_step(c, l);
+  for (int l = 0; l < c->L; ++l) PD_TRY(w_and_b_step(c, l));
   // z-, q-, u-update (q_l and u_l need p_{l+1} of this iteration)
   for (int l = 0; l < c->L; ++l) zqu_step(c, l);
   return PDADMM_OK;
@@ -391,10 +500,13 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
   c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, 4); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
+  c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
   PD_CUDA(cudaSetDevice(cfg->device));
   PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
   cudaStream_t st = c->scr.st;
   PD_CUDA(cudaMallocHost((void **)&c->h_pinned, 64 * sizeof(int)));
+  PD_CUDA(cudaEventCreate(&c->ev_begin));
+  PD_CUDA(cudaEventCreate(&c->ev_end));
   PD_TRY(dev_alloc(c, &c->d_flag, 4));
 
   // graph: CSR pattern on the host, values and sparse products on the device
@@ -431,6 +543,12 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &ly.p, e_in));
     PD_TRY(dev_alloc(c, &ly.W, (size_t)ly.n_out * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.gradW, (size_t)ly.n_out * ly.ld_in));
+    if (c->use_tc) {
+      PD_TRY(dev_alloc(c, &ly.W_hi, (size_t)ly.n_out * ly.ld_in));
+      PD_TRY(dev_alloc(c, &ly.W_lo, (size_t)ly.n_out * ly.ld_in));
+      PD_TRY(dev_alloc(c, &ly.G_hi, (size_t)ly.n_out * ly.ld_in));
+      PD_TRY(dev_alloc(c, &ly.G_lo, (size_t)ly.n_out * ly.ld_in));
+    }
     PD_TRY(dev_alloc(c, &ly.b, (size_t)ly.ld_out));
     PD_TRY(dev_alloc(c, &ly.shift, (size_t)ly.ld_out));
     PD_TRY(dev_alloc(c, &ly.z, e_out));
@@ -440,9 +558,9 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &ly.sc, 1));
     PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
     // node slices of the W-gradient product: enough blocks to fill the device twice, slices >= 256 nodes
-    const int64_t tiles = ceil_div(ly.n_in, SG_BN) * ceil_div(ly.n_out, SG_BM);
+    const int64_t tiles = ceil_div(ly.n_in, SG_BN) * ceil_div(ly.n_out, SG_BM);   // same tile for both kernels
     int split = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(2 * 148, tiles), ceil_div(N, 256)));
-    ly.k_chunk = round_up((int)ceil_div(N, split), SG_BK);
+    ly.k_chunk = round_up((int)ceil_div(N, split), TC_BK);      // multiple of both kernels' K blocks
     ly.n_split = (int)ceil_div(N, ly.k_chunk);
     max_part = std::max(max_part, (size_t)ly.n_split * ly.n_out * ly.ld_in);
   }
@@ -471,8 +589,9 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   for (int l = 0; l < c->L; ++l) {
     Layer &ly = c->layers[l];
     EpiStore epi{ly.z, ly.ld_out};
-    gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, epi, nullptr,
-                      nullptr, 0);
+    split_planes(c, st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.W_hi, ly.W_lo,
+                             ly.ld_in, epi, nullptr, nullptr, 0));
     if (l + 1 == c->L) break;
     Layer &nx = c->layers[l + 1];
     const size_t n4 = (size_t)N * ly.ld_out / 4;
@@ -494,6 +613,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   PD_CUDA(cudaStreamSynchronize(st));
   PD_CUDA(cudaGetLastError());
   c->r_valid = true;                        // z = W p + b exactly by construction, r = 0 (allocated as zero)
+  c->w_planes_valid = true;
   c->launches = 0;
   return PDADMM_OK;
 }
@@ -506,6 +626,8 @@ static void destroy(pdadmm_ctx *c) {
   for (auto e : c->ev_pool) cudaEventDestroy(e);
   for (void *p : c->allocs) cudaFree(p);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
+  if (c->ev_begin) cudaEventDestroy(c->ev_begin);
+  if (c->ev_end) cudaEventDestroy(c->ev_end);
   if (c->scr.st) cudaStreamDestroy(c->scr.st);
   delete c;
 }
@@ -548,8 +670,12 @@ extern "C" int pdadmm_destroy(pdadmm_ctx *c) {
 }
 
 static int ensure_residual(pdadmm_ctx *c) {
+  if (!c->w_planes_valid) {
+    for (auto &ly : c->layers) split_planes(c, c->scr.st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
+    c->w_planes_valid = true;
+  }
   if (c->r_valid) return PDADMM_OK;
-  for (int l = 0; l < c->L; ++l) refresh_residual(c, c->layers[l], c->scr.st);
+  for (int l = 0; l < c->L; ++l) PD_TRY(refresh_residual(c, c->layers[l], c->scr.st));
   c->r_valid = true;
   return PDADMM_OK;
 }
@@ -558,14 +684,22 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
   if (!c) return fail(PDADMM_EINVAL, "context is null");
   if (n_iters < 0) return fail(PDADMM_EINVAL, "n_iters is negative");
   PD_CUDA(cudaSetDevice(c->device));
-  PD_CUDA(cudaMemsetAsync(c->d_flag, 0, sizeof(int), c->scr.st));
+  PD_CUDA(cudaEventRecord(c->ev_begin, c->scr.st));
+  PD_CUDA(cudaMemsetAsync(c->d_flag, 0, 2 * sizeof(int), c->scr.st));
   PD_TRY(ensure_residual(c));
   bool hit_cap = false;
   for (int k = 0; k < n_iters; ++k) PD_TRY(iterate_once(c, &hit_cap));
-  PD_CUDA(cudaMemcpyAsync(c->h_pinned + 8, c->d_flag, sizeof(int), cudaMemcpyDeviceToHost, c->scr.st));
+  PD_CUDA(cudaMemcpyAsync(c->h_pinned + 8, c->d_flag, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->scr.st));
+  PD_CUDA(cudaEventRecord(c->ev_end, c->scr.st));
   PD_CUDA(cudaStreamSynchronize(c->scr.st));
   PD_CUDA(cudaGetLastError());
+  {
+    float ms = 0.f;
+    PD_CUDA(cudaEventElapsedTime(&ms, c->ev_begin, c->ev_end));
+    c->last_step_ms = ms;
+  }
   if (c->profiling) PD_TRY(prof_collect(c));
+  if (c->h_pinned[9] != 0) return fail(PDADMM_ETIMEOUT, "a bounded wait inside a tensor-core product expired");
   if (c->h_pinned[8] != 0)
     return fail(PDADMM_ENOTCONV, "the last-layer z solver did not converge on %d nodes", c->h_pinned[8]);
   if (hit_cap) return fail(PDADMM_ENOTCONV, "the tau search of a quantised p-update reached its trial cap");
@@ -702,6 +836,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
   PD_CUDA(cudaStreamSynchronize(c->scr.st));
   if (kind == PDADMM_T_X || kind == PDADMM_T_P || kind == PDADMM_T_W || kind == PDADMM_T_B || kind == PDADMM_T_Z)
     c->r_valid = false;
+  if (kind == PDADMM_T_W) c->w_planes_valid = false;
   if (kind == PDADMM_T_P && c->levels && layer >= 2) {
     Layer &y = c->layers[layer - 1];
     const size_t n = (size_t)c->N * y.ld_in;
@@ -776,6 +911,80 @@ extern "C" int pdadmm_spmm(int device, int64_t n_rows, const int32_t *row_ptr, c
   return rc;
 }
 
+extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const float *A, const float *B, float *C,
+                             double *sumsq, uint32_t flags) {
+  if (mode < 0 || mode > 2 || M < 1 || N < 1 || K < 1 || !A || !B || !C) return fail(PDADMM_EINVAL, "bad argument");
+  PD_CUDA(cudaSetDevice(device));
+  pdadmm_ctx *c = new (std::nothrow) pdadmm_ctx();
+  if (!c) return fail(PDADMM_ENOMEM, "out of host memory");
+  c->device = device;
+  c->use_tc = (flags & PDADMM_FLAG_SIMT_GEMM) == 0;
+  auto body = [&]() -> int {
+    PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
+    cudaStream_t st = c->scr.st;
+    PD_TRY(dev_alloc(c, &c->d_flag, 4));
+    // operand shapes as stored: rows x cols
+    const int a_rows = mode == 2 ? K : M, a_cols = mode == 2 ? M : K;
+    const int b_rows = mode == 0 ? N : K, b_cols = mode == 0 ? K : N;
+    const int lda = round_up(a_cols, 4), ldb = round_up(b_cols, 4), ldc = round_up(N, 4);
+    float *dA, *dB, *dBh, *dBl, *dC, *part = nullptr;
+    double *slots;
+    PD_TRY(dev_alloc(c, &dA, (size_t)a_rows * lda));
+    PD_TRY(dev_alloc(c, &dB, (size_t)b_rows * ldb));
+    PD_TRY(dev_alloc(c, &dBh, (size_t)b_rows * ldb));
+    PD_TRY(dev_alloc(c, &dBl, (size_t)b_rows * ldb));
+    PD_TRY(dev_alloc(c, &dC, (size_t)M * ldc));
+    const int n_slots = (int)(ceil_div(M, 128) * ceil_div(N, 128)) + 2048;
+    PD_TRY(dev_alloc(c, &slots, (size_t)n_slots));
+    PD_TRY(upload_rows(st, dA, lda, A, a_cols, a_rows));
+    PD_TRY(upload_rows(st, dB, ldb, B, b_cols, b_rows));
+    split_planes(c, st, dB, dBh, dBl, (size_t)b_rows * ldb);
+    int np = 0;
+    if (mode == 0) {
+      EpiStoreSumsq epi{dC, ldc};
+      PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, st, M, N, K, dA, lda, dB, dBh, dBl, ldb, epi, slots, &np, 0));
+    } else if (mode == 1) {
+      EpiStoreSumsq epi{dC, ldc};
+      PD_TRY(gemm_nodes<true>(c, KC_GEMM_WG, st, M, N, K, dA, lda, dB, dBh, dBl, ldb, epi, slots, &np, 0));
+    } else {
+      const int split = (int)std::max<int64_t>(1, std::min<int64_t>(8, ceil_div(K, 64)));
+      const int k_chunk = round_up((int)ceil_div(K, split), TC_BK);
+      const int n_split = (int)ceil_div(K, k_chunk);
+      PD_TRY(dev_alloc(c, &part, (size_t)n_split * M * ldc));
+      if (!c->use_tc) {
+        dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM), (unsigned)n_split);
+        gemm_tn_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, k_chunk, dA, lda, dB, ldb, part, ldc);
+      } else {
+        dim3 grid((unsigned)ceil_div(N, TC_BN), (unsigned)ceil_div(M, TC_BM), (unsigned)n_split);
+        CUtensorMap ma, mb;
+        PD_TRY(get_tmap(c, dA, (uint64_t)M, (uint64_t)K, (uint64_t)lda, 32, TC_BK, true, &ma));
+        PD_TRY(get_tmap(c, dB, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mb));
+        TcParams prm{M, N, K, k_chunk, (size_t)M * ldc, c->d_flag + 1};
+        EpiStore epi{part, ldc};
+        PD_TRY((launch_tc<true, true, true, EpiStore>(c, st, ma, mb, mb, prm, epi, nullptr, grid)));
+      }
+      const size_t n4 = (size_t)M * ldc / 4;
+      np = ew_grid(n4);
+      reduce_gradW_kernel<<<np, EW_THREADS, 0, st>>>(part, n_split, n4, 1.0f, dC, slots);
+    }
+    double *res = slots + n_slots - 1;
+    reduce_slots_kernel<<<1, 32, 0, st>>>(slots, np, 1, 1, res);
+    double h = 0;
+    PD_CUDA(cudaMemcpyAsync(&h, res, 8, cudaMemcpyDeviceToHost, st));
+    PD_CUDA(cudaMemcpy2DAsync(C, (size_t)N * 4, dC, (size_t)ldc * 4, (size_t)N * 4, (size_t)M, cudaMemcpyDeviceToHost, st));
+    int err = 0;
+    PD_CUDA(cudaMemcpyAsync(&err, c->d_flag + 1, 4, cudaMemcpyDeviceToHost, st));
+    PD_CUDA(cudaStreamSynchronize(st));
+    PD_CUDA(cudaGetLastError());
+    if (sumsq) *sumsq = h;
+    if (err) return fail(PDADMM_ETIMEOUT, "a bounded wait inside a tensor-core product expired");
+    return PDADMM_OK;
+  };
+  const int rc = body();
+  destroy(c);
+  return rc;
+}
+
 // ---- timing ----------------------------------------------------------------------------------------------------
 extern "C" int pdadmm_profile(pdadmm_ctx *c, int enable) {
   if (!c) return fail(PDADMM_EINVAL, "context is null");
@@ -794,6 +1003,11 @@ extern "C" int pdadmm_profile_read(pdadmm_ctx *c, int k, double *ms, int64_t *la
   if (launches) *launches = c->prof_n[k];
   if (bytes) *bytes = c->prof_bytes[k];
   if (flops) *flops = c->prof_flops[k];
+  return PDADMM_OK;
+}
+extern "C" int pdadmm_last_step_ms(pdadmm_ctx *c, double *ms) {
+  if (!c || !ms) return fail(PDADMM_EINVAL, "null argument");
+  *ms = c->last_step_ms;
   return PDADMM_OK;
 }
 extern "C" int pdadmm_launches(pdadmm_ctx *c, int64_t *count) {
