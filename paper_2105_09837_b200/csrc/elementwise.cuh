@@ -34,13 +34,23 @@ __device__ __forceinline__ float4 ld4(const float *p, size_t i) { return reinter
 __device__ __forceinline__ void st4(float *p, size_t i, float4 v) { reinterpret_cast<float4 *>(p)[i] = v; }
 
 // ---- final, fixed-order reduction of per-block slots -------------------------------------------
-// out[j] = sum_i slots[i * stride + j], j < n_out, i < n_slots   (one block; thread j strides over outputs)
-__global__ void reduce_slots_kernel(const double *__restrict__ slots, int n_slots, int stride, int n_out,
-                                    double *__restrict__ out) {
-  for (int j = threadIdx.x; j < n_out; j += blockDim.x) {
+// out[j] = sum_i slots[i * stride + j], j < n_out, i < n_slots.  One block of 256 threads: thread t adds the
+// slots t, t+256, ... in that order, then the 256 partial sums are combined in a fixed tree, so the result
+// does not depend on scheduling.
+__global__ void __launch_bounds__(256)
+reduce_slots_kernel(const double *__restrict__ slots, int n_slots, int stride, int n_out, double *__restrict__ out) {
+  __shared__ double sh[256];
+  for (int j = 0; j < n_out; ++j) {
     double s = 0.0;
-    for (int i = 0; i < n_slots; ++i) s += slots[(size_t)i * stride + j];
-    out[j] = s;
+    for (int i = threadIdx.x; i < n_slots; i += 256) s += slots[(size_t)i * stride + j];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+      if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) out[j] = sh[0];
+    __syncthreads();
   }
 }
 

@@ -108,6 +108,7 @@ struct pdadmm_ctx {
   int64_t prof_n[pd::KC_COUNT] = {0};
   std::vector<void *> allocs;
   bool use_tc = true;               // dense products on the tensor cores
+  int n_sms = 148;
   bool w_planes_valid = false;
   std::map<std::tuple<const void *, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t>, CUtensorMap> tmaps;
 };
@@ -172,7 +173,7 @@ static int prof_collect(pdadmm_ctx *c) {
 // ---- fixed-order sum of per-block slots into a field of the layer's scalars ---------------------------
 static void sum_slots(pdadmm_ctx *c, cudaStream_t st, const double *slots, int n_slots, double *dst) {
   Launch l(c, KC_SMALL, st, 8.0 * n_slots, 0);
-  reduce_slots_kernel<<<1, 32, 0, st>>>(slots, n_slots, 1, 1, dst);
+  reduce_slots_kernel<<<1, 256, 0, st>>>(slots, n_slots, 1, 1, dst);
 }
 
 
@@ -220,8 +221,9 @@ static int get_tmap(pdadmm_ctx *c, const float *base, uint64_t inner, uint64_t o
 
 template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
 static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mbl,
-                     const TcParams &prm, const Epi &epi, double *partials, dim3 grid) {
+                     const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
   auto kern = gemm_tc_kernel<A_MN, B_MN, B_SPLIT, Epi>;
+  const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
   static bool configured = false;
   if (!configured) {
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
@@ -246,8 +248,8 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     gemm_nt_kernel<B_NMAJOR, Epi><<<grid, SG_THREADS, 0, st>>>(M, N, K, A, lda, B, ldb, epi, partials);
     return PDADMM_OK;
   }
-  dim3 grid((unsigned)ceil_div(N, TC_BN), (unsigned)ceil_div(M, TC_BM), 1);
-  if (n_partials) *n_partials = (int)(grid.x * grid.y);
+  const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM));
+  if (n_partials) *n_partials = 8 * n_tiles;        // one slot per tile and epilogue warp
   CUtensorMap ma, mb, mbl;
   PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TC_BK, TC_BM, false, &ma));
   if (B_NMAJOR) {
@@ -257,9 +259,9 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     PD_TRY(get_tmap(c, B_hi, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mb));
     PD_TRY(get_tmap(c, B_lo, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mbl));
   }
-  TcParams prm{M, N, K, round_up(K, TC_BK), 0, c->d_flag + 1};
+  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1};
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
-  return launch_tc<false, B_NMAJOR, false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, grid);
+  return launch_tc<false, B_NMAJOR, false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, n_tiles);
 }
 
 // hi/lo planes of a weight-sized matrix for the tensor-core path
@@ -373,14 +375,14 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
                                                  s.part, ly.ld_in);
   } else {
     // both operands are node-major, i.e. contiguous along their output index: r is [nodes][n_out], p+ is [nodes][n_in]
-    dim3 grid((unsigned)ceil_div(ly.n_in, TC_BN), (unsigned)ceil_div(ly.n_out, TC_BM), (unsigned)ly.n_split);
+    const int n_tiles = (int)(ceil_div(ly.n_in, TC_BN) * ceil_div(ly.n_out, TC_BM)) * ly.n_split;
     CUtensorMap ma, mb;
     PD_TRY(get_tmap(c, ly.r, (uint64_t)ly.n_out, (uint64_t)N, (uint64_t)ly.ld_out, 32, TC_BK, true, &ma));
     PD_TRY(get_tmap(c, ly.p, (uint64_t)ly.n_in, (uint64_t)N, (uint64_t)ly.ld_in, 32, TC_BK, true, &mb));
-    TcParams prm{ly.n_out, ly.n_in, N, ly.k_chunk, (size_t)ly.n_out * ly.ld_in, c->d_flag + 1};
+    TcParams prm{ly.n_out, ly.n_in, N, ly.k_chunk, ly.n_split, (size_t)ly.n_out * ly.ld_in, c->d_flag + 1};
     EpiStore epi{s.part, ly.ld_in};
     Launch k(c, KC_GEMM_GRADW, s.st, 4.0 * ((double)N * ly.n_in + (double)N * ly.n_out), 2.0 * N * ly.n_in * ly.n_out);
-    PD_TRY((launch_tc<true, true, true, EpiStore>(c, s.st, ma, mb, mb, prm, epi, nullptr, grid)));
+    PD_TRY((launch_tc<true, true, true, EpiStore>(c, s.st, ma, mb, mb, prm, epi, nullptr, n_tiles)));
   }
   const size_t n4w = (size_t)ly.n_out * ly.ld_in / 4;
   const int gw = ew_grid(n4w);
@@ -502,6 +504,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
   PD_CUDA(cudaSetDevice(cfg->device));
+  PD_CUDA(cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, cfg->device));
   PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
   cudaStream_t st = c->scr.st;
   PD_CUDA(cudaMallocHost((void **)&c->h_pinned, 64 * sizeof(int)));
@@ -575,7 +578,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &s.codes_new, (size_t)N * max_in));
   }
   PD_TRY(dev_alloc(c, &s.part, max_part));
-  s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
+  s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
   PD_TRY(dev_alloc(c, &s.slots, s.n_slots));
 
   // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
@@ -708,7 +711,7 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
 
 static int read_slots(pdadmm_ctx *c, int n_slots, int stride, int n_out, double *host) {
   double *dst = c->scr.slots + c->scr.n_slots - 8;            // tail of the slot buffer: results
-  reduce_slots_kernel<<<1, 32, 0, c->scr.st>>>(c->scr.slots, n_slots, stride, n_out, dst);
+  reduce_slots_kernel<<<1, 256, 0, c->scr.st>>>(c->scr.slots, n_slots, stride, n_out, dst);
   PD_CUDA(cudaMemcpyAsync(host, dst, n_out * sizeof(double), cudaMemcpyDeviceToHost, c->scr.st));
   PD_CUDA(cudaStreamSynchronize(c->scr.st));
   return PDADMM_OK;
@@ -920,6 +923,7 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
   c->device = device;
   c->use_tc = (flags & PDADMM_FLAG_SIMT_GEMM) == 0;
   auto body = [&]() -> int {
+    PD_CUDA(cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, device));
     PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
     cudaStream_t st = c->scr.st;
     PD_TRY(dev_alloc(c, &c->d_flag, 4));
@@ -934,7 +938,7 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
     PD_TRY(dev_alloc(c, &dBh, (size_t)b_rows * ldb));
     PD_TRY(dev_alloc(c, &dBl, (size_t)b_rows * ldb));
     PD_TRY(dev_alloc(c, &dC, (size_t)M * ldc));
-    const int n_slots = (int)(ceil_div(M, 128) * ceil_div(N, 128)) + 2048;
+    const int n_slots = 8 * (int)(ceil_div(M, 128) * ceil_div(N, 128)) + 2048;
     PD_TRY(dev_alloc(c, &slots, (size_t)n_slots));
     PD_TRY(upload_rows(st, dA, lda, A, a_cols, a_rows));
     PD_TRY(upload_rows(st, dB, ldb, B, b_cols, b_rows));
@@ -955,20 +959,20 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
         dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM), (unsigned)n_split);
         gemm_tn_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, k_chunk, dA, lda, dB, ldb, part, ldc);
       } else {
-        dim3 grid((unsigned)ceil_div(N, TC_BN), (unsigned)ceil_div(M, TC_BM), (unsigned)n_split);
+        const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM)) * n_split;
         CUtensorMap ma, mb;
         PD_TRY(get_tmap(c, dA, (uint64_t)M, (uint64_t)K, (uint64_t)lda, 32, TC_BK, true, &ma));
         PD_TRY(get_tmap(c, dB, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mb));
-        TcParams prm{M, N, K, k_chunk, (size_t)M * ldc, c->d_flag + 1};
+        TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1};
         EpiStore epi{part, ldc};
-        PD_TRY((launch_tc<true, true, true, EpiStore>(c, st, ma, mb, mb, prm, epi, nullptr, grid)));
+        PD_TRY((launch_tc<true, true, true, EpiStore>(c, st, ma, mb, mb, prm, epi, nullptr, n_tiles)));
       }
       const size_t n4 = (size_t)M * ldc / 4;
       np = ew_grid(n4);
       reduce_gradW_kernel<<<np, EW_THREADS, 0, st>>>(part, n_split, n4, 1.0f, dC, slots);
     }
     double *res = slots + n_slots - 1;
-    reduce_slots_kernel<<<1, 32, 0, st>>>(slots, np, 1, 1, res);
+    reduce_slots_kernel<<<1, 256, 0, st>>>(slots, np, 1, 1, res);
     double h = 0;
     PD_CUDA(cudaMemcpyAsync(&h, res, 8, cudaMemcpyDeviceToHost, st));
     PD_CUDA(cudaMemcpy2DAsync(C, (size_t)N * 4, dC, (size_t)ldc * 4, (size_t)N * 4, (size_t)M, cudaMemcpyDeviceToHost, st));
