@@ -173,6 +173,31 @@ int pdadmm_matmul(int device, int mode, int M, int N, int K, const float *A, con
                   double *sumsq, uint32_t flags);
 
 /*
+ * pdadmm_matmul_tn_static -- (no counterpart in the paper: an interface for callers that cannot allocate.)
+ * C[M][ldc] = A[K][lda]^T * B[K][ldb] on DEVICE buffers of the caller, fp32 on the CUDA cores, ldc = N rounded
+ * up to a multiple of 4 (rows of C are padded to that width and the padding is written as zero).  This is
+ * the contraction over the node index that the W-gradient needs; like pdadmm_matmul mode 2 it cuts the nodes
+ * into slices and adds the slices' partial tiles in slice order, but the partial tiles live in a fixed 4 MiB
+ * array inside the library image, so the call performs no cudaMalloc, cudaFree or other allocation.  Meant
+ * for callers that must not allocate: code running inside a stream capture, a latency-critical loop that may
+ * not take the allocator lock or cause an implicit device synchronisation, or a layer that was given all of
+ * its buffers up front.
+ *  - dA, dB, dC: device pointers on `device`, 16-byte aligned; lda >= M, ldb >= N, both multiples of 4.
+ *  - Limit: M * ldc <= 1048576 floats (one partial tile must fit the built-in array); larger outputs are
+ *    rejected with PDADMM_EINVAL and a message that names both sizes.  Every GPU that loads the library holds
+ *    the 4 MiB until the process exits.
+ *  - The two kernels are enqueued on `stream` (a cudaStream_t, or null for the default stream) and the call
+ *    returns without waiting for them.
+ *  - The first call on each device looks up the device address of the built-in array (once per device); make
+ *    that first call before beginning any stream capture.
+ *  - All calls share the array and it keeps the contents of the last call.  Nothing in it has to start at
+ *    zero: every element that a call reads was written earlier in the same call.  Two calls whose kernels
+ *    overlap on the GPU (different streams, or different host threads) race on the array: serialise them.
+ */
+int pdadmm_matmul_tn_static(int device, int M, int N, int K, const float *dA, int lda, const float *dB, int ldb,
+                            float *dC, void *stream);
+
+/*
  * Per-kernel timing.  pdadmm_profile(ctx, 1) makes every later kernel launch of pdadmm_step be
  * bracketed by CUDA events on its own stream (the layers then run one after another);
  * pdadmm_profile(ctx, 0) turns it off; either call clears the counters.

@@ -25,7 +25,7 @@ OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5,
 
 EXPORTS = [
     "pdadmm_init", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
-    "pdadmm_set_tensor", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_profile", "pdadmm_profile_classes",
+    "pdadmm_set_tensor", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_profile", "pdadmm_profile_classes",
     "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_destroy", "pdadmm_last_error",
 ]
 
@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
         L.pdadmm_spmm.argtypes = [C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.pdadmm_matmul.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.POINTER(C.c_double), C.c_uint32]
+        L.pdadmm_matmul_tn_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_int,
+                                              C.c_void_p, C.c_void_p]
         L.pdadmm_profile.argtypes = [C.c_void_p, C.c_int]
         L.pdadmm_profile_name.argtypes = [C.c_int]
         L.pdadmm_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64),
@@ -264,3 +266,13 @@ def matmul(mode: int, A, B, flags: int = 0, device: int = 0):
     _check(lib().pdadmm_matmul(device, mode, M, N, K, a.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p),
                                c.ctypes.data_as(C.c_void_p), C.byref(ss), flags))
     return c, ss.value
+
+
+def matmul_tn_static(dA: int, lda: int, dB: int, ldb: int, dC: int, M: int, N: int, K: int, stream: int = 0,
+                     device: int = 0):
+    """``pdadmm_matmul_tn_static``: C = A^T B on device buffers given by their addresses; allocates nothing.
+
+    The kernels are only enqueued on ``stream``; the caller synchronises before reading C.
+    """
+    _check(lib().pdadmm_matmul_tn_static(device, M, N, K, C.c_void_p(dA), lda, C.c_void_p(dB), ldb, C.c_void_p(dC),
+                                         C.c_void_p(stream)))

@@ -1019,3 +1019,5 @@ extern "C" int pdadmm_launches(pdadmm_ctx *c, int64_t *count) {
   *count = c->launches;
   return PDADMM_OK;
 }
+
+#include "no_alloc.cuh"
