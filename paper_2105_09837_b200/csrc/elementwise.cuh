@@ -31,6 +31,7 @@ struct LayerScalars {
 };
 
 __device__ __forceinline__ float4 ld4(const float *p, size_t i) { return reinterpret_cast<const float4 *>(p)[i]; }
+__device__ __forceinline__ float4 ld4f(const float *p, size_t i) { return reinterpret_cast<const float4 *>(p)[i]; }
 __device__ __forceinline__ void st4(float *p, size_t i, float4 v) { reinterpret_cast<float4 *>(p)[i] = v; }
 
 // ---- final, fixed-order reduction of per-block slots -------------------------------------------
@@ -179,32 +180,64 @@ reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, floa
 }
 
 // ---- column sums of r - gp * inv_theta  (for the b-update) ----------------------------------------
-// Block b handles rows [b*rows_per_block, ...); thread c strides over columns.  slots[b][ld].
+// Block b handles rows [b*rows_per_block, ...).  A thread owns one group of 4 columns (float4) and one row
+// subgroup: with ld/4 <= 128 column groups the block's 256 threads cover several rows per pass.  The row
+// subgroups' sums are combined in subgroup order, then written to slots[b][ld].
+constexpr int COLSUM_MAX_SUB = 8;
 __global__ void __launch_bounds__(EW_THREADS)
 resid_colsum_kernel(float *__restrict__ r, const float *__restrict__ gp, const LayerScalars *__restrict__ sc,
                     int n_rows, int ld, int rows_per_block, double *__restrict__ slots) {
+  extern __shared__ double colsum_sh[];                       // [n_sub][ld] when n_sub > 1
   const float a = sc->inv_theta;
+  const int ld4 = ld >> 2;
+  const int cols_per_pass = min(ld4, EW_THREADS);
+  const int n_sub = min(EW_THREADS / cols_per_pass, COLSUM_MAX_SUB);
+  const int sub = threadIdx.x / cols_per_pass, c0 = threadIdx.x % cols_per_pass;
   const int r0 = blockIdx.x * rows_per_block, r1 = min(n_rows, r0 + rows_per_block);
-  for (int c = threadIdx.x; c < ld; c += blockDim.x) {
-    double s = 0.0;
-    for (int j = r0; j < r1; ++j) {
-      const size_t o = (size_t)j * ld + c;
-      const float v = fmaf(-a, gp[o], r[o]);
-      r[o] = v;
-      s += (double)v;
+  double *out = slots + (size_t)blockIdx.x * ld;
+  if (sub < n_sub) {
+    for (int cg = c0; cg < ld4; cg += cols_per_pass) {
+      double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+#pragma unroll 4
+      for (int j = r0 + sub; j < r1; j += n_sub) {
+        const size_t o = (size_t)j * ld4 + cg;
+        float4 v = ld4f(r, o);
+        const float4 g = ld4f(gp, o);
+        v.x = fmaf(-a, g.x, v.x); v.y = fmaf(-a, g.y, v.y); v.z = fmaf(-a, g.z, v.z); v.w = fmaf(-a, g.w, v.w);
+        st4(r, o, v);
+        s0 += (double)v.x; s1 += (double)v.y; s2 += (double)v.z; s3 += (double)v.w;
+      }
+      double *dst = (n_sub > 1 ? colsum_sh + (size_t)sub * ld : out) + 4 * cg;
+      dst[0] = s0; dst[1] = s1; dst[2] = s2; dst[3] = s3;
     }
-    slots[(size_t)blockIdx.x * ld + c] = s;
+  }
+  if (n_sub > 1) {
+    __syncthreads();
+    for (int c = threadIdx.x; c < ld; c += blockDim.x) {
+      double s = 0.0;
+      for (int k = 0; k < n_sub; ++k) s += colsum_sh[(size_t)k * ld + c];
+      out[c] = s;
+    }
   }
 }
 
 // b+ = b - mean_j r[j][:]  (Eq. "update b" with the step 1/(nu N), i.e. the exact minimiser);
-// shift[c] = that mean, which the z-update subtracts from r.
-__global__ void finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int width, double inv_n,
-                                     float *__restrict__ b, float *__restrict__ shift) {
-  for (int c = threadIdx.x + blockIdx.x * blockDim.x; c < ld; c += blockDim.x * gridDim.x) {
-    double s = 0.0;
-    for (int i = 0; i < n_slots; ++i) s += slots[(size_t)i * ld + c];
-    const float m = c < width ? (float)(s * inv_n) : 0.0f;
+// shift[c] = that mean, which the z-update subtracts from r.  blockDim = (32 columns, 8 slot groups): group g adds
+// the slots g, g+8, ... of its column, the 8 group sums are then added in group order.
+__global__ void __launch_bounds__(256)
+finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int width, double inv_n,
+                     float *__restrict__ b, float *__restrict__ shift) {
+  __shared__ double sh[8][33];
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  double s = 0.0;
+  if (c < ld)
+    for (int i = threadIdx.y; i < n_slots; i += 8) s += slots[(size_t)i * ld + c];
+  sh[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && c < ld) {
+    double t = 0.0;
+    for (int k = 0; k < 8; ++k) t += sh[k][threadIdx.x];
+    const float m = c < width ? (float)(t * inv_n) : 0.0f;
     shift[c] = m;
     if (c < width) b[c] -= m;
   }

@@ -406,17 +406,20 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
     wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w);
   }
   split_planes(c, s.st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
-  const int n_blocks = (int)std::min<int64_t>(148 * 4, ceil_div(N, 8));
+  const int n_blocks = (int)std::min<int64_t>(c->n_sms * 2, ceil_div(N, 16));
   const int rows_per_block = (int)ceil_div(N, n_blocks);
   const int used_blocks = (int)ceil_div(N, rows_per_block);
   {
+    const int ld4 = ly.ld_out / 4, cols_per_pass = std::min(ld4, EW_THREADS);
+    const int n_sub = std::min(EW_THREADS / cols_per_pass, COLSUM_MAX_SUB);
+    const size_t sh = n_sub > 1 ? (size_t)n_sub * ly.ld_out * sizeof(double) : 0;
     Launch k(c, KC_COLSUM, s.st, 12.0 * N * ly.n_out, 0);
-    resid_colsum_kernel<<<used_blocks, EW_THREADS, 0, s.st>>>(ly.r, s.s1, ly.sc, N, ly.ld_out, rows_per_block, s.slots);
+    resid_colsum_kernel<<<used_blocks, EW_THREADS, sh, s.st>>>(ly.r, s.s1, ly.sc, N, ly.ld_out, rows_per_block, s.slots);
   }
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * used_blocks * ly.ld_out, 0);
-    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 128), 128, 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
-                                                                          1.0 / (double)N, ly.b, ly.shift);
+    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
+                                                                                1.0 / (double)N, ly.b, ly.shift);
   }
   return PDADMM_OK;
 }
