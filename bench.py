@@ -159,11 +159,9 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2105_09837_b200 import replicas, synth
+    rank, world, local_rank = replicas.env_rank_world()
 
-    from paper_2105_09837_b200 import synth
     w = synth.get(args.workload)
     config = {"workload": f"{w.name}: N={w.n_nodes} {w.graph.upper()} graph, d={w.feat_dim} x {w.n_blocks} hop blocks "
                           f"(n0={w.n0}), {w.n_layers} layers x {w.hidden}, {w.n_classes} classes, "
@@ -205,7 +203,7 @@ def main():
         import torch.distributed as dist
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    device = local_rank if world > 1 else 0
+    device = replicas.device_for(local_rank, world)
     flags = B.FLAG_SIMT_GEMM if args.simt else 0
 
     inp = synth.make_inputs(w)
@@ -227,11 +225,8 @@ def main():
         barrier()
         wall = time.perf_counter() - t0
     launches = ctx.launches() - launches0
-    if dist is not None:
-        tms = torch.tensor([ms], device=f"cuda:{device}", dtype=torch.float64)
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms = float(tms.item())
-    value = world * args.steps / (ms * 1e-3)
+    ms = replicas.max_over_ranks(ms, dist, f"cuda:{device}")
+    value = replicas.job_throughput(world, args.steps, ms)
     obj = ctx.objective()
 
     # per-kernel device times (second pass with an event pair around every launch)
@@ -284,11 +279,8 @@ def main():
     torch.cuda.synchronize(device)
     e2e_s = time.perf_counter() - t0
     ctx2.destroy()
-    if dist is not None:
-        te = torch.tensor([e2e_s], device=f"cuda:{device}", dtype=torch.float64)
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e_s = float(te.item())
-    e2e = {"value": world * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d / args.steps,
+    e2e_s = replicas.max_over_ranks(e2e_s, dist, f"cuda:{device}")
+    e2e = {"value": replicas.job_throughput(world, args.steps, e2e_s * 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d / args.steps,
            "d2h_bytes_per_step": d2h / args.steps,
            "note": "pdadmm_init from host buffers + K iterations + objective and W,b read back"}
 

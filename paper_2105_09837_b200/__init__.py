@@ -8,7 +8,7 @@ input generators (``synth``).  Sub-modules are imported on demand so that
 
 import importlib
 
-__all__ = ["synth", "binding", "build"]
+__all__ = ["synth", "binding", "build", "replicas"]
 
 
 def __getattr__(name):
