@@ -1,0 +1,97 @@
+"""GPU parity at the full sizes of the five workloads, in the launch configuration bench.py times.
+
+c1, c2, c3: the oracle can afford whole iterations, so one teacher-forced iteration (after two oracle
+iterations, when every layer has started to move) is compared variable by variable, and c1 also runs its
+20 free iterations.  c4, c5: the oracle cannot afford an iteration (1e13..1e14 flop in fp64, >200 GB), so the
+parts it can compute are compared (the whole augmented input, the forward pass on sampled nodes) and the state
+after two device iterations is checked against properties that hold at any size (Lemma "q_opt", p on the level
+set, finite and decreasing objective).
+"""
+
+import numpy as np
+import pytest
+
+import oracle.pdadmm_oracle as o
+from paper_2105_09837_b200 import binding as B
+from paper_2105_09837_b200 import synth
+import parity_util as U
+from test_gpu_parity import _compare_iteration
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c1_full_teacher_forced_and_20_free_iterations():
+    inp = synth.make_inputs(synth.get("c1"))
+    prm, s, _ = U.oracle_problem(inp)
+    ctx = B.from_inputs(inp)
+    free = B.from_inputs(inp)
+    free.step(20)
+    for k in range(20):
+        if k in (2, 7, 15):
+            prev = U.round_state(s)
+            U.load_state(ctx, prev, False)
+            _compare_iteration(ctx, prev, prm, f"c1/k={k}")
+        s = o.iterate(s, prm)
+    want, got = o.objective(s, prm), free.objective()
+    assert abs(got[5] - want[5]) <= 1e-3 * abs(want[5]), (got, want)
+    ctx.destroy()
+    free.destroy()
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_c2_c3_full_one_teacher_forced_iteration(name):
+    inp = synth.make_inputs(synth.get(name))
+    prm, s, A = U.oracle_problem(inp)
+    ctx = B.from_inputs(inp)
+    X = ctx.get_tensor(B.T_X).T.astype(np.float64)
+    assert U.rel_err(X, s.p[0]) < 1e-6
+    del X
+    for _ in range(2):
+        s = o.iterate(s, prm)
+    prev = U.round_state(s)
+    del s
+    U.load_state(ctx, prev, prm.quant_levels > 0)
+    _compare_iteration(ctx, prev, prm, f"{name}/k=2")
+    ctx.destroy()
+
+
+@pytest.mark.parametrize("name", ["c4", "c5"])
+def test_c4_c5_full_size_parts_and_invariants(name):
+    w = synth.get(name)
+    inp = synth.make_inputs(w)
+    ctx = B.from_inputs(inp)
+    # the whole augmented input against the oracle (sparse products are cheap for it)
+    A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
+    assert np.array_equal(ctx.get_tensor(B.T_CSR_ROWPTR), A.indptr.astype(np.int32))
+    assert np.array_equal(ctx.get_tensor(B.T_CSR_COLIDX), A.indices.astype(np.int32))
+    X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
+    Xg = ctx.get_tensor(B.T_X)
+    assert U.rel_err(Xg.T.astype(np.float64), X) < 1e-6
+    # forward pass of layer 1 on sampled nodes, one by one
+    rng = np.random.default_rng(7)
+    nodes = rng.choice(w.n_nodes, size=64, replace=False)
+    z1 = ctx.get_tensor(B.T_Z, 1)
+    want = (inp.init_W[0].astype(np.float64) @ X[:, nodes]).T
+    assert U.rel_err(z1[nodes].astype(np.float64), want) < 1e-5
+    del X, Xg, z1
+    L, m = w.n_layers, w.quant_levels
+    obj0 = ctx.objective()
+    ctx.step(2)
+    obj2 = ctx.objective()
+    assert np.all(np.isfinite(obj2)) and obj2[5] < obj0[5]
+    res = ctx.residuals()
+    assert res.shape == (L - 1,) and np.all(np.isfinite(res))
+    for l in (1, L // 2, L - 1):
+        # Lemma q_opt: u_l = nu (q_l - ReLU(z_l)) after every iteration
+        u, q, z = ctx.get_tensor(B.T_U, l), ctx.get_tensor(B.T_Q, l), ctx.get_tensor(B.T_Z, l)
+        rhs = np.float32(w.nu) * (q - np.maximum(z, 0))
+        assert np.linalg.norm((u - rhs).ravel()) <= 1e-4 * max(np.linalg.norm(rhs.ravel()), 1e-12)
+        del u, q, z, rhs
+        # p on the level set, bit for bit
+        codes, p = ctx.get_tensor(B.T_CODES, l + 1), ctx.get_tensor(B.T_P, l + 1)
+        scale = ctx.get_tensor(B.T_QSCALE, l + 1)[0]
+        assert int(codes.max()) <= m - 1
+        assert np.array_equal(p, codes.astype(np.float32) * scale)
+        del codes, p
+        assert 1 <= int(ctx.get_tensor(B.T_TRIALS, l + 1)[0]) <= 30
+    ctx.destroy()

@@ -114,8 +114,6 @@ def _compare_iteration(ctx, prev, prm, label):
         if np.linalg.norm(nxt.p[l] - prev.p[l]) > 1e-3 * np.linalg.norm(prev.p[l]):
             tau = float(ctx.get_tensor(B.T_TAU, l + 1)[0])
             assert abs(tau - nxt.tau[l]) <= 1e-3 * nxt.tau[l], f"{label}: tau_{l + 1} {tau} vs {nxt.tau[l]}"
-    if not clean:
-        pytest.skip(f"{label}: a code flipped at a rounding boundary; later variables are not comparable")
     for l in range(L):
         worst[f"W{l + 1}"] = U.rel_err(got["W"][l], nxt.W[l])
         # b_l = mean_j (z - W p)_j is a difference of two terms of the size of W p: in single precision its
@@ -142,6 +140,10 @@ def _compare_iteration(ctx, prev, prm, label):
         else:
             worst[f"z{l + 1}"] = U.rel_err(got["z"][l], nxt.z[l])
     bad = {k: v for k, v in worst.items() if not v <= TOL}
+    if bad and not clean:
+        # a code flipped at a rounding boundary: one entry of p differs by a whole level, which the variables
+        # computed from p inherit; in a small problem that alone can exceed the tolerance
+        pytest.skip(f"{label}: a code flipped at a rounding boundary and later variables differ: {bad}")
     assert not bad, f"{label}: relative errors above {TOL}: {bad} (all: {worst})"
     return nxt
 
