@@ -64,6 +64,7 @@ typedef enum {
 /* Bits of pdadmm_config.flags. */
 #define PDADMM_FLAG_SIMT_GEMM 1u     /* run the dense products on CUDA cores (fp32 FMA) instead of tensor cores */
 #define PDADMM_FLAG_ONE_STREAM 2u    /* issue all layers on one stream (no concurrency across layers)           */
+#define PDADMM_FLAG_NO_GRAPH 4u      /* launch every kernel of an iteration directly instead of replaying a CUDA graph */
 
 /*
  * Problem statement (paper: Problem 2 / Problem 3, Algorithm 1 "Require", and the experimental

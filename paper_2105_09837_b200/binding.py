@@ -20,6 +20,7 @@ _lib = None
 T_X, T_P, T_W, T_B, T_Z, T_Q, T_U, T_CODES, T_TAU, T_THETA, T_QSCALE, T_CSR_ROWPTR, T_CSR_COLIDX, T_CSR_VAL, T_TRIALS = range(15)
 FLAG_SIMT_GEMM = 1
 FLAG_ONE_STREAM = 2
+FLAG_NO_GRAPH = 4
 
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 

@@ -108,6 +108,9 @@ struct pdadmm_ctx {
   int64_t prof_n[pd::KC_COUNT] = {0};
   std::vector<void *> allocs;
   bool use_tc = true;               // dense products on the tensor cores
+  cudaGraphExec_t iter_graph = nullptr;   // one captured pdADMM-G iteration (no host round trips in it)
+  int64_t iter_graph_launches = 0;
+  bool graph_failed = false;
   int n_sms = 148;
   bool w_planes_valid = false;
   std::map<std::tuple<const void *, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t>, CUtensorMap> tmaps;
@@ -634,6 +637,7 @@ static void destroy(pdadmm_ctx *c) {
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   if (c->ev_begin) cudaEventDestroy(c->ev_begin);
   if (c->ev_end) cudaEventDestroy(c->ev_end);
+  if (c->iter_graph) cudaGraphExecDestroy(c->iter_graph);
   if (c->scr.st) cudaStreamDestroy(c->scr.st);
   delete c;
 }
@@ -694,7 +698,40 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
   PD_CUDA(cudaMemsetAsync(c->d_flag, 0, 2 * sizeof(int), c->scr.st));
   PD_TRY(ensure_residual(c));
   bool hit_cap = false;
-  for (int k = 0; k < n_iters; ++k) PD_TRY(iterate_once(c, &hit_cap));
+  // pdADMM-G has no host decision inside an iteration, so after a first eager iteration the sequence of launches
+  // is captured once into a CUDA graph and replayed; pointers and tensor maps never change in that mode.
+  // pdADMM-G-Q reads the accept flag of every tau trial on the host, and per-kernel timing needs its events:
+  // both stay eager.
+  const bool may_graph = c->levels == 0 && !c->profiling && !c->graph_failed && !(c->flags & PDADMM_FLAG_NO_GRAPH);
+  int k = 0;
+  if (may_graph && c->iter_graph == nullptr && n_iters > 1) {
+    PD_TRY(iterate_once(c, &hit_cap));
+    ++k;
+    const int64_t before = c->launches;
+    cudaGraph_t g = nullptr;
+    if (cudaStreamBeginCapture(c->scr.st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+      const int rc = iterate_once(c, &hit_cap);
+      const cudaError_t e = cudaStreamEndCapture(c->scr.st, &g);
+      if (rc != PDADMM_OK || e != cudaSuccess || cudaGraphInstantiate(&c->iter_graph, g, 0) != cudaSuccess) {
+        c->iter_graph = nullptr;
+        c->graph_failed = true;
+      }
+      if (g) cudaGraphDestroy(g);
+    } else {
+      c->graph_failed = true;
+    }
+    cudaGetLastError();
+    c->iter_graph_launches = c->launches - before;
+    c->launches = before;                       // capturing launched nothing
+  }
+  for (; k < n_iters; ++k) {
+    if (may_graph && c->iter_graph != nullptr) {
+      PD_CUDA(cudaGraphLaunch(c->iter_graph, c->scr.st));
+      c->launches += c->iter_graph_launches;
+    } else {
+      PD_TRY(iterate_once(c, &hit_cap));
+    }
+  }
   PD_CUDA(cudaMemcpyAsync(c->h_pinned + 8, c->d_flag, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->scr.st));
   PD_CUDA(cudaEventRecord(c->ev_end, c->scr.st));
   PD_CUDA(cudaStreamSynchronize(c->scr.st));

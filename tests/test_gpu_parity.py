@@ -210,6 +210,20 @@ def test_objective_after_20_free_iterations(case, levels, tol):
     ctx.destroy()
 
 
+def test_graph_replay_equals_direct_launches():
+    inp = _inputs("ba-ragged", quant_levels=0)
+    a, b = B.from_inputs(inp), B.from_inputs(inp, flags=B.FLAG_NO_GRAPH)
+    a.step(5)
+    b.step(5)
+    assert a.launches() == b.launches() > 0
+    sa, sb = U.read_state(a), U.read_state(b)
+    for k in sa:
+        for x, y in zip(sa[k], sb[k]):
+            assert np.array_equal(x, y), k
+    a.destroy()
+    b.destroy()
+
+
 def test_step_is_deterministic_and_split_calls_agree():
     inp = _inputs("ba-ragged", quant_levels=0)
     a, b = B.from_inputs(inp), B.from_inputs(inp)
