@@ -129,40 +129,89 @@ quantize_kernel(const float *__restrict__ x, size_t n, float scale, int levels, 
   }
 }
 
-// ---- single-thread finalisers of the step parameters ---------------------------------------------
+// ---- finalisers of the step parameters (one block of 256 threads) ---------------------------------
+// Fixed-order sum of n slots by one block: thread t adds slots t, t+256, ..., then a fixed tree.  Result in thread 0.
+__device__ __forceinline__ double block_sum_slots(const double *__restrict__ slots, int n, double *sh /* 256 */) {
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 256) s += slots[i];
+  __syncthreads();
+  sh[threadIdx.x] = s;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+    __syncthreads();
+  }
+  return sh[0];
+}
+// ||g||^2 and ||W g||^2 from their slots, then
 // tau = rho + nu ||W g||^2 / ||g||^2 : the smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
-__global__ void finalize_tau_kernel(LayerScalars *sc, double rho, double nu) {
-  const double gg = sc->sum_g2;
-  const double tau = gg > 0.0 ? rho + nu * sc->sum_wg2 / gg : rho;
-  sc->tau = tau;
-  sc->inv_tau = (float)(1.0 / tau);
-  sc->accepted = 0;
-  sc->trials = 0;
+__global__ void __launch_bounds__(256)
+finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots_g, int n_g, const double *slots_wg, int n_wg) {
+  __shared__ double sh[256];
+  const double gg = block_sum_slots(slots_g, n_g, sh);
+  const double wg = block_sum_slots(slots_wg, n_wg, sh);
+  if (threadIdx.x == 0) {
+    sc->sum_g2 = gg;
+    sc->sum_wg2 = wg;
+    const double tau = gg > 0.0 ? rho + nu * wg / gg : rho;
+    sc->tau = tau;
+    sc->inv_tau = (float)(1.0 / tau);
+    sc->accepted = 0;
+    sc->trials = 0;
+  }
 }
 // Stop condition of the quantised step in its quadratic form: nu||W d||^2 + rho||d||^2 <= tau||d||^2 (1 + slack).
 // Not accepted: tau is doubled for the next trial.
-__global__ void finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack) {
-  const double dd = sc->sum_d2;
-  const bool ok = nu * sc->sum_wd2 + rho * dd <= sc->tau * dd * (1.0 + slack);
-  sc->trials += 1;
-  sc->accepted = ok ? 1 : 0;
-  if (!ok) {
-    sc->tau *= 2.0;
-    sc->inv_tau = (float)(1.0 / sc->tau);
+__global__ void __launch_bounds__(256)
+finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack, const double *slots_d, int n_d,
+                      const double *slots_wd, int n_wd) {
+  __shared__ double sh[256];
+  const double dd = block_sum_slots(slots_d, n_d, sh);
+  const double wd = block_sum_slots(slots_wd, n_wd, sh);
+  if (threadIdx.x == 0) {
+    sc->sum_d2 = dd;
+    sc->sum_wd2 = wd;
+    const bool ok = nu * wd + rho * dd <= sc->tau * dd * (1.0 + slack);
+    sc->trials += 1;
+    sc->accepted = ok ? 1 : 0;
+    if (!ok) {
+      sc->tau *= 2.0;
+      sc->inv_tau = (float)(1.0 / sc->tau);
+    }
   }
 }
+// ||grad_W||^2 and ||grad_W p+||^2 from their slots, then
 // theta = nu ||grad_W p+||^2 / ||grad_W||^2 : the smallest theta with phi(W+) <= V_l(W+; theta).
-__global__ void finalize_theta_kernel(LayerScalars *sc, double nu) {
-  const double GG = sc->sum_G2;
-  const double theta = GG > 0.0 ? nu * sc->sum_Gp2 / GG : 0.0;
-  sc->theta = theta;
-  sc->inv_theta = theta > 0.0 ? (float)(1.0 / theta) : 0.0f;
+__global__ void __launch_bounds__(256)
+finalize_theta_kernel(LayerScalars *sc, double nu, const double *slots_G, int n_G, const double *slots_Gp, int n_Gp) {
+  __shared__ double sh[256];
+  const double GG = block_sum_slots(slots_G, n_G, sh);
+  const double Gp = block_sum_slots(slots_Gp, n_Gp, sh);
+  if (threadIdx.x == 0) {
+    sc->sum_G2 = GG;
+    sc->sum_Gp2 = Gp;
+    const double theta = GG > 0.0 ? nu * Gp / GG : 0.0;
+    sc->theta = theta;
+    sc->inv_theta = theta > 0.0 ? (float)(1.0 / theta) : 0.0f;
+  }
+}
+
+// hi = value rounded to tf32 (11 significant bits), lo = value - hi (exact): the operand planes of the
+// tensor-core products for weight-sized matrices
+__device__ __forceinline__ void store_planes(float *__restrict__ hi, float *__restrict__ lo, size_t i, float4 v) {
+  float4 h;
+  h.x = __uint_as_float((__float_as_uint(v.x) + 0x1000u) & 0xFFFFE000u);
+  h.y = __uint_as_float((__float_as_uint(v.y) + 0x1000u) & 0xFFFFE000u);
+  h.z = __uint_as_float((__float_as_uint(v.z) + 0x1000u) & 0xFFFFE000u);
+  h.w = __uint_as_float((__float_as_uint(v.w) + 0x1000u) & 0xFFFFE000u);
+  st4(hi, i, h);
+  st4(lo, i, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
 }
 
 // ---- reduction of the split partial tiles of grad_W, scaling by nu, ||grad_W||^2 ------------------
 __global__ void __launch_bounds__(EW_THREADS)
 reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, float nu, float *__restrict__ G,
-                    double *__restrict__ slots) {
+                    float *__restrict__ G_hi, float *__restrict__ G_lo, double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   double ss = 0.0;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
@@ -174,6 +223,7 @@ reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, floa
     a.x *= nu; a.y *= nu; a.z *= nu; a.w *= nu;
     ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
     st4(G, i, a);
+    if (G_hi != nullptr) store_planes(G_hi, G_lo, i, a);      // tf32 planes for the tensor-core product G p+
   }
   const double tot = block_sum<EW_THREADS>(ss, red);
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
@@ -416,13 +466,15 @@ risk_kernel(const float *__restrict__ z, const int *__restrict__ labels, const u
 
 // W+ = W - grad_W * inv_theta  (Eq. "update W")
 __global__ void __launch_bounds__(EW_THREADS)
-wstep_kernel(float *__restrict__ W, const float *__restrict__ G, const LayerScalars *__restrict__ sc, size_t n4) {
+wstep_kernel(float *__restrict__ W, const float *__restrict__ G, const LayerScalars *__restrict__ sc, size_t n4,
+             float *__restrict__ W_hi, float *__restrict__ W_lo) {
   const float a = sc->inv_theta;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = ld4(W, i);
     const float4 g = ld4(G, i);
     v.x = fmaf(-a, g.x, v.x); v.y = fmaf(-a, g.y, v.y); v.z = fmaf(-a, g.z, v.z); v.w = fmaf(-a, g.w, v.w);
     st4(W, i, v);
+    if (W_hi != nullptr) store_planes(W_hi, W_lo, i, v);
   }
 }
 

@@ -173,13 +173,6 @@ static int prof_collect(pdadmm_ctx *c) {
   return PDADMM_OK;
 }
 
-// ---- fixed-order sum of per-block slots into a field of the layer's scalars ---------------------------
-static void sum_slots(pdadmm_ctx *c, cudaStream_t st, const double *slots, int n_slots, double *dst) {
-  Launch l(c, KC_SMALL, st, 8.0 * n_slots, 0);
-  reduce_slots_kernel<<<1, 256, 0, st>>>(slots, n_slots, 1, 1, dst);
-}
-
-
 // ---- tensor maps -------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -297,14 +290,14 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   EpiGradP epi{s.s1, ly.ld_in, prev.u, ly.p, prev.q, c->nu, c->rho};
   PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
                           epi, s.slots, &np, 3.0 * 4.0 * N * ly.n_in));
-  sum_slots(c, s.st, s.slots, np, &ly.sc->sum_g2);
+  int np2 = 0;
+  double *slots_b = s.slots + s.n_slots / 2;          // second half of the slot buffer
   EpiStoreSumsq epi2{s.s2, ly.ld_out};
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
-                           epi2, s.slots, &np, 0));
-  sum_slots(c, s.st, s.slots, np, &ly.sc->sum_wg2);
+                           epi2, slots_b, &np2, 0));
   {
-    Launch k(c, KC_SMALL, s.st, 0, 0);
-    finalize_tau_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu);
+    Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
+    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2);
   }
   return PDADMM_OK;
 }
@@ -339,15 +332,14 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
       quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, c->levels, s.p_new, s.d,
                                                        s.codes_new, n4p, s.slots);
     }
-    sum_slots(c, s.st, s.slots, grid, &ly.sc->sum_d2);
     int np = 0;
+    double *slots_b = s.slots + s.n_slots / 2;
     EpiStoreSumsq epi{s.s2, ly.ld_out};
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in, epi,
-                             s.slots, &np, 0));
-    sum_slots(c, s.st, s.slots, np, &ly.sc->sum_wd2);
+                             slots_b, &np, 0));
     {
-      Launch k(c, KC_SMALL, s.st, 0, 0);
-      finalize_trial_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6);
+      Launch k(c, KC_SMALL, s.st, 8.0 * (grid + np), 0);
+      finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
     }
     PD_CUDA(cudaMemcpyAsync(c->h_pinned, &ly.sc->accepted, sizeof(int), cudaMemcpyDeviceToHost, s.st));
     PD_CUDA(cudaStreamSynchronize(s.st));
@@ -391,24 +383,21 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
   const int gw = ew_grid(n4w);
   {
     Launch k(c, KC_GRADW_REDUCE, s.st, 4.0 * (ly.n_split + 1.0) * ly.n_out * ly.n_in, 0);
-    reduce_gradW_kernel<<<gw, EW_THREADS, 0, s.st>>>(s.part, ly.n_split, n4w, c->nu, ly.gradW, s.slots);
+    reduce_gradW_kernel<<<gw, EW_THREADS, 0, s.st>>>(s.part, ly.n_split, n4w, c->nu, ly.gradW, ly.G_hi, ly.G_lo, s.slots);
   }
-  sum_slots(c, s.st, s.slots, gw, &ly.sc->sum_G2);
   int np = 0;
+  double *slots_b = s.slots + s.n_slots / 2;
   EpiStoreSumsq epi{s.s1, ly.ld_out};
-  split_planes(c, s.st, ly.gradW, ly.G_hi, ly.G_lo, (size_t)ly.n_out * ly.ld_in);
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.G_hi, ly.G_lo, ly.ld_in,
-                           epi, s.slots, &np, 0));
-  sum_slots(c, s.st, s.slots, np, &ly.sc->sum_Gp2);
+                           epi, slots_b, &np, 0));
   {
-    Launch k(c, KC_SMALL, s.st, 0, 0);
-    finalize_theta_kernel<<<1, 1, 0, s.st>>>(ly.sc, (double)c->nu);
+    Launch k(c, KC_SMALL, s.st, 8.0 * (gw + np), 0);
+    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np);
   }
   {
-    Launch k(c, KC_WSTEP, s.st, 12.0 * ly.n_out * ly.n_in, 0);
-    wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w);
+    Launch k(c, KC_WSTEP, s.st, 20.0 * ly.n_out * ly.n_in, 0);
+    wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w, ly.W_hi, ly.W_lo);
   }
-  split_planes(c, s.st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
   const int n_blocks = (int)std::min<int64_t>(c->n_sms * 2, ceil_div(N, 16));
   const int rows_per_block = (int)ceil_div(N, n_blocks);
   const int used_blocks = (int)ceil_div(N, rows_per_block);
@@ -440,7 +429,6 @@ static void zqu_step(pdadmm_ctx *c, int l) {
       zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, c->layers[l + 1].p, ly.shift, ly.ld_out / 4, n4,
                                                c->rho, c->nu, s.slots);
     }
-    sum_slots(c, s.st, s.slots, grid, &ly.sc->res2);
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
     zlast_kernel<<<(int)ceil_div(N, 128), 128, 0, s.st>>>(ly.r, ly.z, ly.shift, c->labels, c->mask, N, ly.n_out,
@@ -585,6 +573,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   }
   PD_TRY(dev_alloc(c, &s.part, max_part));
   s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
+  s.n_slots *= 2;                       // two halves: consecutive reductions of one layer use different halves
   PD_TRY(dev_alloc(c, &s.slots, s.n_slots));
 
   // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
@@ -1009,7 +998,7 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
       }
       const size_t n4 = (size_t)M * ldc / 4;
       np = ew_grid(n4);
-      reduce_gradW_kernel<<<np, EW_THREADS, 0, st>>>(part, n_split, n4, 1.0f, dC, slots);
+      reduce_gradW_kernel<<<np, EW_THREADS, 0, st>>>(part, n_split, n4, 1.0f, dC, nullptr, nullptr, slots);
     }
     double *res = slots + n_slots - 1;
     reduce_slots_kernel<<<1, 256, 0, st>>>(slots, np, 1, 1, res);
