@@ -40,6 +40,23 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def measured_traffic(workload: str, kernel_class: str):
+    """DRAM bytes per launch of a kernel class from the committed ncu capture of this workload, or None if there
+    is no capture or the kernel sources have changed since it was taken."""
+    import glob
+    import hashlib
+    path = os.path.join(ROOT, "profiles", f"{workload}_kernel_traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path))
+    h = hashlib.sha256()
+    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2105_09837_b200", "csrc", "*"))):
+        h.update(open(f, "rb").read())
+    if h.hexdigest() != rec.get("csrc_sha256"):
+        return None
+    return rec.get("traffic_bytes_per_launch", {}).get(kernel_class)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
 
@@ -264,7 +281,7 @@ def main():
                 "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["kernel"] = dom
-    roof["traffic"] = None
+    roof["traffic"] = measured_traffic(args.workload, dom)
     ctx.destroy()
 
     # end to end through the public API from host buffers: init (H2D of graph, features, weights), K iterations,

@@ -1,7 +1,7 @@
 """Small, self-contained invocations for kernel profilers (one kernel class each, a few launches).
 
     python -m paper_2105_09837_b200.profile_case matmul MODE M N K [--simt]    # one dense product, run twice
-    python -m paper_2105_09837_b200.profile_case iterate WORKLOAD N_NODES ITERS  # a reduced workload, ITERS iterations
+    python -m paper_2105_09837_b200.profile_case iterate WORKLOAD N_NODES ITERS [--no-graph]  # a (reduced) workload
 """
 
 import sys
@@ -25,7 +25,7 @@ def main(argv):
         return 0
     if argv and argv[0] == "iterate":
         w = synth.small(argv[1], int(argv[2]))
-        ctx = B.from_inputs(synth.make_inputs(w))
+        ctx = B.from_inputs(synth.make_inputs(w), flags=B.FLAG_NO_GRAPH if "--no-graph" in argv else 0)
         ctx.step(int(argv[3]))
         print("objective", ctx.objective()[5])
         ctx.destroy()
