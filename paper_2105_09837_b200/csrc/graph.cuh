@@ -1,44 +1,150 @@
-// Graph pre-processing: CSR structure of A + I (host), values of the renormalised adjacency
+// Graph pre-processing: CSR structure of A + I, values of the renormalised adjacency
 // A~ = (D+I)^{-1/2}(A+I)(D+I)^{-1/2} (device), and the sparse product Y = A~ X used to build the
 // multi-hop input X = [H; H A~; H A~^2; ...] (A~ is symmetric, so in node-major storage the
 // k-th block is A~ times the (k-1)-th block).
 #pragma once
 
-#include <algorithm>
-#include <vector>
+#include <cstdint>
 
 #include "common.cuh"
 
 namespace pd {
 
-// Host: undirected edge list -> CSR pattern of A + I with ascending columns; repeats and self-loops
-// in the input are dropped.  Returns EINVAL on an out-of-range node id.
-inline int build_csr_pattern(int64_t n, int64_t n_edges, const int32_t *src, const int32_t *dst,
-                             std::vector<int32_t> &row_ptr, std::vector<int32_t> &col_idx) {
-  std::vector<uint64_t> keys;
-  keys.reserve((size_t)(2 * n_edges + n));
-  for (int64_t e = 0; e < n_edges; ++e) {
-    const int64_t a = src[e], b = dst[e];
-    if (a < 0 || a >= n || b < 0 || b >= n)
-      return fail(PDADMM_EINVAL, "edge %lld = (%lld, %lld) is outside [0, %lld)", (long long)e, (long long)a,
-                  (long long)b, (long long)n);
-    if (a == b) continue;
-    keys.push_back((uint64_t)a * (uint64_t)n + (uint64_t)b);
-    keys.push_back((uint64_t)b * (uint64_t)n + (uint64_t)a);
+// ---- CSR pattern of A + I on the device ---------------------------------------------------------------
+// Undirected edge list -> rows with ascending, unique columns; self-loops and repeats in the input are
+// dropped and every row gets its diagonal entry.  Steps: count the raw entries of each row, prefix-sum them,
+// scatter the edges (any order within a row), sort each row and drop its repeats, prefix-sum the final row
+// lengths and compact.  The result does not depend on the order in which the scatter's atomics land.
+// meta[0] = error word (1 bad node id, 2 more than 2^31-1 entries, 3 a row above CSR_MAX_ROW),
+// meta[1] = number of long rows; bad_edge = smallest index of an edge with a node id outside [0, n).
+
+constexpr int CSR_WARP_ROW = 512;        // longer rows are sorted by a whole block
+constexpr int CSR_MAX_ROW = 1 << 16;     // the row sort is quadratic in the row length
+
+__global__ void edge_count_kernel(const int *__restrict__ src, const int *__restrict__ dst, long long n_edges, int n,
+                                  int *__restrict__ deg, int *__restrict__ meta, unsigned long long *bad_edge) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n_edges) return;
+  const int a = src[e], b = dst[e];
+  if ((unsigned)a >= (unsigned)n || (unsigned)b >= (unsigned)n) {
+    meta[0] = 1;
+    atomicMin(bad_edge, (unsigned long long)e);
+    return;
   }
-  for (int64_t i = 0; i < n; ++i) keys.push_back((uint64_t)i * (uint64_t)n + (uint64_t)i);
-  std::sort(keys.begin(), keys.end());
-  keys.erase(std::unique(keys.begin(), keys.end()), keys.end());
-  if (keys.size() > (size_t)INT32_MAX) return fail(PDADMM_EINVAL, "more than 2^31-1 non-zeros");
-  row_ptr.assign((size_t)n + 1, 0);
-  col_idx.resize(keys.size());
-  for (size_t i = 0; i < keys.size(); ++i) {
-    const uint64_t r = keys[i] / (uint64_t)n;
-    col_idx[i] = (int32_t)(keys[i] % (uint64_t)n);
-    row_ptr[r + 1]++;
+  if (a == b) return;
+  atomicAdd(deg + a, 1);
+  atomicAdd(deg + b, 1);
+}
+
+// out[i] = sum_{j<i} (in[j] + add) for i = 0..n (out[n] is the total); one block, chunks of blockDim.x.
+__global__ void __launch_bounds__(1024)
+exclusive_scan_kernel(const int *__restrict__ in, int n, int add, int *__restrict__ out, int *__restrict__ meta) {
+  __shared__ int warp_sum[32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  long long carry = 0;
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int v = i < n ? in[i] + add : 0;
+    int x = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, d);
+      if (lane >= d) x += y;
+    }
+    if (lane == 31) warp_sum[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      int t = warp_sum[lane];
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, t, d);
+        if (lane >= d) t += y;
+      }
+      warp_sum[lane] = t;
+    }
+    __syncthreads();
+    if (i < n) out[i] = (int)(carry + (warp ? warp_sum[warp - 1] : 0) + x - v);
+    carry += warp_sum[31];
+    __syncthreads();
   }
-  for (int64_t i = 0; i < n; ++i) row_ptr[i + 1] += row_ptr[i];
-  return PDADMM_OK;
+  if (threadIdx.x == 0) {
+    out[n] = (int)carry;
+    if (carry > (long long)INT32_MAX) meta[0] = 2;
+  }
+}
+
+__global__ void edge_scatter_kernel(const int *__restrict__ src, const int *__restrict__ dst, long long n_edges, int n,
+                                    const int *__restrict__ raw_ptr, int *__restrict__ cursor, int *__restrict__ raw) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n_edges) return;
+  const int a = src[e], b = dst[e];
+  if ((unsigned)a >= (unsigned)n || (unsigned)b >= (unsigned)n || a == b) return;
+  raw[raw_ptr[a] + atomicAdd(cursor + a, 1)] = b;
+  raw[raw_ptr[b] + atomicAdd(cursor + b, 1)] = a;
+}
+
+// One row: raw[b .. b+d) holds the neighbours in any order, its last slot is free for the diagonal.
+// Writes the distinct columns in ascending order to sorted[b ..] and their number to len[row].
+// Each of the `nt` threads of the group (a warp or a block) takes the entries k = t, t+nt, ...
+template <bool BLOCK>
+__device__ __forceinline__ void sort_unique_row(int row, int b, int d, int *raw, int *sorted, int *len, int t, int nt) {
+  auto group_sync = [] { if constexpr (BLOCK) __syncthreads(); else __syncwarp(); };
+  if (t == 0) raw[b + d - 1] = row;
+  group_sync();
+  // an entry is a repeat when an equal column stands before it
+  for (int k = t; k < d; k += nt) {
+    const int ck = raw[b + k];
+    int rep = 0;
+    for (int j = 0; j < k; ++j) rep |= (raw[b + j] == ck);
+    sorted[b + k] = rep;
+  }
+  group_sync();
+  int kept = 0;
+  for (int k = t; k < d; k += nt) {
+    if (sorted[b + k]) raw[b + k] = INT32_MAX; else ++kept;
+  }
+  group_sync();
+  // rank = number of distinct smaller columns (repeats now compare as +infinity)
+  for (int k = t; k < d; k += nt) {
+    const int ck = raw[b + k];
+    if (ck == INT32_MAX) continue;
+    int rank = 0;
+    for (int j = 0; j < d; ++j) rank += (raw[b + j] < ck);
+    sorted[b + rank] = ck;
+  }
+  if (kept) atomicAdd(len + row, kept);
+}
+
+// Rows up to CSR_WARP_ROW entries: one warp each.  Longer rows are appended to `long_rows`.
+__global__ void __launch_bounds__(256)
+row_sort_warp_kernel(const int *__restrict__ raw_ptr, int n, int *raw, int *sorted, int *__restrict__ len,
+                     int *__restrict__ long_rows, int *__restrict__ meta) {
+  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (row >= n) return;
+  const int b = raw_ptr[row], d = raw_ptr[row + 1] - b;
+  if (d > CSR_MAX_ROW) { if (lane == 0) meta[0] = 3; return; }
+  if (d > CSR_WARP_ROW) { if (lane == 0) long_rows[atomicAdd(meta + 1, 1)] = row; return; }
+  sort_unique_row<false>(row, b, d, raw, sorted, len, lane, 32);
+}
+
+__global__ void __launch_bounds__(1024)
+row_sort_block_kernel(const int *__restrict__ raw_ptr, int *raw, int *sorted, int *__restrict__ len,
+                      const int *__restrict__ long_rows, const int *__restrict__ meta) {
+  const int n_long = meta[1];
+  for (int i = blockIdx.x; i < n_long; i += gridDim.x) {
+    const int row = long_rows[i], b = raw_ptr[row], d = raw_ptr[row + 1] - b;
+    sort_unique_row<true>(row, b, d, raw, sorted, len, threadIdx.x, blockDim.x);
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(256)
+row_compact_kernel(const int *__restrict__ raw_ptr, const int *__restrict__ row_ptr, int n,
+                   const int *__restrict__ sorted, int *__restrict__ col_idx) {
+  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (row >= n) return;
+  const int src = raw_ptr[row], dst = row_ptr[row], d = row_ptr[row + 1] - dst;
+  for (int k = lane; k < d; k += 32) col_idx[dst + k] = sorted[src + k];
 }
 
 // val[e] = 1 / sqrt((d_i + 1)(d_j + 1)) for the entry e = (i, j); d_i = row length - 1 (the self-loop).

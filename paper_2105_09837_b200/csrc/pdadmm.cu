@@ -491,6 +491,75 @@ static int upload_rows(cudaStream_t st, float *dst, int ld, const float *src, in
   return PDADMM_OK;
 }
 
+// Temporary device buffers of the CSR construction, released when the builder returns.
+struct TempBuffers {
+  std::vector<void *> ptrs;
+  ~TempBuffers() { for (void *p : ptrs) cudaFree(p); }
+  template <class T>
+  int get(T **out, size_t count) {
+    void *p = nullptr;
+    const size_t bytes = std::max<size_t>(count * sizeof(T), 16);
+    const cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return fail(PDADMM_ENOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+    }
+    ptrs.push_back(p);
+    *out = (T *)p;
+    return PDADMM_OK;
+  }
+};
+
+// Edge list (host) -> c->row_ptr, c->col_idx (device), c->nnz; c->csr_val is allocated, not filled.
+static int build_csr(pdadmm_ctx *c, const pdadmm_config *cfg) {
+  const int64_t N = c->N, E = cfg->n_edges;
+  const size_t raw_cap = (size_t)(2 * E + N);
+  if (raw_cap > (size_t)INT32_MAX) return fail(PDADMM_EINVAL, "more than 2^31-1 non-zeros");
+  cudaStream_t st = c->scr.st;
+  TempBuffers tmp;
+  int *d_src, *d_dst, *deg, *cursor, *raw_ptr, *raw, *sorted, *len, *long_rows, *meta;
+  unsigned long long *bad_edge;
+  PD_TRY(tmp.get(&d_src, (size_t)E)); PD_TRY(tmp.get(&d_dst, (size_t)E));
+  PD_TRY(tmp.get(&deg, (size_t)N)); PD_TRY(tmp.get(&cursor, (size_t)N)); PD_TRY(tmp.get(&len, (size_t)N));
+  PD_TRY(tmp.get(&raw_ptr, (size_t)N + 1)); PD_TRY(tmp.get(&long_rows, (size_t)N));
+  PD_TRY(tmp.get(&raw, raw_cap)); PD_TRY(tmp.get(&sorted, raw_cap));
+  PD_TRY(tmp.get(&meta, 4)); PD_TRY(tmp.get(&bad_edge, 1));
+  PD_TRY(dev_alloc(c, &c->row_ptr, (size_t)N + 1, false));
+  PD_CUDA(cudaMemsetAsync(deg, 0, (size_t)N * 4, st));
+  PD_CUDA(cudaMemsetAsync(cursor, 0, (size_t)N * 4, st));
+  PD_CUDA(cudaMemsetAsync(len, 0, (size_t)N * 4, st));
+  PD_CUDA(cudaMemsetAsync(meta, 0, 16, st));
+  PD_CUDA(cudaMemsetAsync(bad_edge, 0xff, 8, st));
+  const int e_grid = (int)std::max<int64_t>(1, ceil_div(E, 256)), r_grid = (int)ceil_div(N * 32, 256);
+  if (E > 0) {
+    PD_CUDA(cudaMemcpyAsync(d_src, cfg->edge_src, (size_t)E * 4, cudaMemcpyHostToDevice, st));
+    PD_CUDA(cudaMemcpyAsync(d_dst, cfg->edge_dst, (size_t)E * 4, cudaMemcpyHostToDevice, st));
+    edge_count_kernel<<<e_grid, 256, 0, st>>>(d_src, d_dst, (long long)E, (int)N, deg, meta, bad_edge);
+  }
+  exclusive_scan_kernel<<<1, 1024, 0, st>>>(deg, (int)N, 1, raw_ptr, meta);
+  if (E > 0) edge_scatter_kernel<<<e_grid, 256, 0, st>>>(d_src, d_dst, (long long)E, (int)N, raw_ptr, cursor, raw);
+  row_sort_warp_kernel<<<r_grid, 256, 0, st>>>(raw_ptr, (int)N, raw, sorted, len, long_rows, meta);
+  row_sort_block_kernel<<<2 * c->n_sms, 1024, 0, st>>>(raw_ptr, raw, sorted, len, long_rows, meta);
+  exclusive_scan_kernel<<<1, 1024, 0, st>>>(len, (int)N, 0, c->row_ptr, meta);
+  int h_meta[4]; unsigned long long h_bad; int h_nnz;
+  PD_CUDA(cudaMemcpyAsync(h_meta, meta, 16, cudaMemcpyDeviceToHost, st));
+  PD_CUDA(cudaMemcpyAsync(&h_bad, bad_edge, 8, cudaMemcpyDeviceToHost, st));
+  PD_CUDA(cudaMemcpyAsync(&h_nnz, c->row_ptr + N, 4, cudaMemcpyDeviceToHost, st));
+  PD_CUDA(cudaStreamSynchronize(st));
+  if (h_meta[0] == 1)
+    return fail(PDADMM_EINVAL, "edge %llu = (%d, %d) is outside [0, %lld)", h_bad, cfg->edge_src[h_bad],
+                cfg->edge_dst[h_bad], (long long)N);
+  if (h_meta[0] == 2) return fail(PDADMM_EINVAL, "more than 2^31-1 non-zeros");
+  if (h_meta[0] == 3) return fail(PDADMM_EINVAL, "a node has more than %d neighbours", CSR_MAX_ROW - 1);
+  c->nnz = h_nnz;
+  PD_TRY(dev_alloc(c, &c->col_idx, (size_t)c->nnz, false));
+  PD_TRY(dev_alloc(c, &c->csr_val, (size_t)c->nnz, false));
+  row_compact_kernel<<<r_grid, 256, 0, st>>>(raw_ptr, c->row_ptr, (int)N, sorted, c->col_idx);
+  PD_CUDA(cudaGetLastError());
+  PD_CUDA(cudaStreamSynchronize(st));     // the temporaries are released on return
+  return PDADMM_OK;
+}
+
 static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   const int64_t N = cfg->n_nodes;
   c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
@@ -506,16 +575,8 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   PD_CUDA(cudaEventCreate(&c->ev_end));
   PD_TRY(dev_alloc(c, &c->d_flag, 4));
 
-  // graph: CSR pattern on the host, values and sparse products on the device
-  std::vector<int32_t> rp, ci;
-  PD_TRY(build_csr_pattern(N, cfg->n_edges, cfg->edge_src, cfg->edge_dst, rp, ci));
-  c->nnz = (int64_t)ci.size();
-  PD_TRY(dev_alloc(c, &c->row_ptr, (size_t)N + 1, false));
-  PD_TRY(dev_alloc(c, &c->col_idx, ci.size(), false));
-  PD_TRY(dev_alloc(c, &c->csr_val, ci.size(), false));
-  PD_CUDA(cudaMemcpyAsync(c->row_ptr, rp.data(), rp.size() * 4, cudaMemcpyHostToDevice, st));
-  PD_CUDA(cudaMemcpyAsync(c->col_idx, ci.data(), ci.size() * 4, cudaMemcpyHostToDevice, st));
-  PD_CUDA(cudaStreamSynchronize(st));
+  // graph: CSR pattern, values and sparse products all on the device
+  PD_TRY(build_csr(c, cfg));
   adjacency_values_kernel<<<(int)ceil_div(N * 32, 256), 256, 0, st>>>(c->row_ptr, c->col_idx, (int)N, c->csr_val);
   PD_TRY(dev_alloc(c, &c->labels, (size_t)N, false));
   PD_TRY(dev_alloc(c, &c->mask, (size_t)N, false));

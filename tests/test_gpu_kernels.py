@@ -87,6 +87,33 @@ def test_graph_without_edges_and_tiny_node_counts():
         ctx.destroy()
 
 
+def test_csr_from_messy_edge_list_with_a_hub_is_bit_exact():
+    """Repeats, both directions, self-loops and a node with more neighbours than one warp sorts."""
+    w = synth.small("c2", 2500, feat_dim=3, hidden=4, n_layers=2)
+    inp = synth.make_inputs(w)
+    hub = 17
+    others = np.setdiff1d(np.arange(w.n_nodes, dtype=np.int32), [hub])[::-1][:1400]      # descending ids
+    src = np.concatenate([inp.edge_src, inp.edge_dst[:300], np.full(others.size, hub, np.int32), [5, 9, 9]])
+    dst = np.concatenate([inp.edge_dst, inp.edge_src[:300], others, [5, 9, 11]])
+    perm = np.random.default_rng(3).permutation(src.size)
+    inp.edge_src, inp.edge_dst = src[perm].astype(np.int32), dst[perm].astype(np.int32)
+    A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
+    ctx = B.from_inputs(inp)
+    assert np.array_equal(ctx.get_tensor(B.T_CSR_ROWPTR), A.indptr.astype(np.int32))
+    assert np.array_equal(ctx.get_tensor(B.T_CSR_COLIDX), A.indices.astype(np.int32))
+    assert np.allclose(ctx.get_tensor(B.T_CSR_VAL), A.data, rtol=3e-7, atol=0)
+    ctx.destroy()
+
+
+def test_edge_with_node_id_out_of_range_is_rejected():
+    w = synth.small("c1", 50, feat_dim=3, hidden=4, n_layers=2)
+    inp = synth.make_inputs(w)
+    inp.edge_dst = inp.edge_dst.copy()
+    inp.edge_dst[4] = 50
+    with pytest.raises(RuntimeError, match="edge 4"):
+        B.from_inputs(inp)
+
+
 def test_all_nodes_unlabelled_keeps_z_equal_to_a():
     inp = synth.make_inputs(synth.small("c1", 200, feat_dim=5, hidden=6, n_layers=2))
     inp.train_mask[:] = 0
