@@ -16,19 +16,31 @@ namespace pd {
 constexpr int SG_BM = 128, SG_BN = 128, SG_BK = 8, SG_THREADS = 256;
 
 // ---- epilogues: called with 4 consecutive columns of one row ------------------------------------
+// prefetch(row, col): optional hint that the 128 bytes of every epilogue input at (row, col .. col+31) will be
+// read soon (the tensor-core kernel issues it when it starts a tile).
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// kDirect: the output is the accumulator itself (the tensor-core kernel then stores the tile by TMA);
+// kSumsq: the epilogue accumulates the sum of squares of the output.
 struct EpiStore {             // C = acc
+  static constexpr bool kDirect = true, kSumsq = false;
   float *C; int ldc;
+  __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ float4 operator()(int, int, float4 a, double &) const { return a; }
 };
 struct EpiStoreSumsq {        // C = acc, accumulates sum(acc^2)
+  static constexpr bool kDirect = true, kSumsq = true;
   float *C; int ldc;
+  __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ float4 operator()(int, int, float4 a, double &ss) const {
     ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
     return a;
   }
 };
 struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b - z)
+  static constexpr bool kDirect = false, kSumsq = false;
   float *C; int ldc; const float *bias; const float *Z;
+  __device__ __forceinline__ void prefetch(int row, int col) const { prefetch_l2(Z + (size_t)row * ldc + col); }
   __device__ __forceinline__ float4 operator()(int row, int col, float4 a, double &) const {
     const float4 z = *reinterpret_cast<const float4 *>(Z + (size_t)row * ldc + col);
     const float4 b = *reinterpret_cast<const float4 *>(bias + col);
@@ -36,7 +48,12 @@ struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b
   }
 };
 struct EpiGradP {             // C = nu*acc + U + rho*(P - Q), accumulates sum(C^2)
+  static constexpr bool kDirect = false, kSumsq = true;
   float *C; int ldc; const float *U, *P, *Q; float nu, rho;
+  __device__ __forceinline__ void prefetch(int row, int col) const {
+    const size_t o = (size_t)row * ldc + col;
+    prefetch_l2(U + o); prefetch_l2(P + o); prefetch_l2(Q + o);
+  }
   __device__ __forceinline__ float4 operator()(int row, int col, float4 a, double &ss) const {
     const size_t o = (size_t)row * ldc + col;
     const float4 u = *reinterpret_cast<const float4 *>(U + o);

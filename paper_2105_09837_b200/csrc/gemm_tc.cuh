@@ -20,7 +20,9 @@
 namespace pd {
 
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 32, TC_STAGES = 3;
+constexpr int TC_FLUSH = 1;                                    // K blocks per read-out of the main accumulator
 constexpr int TC_TILE_BYTES = 128 * TC_BK * 4;                 // 16 KB: one 128 x 32 fp32 operand tile
+constexpr int TC_MN_CHUNK = TC_BK * 128;                       // MN-major tiles: 32 output indices x TC_BK rows
 constexpr int TC_STAGE_BYTES = 4 * TC_TILE_BYTES;              // A_hi, A_lo, B_hi, B_lo
 // warp 0: TMA, warp 1: MMA, warps 2..5: operand split, warps 6..13: accumulate + epilogue
 // (two warps per 32-lane quarter of tensor memory, 64 columns each)
@@ -41,6 +43,13 @@ struct TcParams {
   int n_split;            // number of contraction slices; slice z writes its own partial output
   size_t c_split_stride;  // elements between the partial outputs of consecutive slices
   int *error;             // set to 1 if a bounded wait expired
+  // Tail balancing (n_split == 1 only): output tiles from tail_begin on are cut into tail_split contraction
+  // slices, one work unit each, so that the last, partly filled round of the persistent grid is shorter.
+  // A slice leaves its accumulators in tail_ws; the warp that finds itself last (tail_count) adds the slices
+  // in slice order and runs the epilogue.  tail_split <= 1 switches this off.
+  int tail_begin, tail_split;
+  float *tail_ws;         // [tiles from tail_begin][tail_split][8 warps][64][32] floats
+  int *tail_count;        // [tiles from tail_begin][8 warps], zero before and after every launch
 };
 
 // A_MN / B_MN: operand is stored contiguous along its output index (rows of the tile are K slices);
@@ -60,7 +69,8 @@ struct TcParams {
 template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_blo, const TcParams prm, Epi epi, double *__restrict__ partials) {
+               const __grid_constant__ CUtensorMap map_blo, const __grid_constant__ CUtensorMap map_c,
+               const TcParams prm, Epi epi, double *__restrict__ partials) {
   if (*reinterpret_cast<volatile int *>(prm.error) != 0) return;   // an earlier block gave up: do not queue behind it
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -74,7 +84,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_n = (prm.N + TC_BN - 1) / TC_BN, tiles_m = (prm.M + TC_BM - 1) / TC_BM;
-  const int n_tiles = tiles_n * tiles_m * prm.n_split;
+  const int n_out_tiles = tiles_n * tiles_m * prm.n_split;
+  const bool tail_on = prm.tail_split > 1;
+  const int tail_begin = tail_on ? prm.tail_begin : n_out_tiles;
+  const int n_tiles = tail_begin + (n_out_tiles - tail_begin) * (tail_on ? prm.tail_split : 1);   // work units
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) {
@@ -93,6 +106,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::prefetch_tmap(&map_a);
     ptx::prefetch_tmap(&map_b);
     if (!B_SPLIT) ptx::prefetch_tmap(&map_blo);
+    if (Epi::kDirect) ptx::prefetch_tmap(&map_c);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, TC_TMEM_COLS);
@@ -103,8 +117,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // tile -> (row tile origin, column tile origin, first and number of K blocks)
-  auto tile_coords = [&](int tile, int &m0, int &n0, int &k_begin, int &n_kb, int &z) {
+  // work unit -> (row tile origin, column tile origin, first and number of K blocks); a unit is an output tile or,
+  // in the tail, one contraction slice of an output tile
+  auto tile_coords = [&](int unit, int &m0, int &n0, int &k_begin, int &n_kb, int &z) {
+    int tile = unit, slice = 0;
+    if (unit >= tail_begin) {
+      tile = tail_begin + (unit - tail_begin) / prm.tail_split;
+      slice = (unit - tail_begin) % prm.tail_split;
+    }
     z = tile / (tiles_m * tiles_n);
     const int rem = tile - z * tiles_m * tiles_n;
     m0 = (rem / tiles_n) * TC_BM;
@@ -112,6 +132,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     k_begin = z * prm.k_chunk;
     const int k_end = min(prm.K, k_begin + prm.k_chunk);
     n_kb = (max(k_end - k_begin, 0) + TC_BK - 1) / TC_BK;
+    if (unit >= tail_begin) {
+      const int kb0 = slice * n_kb / prm.tail_split, kb1 = (slice + 1) * n_kb / prm.tail_split;
+      k_begin += kb0 * TC_BK;
+      n_kb = kb1 - kb0;
+    }
   };
 
   if (warp == 0) {
@@ -129,15 +154,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int k0 = k_begin + kb * TC_BK;
           ptx::mbar_expect_tx(&full_bar[s], (B_SPLIT ? 2 : 3) * TC_TILE_BYTES);
           if (A_MN) {
-            for (int j = 0; j < 4; ++j) ptx::tma_load_2d(st + j * 4096, &map_a, m0 + 32 * j, k0, &full_bar[s]);
+            for (int j = 0; j < 4; ++j) ptx::tma_load_2d(st + j * TC_MN_CHUNK, &map_a, m0 + 32 * j, k0, &full_bar[s]);
           } else {
             ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
           }
           uint8_t *bh = st + 2 * TC_TILE_BYTES, *bl = st + 3 * TC_TILE_BYTES;
           if (B_MN) {
-            for (int j = 0; j < 4; ++j) ptx::tma_load_2d(bh + j * 4096, &map_b, n0 + 32 * j, k0, &full_bar[s]);
+            for (int j = 0; j < 4; ++j) ptx::tma_load_2d(bh + j * TC_MN_CHUNK, &map_b, n0 + 32 * j, k0, &full_bar[s]);
             if (!B_SPLIT)
-              for (int j = 0; j < 4; ++j) ptx::tma_load_2d(bl + j * 4096, &map_blo, n0 + 32 * j, k0, &full_bar[s]);
+              for (int j = 0; j < 4; ++j) ptx::tma_load_2d(bl + j * TC_MN_CHUNK, &map_blo, n0 + 32 * j, k0, &full_bar[s]);
           } else {
             ptx::tma_load_2d(bh, &map_b, k0, n0, &full_bar[s]);
             if (!B_SPLIT) ptx::tma_load_2d(bl, &map_blo, k0, n0, &full_bar[s]);
@@ -155,36 +180,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::idesc_tf32(TC_BM, TC_BN, A_MN, B_MN);
       const uint32_t d_corr = tmem_base + (uint32_t)(TC_ACC_BUFS * TC_BN);
+      // descriptors: constant high words; the low word of stage 0 advances by whole stages / K steps
+      const uint32_t hi_a = ptx::smem_desc_hi(A_MN, TC_BK * 4), hi_b = ptx::smem_desc_hi(B_MN, TC_BK * 4);
+      const uint32_t lo_a0 = ptx::smem_desc_lo(ptx::smem_u32(smem), A_MN, TC_MN_CHUNK);
+      const uint32_t lo_b0 = ptx::smem_desc_lo(ptx::smem_u32(smem) + 2 * TC_TILE_BYTES, B_MN, TC_MN_CHUNK);
+      constexpr uint32_t step_a = (A_MN ? 1024u : 32u) >> 4, step_b = (B_MN ? 1024u : 32u) >> 4;
       bool ok = true;
-      int it = 0, ti = 0;
+      // running state: stage s with phase bit sp, accumulator buffer b with phase bit bp (of its *previous* use),
+      // and whether the barriers of the coming K block were already seen complete by the probe below
+      int s = 0, b = 0, ti = 0;
+      uint32_t sp = 0, bp = 1;
+      bool first_round = true, seen_conv = false, seen_acc = false;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++ti) {
         int m0, n0, k_begin, n_kb, z;
         tile_coords(tile, m0, n0, k_begin, n_kb, z);
         // the correction tile of the previous output tile must have been read before it is overwritten
         if (ti > 0 && n_kb > 0) ok = ptx::mbar_wait(corr_empty, (ti - 1) & 1, abort_flag);
-        for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
-          const int s = it % TC_STAGES, use = it / TC_STAGES;
-          const int b = it % TC_ACC_BUFS, buse = it / TC_ACC_BUFS;
-          ok = ptx::mbar_wait(&conv_bar[s], use & 1, abort_flag);
-          if (ok && buse > 0) ok = ptx::mbar_wait(&acc_empty[b], (buse - 1) & 1, abort_flag);
+        for (int kb = 0; kb < n_kb && ok; ++kb) {
+          const bool first = kb % TC_FLUSH == 0, last = kb % TC_FLUSH == TC_FLUSH - 1 || kb == n_kb - 1;
+          if (!seen_conv) ok = ptx::mbar_wait(&conv_bar[s], sp, abort_flag);
+          if (ok && first && !first_round && !seen_acc) ok = ptx::mbar_wait(&acc_empty[b], bp, abort_flag);
           if (!ok) break;
           ptx::tc_fence_after_sync();
-          const uint32_t st = ptx::smem_u32(smem + s * TC_STAGE_BYTES);
-          const uint32_t a_hi = st, a_lo = st + TC_TILE_BYTES, b_hi = st + 2 * TC_TILE_BYTES, b_lo = st + 3 * TC_TILE_BYTES;
+          const uint32_t la = lo_a0 + (uint32_t)s * (TC_STAGE_BYTES >> 4), lb = lo_b0 + (uint32_t)s * (TC_STAGE_BYTES >> 4);
           const uint32_t d = tmem_base + (uint32_t)(b * TC_BN);
+          // next K block's stage and, if it starts a new group, its accumulator buffer
+          const int s_next = s + 1 == TC_STAGES ? 0 : s + 1;
+          const uint32_t sp_next = s + 1 == TC_STAGES ? sp ^ 1u : sp;
+          const int b_next = b + 1 == TC_ACC_BUFS ? 0 : b + 1;
+          const uint32_t bp_next = b + 1 == TC_ACC_BUFS ? bp ^ 1u : bp;
+          const bool round_next = first_round && b + 1 != TC_ACC_BUFS;
 #pragma unroll
           for (int kk = 0; kk < TC_BK / 8; ++kk) {
-            const uint32_t ao = A_MN ? kk * 1024 : kk * 32, bo = B_MN ? kk * 1024 : kk * 32;
-            const uint64_t dah = ptx::smem_desc(a_hi + ao, A_MN, 4096);
-            const uint64_t dal = ptx::smem_desc(a_lo + ao, A_MN, 4096);
-            const uint64_t dbh = ptx::smem_desc(b_hi + bo, B_MN, 4096);
-            const uint64_t dbl = ptx::smem_desc(b_lo + bo, B_MN, 4096);
+            const uint64_t dah = ptx::smem_desc(hi_a, la + kk * step_a);
+            const uint64_t dal = ptx::smem_desc(hi_a, la + (TC_TILE_BYTES >> 4) + kk * step_a);
+            const uint64_t dbh = ptx::smem_desc(hi_b, lb + kk * step_b);
+            const uint64_t dbl = ptx::smem_desc(hi_b, lb + (TC_TILE_BYTES >> 4) + kk * step_b);
             ptx::mma_tf32(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
             ptx::mma_tf32(d_corr, dah, dbl, idesc, true);
-            ptx::mma_tf32(d, dah, dbh, idesc, kk > 0);
+            ptx::mma_tf32(d, dah, dbh, idesc, !first || kk > 0);
+            if (kk == TC_BK / 8 - 2) {
+              // probe the coming block's barriers while the tensor pipe still has work queued
+              seen_conv = ptx::mbar_test_wait(&conv_bar[s_next], sp_next);
+              seen_acc = last ? (round_next ? true : ptx::mbar_test_wait(&acc_empty[b_next], bp_next)) : true;
+            }
           }
           ptx::mma_commit(&empty_bar[s]);          // stage can be refilled once these MMAs have read it
-          ptx::mma_commit(&acc_full[b]);           // this block's partial product is complete
+          if (last) {
+            ptx::mma_commit(&acc_full[b]);         // this group's partial product is complete
+            if (b + 1 == TC_ACC_BUFS) first_round = false;
+            b = b_next; bp = bp_next;
+          }
+          s = s_next; sp = sp_next;
         }
       }
       if (!ok) {
@@ -240,6 +287,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       int m0, n0, k_begin, n_kb, z;
       tile_coords(tile, m0, n0, k_begin, n_kb, z);
+      if (m0 + lane_base + lane < prm.M) {          // this thread's row of the epilogue inputs, on its way to L2
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int col = n0 + chalf * 64 + h * 32;
+          if (col < n_pad) epi.prefetch(m0 + lane_base + lane, col);
+        }
+      }
       float acc[64];
 #pragma unroll
       for (int j = 0; j < 64; ++j) acc[j] = 0.f;
@@ -252,7 +306,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
         for (int j = 0; j < 32; ++j) { acc[j] += __uint_as_float(v0[j]); acc[32 + j] += __uint_as_float(v1[j]); }
       };
-      for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+      const int n_grp = (n_kb + TC_FLUSH - 1) / TC_FLUSH;
+      for (int g = 0; g < n_grp && ok; ++g, ++it) {
         const int b = it % TC_ACC_BUFS, buse = it / TC_ACC_BUFS;
         ok = ptx::mbar_wait(&acc_full[b], buse & 1, abort_flag);
         if (!ok) break;
@@ -268,40 +323,95 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(corr_empty);
       }
-      // Epilogue.  Thread i of the warp holds row (lane_base + i), 64 columns.  For coalesced global accesses the
-      // warp's piece goes through shared memory 32 columns at a time: thread i writes its 8 float4 groups with the
-      // group index XOR-ed by (i mod 8) (conflict-free 128-bit stores), then the warp walks over its rows four at a
-      // time: lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane (one 128-byte line per row).
-      double ss = 0.0;
-      float *C = epi.C + (size_t)z * prm.c_split_stride;
+      int out_tile = tile;
+      if (tile >= tail_begin) {
+        // contraction slice of a tail tile: park the accumulators; the last warp to arrive sums the slices
+        const int u = tile - tail_begin, t_idx = u / prm.tail_split;
+        out_tile = tail_begin + t_idx;
+        float *mine = prm.tail_ws + ((size_t)u * 8 + (warp - 6)) * 2048;
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
+        for (int j = 0; j < 64; ++j) mine[j * 32 + lane] = acc[j];
+        __threadfence();
         __syncwarp();
+        int prev = 0;
+        if (lane == 0) prev = atomicAdd(prm.tail_count + t_idx * 8 + (warp - 6), 1);
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        if (prev != prm.tail_split - 1) continue;
+        __threadfence();
+        if (lane == 0) prm.tail_count[t_idx * 8 + (warp - 6)] = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int jj = h * 8 + j;
-          tr[lane * 8 + (j ^ (lane & 7))] = make_float4(acc[4 * jj], acc[4 * jj + 1], acc[4 * jj + 2], acc[4 * jj + 3]);
+        for (int j = 0; j < 64; ++j) acc[j] = 0.f;
+        for (int sl = 0; sl < prm.tail_split; ++sl) {
+          const float *part = prm.tail_ws + ((size_t)(t_idx * prm.tail_split + sl) * 8 + (warp - 6)) * 2048;
+#pragma unroll
+          for (int j = 0; j < 64; ++j) acc[j] += __ldcg(part + j * 32 + lane);
         }
-        __syncwarp();
-        const int col = n0 + chalf * 64 + h * 32 + 4 * (lane & 7);
-        if (col < n_pad) {
+      }
+      // Epilogue.  Thread i of the warp holds row (lane_base + i), 64 columns.  The warp's piece goes through shared
+      // memory 32 columns at a time: thread i writes its 8 float4 groups with the group index XOR-ed by (i mod 8)
+      // (conflict-free 128-bit stores; this is also the 128-byte swizzle of the output tensor map).
+      double ss = 0.0;
+      if constexpr (Epi::kDirect) {
+        // The output is the accumulator: sum of squares straight from the registers (four fp32 partial sums of 16
+        // squares each, added in double), and the 32 x 32 pieces leave shared memory as TMA stores, which clip at the
+        // matrix edges.  Rows and columns outside the matrix hold exact zeros (zero-filled operand tiles).
+        if constexpr (Epi::kSumsq) {
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int j = 0; j < 64; ++j) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
+          ss = ((double)s4[0] + (double)s4[1]) + ((double)s4[2] + (double)s4[3]);
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (lane == 0) ptx::bulk_wait_read();       // the previous store has read the staging buffer
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int jj = h * 8 + j;
+            tr[lane * 8 + (j ^ (lane & 7))] = make_float4(acc[4 * jj], acc[4 * jj + 1], acc[4 * jj + 2], acc[4 * jj + 3]);
+          }
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            const int x = n0 + chalf * 64 + h * 32, y = m0 + lane_base;
+            if (x < epi.ldc && y < prm.M) ptx::tma_store_3d(&map_c, tr, x, y, z);
+            ptx::bulk_commit();
+          }
+        }
+      } else {
+        // Inputs of the epilogue are read with the same coalesced pattern as the output is written: the warp walks
+        // over its rows four at a time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.
+        float *C = epi.C + (size_t)z * prm.c_split_stride;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int jj = h * 8 + j;
+            tr[lane * 8 + (j ^ (lane & 7))] = make_float4(acc[4 * jj], acc[4 * jj + 1], acc[4 * jj + 2], acc[4 * jj + 3]);
+          }
+          __syncwarp();
+          const int col = n0 + chalf * 64 + h * 32 + 4 * (lane & 7);
+          if (col < n_pad) {
 #pragma unroll 4
-          for (int step = 0; step < 8; ++step) {
-            const int r = 4 * step + (lane >> 3);
-            const int row = m0 + lane_base + r;
-            if (row < prm.M) {
-              const float4 a = tr[r * 8 + ((lane & 7) ^ (r & 7))];
-              const float4 o = epi(row, col, a, ss);
-              *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
+            for (int step = 0; step < 8; ++step) {
+              const int r = 4 * step + (lane >> 3);
+              const int row = m0 + lane_base + r;
+              if (row < prm.M) {
+                const float4 a = tr[r * 8 + ((lane & 7) ^ (r & 7))];
+                const float4 o = epi(row, col, a, ss);
+                *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
+              }
             }
           }
         }
       }
       if (partials != nullptr) {          // one slot per tile and warp; the host adds the slots in index order
         ss = warp_sum(ss);
-        if (lane == 0) partials[(size_t)tile * 8 + (warp - 6)] = ss;
+        if (lane == 0) partials[(size_t)out_tile * 8 + (warp - 6)] = ss;
       }
     }
+    if (Epi::kDirect && lane == 0) ptx::bulk_wait_all();
   }
   ptx::tc_fence_before_sync();
   __syncthreads();

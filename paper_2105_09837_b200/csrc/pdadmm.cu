@@ -76,6 +76,8 @@ struct Scratch {
   float *part = nullptr;    // partial tiles of grad_W
   double *slots = nullptr;  // per-block partial sums
   size_t n_slots = 0;
+  float *tail_ws = nullptr; // accumulators of the contraction slices of tail tiles (one tile per SM at most)
+  int *tail_count = nullptr;
 };
 
 struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
@@ -205,7 +207,8 @@ static int get_tmap(pdadmm_ctx *c, const float *base, uint64_t inner, uint64_t o
   cuuint32_t estr[2] = {1, 1};
   CUtensorMap m;
   CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)base, dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
+                           : (box_inner * 4 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
@@ -215,9 +218,36 @@ static int get_tmap(pdadmm_ctx *c, const float *base, uint64_t inner, uint64_t o
   return PDADMM_OK;
 }
 
+// Output of a product as a 3-D tensor [n_split][rows][ld] for the TMA stores of the epilogue: 32 x 32 boxes,
+// 128-byte swizzle (the layout the epilogue leaves in shared memory).
+static int get_tmap_out(pdadmm_ctx *c, const float *base, uint64_t ld, uint64_t rows, uint64_t n_split,
+                        uint64_t split_stride, CUtensorMap *out) {
+  auto key = std::make_tuple((const void *)base, ld, rows, n_split, 0xC0000000u, (uint32_t)(split_stride & 0xffffffffu));
+  auto it = c->tmaps.find(key);
+  if (it != c->tmaps.end()) { *out = it->second; return PDADMM_OK; }
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled is not available in this driver");
+  cuuint64_t dims[3] = {ld, rows, n_split};
+  cuuint64_t strides[2] = {ld * 4, (n_split > 1 ? split_stride : rows * ld) * 4};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUtensorMap m;
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void *)base, dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled (output) failed with code %d", (int)r);
+  if (c->tmaps.size() > 4096) c->tmaps.clear();
+  c->tmaps[key] = m;
+  *out = m;
+  return PDADMM_OK;
+}
+
 template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
 static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mbl,
                      const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
+  CUtensorMap mc = ma;                 // not used unless the epilogue stores the accumulator itself
+  if (Epi::kDirect)
+    PD_TRY(get_tmap_out(c, epi.C, (uint64_t)epi.ldc, (uint64_t)prm.M, (uint64_t)prm.n_split, prm.c_split_stride, &mc));
   auto kern = gemm_tc_kernel<A_MN, B_MN, B_SPLIT, Epi>;
   const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
   static bool configured = false;
@@ -225,7 +255,7 @@ static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, cons
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     configured = true;
   }
-  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, prm, epi, partials);
+  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, mc, prm, epi, partials);
   return PDADMM_OK;
 }
 
@@ -256,8 +286,20 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     PD_TRY(get_tmap(c, B_lo, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mbl));
   }
   TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1};
+  // The persistent grid works through the tiles in rounds of n_sms; a last round that fills only part of the
+  // SMs costs as much as a full one, so its tiles are cut along the contraction into as many slices as fit.
+  int n_units = n_tiles;
+  const int tail = n_tiles % c->n_sms, n_kb = (int)ceil_div(K, TC_BK);
+  if (tail > 0 && c->scr.tail_ws != nullptr) {
+    const int split = std::min(std::min(c->n_sms / tail, n_kb / 4), 8);     // at least 4 K blocks per slice
+    if (split > 1) {
+      prm.tail_begin = n_tiles - tail; prm.tail_split = split;
+      prm.tail_ws = c->scr.tail_ws; prm.tail_count = c->scr.tail_count;
+      n_units = prm.tail_begin + tail * split;
+    }
+  }
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
-  return launch_tc<false, B_NMAJOR, false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, n_tiles);
+  return launch_tc<false, B_NMAJOR, false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, n_units);
 }
 
 // hi/lo planes of a weight-sized matrix for the tensor-core path
@@ -636,6 +678,10 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
   s.n_slots *= 2;                       // two halves: consecutive reductions of one layer use different halves
   PD_TRY(dev_alloc(c, &s.slots, s.n_slots));
+  if (c->use_tc) {
+    PD_TRY(dev_alloc(c, &s.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
+    PD_TRY(dev_alloc(c, &s.tail_count, (size_t)c->n_sms * 8));
+  }
 
   // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
   Layer &l0 = c->layers[0];
@@ -1017,6 +1063,10 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
     PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
     cudaStream_t st = c->scr.st;
     PD_TRY(dev_alloc(c, &c->d_flag, 4));
+    if (c->use_tc) {
+      PD_TRY(dev_alloc(c, &c->scr.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
+      PD_TRY(dev_alloc(c, &c->scr.tail_count, (size_t)c->n_sms * 8));
+    }
     // operand shapes as stored: rows x cols
     const int a_rows = mode == 2 ? K : M, a_cols = mode == 2 ? M : K;
     const int b_rows = mode == 0 ? N : K, b_cols = mode == 0 ? K : N;

@@ -32,6 +32,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// Non-blocking probe of a phase (mbarrier.try_wait may suspend the thread for a while; this never does).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait: gives up after about `limit_cycles` SM cycles (or, with heed_abort, as soon as another
 // thread of the block has given up) and raises *abort_flag (shared memory).  Returns false if the wait
 // was abandoned.
@@ -55,6 +65,17 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
 }
+// ---- TMA: 3-D tile store shared -> global (bulk async group of the issuing thread) ---------------------
+// Parts of the box outside the tensor are not written.  Coordinates must not be negative.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, const void *src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all bulk groups of this thread have finished reading shared memory / have completed
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -103,19 +124,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---- descriptors -------------------------------------------------------------------------------------------
-// Shared-memory matrix descriptor for tiles whose rows are 128 bytes (the tile base must be 1024-byte aligned).
-// K-major operand  (rows = output index, 32 floats of K per row): 128-byte swizzle with 16-byte atoms,
-//                   8-row groups 1024 bytes apart (sbo); lbo is not used by the hardware for this form.
+// Shared-memory matrix descriptor (the tile base must be aligned to the swizzle period).
+// K-major operand  (rows = output index, k_row_bytes = 64 or 128 bytes of K per row): swizzle of the row width
+//                   with 16-byte atoms, 8-row groups 8 rows apart (sbo); lbo is not used by the hardware here.
 // MN-major operand (rows = K index, 32 floats of the output index per row): for 32-bit types the only
 //                   layout is the 128-byte swizzle with 32-byte atoms; 4-row groups 512 bytes apart (sbo),
 //                   the next 32 output indices lbo bytes further.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, bool mn_major, uint32_t lbo_mn) {
-  const uint32_t lbo = mn_major ? lbo_mn : 16u, sbo = mn_major ? 512u : 1024u;
-  const uint32_t layout = mn_major ? 1u /* 128B swizzle, 32B atoms */ : 2u /* 128B swizzle */;
-  const uint32_t lo = ((saddr >> 4) & 0x3FFFu) | (((lbo >> 4) & 0x3FFFu) << 16);
-  const uint32_t hi = ((sbo >> 4) & 0x3FFFu) | (1u << 14) /* descriptor version */ | (layout << 29);
-  return ((uint64_t)hi << 32) | lo;
+// The descriptor is built from two words so that a loop only has to add to the low one: the start address
+// field counts 16-byte units and shared-memory addresses stay below 2^18, so (address >> 4) needs no mask.
+__device__ __forceinline__ uint32_t smem_desc_hi(bool mn_major, uint32_t k_row_bytes) {
+  const uint32_t sbo = mn_major ? 512u : 8u * k_row_bytes;
+  const uint32_t layout = mn_major ? 1u /* 128B swizzle, 32B atoms */ : (k_row_bytes == 128u ? 2u /* 128B */ : 4u /* 64B */);
+  return ((sbo >> 4) & 0x3FFFu) | (1u << 14) /* descriptor version */ | (layout << 29);
 }
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, bool mn_major, uint32_t lbo_mn) {
+  const uint32_t lbo = mn_major ? lbo_mn : 16u;
+  return (saddr >> 4) | (((lbo >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t smem_desc(uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; }
 // Instruction descriptor: tf32 x tf32 -> fp32, M x N tile, operand majors (false = K-major, true = MN-major).
 __host__ __device__ constexpr uint32_t idesc_tf32(int M, int N, bool a_mn_major, bool b_mn_major) {
   return (1u << 4) | (2u << 7) | (2u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
