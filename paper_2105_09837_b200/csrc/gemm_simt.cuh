@@ -24,12 +24,14 @@ __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefe
 // kSumsq: the epilogue accumulates the sum of squares of the output.
 struct EpiStore {             // C = acc
   static constexpr bool kDirect = true, kSumsq = false;
+  static constexpr int kInputs = 0;
   float *C; int ldc;
   __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ float4 operator()(int, int, float4 a, double &) const { return a; }
 };
 struct EpiStoreSumsq {        // C = acc, accumulates sum(acc^2)
   static constexpr bool kDirect = true, kSumsq = true;
+  static constexpr int kInputs = 0;
   float *C; int ldc;
   __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ float4 operator()(int, int, float4 a, double &ss) const {
@@ -39,8 +41,16 @@ struct EpiStoreSumsq {        // C = acc, accumulates sum(acc^2)
 };
 struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b - z)
   static constexpr bool kDirect = false, kSumsq = false;
+  static constexpr int kInputs = 1;        // float4 loads per output group: load() fetches, apply() combines
   float *C; int ldc; const float *bias; const float *Z;
   __device__ __forceinline__ void prefetch(int row, int col) const { prefetch_l2(Z + (size_t)row * ldc + col); }
+  __device__ __forceinline__ void load(int row, int col, float4 *in) const {
+    in[0] = *reinterpret_cast<const float4 *>(Z + (size_t)row * ldc + col);
+  }
+  __device__ __forceinline__ float4 apply(int col, float4 a, const float4 *in) const {
+    const float4 b = *reinterpret_cast<const float4 *>(bias + col);
+    return make_float4(a.x + b.x - in[0].x, a.y + b.y - in[0].y, a.z + b.z - in[0].z, a.w + b.w - in[0].w);
+  }
   __device__ __forceinline__ float4 operator()(int row, int col, float4 a, double &) const {
     const float4 z = *reinterpret_cast<const float4 *>(Z + (size_t)row * ldc + col);
     const float4 b = *reinterpret_cast<const float4 *>(bias + col);
@@ -49,7 +59,18 @@ struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b
 };
 struct EpiGradP {             // C = nu*acc + U + rho*(P - Q), accumulates sum(C^2)
   static constexpr bool kDirect = false, kSumsq = true;
+  static constexpr int kInputs = 3;
   float *C; int ldc; const float *U, *P, *Q; float nu, rho;
+  __device__ __forceinline__ void load(int row, int col, float4 *in) const {
+    const size_t o = (size_t)row * ldc + col;
+    in[0] = *reinterpret_cast<const float4 *>(U + o);
+    in[1] = *reinterpret_cast<const float4 *>(P + o);
+    in[2] = *reinterpret_cast<const float4 *>(Q + o);
+  }
+  __device__ __forceinline__ float4 apply(int, float4 a, const float4 *in) const {
+    return make_float4(nu * a.x + in[0].x + rho * (in[1].x - in[2].x), nu * a.y + in[0].y + rho * (in[1].y - in[2].y),
+                       nu * a.z + in[0].z + rho * (in[1].z - in[2].z), nu * a.w + in[0].w + rho * (in[1].w - in[2].w));
+  }
   __device__ __forceinline__ void prefetch(int row, int col) const {
     const size_t o = (size_t)row * ldc + col;
     prefetch_l2(U + o); prefetch_l2(P + o); prefetch_l2(Q + o);

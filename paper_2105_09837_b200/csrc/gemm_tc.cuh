@@ -154,15 +154,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int k0 = k_begin + kb * TC_BK;
           ptx::mbar_expect_tx(&full_bar[s], (B_SPLIT ? 2 : 3) * TC_TILE_BYTES);
           if (A_MN) {
-            for (int j = 0; j < 4; ++j) ptx::tma_load_2d(st + j * TC_MN_CHUNK, &map_a, m0 + 32 * j, k0, &full_bar[s]);
+            ptx::tma_load_3d(st, &map_a, 0, k0, m0 / 32, &full_bar[s]);
           } else {
             ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
           }
           uint8_t *bh = st + 2 * TC_TILE_BYTES, *bl = st + 3 * TC_TILE_BYTES;
           if (B_MN) {
-            for (int j = 0; j < 4; ++j) ptx::tma_load_2d(bh + j * TC_MN_CHUNK, &map_b, n0 + 32 * j, k0, &full_bar[s]);
-            if (!B_SPLIT)
-              for (int j = 0; j < 4; ++j) ptx::tma_load_2d(bl + j * TC_MN_CHUNK, &map_blo, n0 + 32 * j, k0, &full_bar[s]);
+            ptx::tma_load_3d(bh, &map_b, 0, k0, n0 / 32, &full_bar[s]);
+            if (!B_SPLIT) ptx::tma_load_3d(bl, &map_blo, 0, k0, n0 / 32, &full_bar[s]);
           } else {
             ptx::tma_load_2d(bh, &map_b, k0, n0, &full_bar[s]);
             if (!B_SPLIT) ptx::tma_load_2d(bl, &map_blo, k0, n0, &full_bar[s]);
@@ -357,8 +356,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // matrix edges.  Rows and columns outside the matrix hold exact zeros (zero-filled operand tiles).
         if constexpr (Epi::kSumsq) {
           float s4[4] = {0.f, 0.f, 0.f, 0.f};
+          const int n_valid = prm.N - (n0 + chalf * 64);      // columns of this thread inside the matrix
 #pragma unroll
-          for (int j = 0; j < 64; ++j) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
+          for (int j = 0; j < 64; ++j)
+            if (j < n_valid) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
           ss = ((double)s4[0] + (double)s4[1]) + ((double)s4[2] + (double)s4[3]);
         }
 #pragma unroll
@@ -380,8 +381,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       } else {
         // Inputs of the epilogue are read with the same coalesced pattern as the output is written: the warp walks
-        // over its rows four at a time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.
+        // over its rows four at a time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.  The
+        // loads of four steps are issued together (rows past the end are clamped, their results dropped).
         float *C = epi.C + (size_t)z * prm.c_split_stride;
+        float ssf = 0.f;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           __syncwarp();
@@ -393,18 +396,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __syncwarp();
           const int col = n0 + chalf * 64 + h * 32 + 4 * (lane & 7);
           if (col < n_pad) {
-#pragma unroll 4
-            for (int step = 0; step < 8; ++step) {
-              const int r = 4 * step + (lane >> 3);
-              const int row = m0 + lane_base + r;
-              if (row < prm.M) {
-                const float4 a = tr[r * 8 + ((lane & 7) ^ (r & 7))];
-                const float4 o = epi(row, col, a, ss);
-                *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
+#pragma unroll
+            for (int s0 = 0; s0 < 8; s0 += 4) {
+              float4 in[4][Epi::kInputs > 0 ? Epi::kInputs : 1];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int r = 4 * (s0 + i) + (lane >> 3);
+                epi.load(min(m0 + lane_base + r, prm.M - 1), col, in[i]);
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int r = 4 * (s0 + i) + (lane >> 3);
+                const int row = m0 + lane_base + r;
+                const float4 o = epi.apply(col, tr[r * 8 + ((lane & 7) ^ (r & 7))], in[i]);
+                if (row < prm.M) {
+                  if (Epi::kSumsq) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
+                  *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
+                }
               }
             }
           }
         }
+        ss = (double)ssf;
       }
       if (partials != nullptr) {          // one slot per tile and warp; the host adds the slots in index order
         ss = warp_sum(ss);

@@ -124,7 +124,7 @@ namespace pd {
 template <class T>
 static int dev_alloc(pdadmm_ctx *c, T **ptr, size_t count, bool zero = true) {
   void *p = nullptr;
-  const size_t bytes = std::max<size_t>(count * sizeof(T), 16);
+  const size_t bytes = count * sizeof(T) + 256;     // slack: operand copies may read up to 31 floats past a matrix
   cudaError_t e = cudaMalloc(&p, bytes);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -201,16 +201,28 @@ static int get_tmap(pdadmm_ctx *c, const float *base, uint64_t inner, uint64_t o
   if (it != c->tmaps.end()) { *out = it->second; return PDADMM_OK; }
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled is not available in this driver");
-  cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {ld * 4};
-  cuuint32_t box[2] = {box_inner, box_outer};
-  cuuint32_t estr[2] = {1, 1};
   CUtensorMap m;
-  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)base, dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
-                           : (box_inner * 4 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r;
+  if (mn_major) {
+    // rows = contraction index, `inner` output indices per row.  Seen as [inner / 32][outer][32] so that one copy
+    // brings four 32-wide column chunks, each as consecutive 128-byte rows (the layout of an MN-major operand).
+    // The last chunk may reach past the row end into the next row (or the slack after the allocation): those
+    // columns only feed output elements outside the matrix, which are never stored.
+    cuuint64_t dims[3] = {32, outer, (inner + 31) / 32};
+    cuuint64_t strides[2] = {ld * 4, 128};
+    cuuint32_t box[3] = {32, box_outer, 4};
+    cuuint32_t estr[3] = {1, 1, 1};
+    r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {ld * 4};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           box_inner * 4 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   if (r != CUDA_SUCCESS) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
   if (c->tmaps.size() > 4096) c->tmaps.clear();
   c->tmaps[key] = m;
