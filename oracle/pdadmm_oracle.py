@@ -76,6 +76,9 @@ class Params:
     quant_levels: int = 0                 # 0: pdADMM-G ; m >= 2: pdADMM-G-Q with m levels per layer
     max_trials: int = 30                  # cap of the tau search in the quantised p-update
     accept_slack: float = 1e-6
+    quantize_q: bool = False              # the variant that also keeps q_l in Delta (end of Sec. "Quantization Extension")
+    level_lo: float = 0.0                 # smallest level delta_0
+    level_step: float = 0.0               # > 0: the same fixed step for every layer; 0: step from max(p) at the start
 
 
 @dataclasses.dataclass
@@ -202,30 +205,32 @@ def update_p(p, W, b, z, nu, q_prev, u_prev, rho):
 # Quantisation set and the quantised p-update (Eq. update p quantized)
 # ----------------------------------------------------------------------------
 
-def level_set(scale: float, m: int) -> np.ndarray:
-    """Delta = {delta_0..delta_{m-1}}, delta_c = fl32(c * s): m uniform levels starting at 0.
+def level_set(scale: float, m: int, lo: float = 0.0) -> np.ndarray:
+    """Delta = {delta_0..delta_{m-1}}, delta_c = fl32(lo + fl32(c * s)): m uniform levels starting at lo.
 
-    The levels are single-precision numbers (one rounded multiply), so that a
-    quantised p is exactly representable in the fp32 state of the CUDA path.
+    The levels are single-precision numbers (one rounded multiply, one rounded
+    add), so that a quantised p is exactly representable in the fp32 state of
+    the CUDA path.  lo = -1, s = 1, m = 22 is the set {-1, 0, ..., 20} of the
+    paper's experiments (Sec. "Datasets and Settings").
     """
-    return (np.arange(m, dtype=np.float32) * np.float32(scale)).astype(np.float64)
+    return (np.float32(lo) + np.arange(m, dtype=np.float32) * np.float32(scale)).astype(np.float64)
 
 
-def quantize(x, scale: float, m: int):
+def quantize(x, scale: float, m: int, lo: float = 0.0):
     """Nearest element of Delta, element by element: argmin_delta |delta - x|.
 
     Since ||delta - x||^2 is separable the argmin of Eq. (update p quantized)
     is taken per element.  For uniform levels it is a rounding:
-    code = clamp(floor(x/s + 1/2), 0, m-1) (ties at half-levels go up).  The
-    rounding decision is taken in single precision, the precision of the
+    code = clamp(floor((x - lo)/s + 1/2), 0, m-1) (ties at half-levels go up).
+    The rounding decision is taken in single precision, the precision of the
     kernel that takes the same decision.  Returns (codes uint8, p in Delta).
     """
     x32 = np.asarray(x, dtype=np.float32)
-    t = x32 / np.float32(scale)
+    t = (x32 - np.float32(lo)) / np.float32(scale)
     c = np.floor(t + np.float32(0.5))
     c = np.clip(c, np.float32(0.0), np.float32(m - 1))
     codes = c.astype(np.uint8)
-    vals = (c * np.float32(scale)).astype(np.float64)
+    vals = (np.float32(lo) + c * np.float32(scale)).astype(np.float64)
     return codes, vals
 
 
@@ -237,7 +242,7 @@ def quantization_scale(x, m: int) -> float:
     return float(np.float32(mx) / np.float32(m - 1))
 
 
-def update_p_quantized(p, W, b, z, nu, q_prev, u_prev, rho, scale, m, max_trials=30, slack=1e-6):
+def update_p_quantized(p, W, b, z, nu, q_prev, u_prev, rho, scale, m, max_trials=30, slack=1e-6, lo=0.0):
     """p^{k+1} = argmin_{delta in Delta} ||delta - (p^k - nabla_p phi / tau)||.
 
     tau starts at the smallest value admissible for the unprojected step and
@@ -249,7 +254,7 @@ def update_p_quantized(p, W, b, z, nu, q_prev, u_prev, rho, scale, m, max_trials
     tau = tau_smallest_admissible(g, W, nu, rho)
     phi_old = phi(p, W, b, z, nu, q_prev, u_prev, rho)
     for trial in range(1, max_trials + 1):
-        codes, p_new = quantize(p - g / tau, scale, m)
+        codes, p_new = quantize(p - g / tau, scale, m, lo)
         d = p_new - p
         dd = float(np.sum(d * d))
         lhs = phi(p_new, W, b, z, nu, q_prev, u_prev, rho)
@@ -500,6 +505,13 @@ def update_q(p_next, u, z, rho, nu):
     return (rho * p_next + u + nu * relu(z)) / (rho + nu)
 
 
+def update_q_quantized(p_next, u, z, rho, nu, scale, m, lo=0.0):
+    """The variant with q_l in Delta as well: q_l^{k+1} = argmin_{delta in Delta}
+    ||delta - (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)||, element by element
+    (Sec. "Quantization Extension", last paragraph).  Delta is the level set of p_{l+1}, which q_l has to equal."""
+    return quantize(update_q(p_next, u, z, rho, nu), scale, m, lo)[1]
+
+
 def update_u(u, p_next, q, rho):
     """u_l^{k+1} = u_l^k + rho (p_{l+1}^{k+1} - q_l^{k+1})."""
     return u + rho * (p_next - q)
@@ -514,7 +526,9 @@ def init_state(X, W0, y, mask, prm: Params) -> State:
 
     b = 0 and a forward pass: z_l = W_l p_l, q_l = relu(z_l), p_{l+1} = q_l, u = 0.
     pdADMM-G-Q: the pass is sequential in l; the step s_{l+1} of p_{l+1} is
-    max(q_l) / (m - 1) and p_{l+1} = Proj_Delta(q_l), so the residual starts non-zero.
+    max(q_l) / (m - 1) (or the fixed prm.level_step) and p_{l+1} = Proj_Delta(q_l), so the
+    residual starts non-zero.  In the variant that keeps q in Delta too, q_l = p_{l+1} =
+    Proj_Delta(relu(z_l)): a feasible start inside Delta.
     """
     L = len(W0)
     p = [np.asarray(X, dtype=np.float64)]
@@ -528,8 +542,11 @@ def init_state(X, W0, y, mask, prm: Params) -> State:
             q.append(relu(z[l]))
             u.append(np.zeros_like(q[l]))
             if prm.quant_levels:
-                scale[l + 1] = quantization_scale(q[l], prm.quant_levels)
-                p.append(quantize(q[l], scale[l + 1], prm.quant_levels)[1])
+                scale[l + 1] = (float(np.float32(prm.level_step)) if prm.level_step > 0
+                                else quantization_scale(q[l], prm.quant_levels))
+                p.append(quantize(q[l], scale[l + 1], prm.quant_levels, prm.level_lo)[1])
+                if prm.quantize_q:
+                    q[l] = p[l + 1].copy()
             else:
                 p.append(q[l].copy())
     return State(p, W, b, z, q, u, np.asarray(y), np.asarray(mask, dtype=bool), scale,
@@ -548,7 +565,7 @@ def iterate(s: State, prm: Params) -> State:
         if prm.quant_levels:
             n.p[l], _, n.tau[l], n.trials[l] = update_p_quantized(
                 s.p[l], s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho,
-                s.scale[l], prm.quant_levels, prm.max_trials, prm.accept_slack)
+                s.scale[l], prm.quant_levels, prm.max_trials, prm.accept_slack, prm.level_lo)
         else:
             n.p[l], n.tau[l] = update_p(s.p[l], s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho)
     # W_l^{k+1} from (p^{k+1}, b^k, z^k)
@@ -566,7 +583,10 @@ def iterate(s: State, prm: Params) -> State:
             n.z[l] = update_z_last(a, s.y, s.mask, nu)
     # q_l^{k+1}, then u_l^{k+1}
     for l in range(L - 1):
-        n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu)
+        if prm.quant_levels and prm.quantize_q:
+            n.q[l] = update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels, prm.level_lo)
+        else:
+            n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu)
     for l in range(L - 1):
         n.u[l] = update_u(s.u[l], n.p[l + 1], n.q[l], rho)
     return n
