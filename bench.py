@@ -175,6 +175,8 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--simt", action="store_true", help="run the dense products on CUDA cores")
+    ap.add_argument("--quant-q", action="store_true",
+                    help="pdADMM-G-Q workloads: keep q on the level set as well (variant of Sec. Quantization Extension)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -186,7 +188,8 @@ def main():
     w = synth.get(args.workload)
     config = {"workload": f"{w.name}: N={w.n_nodes} {w.graph.upper()} graph, d={w.feat_dim} x {w.n_blocks} hop blocks "
                           f"(n0={w.n0}), {w.n_layers} layers x {w.hidden}, {w.n_classes} classes, "
-                          f"{'pdADMM-G' if not w.quant_levels else f'pdADMM-G-Q {w.quant_levels} levels'}, rho=nu={w.rho}",
+                          f"{'pdADMM-G' if not w.quant_levels else f'pdADMM-G-Q {w.quant_levels} levels'}"
+                          f"{' (p and q quantised)' if args.quant_q else ''}, rho=nu={w.rho}",
               "replicas": args.gpus,
               "l2": "state (about %.1f GB per replica) is far larger than the 126 MB L2" %
                     (5 * 4e-9 * w.n_nodes * w.hidden * w.n_layers)}
@@ -225,7 +228,7 @@ def main():
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     device = replicas.device_for(local_rank, world)
-    flags = B.FLAG_SIMT_GEMM if args.simt else 0
+    flags = (B.FLAG_SIMT_GEMM if args.simt else 0) | (B.FLAG_QUANT_Q if args.quant_q else 0)
 
     inp = synth.make_inputs(w)
     ctx = B.from_inputs(inp, device=device, flags=flags)

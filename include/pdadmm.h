@@ -63,7 +63,7 @@ typedef enum {
 
 /* Bits of pdadmm_config.flags. */
 #define PDADMM_FLAG_SIMT_GEMM 1u     /* run the dense products on CUDA cores (fp32 FMA) instead of tensor cores */
-#define PDADMM_FLAG_ONE_STREAM 2u    /* issue all layers on one stream (no concurrency across layers)           */
+#define PDADMM_FLAG_QUANT_Q 2u       /* pdADMM-G-Q variant that keeps q_l on the level set of p_{l+1} as well   */
 #define PDADMM_FLAG_NO_GRAPH 4u      /* launch every kernel of an iteration directly instead of replaying a CUDA graph */
 
 /*
@@ -86,6 +86,9 @@ typedef struct {
   float rho;                     /* > 0                                                                 */
   float nu;                      /* > 0                                                                 */
   int32_t quant_levels;          /* 0: pdADMM-G;  2..256: pdADMM-G-Q with that many uniform levels      */
+  int32_t quant_neg_levels;      /* levels below zero: Delta = {(c - quant_neg_levels) s, c = 0..m-1}; 0 = levels
+                                    start at 0.  A value > 0 needs quant_step > 0.  ({-1..20}: m=22, 1, step 1) */
+  float quant_step;              /* > 0: the same level spacing s for every layer; 0: s_l = max(p_l^0)/(m-1)  */
   const float *const *init_W;    /* [L] pointers: W_l^0 as [n_l][n_{l-1}] (required; the caller draws them) */
   int32_t device;                /* CUDA device ordinal                                                 */
   uint32_t flags;                /* PDADMM_FLAG_*                                                       */
@@ -146,11 +149,13 @@ int pdadmm_set_tensor(pdadmm_ctx *ctx, int kind, int layer, const void *host_src
 
 /*
  * pdadmm_quantize -- the projection used by Eq. "update p quantized" on its own: for n host floats x,
- * code = clamp(floor(x/scale + 1/2), 0, levels-1) as uint8 and p = code * scale (one rounded
- * single-precision multiply), computed by the same device function as inside pdadmm_step.
- * codes_out and p_out are host buffers of n elements (either may be null).
+ * code = clamp(floor((x - lo)/scale + 1/2), 0, levels-1) as uint8 and p = lo + code * scale (one rounded
+ * single-precision multiply, one rounded add), computed by the same device function as inside
+ * pdadmm_step.  lo is the smallest level (0 for levels that start at zero, -1 with scale 1 and 22 levels
+ * for the set {-1..20} of the paper's experiments).  codes_out and p_out are host buffers of n elements
+ * (either may be null).
  */
-int pdadmm_quantize(int device, const float *x, size_t n, float scale, int levels,
+int pdadmm_quantize(int device, const float *x, size_t n, float scale, float lo, int levels,
                     uint8_t *codes_out, float *p_out);
 
 /*

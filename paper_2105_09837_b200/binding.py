@@ -19,7 +19,7 @@ _lib = None
 # tensor kinds (pdadmm_tensor)
 T_X, T_P, T_W, T_B, T_Z, T_Q, T_U, T_CODES, T_TAU, T_THETA, T_QSCALE, T_CSR_ROWPTR, T_CSR_COLIDX, T_CSR_VAL, T_TRIALS = range(15)
 FLAG_SIMT_GEMM = 1
-FLAG_ONE_STREAM = 2
+FLAG_QUANT_Q = 2
 FLAG_NO_GRAPH = 4
 
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
@@ -46,6 +46,7 @@ class _Config(C.Structure):
         ("labels", C.POINTER(C.c_int32)), ("train_mask", C.POINTER(C.c_uint8)),
         ("n_layers", C.c_int32), ("layer_widths", C.POINTER(C.c_int32)),
         ("rho", C.c_float), ("nu", C.c_float), ("quant_levels", C.c_int32),
+        ("quant_neg_levels", C.c_int32), ("quant_step", C.c_float),
         ("init_W", C.POINTER(C.POINTER(C.c_float))),
         ("device", C.c_int32), ("flags", C.c_uint32),
     ]
@@ -67,7 +68,8 @@ def lib() -> C.CDLL:
         L.pdadmm_residuals.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.c_int]
         L.pdadmm_get_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
         L.pdadmm_set_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
-        L.pdadmm_quantize.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_float, C.c_int, C.c_void_p, C.c_void_p]
+        L.pdadmm_quantize.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_float, C.c_float, C.c_int, C.c_void_p,
+                                      C.c_void_p]
         L.pdadmm_spmm.argtypes = [C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.pdadmm_matmul.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.POINTER(C.c_double), C.c_uint32]
@@ -97,7 +99,7 @@ class Context:
 
     def __init__(self, n_nodes: int, edge_src, edge_dst, features, n_hops: int, n_classes: int, labels, train_mask,
                  layer_widths: Sequence[int], rho: float, nu: float, quant_levels: int, init_W: List[np.ndarray],
-                 device: int = 0, flags: int = 0):
+                 device: int = 0, flags: int = 0, quant_neg_levels: int = 0, quant_step: float = 0.0):
         self._h = C.c_void_p()
         src = np.ascontiguousarray(edge_src, dtype=np.int32)
         dst = np.ascontiguousarray(edge_dst, dtype=np.int32)
@@ -120,7 +122,8 @@ class Context:
         wp = (C.POINTER(C.c_float) * len(Ws))(*[_ptr(w, C.c_float) for w in Ws])
         cfg = _Config(n_nodes, src.size, _ptr(src, C.c_int32), _ptr(dst, C.c_int32), feat.shape[1],
                       _ptr(feat, C.c_float), n_hops, n_classes, _ptr(lab, C.c_int32), _ptr(msk, C.c_uint8),
-                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, wp, device, flags)
+                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, quant_neg_levels, quant_step, wp,
+                      device, flags)
         self.n_nodes, self.n_layers = int(n_nodes), len(widths)
         self.n0 = (n_hops + 1) * feat.shape[1]
         self.widths = [int(x) for x in widths]
@@ -219,20 +222,21 @@ class Context:
 
 
 def from_inputs(inp, device: int = 0, flags: int = 0, rho: Optional[float] = None, nu: Optional[float] = None,
-                quant_levels: Optional[int] = None) -> Context:
+                quant_levels: Optional[int] = None, quant_neg_levels: int = 0, quant_step: float = 0.0) -> Context:
     """Context for a ``synth.Inputs`` bundle."""
     w = inp.workload
     return Context(w.n_nodes, inp.edge_src, inp.edge_dst, inp.features, w.n_hops, w.n_classes, inp.labels,
                    inp.train_mask, w.widths, w.rho if rho is None else rho, w.nu if nu is None else nu,
-                   w.quant_levels if quant_levels is None else quant_levels, inp.init_W, device, flags)
+                   w.quant_levels if quant_levels is None else quant_levels, inp.init_W, device, flags,
+                   quant_neg_levels, quant_step)
 
 
-def quantize(x, scale: float, levels: int, device: int = 0):
-    """``pdadmm_quantize``: (codes uint8, p float32) for a float32 array."""
+def quantize(x, scale: float, levels: int, device: int = 0, lo: float = 0.0):
+    """``pdadmm_quantize``: (codes uint8, p float32) for a float32 array; ``lo`` is the smallest level."""
     a = np.ascontiguousarray(x, dtype=np.float32)
     codes = np.empty(a.shape, dtype=np.uint8)
     p = np.empty(a.shape, dtype=np.float32)
-    _check(lib().pdadmm_quantize(device, a.ctypes.data_as(C.c_void_p), a.size, scale, levels,
+    _check(lib().pdadmm_quantize(device, a.ctypes.data_as(C.c_void_p), a.size, scale, lo, levels,
                                  codes.ctypes.data_as(C.c_void_p), p.ctypes.data_as(C.c_void_p)))
     return codes, p
 

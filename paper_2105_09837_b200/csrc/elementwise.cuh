@@ -55,13 +55,13 @@ reduce_slots_kernel(const double *__restrict__ slots, int n_slots, int stride, i
   }
 }
 
-// Quantisation to m uniform levels starting at 0 (Eq. "update p quantized", elementwise argmin):
-// code = clamp(floor(x/s + 1/2), 0, m-1), value = float(code) * s with a single rounding.
-__device__ __forceinline__ float quantize_one(float x, float s, float top, unsigned &code) {
-  float c = floorf(__fdiv_rn(x, s) + 0.5f);
+// Quantisation to m uniform levels lo, lo + s, ... (Eq. "update p quantized", elementwise argmin):
+// code = clamp(floor((x - lo)/s + 1/2), 0, m-1), value = lo + float(code) * s, every operation rounded once.
+__device__ __forceinline__ float quantize_one(float x, float s, float lo, float top, unsigned &code) {
+  float c = floorf(__fdiv_rn(__fsub_rn(x, lo), s) + 0.5f);
   c = fminf(fmaxf(c, 0.0f), top);
   code = (unsigned)c;
-  return __fmul_rn(c, s);
+  return __fadd_rn(lo, __fmul_rn(c, s));
 }
 
 // ---- y -= x * (*inv) ----------------------------------------------------------------------------
@@ -93,7 +93,7 @@ add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4) {
 // x = p - g/tau; p_new = nearest level; d = p_new - p; codes; per-block sum of d^2.
 __global__ void __launch_bounds__(EW_THREADS)
 quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, const LayerScalars *__restrict__ sc,
-                   float scale, int levels, float *__restrict__ p_new, float *__restrict__ d,
+                   float scale, float lo, int levels, float *__restrict__ p_new, float *__restrict__ d,
                    uint8_t *__restrict__ codes, size_t n4, double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_tau = sc->inv_tau, top = (float)(levels - 1);
@@ -102,10 +102,10 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
     const float4 pv = ld4(p, i), gv = ld4(g, i);
     unsigned c0, c1, c2, c3;
     float4 nv, dv;
-    nv.x = quantize_one(fmaf(-inv_tau, gv.x, pv.x), scale, top, c0);
-    nv.y = quantize_one(fmaf(-inv_tau, gv.y, pv.y), scale, top, c1);
-    nv.z = quantize_one(fmaf(-inv_tau, gv.z, pv.z), scale, top, c2);
-    nv.w = quantize_one(fmaf(-inv_tau, gv.w, pv.w), scale, top, c3);
+    nv.x = quantize_one(fmaf(-inv_tau, gv.x, pv.x), scale, lo, top, c0);
+    nv.y = quantize_one(fmaf(-inv_tau, gv.y, pv.y), scale, lo, top, c1);
+    nv.z = quantize_one(fmaf(-inv_tau, gv.z, pv.z), scale, lo, top, c2);
+    nv.w = quantize_one(fmaf(-inv_tau, gv.w, pv.w), scale, lo, top, c3);
     dv.x = nv.x - pv.x; dv.y = nv.y - pv.y; dv.z = nv.z - pv.z; dv.w = nv.w - pv.w;
     ss += (double)dv.x * dv.x + (double)dv.y * dv.y + (double)dv.z * dv.z + (double)dv.w * dv.w;
     st4(p_new, i, nv);
@@ -118,12 +118,12 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
 
 // Plain projection of an array (initial forward pass, pdadmm_quantize, pdadmm_set_tensor).
 __global__ void __launch_bounds__(EW_THREADS)
-quantize_kernel(const float *__restrict__ x, size_t n, float scale, int levels, float *__restrict__ p_out,
+quantize_kernel(const float *__restrict__ x, size_t n, float scale, float lo, int levels, float *__restrict__ p_out,
                 uint8_t *__restrict__ codes_out) {
   const float top = (float)(levels - 1);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     unsigned c;
-    const float v = quantize_one(x[i], scale, top, c);
+    const float v = quantize_one(x[i], scale, lo, top, c);
     if (p_out) p_out[i] = v;
     if (codes_out) codes_out[i] = (uint8_t)c;
   }
@@ -295,12 +295,13 @@ finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int 
 
 // ---- z-, q-, u-update of a hidden layer, fused ----------------------------------------------------
 // a = W+ p+ + b+ = (r - shift) + z.  z+ by the ReLU closed form of Eq. "update z" (better of the two
-// half-line minimisers; a tie keeps the non-positive one), q+ by Eq. "update q", residual p_{l+1} - q+,
+// half-line minimisers; a tie keeps the non-positive one), q+ by Eq. "update q" (q_top >= 0: projected onto
+// the level set of p_{l+1}, the variant at the end of Sec. "Quantization Extension"), residual p_{l+1} - q+,
 // u+ by Eq. "update u", and the linear residual of the next iteration r = a - z+.
 __global__ void __launch_bounds__(EW_THREADS)
 zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
            const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
-           float rho, float nu, double *__restrict__ slots) {
+           float rho, float nu, float q_scale, float q_lo, float q_top, double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_rn = 1.0f / (rho + nu);
   double ss = 0.0;
@@ -316,7 +317,8 @@ zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, 
       const float fneg = (zneg - a) * (zneg - a) + qv.f * qv.f + (zneg - zv.f) * (zneg - zv.f); \
       const float fpos = (zpos - a) * (zpos - a) + (qv.f - zpos) * (qv.f - zpos) + (zpos - zv.f) * (zpos - zv.f); \
       const float zz = fpos < fneg ? zpos : zneg;                                   \
-      const float qq = (rho * pv.f + uv.f + nu * fmaxf(zz, 0.0f)) * inv_rn;         \
+      float qq = (rho * pv.f + uv.f + nu * fmaxf(zz, 0.0f)) * inv_rn;               \
+      if (q_top >= 0.0f) { unsigned code; qq = quantize_one(qq, q_scale, q_lo, q_top, code); } \
       const float res = pv.f - qq;                                                  \
       zn.f = zz; qn.f = qq; un.f = fmaf(rho, res, uv.f); rn.f = a - zz;             \
       ss += (double)res * res;                                                      \

@@ -61,7 +61,8 @@ struct Layer {
   float *G_hi = nullptr, *G_lo = nullptr;   // tf32 split planes of grad_W
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in], quantised mode, l >= 2
-  float scale = 1.0f;
+  float scale = 1.0f;       // level spacing s_l of p_l
+  float lo = 0.0f;          // smallest level of p_l: -(levels below zero) * s_l
   LayerScalars *sc = nullptr;
   int n_split = 1, k_chunk = 0;
 };
@@ -88,6 +89,9 @@ struct pdadmm_ctx {
   int device = 0;
   int64_t N = 0;
   int L = 0, d = 0, n_blocks = 0, n0 = 0, ld0 = 0, C = 0, levels = 0;
+  int neg_levels = 0;              // levels below zero
+  float fixed_step = 0.f;          // > 0: the same level spacing for every layer
+  bool quant_q = false;            // q_l is kept on the level set of p_{l+1} as well
   float rho = 0, nu = 0;
   uint32_t flags = 0;
   int64_t nnz = 0;
@@ -383,7 +387,7 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
     const int grid = ew_grid(n4p);
     {
       Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
-      quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, c->levels, s.p_new, s.d,
+      quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
                                                        s.codes_new, n4p, s.slots);
     }
     int np = 0;
@@ -480,8 +484,9 @@ static void zqu_step(pdadmm_ctx *c, int l) {
     const int grid = ew_grid(n4);
     {
       Launch k(c, KC_ZQU, s.st, 36.0 * N * ly.n_out, 0);
-      zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, c->layers[l + 1].p, ly.shift, ly.ld_out / 4, n4,
-                                               c->rho, c->nu, s.slots);
+      const Layer &nx = c->layers[l + 1];
+      zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu,
+                                               nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, s.slots);
     }
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
@@ -530,6 +535,12 @@ static int check_config(const pdadmm_config *cfg) {
   if (!(cfg->rho > 0.f) || !(cfg->nu > 0.f)) return fail(PDADMM_EINVAL, "rho and nu must be positive");
   if (cfg->quant_levels != 0 && (cfg->quant_levels < 2 || cfg->quant_levels > 256))
     return fail(PDADMM_EINVAL, "quant_levels must be 0 or in [2, 256]");
+  if (cfg->quant_neg_levels < 0 || cfg->quant_neg_levels >= std::max(cfg->quant_levels, 1))
+    return fail(PDADMM_EINVAL, "quant_neg_levels must be in [0, quant_levels)");
+  if (cfg->quant_step < 0.f || (cfg->quant_neg_levels > 0 && !(cfg->quant_step > 0.f)))
+    return fail(PDADMM_EINVAL, "quant_step must be >= 0, and > 0 when quant_neg_levels > 0");
+  if ((cfg->flags & PDADMM_FLAG_QUANT_Q) && cfg->quant_levels == 0)
+    return fail(PDADMM_EINVAL, "PDADMM_FLAG_QUANT_Q needs quant_levels >= 2");
   for (int64_t j = 0; j < cfg->n_nodes; ++j)
     if (cfg->labels[j] < 0 || cfg->labels[j] >= cfg->n_classes)
       return fail(PDADMM_EINVAL, "label of node %lld is outside [0, %d)", (long long)j, cfg->n_classes);
@@ -618,6 +629,8 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   const int64_t N = cfg->n_nodes;
   c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
   c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, 4); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
+  c->neg_levels = cfg->quant_neg_levels; c->fixed_step = cfg->quant_step;
+  c->quant_q = (cfg->flags & PDADMM_FLAG_QUANT_Q) != 0;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
   PD_CUDA(cudaSetDevice(cfg->device));
@@ -721,8 +734,11 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
       PD_CUDA(cudaStreamSynchronize(st));
       float mx = 0.f;
       for (float v : hm) mx = std::max(mx, v);
-      nx.scale = mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f;
-      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, c->levels, nx.p, nx.codes);
+      nx.scale = c->fixed_step > 0.f ? c->fixed_step : (mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f);
+      nx.lo = -(float)c->neg_levels * nx.scale;
+      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes);
+      if (c->quant_q)      // start inside the level set: q_l = p_{l+1}
+        PD_CUDA(cudaMemcpyAsync(ly.q, nx.p, n4 * 16, cudaMemcpyDeviceToDevice, st));
     } else {
       PD_CUDA(cudaMemcpyAsync(nx.p, ly.q, n4 * 16, cudaMemcpyDeviceToDevice, st));
     }
@@ -974,6 +990,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
     memcpy(&v, host_src, 4);
     if (!(v > 0.f)) return fail(PDADMM_EINVAL, "QSCALE must be positive");
     c->layers[layer - 1].scale = v;
+    c->layers[layer - 1].lo = -(float)c->neg_levels * v;
     return PDADMM_OK;
   }
   TensorRef t;
@@ -991,14 +1008,14 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
   if (kind == PDADMM_T_P && c->levels && layer >= 2) {
     Layer &y = c->layers[layer - 1];
     const size_t n = (size_t)c->N * y.ld_in;
-    quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, c->levels, nullptr, y.codes);
+    quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, y.lo, c->levels, nullptr, y.codes);
     PD_CUDA(cudaStreamSynchronize(c->scr.st));
   }
   return PDADMM_OK;
 }
 
 // ---- stand-alone entry points for single kernels ------------------------------------------------------------------
-extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale, int levels, uint8_t *codes_out,
+extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale, float lo, int levels, uint8_t *codes_out,
                                float *p_out) {
   if (!x && n) return fail(PDADMM_EINVAL, "x is null");
   if (levels < 2 || levels > 256 || !(scale > 0.f)) return fail(PDADMM_EINVAL, "levels in [2,256], scale > 0");
@@ -1012,7 +1029,7 @@ extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale
     PD_CUDA(cudaMalloc((void **)&dp, n * 4));
     PD_CUDA(cudaMalloc((void **)&dc, n));
     PD_CUDA(cudaMemcpy(dx, x, n * 4, cudaMemcpyHostToDevice));
-    quantize_kernel<<<ew_grid(n), EW_THREADS>>>(dx, n, scale, levels, dp, dc);
+    quantize_kernel<<<ew_grid(n), EW_THREADS>>>(dx, n, scale, lo, levels, dp, dc);
     PD_CUDA(cudaGetLastError());
     PD_CUDA(cudaDeviceSynchronize());
     if (p_out) PD_CUDA(cudaMemcpy(p_out, dp, n * 4, cudaMemcpyDeviceToHost));

@@ -9,11 +9,14 @@ import oracle.pdadmm_oracle as o
 from paper_2105_09837_b200 import binding as B
 
 
-def oracle_problem(inp, rho=None, nu=None, quant_levels=None):
-    """(Params, initial oracle State) for a synth.Inputs bundle."""
+def oracle_problem(inp, rho=None, nu=None, quant_levels=None, quantize_q=False, neg_levels=0, step=0.0):
+    """(Params, initial oracle State) for a synth.Inputs bundle.  neg_levels / step: a fixed level set
+    {(c - neg_levels) step} as the C ABI's quant_neg_levels / quant_step describe it."""
     w = inp.workload
+    lo = float(np.float32(-neg_levels) * np.float32(step))
     prm = o.Params(w.rho if rho is None else rho, w.nu if nu is None else nu,
-                   w.quant_levels if quant_levels is None else quant_levels)
+                   w.quant_levels if quant_levels is None else quant_levels,
+                   quantize_q=quantize_q, level_lo=lo, level_step=step)
     A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
     X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
     s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels, inp.train_mask, prm)
@@ -88,6 +91,14 @@ def z_tie_mask(prev: o.State, nxt: o.State, l: int, tol=1e-5):
 def boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=2e-4):
     """Elements of p_l (0-based l >= 1) whose pre-quantisation value lies within `tol` levels of a rounding boundary."""
     g = o.grad_p_phi(prev.p[l], prev.W[l], prev.b[l], prev.z[l], prm.nu, prev.q[l - 1], prev.u[l - 1], prm.rho)
-    t = (prev.p[l] - g / nxt.tau[l]) / prev.scale[l]
+    t = (prev.p[l] - g / nxt.tau[l] - prm.level_lo) / prev.scale[l]
+    frac = t - np.floor(t)
+    return np.abs(frac - 0.5) <= tol
+
+
+def q_boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=2e-4):
+    """Elements of q_l (0-based l) whose value before the projection lies within `tol` levels of a rounding boundary."""
+    v = o.update_q(nxt.p[l + 1], prev.u[l], nxt.z[l], prm.rho, prm.nu)
+    t = (v - prm.level_lo) / prev.scale[l + 1]
     frac = t - np.floor(t)
     return np.abs(frac - 0.5) <= tol

@@ -29,6 +29,19 @@ def test_quantise_kernel_is_bit_exact(m, scale):
     assert np.all(np.isin(p.astype(np.float64), lev))
 
 
+@pytest.mark.parametrize("m,scale,lo", [(22, 1.0, -1.0), (16, 0.0173, -0.0346), (256, 0.011, 0.25)])
+def test_quantise_kernel_with_offset_is_bit_exact(m, scale, lo):
+    """Level sets that do not start at zero, e.g. {-1, ..., 20}: same codes and values as the oracle's projection."""
+    rng = np.random.default_rng(m)
+    scale, lo = float(np.float32(scale)), float(np.float32(lo))
+    x = rng.uniform(lo - 2 * scale, lo + (m + 1) * scale, size=200003).astype(np.float32)
+    x[:m] = (lo + (np.arange(m) + 0.5) * scale).astype(np.float32)
+    codes, p = B.quantize(x, scale, m, lo=lo)
+    want_codes, want_p = o.quantize(x, scale, m, lo)
+    assert np.array_equal(codes, want_codes)
+    assert np.array_equal(p, want_p.astype(np.float32))
+
+
 def test_quantise_empty_input():
     codes, p = B.quantize(np.zeros(0, np.float32), 1.0, 4)
     assert codes.size == 0 and p.size == 0
