@@ -612,3 +612,30 @@ def objective(s: State, prm: Params) -> np.ndarray:
 
 def lagrangian(s: State, prm: Params) -> float:
     return float(objective(s, prm)[5])
+
+
+# ----------------------------------------------------------------------------
+# The trained model: forward pass, prediction, accuracy
+# ----------------------------------------------------------------------------
+
+def forward(X, W, b) -> np.ndarray:
+    """z_L of the GA-MLP of Problem 1 with the constraints enforced: p_1 = X,
+    z_l = W_l p_l + b_l, p_{l+1} = f_l(z_l) = relu(z_l) (l < L).  Returns z_L (n_L x |V|)."""
+    p = np.asarray(X, dtype=np.float64)
+    for l in range(len(W)):
+        z = W[l] @ p + np.asarray(b[l])[:, None]
+        p = relu(z)
+    return z
+
+
+def predict(X, W, b) -> np.ndarray:
+    """Class of every node: the largest entry of z_L (the class the cross-entropy risk R(z_L; y) rewards);
+    the first one if several are equal."""
+    return np.argmax(forward(X, W, b), axis=0)
+
+
+def accuracy(pred, y, mask) -> float:
+    """Fraction of the nodes selected by `mask` whose predicted class equals the label (the paper's tables
+    report it on the training, validation and test nodes)."""
+    mask = np.asarray(mask, dtype=bool)
+    return float(np.mean(np.asarray(pred)[mask] == np.asarray(y)[mask])) if mask.any() else float("nan")

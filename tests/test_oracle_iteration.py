@@ -161,3 +161,22 @@ def test_single_layer_model_fixed_point_condition():
     lab = s.mask
     assert np.allclose(s.z[0][:, lab], (a + (E - S) / prm.nu)[:, lab], atol=1e-9)
     assert np.array_equal(s.z[0][:, ~lab], a[:, ~lab])
+
+
+def test_forward_pass_golden_and_consistency_with_a_feasible_state():
+    import os
+    want = np.loadtxt(os.path.join(os.path.dirname(__file__), "golden", "forward_two_layers.txt"))
+    X = np.array([[1.0, 2.0], [-1.0, 0.0]])
+    W = [np.array([[1.0, 0], [0, 1], [1, 1]]), np.array([[1.0, -1, 0], [0, 2, 1]])]
+    b = [np.array([0.0, 1.0, -1.0]), np.array([0.5, 0.0])]
+    assert np.array_equal(o.forward(X, W, b), want)
+    assert o.predict(X, W, b).tolist() == [0, 1]
+    assert o.accuracy([0, 1], [0, 0], [True, True]) == 0.5 and o.accuracy([0, 1], [0, 0], [True, False]) == 1.0
+    # the start of Algorithm 1 is a forward pass with b = 0: its z_L is the model's output
+    w, X, W0, y, mask = _problem()
+    s = o.init_state(X, W0, y, mask, o.Params(1e-3, 1e-3, 0))
+    assert np.allclose(o.forward(X, s.W, s.b), s.z[-1], rtol=1e-12, atol=1e-12)
+    # a bias on the last layer only shifts the logits; a large one decides the class
+    b2 = [x.copy() for x in s.b]
+    b2[-1][3] += 1e6
+    assert np.all(o.predict(X, s.W, b2) == 3)
