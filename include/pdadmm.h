@@ -138,6 +138,20 @@ int pdadmm_objective(pdadmm_ctx *ctx, double out[6]);
 int pdadmm_residuals(pdadmm_ctx *ctx, double *per_layer_sq, int n);
 
 /*
+ * pdadmm_predict -- the trained model on every node (paper, Problem 1: p_1 = X, z_l = W_l p_l + b_l,
+ * p_{l+1} = f_l(z_l) = ReLU(z_l); the class of a node is the largest entry of z_L, the quantity the
+ * cross-entropy risk R(z_L; y) scores and the "Performance" section reports as accuracy).  A forward pass
+ * with the current W and b, run with the same dense-product kernels as the iteration; the state of the
+ * iteration (p, z, q, u) is neither read nor changed.
+ *   logits_out : host [N][C] fp32, z_L of the forward pass                     (may be null)
+ *   pred_out   : host [N] int32, argmax over the C classes, first one if equal (may be null)
+ *   counts_out : host [4] int64: correct and total among nodes with train_mask = 1, correct and
+ *                total among the other nodes                                   (may be null)
+ * Returns 0, EINVAL, ECUDA or ETIMEOUT.
+ */
+int pdadmm_predict(pdadmm_ctx *ctx, float *logits_out, int32_t *pred_out, int64_t counts_out[4]);
+
+/*
  * pdadmm_get_tensor / pdadmm_set_tensor -- copy one tensor of the state to / from a host buffer of
  * exactly `bytes` bytes (dense, without the device's row padding).  Together they are the
  * checkpoint / resume interface.  Setting P, W, B or Z invalidates the cached linear residual

@@ -26,7 +26,7 @@ OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5,
 
 EXPORTS = [
     "pdadmm_init", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
-    "pdadmm_set_tensor", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_profile", "pdadmm_profile_classes",
+    "pdadmm_set_tensor", "pdadmm_predict", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_profile", "pdadmm_profile_classes",
     "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_destroy", "pdadmm_last_error",
 ]
 
@@ -68,6 +68,7 @@ def lib() -> C.CDLL:
         L.pdadmm_residuals.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.c_int]
         L.pdadmm_get_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
         L.pdadmm_set_tensor.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
+        L.pdadmm_predict.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.pdadmm_quantize.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_float, C.c_float, C.c_int, C.c_void_p,
                                       C.c_void_p]
         L.pdadmm_spmm.argtypes = [C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
@@ -149,6 +150,15 @@ class Context:
         out = (C.c_double * max(n, 1))()
         _check(lib().pdadmm_residuals(self._h, out if n else None, n))
         return np.array(out[:n])
+
+    def predict(self):
+        """``pdadmm_predict``: (logits [N][C] float32, classes [N] int32, counts [4] int64)."""
+        logits = np.empty((self.n_nodes, self.widths[-1]), dtype=np.float32)
+        pred = np.empty(self.n_nodes, dtype=np.int32)
+        counts = np.zeros(4, dtype=np.int64)
+        _check(lib().pdadmm_predict(self._h, logits.ctypes.data_as(C.c_void_p), pred.ctypes.data_as(C.c_void_p),
+                                    counts.ctypes.data_as(C.c_void_p)))
+        return logits, pred, counts
 
     def _shape(self, kind: int, layer: int):
         n_in = self.n0 if layer <= 1 else self.widths[layer - 2]

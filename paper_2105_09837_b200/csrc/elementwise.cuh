@@ -466,6 +466,32 @@ risk_kernel(const float *__restrict__ z, const int *__restrict__ labels, const u
   if (threadIdx.x == 0) slots[blockIdx.x] = t;
 }
 
+// Predicted class of every node: the largest of its C logits, the first one among equals.  counts[0..3] (zeroed
+// by the caller) receive: correct and total over the nodes with mask = 1, correct and total over the others.
+__global__ void __launch_bounds__(EW_THREADS)
+argmax_kernel(const float *__restrict__ z, const int *__restrict__ labels, const uint8_t *__restrict__ mask, int n_rows,
+              int C, int ld, int *__restrict__ pred, unsigned long long *__restrict__ counts) {
+  unsigned long long c_in = 0, n_in = 0, c_out = 0, n_out = 0;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n_rows; j += gridDim.x * blockDim.x) {
+    const float *zj = z + (size_t)j * ld;
+    int best = 0;
+    float vbest = zj[0];
+    for (int c = 1; c < C; ++c) {
+      const float v = zj[c];
+      if (v > vbest) { vbest = v; best = c; }
+    }
+    pred[j] = best;
+    const bool hit = best == labels[j];
+    if (mask[j]) { ++n_in; c_in += hit; } else { ++n_out; c_out += hit; }
+  }
+  // integer sums: the order of the atomics does not matter
+  c_in = warp_sum_u64(c_in); n_in = warp_sum_u64(n_in); c_out = warp_sum_u64(c_out); n_out = warp_sum_u64(n_out);
+  if ((threadIdx.x & 31) == 0) {
+    if (n_in) { atomicAdd(counts + 0, c_in); atomicAdd(counts + 1, n_in); }
+    if (n_out) { atomicAdd(counts + 2, c_out); atomicAdd(counts + 3, n_out); }
+  }
+}
+
 // W+ = W - grad_W * inv_theta  (Eq. "update W")
 __global__ void __launch_bounds__(EW_THREADS)
 wstep_kernel(float *__restrict__ W, const float *__restrict__ G, const LayerScalars *__restrict__ sc, size_t n4,

@@ -910,6 +910,49 @@ extern "C" int pdadmm_objective(pdadmm_ctx *c, double out[6]) {
   return PDADMM_OK;
 }
 
+extern "C" int pdadmm_predict(pdadmm_ctx *c, float *logits_out, int32_t *pred_out, int64_t counts_out[4]) {
+  if (!c) return fail(PDADMM_EINVAL, "context is null");
+  PD_CUDA(cudaSetDevice(c->device));
+  cudaStream_t st = c->scr.st;
+  if (!c->w_planes_valid) {
+    for (auto &ly : c->layers) split_planes(c, st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
+    c->w_planes_valid = true;
+  }
+  // forward pass with the constraints enforced: activations alternate between the two scratch matrices
+  const int N = (int)c->N;
+  const float *in = c->layers[0].p;
+  float *bufs[2] = {c->scr.s1, c->scr.s2};
+  float *out = nullptr;
+  for (int l = 0; l < c->L; ++l) {
+    Layer &ly = c->layers[l];
+    out = bufs[l & 1];
+    EpiBiasAct epi{out, ly.ld_out, ly.b, l + 1 < c->L ? 1 : 0};
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, N, ly.n_out, ly.n_in, in, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
+                             epi, nullptr, nullptr, 0));
+    in = out;
+  }
+  const Layer &last = c->layers[c->L - 1];
+  int *d_pred = reinterpret_cast<int *>(bufs[c->L & 1]);              // the scratch matrix the logits are not in
+  unsigned long long *d_counts = reinterpret_cast<unsigned long long *>(c->scr.slots);
+  PD_CUDA(cudaMemsetAsync(d_counts, 0, 4 * sizeof(unsigned long long), st));
+  argmax_kernel<<<(int)std::min<int64_t>(1184, ceil_div(N, EW_THREADS)), EW_THREADS, 0, st>>>(
+      out, c->labels, c->mask, N, last.n_out, last.ld_out, d_pred, d_counts);
+  PD_CUDA(cudaGetLastError());
+  if (logits_out)
+    PD_CUDA(cudaMemcpy2DAsync(logits_out, (size_t)last.n_out * 4, out, (size_t)last.ld_out * 4, (size_t)last.n_out * 4,
+                              (size_t)N, cudaMemcpyDeviceToHost, st));
+  if (pred_out) PD_CUDA(cudaMemcpyAsync(pred_out, d_pred, (size_t)N * 4, cudaMemcpyDeviceToHost, st));
+  unsigned long long h_counts[4];
+  PD_CUDA(cudaMemcpyAsync(h_counts, d_counts, sizeof(h_counts), cudaMemcpyDeviceToHost, st));
+  PD_CUDA(cudaStreamSynchronize(st));
+  if (counts_out)
+    for (int i = 0; i < 4; ++i) counts_out[i] = (int64_t)h_counts[i];
+  int h_err = 0;
+  PD_CUDA(cudaMemcpy(&h_err, c->d_flag + 1, 4, cudaMemcpyDeviceToHost));
+  if (h_err) return fail(PDADMM_ETIMEOUT, "a bounded wait inside a tensor-core product expired");
+  return PDADMM_OK;
+}
+
 extern "C" int pdadmm_residuals(pdadmm_ctx *c, double *per_layer_sq, int n) {
   if (!c) return fail(PDADMM_EINVAL, "context is null");
   if (n != c->L - 1 || (n > 0 && !per_layer_sq)) return fail(PDADMM_EINVAL, "n must be L-1 = %d", c->L - 1);

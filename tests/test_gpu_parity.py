@@ -289,3 +289,45 @@ def test_step_is_deterministic_and_split_calls_agree():
             assert np.array_equal(x, y), k                      # fixed-order reductions: bit-identical runs
     a.destroy()
     b.destroy()
+
+
+# ----------------------------------------------------------------------------- the trained model: forward pass, classes
+
+@pytest.mark.parametrize("case,levels,flags", [("er-small", 0, 0), ("ba-ragged", 0, 0), ("c4-like", 256, 0),
+                                               ("ba-ragged", 0, B.FLAG_SIMT_GEMM)])
+def test_prediction_matches_the_oracle_forward_pass(case, levels, flags):
+    inp = _inputs(case, quant_levels=levels)
+    prm, s, _ = U.oracle_problem(inp)
+    ctx = B.from_inputs(inp, flags=flags)
+    mask = inp.train_mask.astype(bool)
+    for k in range(3):
+        if k:                                   # weights after some iterations, carried over from the oracle
+            for _ in range(2):
+                s = o.iterate(s, prm)
+            U.load_state(ctx, U.round_state(s), levels > 0)
+        Wf = [U.f32(w) for w in s.W]
+        bf = [U.f32(b) for b in s.b]
+        want = o.forward(s.p[0], Wf, bf)
+        logits, pred, counts = ctx.predict()
+        assert U.rel_err(logits.T.astype(np.float64), want) < TOL
+        # classes: equal wherever the two largest logits are further apart than the tolerance allows them to move
+        srt = np.sort(want, axis=0)
+        clear = (srt[-1] - srt[-2]) > 4 * TOL * np.abs(want).max()
+        want_pred = np.argmax(want, axis=0)
+        assert clear.mean() > 0.9
+        assert np.array_equal(pred[clear], want_pred[clear])
+        assert np.array_equal(pred, np.argmax(logits, axis=1))          # the device's own logits decide, first one wins
+        hit = pred == inp.labels
+        assert counts.tolist() == [int(hit[mask].sum()), int(mask.sum()), int(hit[~mask].sum()), int((~mask).sum())]
+        assert abs(counts[0] / counts[1] - o.accuracy(want_pred, inp.labels, mask)) <= (~clear).mean() + 1e-12
+    # the state of the iteration is untouched: one more step gives what it gives without the call in between
+    ref = B.from_inputs(inp, flags=flags)
+    U.load_state(ref, U.round_state(s), levels > 0)
+    ref.step(1)
+    ctx.step(1)
+    a, b = U.read_state(ctx), U.read_state(ref)
+    for name in ("p", "W", "b", "z", "q", "u"):
+        for x, y in zip(a[name], b[name]):
+            assert np.array_equal(x, y)
+    ctx.destroy()
+    ref.destroy()
