@@ -51,7 +51,8 @@ typedef enum {
   PDADMM_T_Z = 4,        /* float  [N][n_l]       l = 1..L                                             */
   PDADMM_T_Q = 5,        /* float  [N][n_l]       l = 1..L-1                                           */
   PDADMM_T_U = 6,        /* float  [N][n_l]       l = 1..L-1                                           */
-  PDADMM_T_CODES = 7,    /* uint8  [N][n_{l-1}]   l = 2..L, pdADMM-G-Q only: p_l = code * QSCALE_l     */
+  PDADMM_T_CODES = 7,    /* uint8 (uint16 above 256 levels) [N][n_{l-1}]  l = 2..L, pdADMM-G-Q only:
+                            p_l = (code - quant_neg_levels) * QSCALE_l (get only)                      */
   PDADMM_T_TAU = 8,      /* double [1]            l = 2..L: tau_l of the last iteration (get only)     */
   PDADMM_T_THETA = 9,    /* double [1]            l = 1..L: theta_l of the last iteration (get only)   */
   PDADMM_T_QSCALE = 10,  /* float  [1]            l = 2..L: level spacing s_l of p_l                   */
@@ -85,7 +86,8 @@ typedef struct {
   const int32_t *layer_widths;   /* [L]: n_1..n_L, n_L == n_classes                                     */
   float rho;                     /* > 0                                                                 */
   float nu;                      /* > 0                                                                 */
-  int32_t quant_levels;          /* 0: pdADMM-G;  2..256: pdADMM-G-Q with that many uniform levels      */
+  int32_t quant_levels;          /* 0: pdADMM-G;  2..65536: pdADMM-G-Q with that many uniform levels (codes
+                                    of one byte up to 256 levels, two bytes above)                      */
   int32_t quant_neg_levels;      /* levels below zero: Delta = {(c - quant_neg_levels) s, c = 0..m-1}; 0 = levels
                                     start at 0.  A value > 0 needs quant_step > 0.  ({-1..20}: m=22, 1, step 1) */
   float quant_step;              /* > 0: the same level spacing s for every layer; 0: s_l = max(p_l^0)/(m-1)  */
@@ -166,11 +168,12 @@ int pdadmm_set_tensor(pdadmm_ctx *ctx, int kind, int layer, const void *host_src
  * code = clamp(floor((x - lo)/scale + 1/2), 0, levels-1) as uint8 and p = lo + code * scale (one rounded
  * single-precision multiply, one rounded add), computed by the same device function as inside
  * pdadmm_step.  lo is the smallest level (0 for levels that start at zero, -1 with scale 1 and 22 levels
- * for the set {-1..20} of the paper's experiments).  codes_out and p_out are host buffers of n elements
- * (either may be null).
+ * for the set {-1..20} of the paper's experiments).  levels in [2, 65536]; codes are uint8 for up to 256
+ * levels and uint16 above (the 8- and 16-bit cases of the paper's "Communication Overheads" experiment).
+ * codes_out and p_out are host buffers of n elements (either may be null).
  */
 int pdadmm_quantize(int device, const float *x, size_t n, float scale, float lo, int levels,
-                    uint8_t *codes_out, float *p_out);
+                    void *codes_out, float *p_out);
 
 /*
  * pdadmm_spmm -- Y = A~ X for a caller-supplied CSR matrix (host arrays, columns in [0, n_rows))

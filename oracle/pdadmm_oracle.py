@@ -223,13 +223,15 @@ def quantize(x, scale: float, m: int, lo: float = 0.0):
     is taken per element.  For uniform levels it is a rounding:
     code = clamp(floor((x - lo)/s + 1/2), 0, m-1) (ties at half-levels go up).
     The rounding decision is taken in single precision, the precision of the
-    kernel that takes the same decision.  Returns (codes uint8, p in Delta).
+    kernel that takes the same decision.  Returns (codes, p in Delta); codes are
+    uint8 for up to 256 levels and uint16 above (the 8- and 16-bit cases of Sec.
+    "Communication Overheads").
     """
     x32 = np.asarray(x, dtype=np.float32)
     t = (x32 - np.float32(lo)) / np.float32(scale)
     c = np.floor(t + np.float32(0.5))
     c = np.clip(c, np.float32(0.0), np.float32(m - 1))
-    codes = c.astype(np.uint8)
+    codes = c.astype(np.uint8 if m <= 256 else np.uint16)
     vals = (np.float32(lo) + c * np.float32(scale)).astype(np.float64)
     return codes, vals
 

@@ -175,7 +175,7 @@ class Context:
         if kind in (T_Z, T_Q, T_U):
             return (N, n_out), np.float32
         if kind == T_CODES:
-            return (N, n_in), np.uint8
+            return (N, n_in), (np.uint16 if self.quant_levels > 256 else np.uint8)
         if kind in (T_TAU, T_THETA):
             return (1,), np.float64
         if kind == T_QSCALE:
@@ -244,7 +244,7 @@ def from_inputs(inp, device: int = 0, flags: int = 0, rho: Optional[float] = Non
 def quantize(x, scale: float, levels: int, device: int = 0, lo: float = 0.0):
     """``pdadmm_quantize``: (codes uint8, p float32) for a float32 array; ``lo`` is the smallest level."""
     a = np.ascontiguousarray(x, dtype=np.float32)
-    codes = np.empty(a.shape, dtype=np.uint8)
+    codes = np.empty(a.shape, dtype=np.uint16 if levels > 256 else np.uint8)
     p = np.empty(a.shape, dtype=np.float32)
     _check(lib().pdadmm_quantize(device, a.ctypes.data_as(C.c_void_p), a.size, scale, lo, levels,
                                  codes.ctypes.data_as(C.c_void_p), p.ctypes.data_as(C.c_void_p)))

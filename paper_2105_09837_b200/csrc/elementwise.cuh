@@ -94,7 +94,7 @@ add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4) {
 __global__ void __launch_bounds__(EW_THREADS)
 quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, const LayerScalars *__restrict__ sc,
                    float scale, float lo, int levels, float *__restrict__ p_new, float *__restrict__ d,
-                   uint8_t *__restrict__ codes, size_t n4, double *__restrict__ slots) {
+                   void *__restrict__ codes, int wide_codes, size_t n4, double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_tau = sc->inv_tau, top = (float)(levels - 1);
   double ss = 0.0;
@@ -110,7 +110,10 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
     ss += (double)dv.x * dv.x + (double)dv.y * dv.y + (double)dv.z * dv.z + (double)dv.w * dv.w;
     st4(p_new, i, nv);
     st4(d, i, dv);
-    reinterpret_cast<uchar4 *>(codes)[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
+    if (wide_codes)      // more than 256 levels: 16-bit codes
+      reinterpret_cast<ushort4 *>(codes)[i] = make_ushort4((unsigned short)c0, (unsigned short)c1, (unsigned short)c2, (unsigned short)c3);
+    else
+      reinterpret_cast<uchar4 *>(codes)[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
   }
   const double tot = block_sum<EW_THREADS>(ss, red);
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
@@ -119,13 +122,16 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
 // Plain projection of an array (initial forward pass, pdadmm_quantize, pdadmm_set_tensor).
 __global__ void __launch_bounds__(EW_THREADS)
 quantize_kernel(const float *__restrict__ x, size_t n, float scale, float lo, int levels, float *__restrict__ p_out,
-                uint8_t *__restrict__ codes_out) {
+                void *__restrict__ codes_out, int wide_codes) {
   const float top = (float)(levels - 1);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     unsigned c;
     const float v = quantize_one(x[i], scale, lo, top, c);
     if (p_out) p_out[i] = v;
-    if (codes_out) codes_out[i] = (uint8_t)c;
+    if (codes_out) {
+      if (wide_codes) reinterpret_cast<uint16_t *>(codes_out)[i] = (uint16_t)c;
+      else reinterpret_cast<uint8_t *>(codes_out)[i] = (uint8_t)c;
+    }
   }
 }
 

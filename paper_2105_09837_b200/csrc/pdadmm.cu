@@ -60,7 +60,7 @@ struct Layer {
   float *W_hi = nullptr, *W_lo = nullptr;   // tf32 split planes of W (tensor-core path)
   float *G_hi = nullptr, *G_lo = nullptr;   // tf32 split planes of grad_W
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
-  uint8_t *codes = nullptr; // [N][ld_in], quantised mode, l >= 2
+  uint8_t *codes = nullptr; // [N][ld_in] codes of 1 byte (up to 256 levels) or 2 bytes, quantised mode, l >= 2
   float scale = 1.0f;       // level spacing s_l of p_l
   float lo = 0.0f;          // smallest level of p_l: -(levels below zero) * s_l
   LayerScalars *sc = nullptr;
@@ -89,6 +89,7 @@ struct pdadmm_ctx {
   int device = 0;
   int64_t N = 0;
   int L = 0, d = 0, n_blocks = 0, n0 = 0, ld0 = 0, C = 0, levels = 0;
+  int code_bytes = 1;              // 1 for up to 256 levels, else 2
   int neg_levels = 0;              // levels below zero
   float fixed_step = 0.f;          // > 0: the same level spacing for every layer
   bool quant_q = false;            // q_l is kept on the level set of p_{l+1} as well
@@ -388,7 +389,7 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
     {
       Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
       quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
-                                                       s.codes_new, n4p, s.slots);
+                                                       s.codes_new, c->code_bytes == 2, n4p, s.slots);
     }
     int np = 0;
     double *slots_b = s.slots + s.n_slots / 2;
@@ -533,8 +534,8 @@ static int check_config(const pdadmm_config *cfg) {
   }
   if (!cfg->labels || !cfg->train_mask) return fail(PDADMM_EINVAL, "labels or mask missing");
   if (!(cfg->rho > 0.f) || !(cfg->nu > 0.f)) return fail(PDADMM_EINVAL, "rho and nu must be positive");
-  if (cfg->quant_levels != 0 && (cfg->quant_levels < 2 || cfg->quant_levels > 256))
-    return fail(PDADMM_EINVAL, "quant_levels must be 0 or in [2, 256]");
+  if (cfg->quant_levels != 0 && (cfg->quant_levels < 2 || cfg->quant_levels > 65536))
+    return fail(PDADMM_EINVAL, "quant_levels must be 0 or in [2, 65536]");
   if (cfg->quant_neg_levels < 0 || cfg->quant_neg_levels >= std::max(cfg->quant_levels, 1))
     return fail(PDADMM_EINVAL, "quant_neg_levels must be in [0, quant_levels)");
   if (cfg->quant_step < 0.f || (cfg->quant_neg_levels > 0 && !(cfg->quant_step > 0.f)))
@@ -630,6 +631,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
   c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, 4); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
   c->neg_levels = cfg->quant_neg_levels; c->fixed_step = cfg->quant_step;
+  c->code_bytes = cfg->quant_levels > 256 ? 2 : 1;
   c->quant_q = (cfg->flags & PDADMM_FLAG_QUANT_Q) != 0;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
@@ -679,7 +681,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &ly.z, e_out));
     PD_TRY(dev_alloc(c, &ly.r, e_out));
     if (l + 1 < c->L) { PD_TRY(dev_alloc(c, &ly.q, e_out)); PD_TRY(dev_alloc(c, &ly.u, e_out)); }
-    if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in));
+    if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in * c->code_bytes));
     PD_TRY(dev_alloc(c, &ly.sc, 1));
     PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
     // node slices of the W-gradient product: enough blocks to fill the device twice, slices >= 256 nodes
@@ -697,7 +699,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   if (c->levels) {
     PD_TRY(dev_alloc(c, &s.p_new, (size_t)N * max_in));
     PD_TRY(dev_alloc(c, &s.d, (size_t)N * max_in));
-    PD_TRY(dev_alloc(c, &s.codes_new, (size_t)N * max_in));
+    PD_TRY(dev_alloc(c, &s.codes_new, (size_t)N * max_in * c->code_bytes));
   }
   PD_TRY(dev_alloc(c, &s.part, max_part));
   s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
@@ -736,7 +738,8 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
       for (float v : hm) mx = std::max(mx, v);
       nx.scale = c->fixed_step > 0.f ? c->fixed_step : (mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f);
       nx.lo = -(float)c->neg_levels * nx.scale;
-      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes);
+      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes,
+                                                              c->code_bytes == 2);
       if (c->quant_q)      // start inside the level set: q_l = p_{l+1}
         PD_CUDA(cudaMemcpyAsync(ly.q, nx.p, n4 * 16, cudaMemcpyDeviceToDevice, st));
     } else {
@@ -993,7 +996,7 @@ static int locate(pdadmm_ctx *c, int kind, int layer, TensorRef *t) {
     case PDADMM_T_CODES: {
       if (!c->levels) return fail(PDADMM_EINVAL, "codes exist only in quantised mode");
       PD_TRY(need(2, L)); Layer &y = c->layers[layer - 1];
-      *t = {y.codes, N, (size_t)y.n_in, (size_t)y.ld_in, 1, false}; return PDADMM_OK;
+      *t = {y.codes, N, (size_t)y.n_in, (size_t)y.ld_in, (size_t)c->code_bytes, false}; return PDADMM_OK;
     }
     case PDADMM_T_TAU: { PD_TRY(need(2, L)); *t = {&c->layers[layer - 1].sc->tau, 1, 1, 1, 8, false}; return PDADMM_OK; }
     case PDADMM_T_THETA: { PD_TRY(need(1, L)); *t = {&c->layers[layer - 1].sc->theta, 1, 1, 1, 8, false}; return PDADMM_OK; }
@@ -1051,17 +1054,19 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
   if (kind == PDADMM_T_P && c->levels && layer >= 2) {
     Layer &y = c->layers[layer - 1];
     const size_t n = (size_t)c->N * y.ld_in;
-    quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, y.lo, c->levels, nullptr, y.codes);
+    quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, y.lo, c->levels, nullptr, y.codes,
+                                                              c->code_bytes == 2);
     PD_CUDA(cudaStreamSynchronize(c->scr.st));
   }
   return PDADMM_OK;
 }
 
 // ---- stand-alone entry points for single kernels ------------------------------------------------------------------
-extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale, float lo, int levels, uint8_t *codes_out,
+extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale, float lo, int levels, void *codes_out,
                                float *p_out) {
   if (!x && n) return fail(PDADMM_EINVAL, "x is null");
-  if (levels < 2 || levels > 256 || !(scale > 0.f)) return fail(PDADMM_EINVAL, "levels in [2,256], scale > 0");
+  if (levels < 2 || levels > 65536 || !(scale > 0.f)) return fail(PDADMM_EINVAL, "levels in [2,65536], scale > 0");
+  const size_t code_bytes = levels > 256 ? 2 : 1;
   if (n == 0) return PDADMM_OK;
   PD_CUDA(cudaSetDevice(device));
   float *dx = nullptr, *dp = nullptr;
@@ -1070,13 +1075,13 @@ extern "C" int pdadmm_quantize(int device, const float *x, size_t n, float scale
   auto body = [&]() -> int {
     PD_CUDA(cudaMalloc((void **)&dx, n * 4));
     PD_CUDA(cudaMalloc((void **)&dp, n * 4));
-    PD_CUDA(cudaMalloc((void **)&dc, n));
+    PD_CUDA(cudaMalloc((void **)&dc, n * code_bytes));
     PD_CUDA(cudaMemcpy(dx, x, n * 4, cudaMemcpyHostToDevice));
-    quantize_kernel<<<ew_grid(n), EW_THREADS>>>(dx, n, scale, lo, levels, dp, dc);
+    quantize_kernel<<<ew_grid(n), EW_THREADS>>>(dx, n, scale, lo, levels, dp, dc, code_bytes == 2);
     PD_CUDA(cudaGetLastError());
     PD_CUDA(cudaDeviceSynchronize());
     if (p_out) PD_CUDA(cudaMemcpy(p_out, dp, n * 4, cudaMemcpyDeviceToHost));
-    if (codes_out) PD_CUDA(cudaMemcpy(codes_out, dc, n, cudaMemcpyDeviceToHost));
+    if (codes_out) PD_CUDA(cudaMemcpy(codes_out, dc, n * code_bytes, cudaMemcpyDeviceToHost));
     return PDADMM_OK;
   };
   rc = body();

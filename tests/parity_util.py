@@ -88,17 +88,28 @@ def z_tie_mask(prev: o.State, nxt: o.State, l: int, tol=1e-5):
     return (np.abs(fp - fn) <= tol * (np.abs(fp) + np.abs(fn) + 1e-30)) & (zp != zn)
 
 
-def boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=2e-4):
+def band(prm: o.Params) -> float:
+    """Half-width, in levels, of the band around a rounding boundary inside which single and double precision may
+    round to different neighbours: 2e-4 levels, or, when there are many levels, four single-precision roundings
+    (2^-24 each) of a value as large as the top level, m * 2.4e-7 levels (4096 levels: 1e-3)."""
+    return max(2e-4, 2.4e-7 * prm.quant_levels)
+
+
+def boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=None):
     """Elements of p_l (0-based l >= 1) whose pre-quantisation value lies within `tol` levels of a rounding boundary."""
+    tol = band(prm) if tol is None else tol
     g = o.grad_p_phi(prev.p[l], prev.W[l], prev.b[l], prev.z[l], prm.nu, prev.q[l - 1], prev.u[l - 1], prm.rho)
     t = (prev.p[l] - g / nxt.tau[l] - prm.level_lo) / prev.scale[l]
     frac = t - np.floor(t)
     return np.abs(frac - 0.5) <= tol
 
 
-def q_boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=2e-4):
+def q_boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=None):
     """Elements of q_l (0-based l) whose value before the projection lies within `tol` levels of a rounding boundary."""
     v = o.update_q(nxt.p[l + 1], prev.u[l], nxt.z[l], prm.rho, prm.nu)
+    # the value to project carries the single-precision error of z+ (a chain of products and sums, about
+    # 1e-6 of the largest value), which with many levels exceeds the band of the storage roundings alone
+    tol = max(band(prm), 1e-6 * float(np.abs(v).max()) / prev.scale[l + 1]) if tol is None else tol
     t = (v - prm.level_lo) / prev.scale[l + 1]
     frac = t - np.floor(t)
     return np.abs(frac - 0.5) <= tol

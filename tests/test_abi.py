@@ -56,7 +56,7 @@ def test_argument_checks_need_no_device():
     assert e.value.code == B.EINVAL
     with pytest.raises(B.PdadmmError) as e:
         B.Context(w.n_nodes, inp.edge_src, inp.edge_dst, inp.features, w.n_hops, w.n_classes, inp.labels,
-                  inp.train_mask, w.widths, 1e-3, 1e-3, 300, inp.init_W)
+                  inp.train_mask, w.widths, 1e-3, 1e-3, 70000, inp.init_W)
     assert e.value.code == B.EINVAL
     with pytest.raises(B.PdadmmError):
         B.quantize(np.zeros(4, np.float32), 0.0, 16)

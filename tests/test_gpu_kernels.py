@@ -29,7 +29,8 @@ def test_quantise_kernel_is_bit_exact(m, scale):
     assert np.all(np.isin(p.astype(np.float64), lev))
 
 
-@pytest.mark.parametrize("m,scale,lo", [(22, 1.0, -1.0), (16, 0.0173, -0.0346), (256, 0.011, 0.25)])
+@pytest.mark.parametrize("m,scale,lo", [(22, 1.0, -1.0), (16, 0.0173, -0.0346), (256, 0.011, 0.25),
+                                        (4096, 0.0007, -0.07), (65536, 0.00004, 0.0)])
 def test_quantise_kernel_with_offset_is_bit_exact(m, scale, lo):
     """Level sets that do not start at zero, e.g. {-1, ..., 20}: same codes and values as the oracle's projection."""
     rng = np.random.default_rng(m)
@@ -37,6 +38,7 @@ def test_quantise_kernel_with_offset_is_bit_exact(m, scale, lo):
     x = rng.uniform(lo - 2 * scale, lo + (m + 1) * scale, size=200003).astype(np.float32)
     x[:m] = (lo + (np.arange(m) + 0.5) * scale).astype(np.float32)
     codes, p = B.quantize(x, scale, m, lo=lo)
+    assert codes.dtype == (np.uint8 if m <= 256 else np.uint16)
     want_codes, want_p = o.quantize(x, scale, m, lo)
     assert np.array_equal(codes, want_codes)
     assert np.array_equal(p, want_p.astype(np.float32))

@@ -99,7 +99,7 @@ def _compare_iteration(ctx, prev, prm, label):
                 pytest.skip(f"{label}: tau search took {trials} trials on the device, {nxt.trials[l]} in the oracle")
             mask = U.boundary_mask(prev, nxt, prm, l)
             codes = ctx.get_tensor(B.T_CODES, l + 1).T
-            want_codes = np.rint((nxt.p[l] - prm.level_lo) / prev.scale[l]).astype(np.uint8)
+            want_codes = np.rint((nxt.p[l] - prm.level_lo) / prev.scale[l]).astype(codes.dtype)
             diff = codes != want_codes
             assert not np.any(diff & ~mask), f"{label}: codes differ away from a rounding boundary (layer {l + 1})"
             assert np.all(np.abs(codes.astype(int) - want_codes.astype(int)) <= 1)
@@ -138,8 +138,15 @@ def _compare_iteration(ctx, prev, prm, label):
                 assert np.all(np.isin(got["q"][l], lev)), f"{label}: q_{l + 1} left the level set"
                 qb = U.q_boundary_mask(prev, nxt, prm, l) | tie
                 dq = np.abs(got["q"][l] - nxt.q[l])
-                assert not np.any((dq > 0) & ~qb), f"{label}: q_{l + 1} differs away from a rounding boundary"
-                assert np.all(dq <= prev.scale[l + 1] * (1 + 1e-4))      # levels are rounded fp32 numbers
+                assert np.all(dq[~tie] <= prev.scale[l + 1] * (1 + 1e-4))      # levels are rounded fp32 numbers
+                if prm.quant_levels > 256:
+                    # 16-bit codes: a level is finer than the single-precision error of z+ that the value to project
+                    # inherits, so neighbouring levels are both right in many places; q is then held to the
+                    # floating-point bar like any other variable (below, outside the boundary band), besides being
+                    # on the level set and within one level of the oracle everywhere
+                    pass
+                else:
+                    assert not np.any((dq > 0) & ~qb), f"{label}: q_{l + 1} differs away from a rounding boundary"
                 # With rho = nu, u = 0 and an inactive ReLU the value to project is p_{l+1}/2: an exact tie between two
                 # levels whenever the code of p_{l+1} is odd, so boundary elements are common here.  Both neighbours
                 # minimise the q-subproblem there; they are left out of the comparison of q and of u (nothing else
@@ -150,9 +157,16 @@ def _compare_iteration(ctx, prev, prm, label):
             # u_l = u_l + rho (p_{l+1} - q_l) is a difference of two terms of size rho ||p||: in single precision
             # it cannot be more accurate than ~1e-7 rho ||p||, so its error is measured against
             # max(||u||, 1e-3 rho ||p_{l+1}||) (a start where p = q to rounding has u = 0 to rounding)
-            floor_u = 1e-3 * prm.rho * np.linalg.norm(nxt.p[l + 1][~tie])
-            worst[f"u{l + 1}"] = float(np.linalg.norm((got["u"][l] - nxt.u[l])[~tie])
-                                       / max(np.linalg.norm(nxt.u[l][~tie]), floor_u))
+            um = tie
+            if quant:
+                um = um | (got["p"][l + 1] != nxt.p[l + 1])      # u_l follows p_{l+1}: a code that took the other
+                #                                                   neighbour at a boundary moves u there by rho s
+            if quant and prm.quantize_q and prm.quant_levels > 256:
+                um = um | (got["q"][l] != nxt.q[l])       # and q_l: where the other neighbour was taken, so does u
+                assert um.mean() < 0.5
+            floor_u = 1e-3 * prm.rho * np.linalg.norm(nxt.p[l + 1][~um])
+            worst[f"u{l + 1}"] = float(np.linalg.norm((got["u"][l] - nxt.u[l])[~um])
+                                       / max(np.linalg.norm(nxt.u[l][~um]), floor_u))
         else:
             worst[f"z{l + 1}"] = U.rel_err(got["z"][l], nxt.z[l])
     bad = {k: v for k, v in worst.items() if not v <= TOL}
@@ -188,6 +202,7 @@ def test_teacher_forced_iterations(case, levels, flags):
     ("er-small", 22, 1, 1.0, False),         # the level set {-1, 0, ..., 20} of the paper's experiments
     ("ba-ragged", 22, 1, 1.0, True),
     ("c4-like", 64, 3, 0.125, True),
+    ("ba-ragged", 4096, 0, 0.0, True),       # 16-bit codes
 ])
 def test_teacher_forced_level_set_variants(case, levels, neg, step, quant_q):
     inp = _inputs(case, quant_levels=levels)

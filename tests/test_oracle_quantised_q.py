@@ -28,7 +28,7 @@ def test_paper_default_level_set():
     assert codes.tolist() == [0, 0, 1, 0, 1, 5, 21, 21]
 
 
-@pytest.mark.parametrize("m,scale,lo", [(22, 1.0, -1.0), (16, 0.0173, -0.0371), (256, 0.011, 0.25)])
+@pytest.mark.parametrize("m,scale,lo", [(22, 1.0, -1.0), (16, 0.0173, -0.0371), (256, 0.011, 0.25), (1000, 0.003, -0.3)])
 def test_quantize_with_offset_is_nearest_level_brute_force(m, scale, lo):
     rng = np.random.default_rng(m)
     scale, lo = float(np.float32(scale)), float(np.float32(lo))
@@ -36,12 +36,13 @@ def test_quantize_with_offset_is_nearest_level_brute_force(m, scale, lo):
     codes, vals = o.quantize(x, scale, m, lo)
     levels = o.level_set(scale, m, lo)
     assert np.array_equal(vals, levels[codes])
+    assert codes.dtype == (np.uint8 if m <= 256 else np.uint16) and int(codes.max()) == m - 1
     x32 = x.astype(np.float32).astype(np.float64)
     dist = np.abs(x32[:, None] - levels[None, :])
     assert np.all(np.abs(x32 - vals) <= dist.min(axis=1) + 1e-6 * scale + 4e-7 * np.abs(x32))
     t = (x32 - lo) / scale
     far = np.abs(np.abs(t - np.floor(t)) - 0.5) > 1e-3
-    assert np.array_equal(codes[far], dist.argmin(axis=1)[far].astype(np.uint8))
+    assert np.array_equal(codes[far], dist.argmin(axis=1)[far].astype(codes.dtype))
 
 
 def test_quantised_q_minimises_the_q_subproblem_over_delta():
