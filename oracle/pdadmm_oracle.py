@@ -79,6 +79,7 @@ class Params:
     quantize_q: bool = False              # the variant that also keeps q_l in Delta (end of Sec. "Quantization Extension")
     level_lo: float = 0.0                 # smallest level delta_0
     level_step: float = 0.0               # > 0: the same fixed step for every layer; 0: step from max(p) at the start
+    slope: float = 0.0                    # 0: f_l = ReLU; in (0, 1): leaky ReLU with that slope for x <= 0
 
 
 @dataclasses.dataclass
@@ -104,8 +105,10 @@ class State:
         return copy.deepcopy(self)
 
 
-def relu(x):
-    return np.maximum(x, 0.0)
+def relu(x, slope: float = 0.0):
+    """f_l: ReLU, or, with 0 < slope < 1, the leaky ReLU f(x) = x (x > 0), slope x (x <= 0), which the paper
+    names beside ReLU as an activation its assumptions cover (Sec. "Convergence Analysis")."""
+    return np.maximum(x, 0.0) if slope == 0.0 else np.where(x > 0, x, slope * x)
 
 
 # ----------------------------------------------------------------------------
@@ -328,23 +331,25 @@ def update_b_literal(p, W, b, z, nu):
 # z-update (Eq. update z, Eq. update zl)
 # ----------------------------------------------------------------------------
 
-def z_objective_hidden(c, a, q, z_old):
+def z_objective_hidden(c, a, q, z_old, slope: float = 0.0):
     """(c - a)^2 + (q - relu(c))^2 + (c - z^k)^2: Eq. (update z) per element, without the common nu/2."""
-    return (c - a) ** 2 + (q - relu(c)) ** 2 + (c - z_old) ** 2
+    return (c - a) ** 2 + (q - relu(c, slope)) ** 2 + (c - z_old) ** 2
 
 
-def update_z_hidden(a, q, z_old):
+def update_z_hidden(a, q, z_old, slope: float = 0.0):
     """ReLU closed form of Eq. (update z), a = W^{k+1} p^{k+1} + b^{k+1}.
 
     The printed case distinction refers to the sign of the unknown; it is
     resolved by minimising on each half-line and keeping the better of the two:
     z- = min((a + z^k)/2, 0) on z <= 0, z+ = max((a + q^k + z^k)/3, 0) on z >= 0.
-    An exact tie keeps z-.
+    An exact tie keeps z-.  Leaky ReLU with slope s: on z <= 0 the objective is
+    (z-a)^2 + (q - s z)^2 + (z - z^k)^2, stationary at (a + s q + z^k)/(2 + s^2), so
+    z- = min((a + s q^k + z^k)/(2 + s^2), 0); z+ is unchanged.
     """
-    z_neg = np.minimum(0.5 * (a + z_old), 0.0)
+    z_neg = np.minimum((a + slope * q + z_old) / (2.0 + slope * slope), 0.0)
     z_pos = np.maximum((a + q + z_old) / 3.0, 0.0)
-    f_neg = z_objective_hidden(z_neg, a, q, z_old)
-    f_pos = z_objective_hidden(z_pos, a, q, z_old)
+    f_neg = z_objective_hidden(z_neg, a, q, z_old, slope)
+    f_pos = z_objective_hidden(z_pos, a, q, z_old, slope)
     return np.where(f_pos < f_neg, z_pos, z_neg)
 
 
@@ -502,16 +507,16 @@ def update_z_last(a, y, mask, nu):
 # q-update (Eq. update q), dual update (Eq. update u)
 # ----------------------------------------------------------------------------
 
-def update_q(p_next, u, z, rho, nu):
+def update_q(p_next, u, z, rho, nu, slope: float = 0.0):
     """q_l^{k+1} = (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)."""
-    return (rho * p_next + u + nu * relu(z)) / (rho + nu)
+    return (rho * p_next + u + nu * relu(z, slope)) / (rho + nu)
 
 
-def update_q_quantized(p_next, u, z, rho, nu, scale, m, lo=0.0):
+def update_q_quantized(p_next, u, z, rho, nu, scale, m, lo=0.0, slope: float = 0.0):
     """The variant with q_l in Delta as well: q_l^{k+1} = argmin_{delta in Delta}
     ||delta - (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)||, element by element
     (Sec. "Quantization Extension", last paragraph).  Delta is the level set of p_{l+1}, which q_l has to equal."""
-    return quantize(update_q(p_next, u, z, rho, nu), scale, m, lo)[1]
+    return quantize(update_q(p_next, u, z, rho, nu, slope), scale, m, lo)[1]
 
 
 def update_u(u, p_next, q, rho):
@@ -541,7 +546,7 @@ def init_state(X, W0, y, mask, prm: Params) -> State:
     for l in range(L):
         z.append(W[l] @ p[l])
         if l < L - 1:
-            q.append(relu(z[l]))
+            q.append(relu(z[l], prm.slope))
             u.append(np.zeros_like(q[l]))
             if prm.quant_levels:
                 scale[l + 1] = (float(np.float32(prm.level_step)) if prm.level_step > 0
@@ -580,15 +585,16 @@ def iterate(s: State, prm: Params) -> State:
     for l in range(L):
         a = n.W[l] @ n.p[l] + n.b[l][:, None]
         if l < L - 1:
-            n.z[l] = update_z_hidden(a, s.q[l], s.z[l])
+            n.z[l] = update_z_hidden(a, s.q[l], s.z[l], prm.slope)
         else:
             n.z[l] = update_z_last(a, s.y, s.mask, nu)
     # q_l^{k+1}, then u_l^{k+1}
     for l in range(L - 1):
         if prm.quant_levels and prm.quantize_q:
-            n.q[l] = update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels, prm.level_lo)
+            n.q[l] = update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels,
+                                        prm.level_lo, prm.slope)
         else:
-            n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu)
+            n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.slope)
     for l in range(L - 1):
         n.u[l] = update_u(s.u[l], n.p[l + 1], n.q[l], rho)
     return n
@@ -605,7 +611,7 @@ def objective(s: State, prm: Params) -> np.ndarray:
     rho, nu, L = prm.rho, prm.nu, s.L
     R = risk(s.z[L - 1], s.y, s.mask)
     lin = sum(float(np.sum((s.z[l] - s.W[l] @ s.p[l] - s.b[l][:, None]) ** 2)) for l in range(L))
-    act = sum(float(np.sum((s.q[l] - relu(s.z[l])) ** 2)) for l in range(L - 1))
+    act = sum(float(np.sum((s.q[l] - relu(s.z[l], prm.slope)) ** 2)) for l in range(L - 1))
     dual = sum(float(np.sum(s.u[l] * (s.p[l + 1] - s.q[l]))) for l in range(L - 1))
     pen = float(np.sum(residuals_sq(s)))
     comps = [R, 0.5 * nu * lin, 0.5 * nu * act, dual, 0.5 * rho * pen]
@@ -620,20 +626,20 @@ def lagrangian(s: State, prm: Params) -> float:
 # The trained model: forward pass, prediction, accuracy
 # ----------------------------------------------------------------------------
 
-def forward(X, W, b) -> np.ndarray:
+def forward(X, W, b, slope: float = 0.0) -> np.ndarray:
     """z_L of the GA-MLP of Problem 1 with the constraints enforced: p_1 = X,
     z_l = W_l p_l + b_l, p_{l+1} = f_l(z_l) = relu(z_l) (l < L).  Returns z_L (n_L x |V|)."""
     p = np.asarray(X, dtype=np.float64)
     for l in range(len(W)):
         z = W[l] @ p + np.asarray(b[l])[:, None]
-        p = relu(z)
+        p = relu(z, slope)
     return z
 
 
-def predict(X, W, b) -> np.ndarray:
+def predict(X, W, b, slope: float = 0.0) -> np.ndarray:
     """Class of every node: the largest entry of z_L (the class the cross-entropy risk R(z_L; y) rewards);
     the first one if several are equal."""
-    return np.argmax(forward(X, W, b), axis=0)
+    return np.argmax(forward(X, W, b, slope), axis=0)
 
 
 def accuracy(pred, y, mask) -> float:

@@ -180,3 +180,24 @@ def test_forward_pass_golden_and_consistency_with_a_feasible_state():
     b2 = [x.copy() for x in s.b]
     b2[-1][3] += 1e6
     assert np.all(o.predict(X, s.W, b2) == 3)
+
+
+def test_leaky_relu_keeps_lemma_q_opt_and_the_objective_decrease():
+    """The proofs only use that f_l is Lipschitz with constant S <= 1, which a leaky ReLU is: Lemma "q_opt" holds
+    at every iteration and, for rho large enough, L_rho does not increase."""
+    w, X, W0, y, mask = _problem()
+    prm = o.Params(1.0, 0.01, 0, slope=0.2)
+    s = o.init_state(X, W0, y, mask, prm)
+    assert np.allclose(o.residuals_sq(s), 0) and np.any(s.q[0] < 0)          # negative activations pass
+    prev = o.lagrangian(s, prm)
+    for _ in range(6):
+        s = o.iterate(s, prm)
+        for l in range(s.L - 1):
+            assert np.allclose(s.u[l], prm.nu * (s.q[l] - np.where(s.z[l] > 0, s.z[l], 0.2 * s.z[l])), rtol=0, atol=1e-13)
+        cur = o.lagrangian(s, prm)
+        assert cur <= prev + 1e-9 * abs(prev)
+        prev = cur
+    # the forward pass uses the same activation
+    z1 = s.W[0] @ s.p[0] + s.b[0][:, None]
+    p2 = np.where(z1 > 0, z1, 0.2 * z1)
+    assert np.allclose(o.forward(s.p[0], s.W[:2], s.b[:2], 0.2), s.W[1] @ p2 + s.b[1][:, None])

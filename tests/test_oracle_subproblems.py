@@ -254,6 +254,26 @@ def test_z_hidden_against_dense_scalar_grid():
     assert np.all(lhs <= rhs + 1e-12)
 
 
+@pytest.mark.parametrize("slope", [0.1, 0.3, 0.9])
+def test_z_hidden_leaky_relu_against_dense_scalar_grid(slope):
+    """f(x) = x for x > 0, slope * x otherwise: the z-subproblem (z-a)^2 + (q-f(z))^2 + (z-z^k)^2 per element,
+    minimised over a dense grid, agrees with the closed form."""
+    rng = np.random.default_rng(int(slope * 100))
+    a = rng.uniform(-3, 3, 200)
+    q = rng.uniform(-2, 3, 200)
+    zk = rng.uniform(-3, 3, 200)
+    got = o.update_z_hidden(a, q, zk, slope)
+    grid = np.arange(-6.0, 6.0 + 1e-9, 1e-4)
+    f_grid = np.where(grid > 0, grid, slope * grid)
+    for i in range(200):
+        vals = (grid - a[i]) ** 2 + (q[i] - f_grid) ** 2 + (grid - zk[i]) ** 2
+        j = int(np.argmin(vals))
+        f_got = (got[i] - a[i]) ** 2 + (q[i] - (got[i] if got[i] > 0 else slope * got[i])) ** 2 + (got[i] - zk[i]) ** 2
+        assert f_got <= vals[j] + 1e-12
+        assert abs(got[i] - grid[j]) <= 1e-4 or abs(f_got - vals[j]) < 1e-7
+    assert np.array_equal(o.update_z_hidden(a, q, zk, 0.0), o.update_z_hidden(a, q, zk))     # slope 0 is ReLU
+
+
 def test_z_hidden_special_cases():
     # q = a = z^k > 0: z stays ; all negative with q = 0: z stays
     assert o.update_z_hidden(np.array([2.0]), np.array([2.0]), np.array([2.0]))[0] == 2.0
