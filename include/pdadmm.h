@@ -91,6 +91,8 @@ typedef struct {
   int32_t quant_neg_levels;      /* levels below zero: Delta = {(c - quant_neg_levels) s, c = 0..m-1}; 0 = levels
                                     start at 0.  A value > 0 needs quant_step > 0.  ({-1..20}: m=22, 1, step 1) */
   float quant_step;              /* > 0: the same level spacing s for every layer; 0: s_l = max(p_l^0)/(m-1)  */
+  float leaky_slope;             /* f_l of the hidden layers: 0 = ReLU; in (0, 1) = leaky ReLU, f(x) = slope x
+                                    for x <= 0 (paper, "Convergence Analysis": both satisfy its assumptions) */
   const float *const *init_W;    /* [L] pointers: W_l^0 as [n_l][n_{l-1}] (required; the caller draws them) */
   int32_t device;                /* CUDA device ordinal                                                 */
   uint32_t flags;                /* PDADMM_FLAG_*                                                       */

@@ -46,7 +46,7 @@ class _Config(C.Structure):
         ("labels", C.POINTER(C.c_int32)), ("train_mask", C.POINTER(C.c_uint8)),
         ("n_layers", C.c_int32), ("layer_widths", C.POINTER(C.c_int32)),
         ("rho", C.c_float), ("nu", C.c_float), ("quant_levels", C.c_int32),
-        ("quant_neg_levels", C.c_int32), ("quant_step", C.c_float),
+        ("quant_neg_levels", C.c_int32), ("quant_step", C.c_float), ("leaky_slope", C.c_float),
         ("init_W", C.POINTER(C.POINTER(C.c_float))),
         ("device", C.c_int32), ("flags", C.c_uint32),
     ]
@@ -100,7 +100,8 @@ class Context:
 
     def __init__(self, n_nodes: int, edge_src, edge_dst, features, n_hops: int, n_classes: int, labels, train_mask,
                  layer_widths: Sequence[int], rho: float, nu: float, quant_levels: int, init_W: List[np.ndarray],
-                 device: int = 0, flags: int = 0, quant_neg_levels: int = 0, quant_step: float = 0.0):
+                 device: int = 0, flags: int = 0, quant_neg_levels: int = 0, quant_step: float = 0.0,
+                 leaky_slope: float = 0.0):
         self._h = C.c_void_p()
         src = np.ascontiguousarray(edge_src, dtype=np.int32)
         dst = np.ascontiguousarray(edge_dst, dtype=np.int32)
@@ -123,7 +124,7 @@ class Context:
         wp = (C.POINTER(C.c_float) * len(Ws))(*[_ptr(w, C.c_float) for w in Ws])
         cfg = _Config(n_nodes, src.size, _ptr(src, C.c_int32), _ptr(dst, C.c_int32), feat.shape[1],
                       _ptr(feat, C.c_float), n_hops, n_classes, _ptr(lab, C.c_int32), _ptr(msk, C.c_uint8),
-                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, quant_neg_levels, quant_step, wp,
+                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, quant_neg_levels, quant_step, leaky_slope, wp,
                       device, flags)
         self.n_nodes, self.n_layers = int(n_nodes), len(widths)
         self.n0 = (n_hops + 1) * feat.shape[1]
@@ -232,13 +233,14 @@ class Context:
 
 
 def from_inputs(inp, device: int = 0, flags: int = 0, rho: Optional[float] = None, nu: Optional[float] = None,
-                quant_levels: Optional[int] = None, quant_neg_levels: int = 0, quant_step: float = 0.0) -> Context:
+                quant_levels: Optional[int] = None, quant_neg_levels: int = 0, quant_step: float = 0.0,
+                leaky_slope: float = 0.0) -> Context:
     """Context for a ``synth.Inputs`` bundle."""
     w = inp.workload
     return Context(w.n_nodes, inp.edge_src, inp.edge_dst, inp.features, w.n_hops, w.n_classes, inp.labels,
                    inp.train_mask, w.widths, w.rho if rho is None else rho, w.nu if nu is None else nu,
                    w.quant_levels if quant_levels is None else quant_levels, inp.init_W, device, flags,
-                   quant_neg_levels, quant_step)
+                   quant_neg_levels, quant_step, leaky_slope)
 
 
 def quantize(x, scale: float, levels: int, device: int = 0, lo: float = 0.0):

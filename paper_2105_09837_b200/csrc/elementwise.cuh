@@ -301,15 +301,16 @@ finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int 
 
 // ---- z-, q-, u-update of a hidden layer, fused ----------------------------------------------------
 // a = W+ p+ + b+ = (r - shift) + z.  z+ by the ReLU closed form of Eq. "update z" (better of the two
-// half-line minimisers; a tie keeps the non-positive one), q+ by Eq. "update q" (q_top >= 0: projected onto
+// half-line minimisers; a tie keeps the non-positive one; slope > 0: leaky ReLU f(x) = slope x for x <= 0, whose
+// minimiser on z <= 0 is (a + slope q + z)/(2 + slope^2)), q+ by Eq. "update q" (q_top >= 0: projected onto
 // the level set of p_{l+1}, the variant at the end of Sec. "Quantization Extension"), residual p_{l+1} - q+,
 // u+ by Eq. "update u", and the linear residual of the next iteration r = a - z+.
 __global__ void __launch_bounds__(EW_THREADS)
 zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
            const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
-           float rho, float nu, float q_scale, float q_lo, float q_top, double *__restrict__ slots) {
+           float rho, float nu, float slope, float q_scale, float q_lo, float q_top, double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
-  const float inv_rn = 1.0f / (rho + nu);
+  const float inv_rn = 1.0f / (rho + nu), inv_neg = 1.0f / (2.0f + slope * slope);
   double ss = 0.0;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 sh = ld4(shift, i % ld4cols);
@@ -318,12 +319,13 @@ zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, 
 #define PD_ZQU(f)                                                                   \
     {                                                                               \
       const float a = (rv.f - sh.f) + zv.f;                                         \
-      const float zneg = fminf(0.5f * (a + zv.f), 0.0f);                            \
+      const float zneg = fminf((fmaf(slope, qv.f, a) + zv.f) * inv_neg, 0.0f);      \
       const float zpos = fmaxf((a + qv.f + zv.f) * (1.0f / 3.0f), 0.0f);            \
-      const float fneg = (zneg - a) * (zneg - a) + qv.f * qv.f + (zneg - zv.f) * (zneg - zv.f); \
+      const float qneg = qv.f - slope * zneg;                                       \
+      const float fneg = (zneg - a) * (zneg - a) + qneg * qneg + (zneg - zv.f) * (zneg - zv.f); \
       const float fpos = (zpos - a) * (zpos - a) + (qv.f - zpos) * (qv.f - zpos) + (zpos - zv.f) * (zpos - zv.f); \
       const float zz = fpos < fneg ? zpos : zneg;                                   \
-      float qq = (rho * pv.f + uv.f + nu * fmaxf(zz, 0.0f)) * inv_rn;               \
+      float qq = (rho * pv.f + uv.f + nu * (zz > 0.0f ? zz : slope * zz)) * inv_rn; \
       if (q_top >= 0.0f) { unsigned code; qq = quantize_one(qq, q_scale, q_lo, q_top, code); } \
       const float res = pv.f - qq;                                                  \
       zn.f = zz; qn.f = qq; un.f = fmaf(rho, res, uv.f); rn.f = a - zz;             \
@@ -410,12 +412,13 @@ zlast_kernel(float *__restrict__ r, float *__restrict__ z, const float *__restri
 
 // ---- elementwise helpers of the initial forward pass ---------------------------------------------
 __global__ void __launch_bounds__(EW_THREADS)
-relu_max_kernel(const float *__restrict__ z, float *__restrict__ q, size_t n4, float *__restrict__ block_max) {
+relu_max_kernel(const float *__restrict__ z, float *__restrict__ q, size_t n4, float slope, float *__restrict__ block_max) {
   __shared__ float red[EW_THREADS / 32];
   float m = 0.0f;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = ld4(z, i);
-    v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f);
+    v.x = v.x > 0.f ? v.x : slope * v.x; v.y = v.y > 0.f ? v.y : slope * v.y;
+    v.z = v.z > 0.f ? v.z : slope * v.z; v.w = v.w > 0.f ? v.w : slope * v.w;
     m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
     st4(q, i, v);
   }
@@ -432,7 +435,7 @@ relu_max_kernel(const float *__restrict__ z, float *__restrict__ q, size_t n4, f
 // slots[b][0..3] = sum r^2, sum (q - relu z)^2, sum u (p_next - q), sum (p_next - q)^2 ; q == nullptr: only r^2.
 __global__ void __launch_bounds__(EW_THREADS)
 objective_layer_kernel(const float *__restrict__ r, const float *__restrict__ z, const float *__restrict__ q,
-                       const float *__restrict__ u, const float *__restrict__ p_next, size_t n,
+                       const float *__restrict__ u, const float *__restrict__ p_next, size_t n, float slope,
                        double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
@@ -440,7 +443,8 @@ objective_layer_kernel(const float *__restrict__ r, const float *__restrict__ z,
     const double rv = r[i];
     s0 += rv * rv;
     if (q != nullptr) {
-      const double qv = q[i], act = fmaxf(z[i], 0.0f), res = (double)p_next[i] - qv;
+      const float zv = z[i];
+      const double qv = q[i], act = zv > 0.0f ? zv : slope * zv, res = (double)p_next[i] - qv;
       s1 += (qv - act) * (qv - act);
       s2 += (double)u[i] * res;
       s3 += res * res;

@@ -57,16 +57,17 @@ struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b
     return make_float4(a.x + b.x - z.x, a.y + b.y - z.y, a.z + b.z - z.z, a.w + b.w - z.w);
   }
 };
-struct EpiBiasAct {           // C = acc + b[col], then ReLU if relu != 0   (forward pass z = W p + b, p' = f(z))
+struct EpiBiasAct {           // C = acc + b[col], then f (ReLU, leaky with `slope`) if relu != 0   (z = W p + b, p' = f(z))
   static constexpr bool kDirect = false, kSumsq = false;
   static constexpr int kInputs = 0;
-  float *C; int ldc; const float *bias; int relu;
+  float *C; int ldc; const float *bias; int relu; float slope;
+  __device__ __forceinline__ float f(float x) const { return x > 0.f ? x : slope * x; }
   __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ void load(int, int, float4 *) const {}
   __device__ __forceinline__ float4 apply(int col, float4 a, const float4 *) const {
     const float4 b = *reinterpret_cast<const float4 *>(bias + col);
     float4 o = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
-    if (relu) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+    if (relu) { o.x = f(o.x); o.y = f(o.y); o.z = f(o.z); o.w = f(o.w); }
     return o;
   }
   __device__ __forceinline__ float4 operator()(int, int col, float4 a, double &) const { return apply(col, a, nullptr); }

@@ -93,6 +93,7 @@ struct pdadmm_ctx {
   int neg_levels = 0;              // levels below zero
   float fixed_step = 0.f;          // > 0: the same level spacing for every layer
   bool quant_q = false;            // q_l is kept on the level set of p_{l+1} as well
+  float slope = 0.f;               // f_l: 0 = ReLU, (0, 1) = leaky ReLU with that slope for x <= 0
   float rho = 0, nu = 0;
   uint32_t flags = 0;
   int64_t nnz = 0;
@@ -487,7 +488,7 @@ static void zqu_step(pdadmm_ctx *c, int l) {
       Launch k(c, KC_ZQU, s.st, 36.0 * N * ly.n_out, 0);
       const Layer &nx = c->layers[l + 1];
       zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu,
-                                               nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, s.slots);
+                                               c->slope, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, s.slots);
     }
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
@@ -540,6 +541,8 @@ static int check_config(const pdadmm_config *cfg) {
     return fail(PDADMM_EINVAL, "quant_neg_levels must be in [0, quant_levels)");
   if (cfg->quant_step < 0.f || (cfg->quant_neg_levels > 0 && !(cfg->quant_step > 0.f)))
     return fail(PDADMM_EINVAL, "quant_step must be >= 0, and > 0 when quant_neg_levels > 0");
+  if (!(cfg->leaky_slope >= 0.f && cfg->leaky_slope < 1.f))
+    return fail(PDADMM_EINVAL, "leaky_slope must be in [0, 1)");
   if ((cfg->flags & PDADMM_FLAG_QUANT_Q) && cfg->quant_levels == 0)
     return fail(PDADMM_EINVAL, "PDADMM_FLAG_QUANT_Q needs quant_levels >= 2");
   for (int64_t j = 0; j < cfg->n_nodes; ++j)
@@ -633,6 +636,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->neg_levels = cfg->quant_neg_levels; c->fixed_step = cfg->quant_step;
   c->code_bytes = cfg->quant_levels > 256 ? 2 : 1;
   c->quant_q = (cfg->flags & PDADMM_FLAG_QUANT_Q) != 0;
+  c->slope = cfg->leaky_slope;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
   PD_CUDA(cudaSetDevice(cfg->device));
@@ -729,7 +733,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     const size_t n4 = (size_t)N * ly.ld_out / 4;
     const int grid = ew_grid(n4);
     float *bm = reinterpret_cast<float *>(s.slots);
-    relu_max_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, ly.q, n4, bm);
+    relu_max_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, ly.q, n4, c->slope, bm);
     if (c->levels) {
       std::vector<float> hm(grid);
       PD_CUDA(cudaMemcpyAsync(hm.data(), bm, grid * sizeof(float), cudaMemcpyDeviceToHost, st));
@@ -896,7 +900,7 @@ extern "C" int pdadmm_objective(pdadmm_ctx *c, double out[6]) {
     const int grid = std::min(ew_grid(n), 512);
     const bool hidden = l + 1 < c->L;
     objective_layer_kernel<<<grid, EW_THREADS, 0, st>>>(ly.r, ly.z, hidden ? ly.q : nullptr, ly.u,
-                                                       hidden ? c->layers[l + 1].p : nullptr, n, c->scr.slots);
+                                                       hidden ? c->layers[l + 1].p : nullptr, n, c->slope, c->scr.slots);
     double h[4];
     PD_TRY(read_slots(c, grid, 4, 4, h));
     lin += h[0]; act += h[1]; dual += h[2]; pen += h[3];
@@ -929,7 +933,7 @@ extern "C" int pdadmm_predict(pdadmm_ctx *c, float *logits_out, int32_t *pred_ou
   for (int l = 0; l < c->L; ++l) {
     Layer &ly = c->layers[l];
     out = bufs[l & 1];
-    EpiBiasAct epi{out, ly.ld_out, ly.b, l + 1 < c->L ? 1 : 0};
+    EpiBiasAct epi{out, ly.ld_out, ly.b, l + 1 < c->L ? 1 : 0, c->slope};
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, N, ly.n_out, ly.n_in, in, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
                              epi, nullptr, nullptr, 0));
     in = out;
@@ -966,7 +970,7 @@ extern "C" int pdadmm_residuals(pdadmm_ctx *c, double *per_layer_sq, int n) {
     const size_t nn = (size_t)c->N * ly.ld_out;
     const int grid = std::min(ew_grid(nn), 512);
     objective_layer_kernel<<<grid, EW_THREADS, 0, c->scr.st>>>(ly.r, ly.z, ly.q, ly.u, c->layers[l + 1].p, nn,
-                                                              c->scr.slots);
+                                                              c->slope, c->scr.slots);
     double h[4];
     PD_TRY(read_slots(c, grid, 4, 4, h));
     per_layer_sq[l] = h[3];

@@ -9,14 +9,14 @@ import oracle.pdadmm_oracle as o
 from paper_2105_09837_b200 import binding as B
 
 
-def oracle_problem(inp, rho=None, nu=None, quant_levels=None, quantize_q=False, neg_levels=0, step=0.0):
+def oracle_problem(inp, rho=None, nu=None, quant_levels=None, quantize_q=False, neg_levels=0, step=0.0, slope=0.0):
     """(Params, initial oracle State) for a synth.Inputs bundle.  neg_levels / step: a fixed level set
     {(c - neg_levels) step} as the C ABI's quant_neg_levels / quant_step describe it."""
     w = inp.workload
     lo = float(np.float32(-neg_levels) * np.float32(step))
     prm = o.Params(w.rho if rho is None else rho, w.nu if nu is None else nu,
                    w.quant_levels if quant_levels is None else quant_levels,
-                   quantize_q=quantize_q, level_lo=lo, level_step=step)
+                   quantize_q=quantize_q, level_lo=lo, level_step=step, slope=slope)
     A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
     X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
     s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels, inp.train_mask, prm)
@@ -76,14 +76,14 @@ def rel_err(got, want, mask=None) -> float:
     return float(num / den)
 
 
-def z_tie_mask(prev: o.State, nxt: o.State, l: int, tol=1e-5):
+def z_tie_mask(prev: o.State, nxt: o.State, l: int, tol=1e-5, slope=0.0):
     """Elements of hidden layer l (0-based) whose two ReLU candidates have (nearly) the same objective:
     both are minimisers there, so single and double precision may pick different ones."""
     a = nxt.W[l] @ nxt.p[l] + nxt.b[l][:, None]
-    zn = np.minimum(0.5 * (a + prev.z[l]), 0.0)
+    zn = np.minimum((a + slope * prev.q[l] + prev.z[l]) / (2.0 + slope * slope), 0.0)
     zp = np.maximum((a + prev.q[l] + prev.z[l]) / 3.0, 0.0)
-    fn = o.z_objective_hidden(zn, a, prev.q[l], prev.z[l])
-    fp = o.z_objective_hidden(zp, a, prev.q[l], prev.z[l])
+    fn = o.z_objective_hidden(zn, a, prev.q[l], prev.z[l], slope)
+    fp = o.z_objective_hidden(zp, a, prev.q[l], prev.z[l], slope)
     # equal candidates (both clamp to 0) are not a tie: either choice gives the same z
     return (np.abs(fp - fn) <= tol * (np.abs(fp) + np.abs(fn) + 1e-30)) & (zp != zn)
 

@@ -127,7 +127,7 @@ def _compare_iteration(ctx, prev, prm, label):
             theta = float(ctx.get_tensor(B.T_THETA, l + 1)[0])
             assert abs(theta - nxt.theta[l]) <= 1e-3 * nxt.theta[l], f"{label}: theta_{l + 1} {theta} vs {nxt.theta[l]}"
         if l < L - 1:
-            tie = U.z_tie_mask(prev, nxt, l)
+            tie = U.z_tie_mask(prev, nxt, l, slope=prm.slope)
             # a coarse fixed level set (integers) makes q exactly 0 or a whole number in many places, and with it
             # exact ties between the two ReLU candidates; elsewhere ties are rare
             assert tie.mean() < (0.1 if prm.level_step else 1e-2)
@@ -232,6 +232,36 @@ def test_teacher_forced_level_set_variants(case, levels, neg, step, quant_q):
             assert np.all(np.isin(st["q"][l - 1], lev))
     assert np.all(np.isfinite(ctx.objective()))
     ctx.destroy()
+
+
+@pytest.mark.parametrize("case,slope,levels,neg,step", [("er-small", 0.2, 0, 0, 0.0), ("ba-ragged", 0.05, 0, 0, 0.0),
+                                                       ("c4-like", 0.3, 64, 8, 0.125)])
+def test_teacher_forced_leaky_relu(case, slope, levels, neg, step):
+    """f_l = leaky ReLU (the other activation the paper names): z-update by its own closed form, q, u, the
+    objective's activation term and the forward pass all use it."""
+    inp = _inputs(case, quant_levels=levels)
+    prm, s, _ = U.oracle_problem(inp, neg_levels=neg, step=step, slope=slope)
+    ctx = B.from_inputs(inp, quant_neg_levels=neg, quant_step=step, leaky_slope=slope)
+    st = U.read_state(ctx)
+    if not levels:
+        for l in range(s.L - 1):
+            assert U.rel_err(st["q"][l], s.q[l]) < 1e-5 and st["q"][l].min() < 0
+    for k in range(4):
+        prev = U.round_state(s)
+        U.load_state(ctx, prev, levels > 0)
+        s = _compare_iteration(ctx, prev, prm, f"{case}/slope={slope}/k={k}")
+    got, want = ctx.objective(), o.objective(s, prm)
+    assert abs(got[2] - want[2]) <= 1e-3 * abs(want[2]) + 1e-12 and abs(got[5] - want[5]) <= 1e-3 * abs(want[5])
+    logits, pred, _ = ctx.predict()
+    want_logits = o.forward(s.p[0], [U.f32(w) for w in ctx_weights(ctx)[0]], [U.f32(b) for b in ctx_weights(ctx)[1]], slope)
+    assert U.rel_err(logits.T.astype(np.float64), want_logits) < TOL
+    ctx.destroy()
+
+
+def ctx_weights(ctx):
+    L = ctx.n_layers
+    return ([ctx.get_tensor(B.T_W, l).astype(np.float64) for l in range(1, L + 1)],
+            [ctx.get_tensor(B.T_B, l).astype(np.float64) for l in range(1, L + 1)])
 
 
 @pytest.mark.parametrize("rho,nu", [(1.0, 0.01), (0.05, 0.5)])
