@@ -24,9 +24,13 @@ constexpr int TC_FLUSH = 1;                                    // K blocks per r
 constexpr int TC_TILE_BYTES = 128 * TC_BK * 4;                 // 16 KB: one 128 x 32 fp32 operand tile
 constexpr int TC_MN_CHUNK = TC_BK * 128;                       // MN-major tiles: 32 output indices x TC_BK rows
 constexpr int TC_STAGE_BYTES = 4 * TC_TILE_BYTES;              // A_hi, A_lo, B_hi, B_lo
-// warp 0: TMA, warp 1: MMA, warps 2..5: operand split, warps 6..13: accumulate + epilogue
+// warp 0: TMA, warp 1: MMA, then 4 (8) operand-split warps, then 8 accumulate + epilogue warps
 // (two warps per 32-lane quarter of tensor memory, 64 columns each)
-constexpr int TC_THREADS = 448;
+constexpr int TC_THREADS = 448;                                // 576 when both operands are split in the kernel
+// number of operand-split warps: twice as many when both operands are split in shared memory (the contraction over
+// nodes), where the split and not the MMA issue sets the pace
+__host__ __device__ constexpr int tc_conv_warps(bool b_split) { return b_split ? 8 : 4; }
+__host__ __device__ constexpr int tc_threads(bool b_split) { return 32 * (2 + tc_conv_warps(b_split) + 8); }
 constexpr int TC_ACC_THREADS = 256;
 constexpr int TC_ACC_BUFS = 3;                                 // main-term accumulator tiles in tensor memory
 constexpr int TC_TMEM_COLS = 512;                              // 3 main tiles + 1 correction tile
@@ -67,7 +71,7 @@ struct TcParams {
 // block fill the other buffer.  The two correction terms are 2^-12 of the main term, so they are summed over
 // the whole contraction in a third tensor-memory tile and added once at the end.
 template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(tc_threads(B_SPLIT), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_blo, const __grid_constant__ CUtensorMap map_c,
                const TcParams prm, Epi epi, double *__restrict__ partials) {
@@ -83,6 +87,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int ACC0 = 2 + tc_conv_warps(B_SPLIT);              // first accumulate warp
+  constexpr int CONV_T = 32 * tc_conv_warps(B_SPLIT);           // operand-split threads
   const int tiles_n = (prm.N + TC_BN - 1) / TC_BN, tiles_m = (prm.M + TC_BM - 1) / TC_BM;
   const int n_out_tiles = tiles_n * tiles_m * prm.n_split;
   const bool tail_on = prm.tail_split > 1;
@@ -92,7 +98,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
-      ptx::mbar_init(&conv_bar[s], 128);
+      ptx::mbar_init(&conv_bar[s], 32 * tc_conv_warps(B_SPLIT));
       ptx::mbar_init(&empty_bar[s], 1);
     }
     for (int b = 0; b < TC_ACC_BUFS; ++b) {
@@ -239,9 +245,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ptx::mbar_wait(drain_bar, 0, abort_flag, 200000000ll, false);
       }
     }
-  } else if (warp < 6) {
-    // ---------------------------------------------------------------- operand split (128 threads)
-    const int t = threadIdx.x - 64;
+  } else if (warp < ACC0) {
+    // ---------------------------------------------------------------- operand split (128 or 256 threads)
+    const int t = threadIdx.x - 64;                       // 0 .. CONV_T-1
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -255,16 +261,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         auto split = [&](uint8_t *hi_buf, uint8_t *lo_buf) {
           uint4 *hi = reinterpret_cast<uint4 *>(hi_buf), *lo = reinterpret_cast<uint4 *>(lo_buf);
 #pragma unroll
-          for (int i = 0; i < TC_TILE_BYTES / 16 / 128; ++i) {
-            const uint4 v = hi[t + 128 * i];
+          for (int i = 0; i < TC_TILE_BYTES / 16 / CONV_T; ++i) {
+            const uint4 v = hi[t + CONV_T * i];
             uint4 h, l;
             h.x = tf32_hi(v.x); h.y = tf32_hi(v.y); h.z = tf32_hi(v.z); h.w = tf32_hi(v.w);
             l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
             l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
             l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
             l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
-            hi[t + 128 * i] = h;
-            lo[t + 128 * i] = l;
+            hi[t + CONV_T * i] = h;
+            lo[t + CONV_T * i] = l;
           }
         };
         split(st, st + TC_TILE_BYTES);
@@ -278,8 +284,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // warp w owns tensor-memory lanes 32 (w mod 4) .. +31 = output rows m0 + that range, and the column half
     // (w - 6) / 4 of the tile (64 columns)
     const int lane_base = (warp & 3) * 32;
-    const int chalf = (warp - 6) >> 2;
-    float4 *tr = reinterpret_cast<float4 *>(tr_base) + (size_t)(warp - 6) * 32 * 8;    // 32 rows x 8 float4 per warp
+    const int chalf = (warp - ACC0) >> 2;
+    float4 *tr = reinterpret_cast<float4 *>(tr_base) + (size_t)(warp - ACC0) * 32 * 8;    // 32 rows x 8 float4 per warp
     const int n_pad = (prm.N + 3) & ~3;
     bool ok = true;
     int it = 0;
@@ -298,12 +304,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int j = 0; j < 64; ++j) acc[j] = 0.f;
       auto add_tile = [&](uint32_t col_base) {
         const uint32_t src = tmem_base + ((uint32_t)lane_base << 16) + col_base + (uint32_t)(chalf * 64);
-        uint32_t v0[32], v1[32];
-        ptx::tmem_ld32(src, v0);
-        ptx::tmem_ld32(src + 32u, v1);
-        ptx::tmem_ld_wait();
+        if constexpr (B_SPLIT) {
+          // 576 threads leave 96 registers per thread: 16 columns at a time
 #pragma unroll
-        for (int j = 0; j < 32; ++j) { acc[j] += __uint_as_float(v0[j]); acc[32 + j] += __uint_as_float(v1[j]); }
+          for (int h = 0; h < 4; ++h) {
+            uint32_t v[16];
+            ptx::tmem_ld16(src + 16u * h, v);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) acc[16 * h + j] += __uint_as_float(v[j]);
+          }
+        } else {
+          uint32_t v0[32], v1[32];
+          ptx::tmem_ld32(src, v0);
+          ptx::tmem_ld32(src + 32u, v1);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) { acc[j] += __uint_as_float(v0[j]); acc[32 + j] += __uint_as_float(v1[j]); }
+        }
       };
       const int n_grp = (n_kb + TC_FLUSH - 1) / TC_FLUSH;
       for (int g = 0; g < n_grp && ok; ++g, ++it) {
@@ -327,21 +345,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // contraction slice of a tail tile: park the accumulators; the last warp to arrive sums the slices
         const int u = tile - tail_begin, t_idx = u / prm.tail_split;
         out_tile = tail_begin + t_idx;
-        float *mine = prm.tail_ws + ((size_t)u * 8 + (warp - 6)) * 2048;
+        float *mine = prm.tail_ws + ((size_t)u * 8 + (warp - ACC0)) * 2048;
 #pragma unroll
         for (int j = 0; j < 64; ++j) mine[j * 32 + lane] = acc[j];
         __threadfence();
         __syncwarp();
         int prev = 0;
-        if (lane == 0) prev = atomicAdd(prm.tail_count + t_idx * 8 + (warp - 6), 1);
+        if (lane == 0) prev = atomicAdd(prm.tail_count + t_idx * 8 + (warp - ACC0), 1);
         prev = __shfl_sync(0xffffffffu, prev, 0);
         if (prev != prm.tail_split - 1) continue;
         __threadfence();
-        if (lane == 0) prm.tail_count[t_idx * 8 + (warp - 6)] = 0;
+        if (lane == 0) prm.tail_count[t_idx * 8 + (warp - ACC0)] = 0;
 #pragma unroll
         for (int j = 0; j < 64; ++j) acc[j] = 0.f;
         for (int sl = 0; sl < prm.tail_split; ++sl) {
-          const float *part = prm.tail_ws + ((size_t)(t_idx * prm.tail_split + sl) * 8 + (warp - 6)) * 2048;
+          const float *part = prm.tail_ws + ((size_t)(t_idx * prm.tail_split + sl) * 8 + (warp - ACC0)) * 2048;
 #pragma unroll
           for (int j = 0; j < 64; ++j) acc[j] += __ldcg(part + j * 32 + lane);
         }
@@ -421,7 +439,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       if (partials != nullptr) {          // one slot per tile and warp; the host adds the slots in index order
         ss = warp_sum(ss);
-        if (lane == 0) partials[(size_t)out_tile * 8 + (warp - 6)] = ss;
+        if (lane == 0) partials[(size_t)out_tile * 8 + (warp - ACC0)] = ss;
       }
     }
     if (Epi::kDirect && lane == 0) ptx::bulk_wait_all();

@@ -273,7 +273,7 @@ static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, cons
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     configured = true;
   }
-  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, mc, prm, epi, partials);
+  kern<<<grid, tc_threads(B_SPLIT), TC_SMEM_BYTES, st>>>(ma, mb, mbl, mc, prm, epi, partials);
   return PDADMM_OK;
 }
 
