@@ -283,6 +283,10 @@ def main():
         roof = {"bound": "hbm", "achieved": d["bytes"] / (d["ms"] * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
                 "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth"}
     roof["frac"] = roof["achieved"] / roof["peak"]
+    if roof["bound"] == "tensor":
+        # every useful product is issued as three tf32 MMAs (hi*hi, hi*lo, lo*hi): the tensor pipe's own load
+        roof["frac_issued"] = 3.0 * roof["frac"]
+        roof["note"] = "achieved counts useful fp32-equivalent flop; the kernel issues three tf32 MMAs per product"
     roof["kernel"] = dom
     roof["traffic"] = measured_traffic(args.workload, dom)
     ctx.destroy()
