@@ -152,13 +152,15 @@ __device__ __forceinline__ double block_sum_slots(const double *__restrict__ slo
 // ||g||^2 and ||W g||^2 from their slots, then
 // tau = rho + nu ||W g||^2 / ||g||^2 : the smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
 __global__ void __launch_bounds__(256)
-finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots_g, int n_g, const double *slots_wg, int n_wg) {
+finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots_g, int n_g, const double *slots_wg, int n_wg,
+                    int *nonfinite) {
   __shared__ double sh[256];
   const double gg = block_sum_slots(slots_g, n_g, sh);
   const double wg = block_sum_slots(slots_wg, n_wg, sh);
   if (threadIdx.x == 0) {
     sc->sum_g2 = gg;
     sc->sum_wg2 = wg;
+    if (!(isfinite(gg) && isfinite(wg))) *nonfinite = 1;      // a NaN or Inf anywhere in the state reaches these sums
     const double tau = gg > 0.0 ? rho + nu * wg / gg : rho;
     sc->tau = tau;
     sc->inv_tau = (float)(1.0 / tau);
@@ -189,13 +191,15 @@ finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack, con
 // ||grad_W||^2 and ||grad_W p+||^2 from their slots, then
 // theta = nu ||grad_W p+||^2 / ||grad_W||^2 : the smallest theta with phi(W+) <= V_l(W+; theta).
 __global__ void __launch_bounds__(256)
-finalize_theta_kernel(LayerScalars *sc, double nu, const double *slots_G, int n_G, const double *slots_Gp, int n_Gp) {
+finalize_theta_kernel(LayerScalars *sc, double nu, const double *slots_G, int n_G, const double *slots_Gp, int n_Gp,
+                      int *nonfinite) {
   __shared__ double sh[256];
   const double GG = block_sum_slots(slots_G, n_G, sh);
   const double Gp = block_sum_slots(slots_Gp, n_Gp, sh);
   if (threadIdx.x == 0) {
     sc->sum_G2 = GG;
     sc->sum_Gp2 = Gp;
+    if (!(isfinite(GG) && isfinite(Gp))) *nonfinite = 1;
     const double theta = GG > 0.0 ? nu * Gp / GG : 0.0;
     sc->theta = theta;
     sc->inv_theta = theta > 0.0 ? (float)(1.0 / theta) : 0.0f;

@@ -357,7 +357,7 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
                            epi2, slots_b, &np2, 0));
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
-    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2);
+    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2);
   }
   return PDADMM_OK;
 }
@@ -452,7 +452,7 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
                            epi, slots_b, &np, 0));
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (gw + np), 0);
-    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np);
+    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2);
   }
   {
     Launch k(c, KC_WSTEP, s.st, 20.0 * ly.n_out * ly.n_in, 0);
@@ -826,7 +826,7 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
   if (n_iters < 0) return fail(PDADMM_EINVAL, "n_iters is negative");
   PD_CUDA(cudaSetDevice(c->device));
   PD_CUDA(cudaEventRecord(c->ev_begin, c->scr.st));
-  PD_CUDA(cudaMemsetAsync(c->d_flag, 0, 2 * sizeof(int), c->scr.st));
+  PD_CUDA(cudaMemsetAsync(c->d_flag, 0, 3 * sizeof(int), c->scr.st));
   PD_TRY(ensure_residual(c));
   bool hit_cap = false;
   // pdADMM-G has no host decision inside an iteration, so after a first eager iteration the sequence of launches
@@ -863,7 +863,7 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
       PD_TRY(iterate_once(c, &hit_cap));
     }
   }
-  PD_CUDA(cudaMemcpyAsync(c->h_pinned + 8, c->d_flag, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->scr.st));
+  PD_CUDA(cudaMemcpyAsync(c->h_pinned + 8, c->d_flag, 3 * sizeof(int), cudaMemcpyDeviceToHost, c->scr.st));
   PD_CUDA(cudaEventRecord(c->ev_end, c->scr.st));
   PD_CUDA(cudaStreamSynchronize(c->scr.st));
   PD_CUDA(cudaGetLastError());
@@ -874,6 +874,7 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
   }
   if (c->profiling) PD_TRY(prof_collect(c));
   if (c->h_pinned[9] != 0) return fail(PDADMM_ETIMEOUT, "a bounded wait inside a tensor-core product expired");
+  if (c->h_pinned[10] != 0) return fail(PDADMM_ENUMERIC, "a non-finite value reached the gradient norms: the state holds NaN or Inf");
   if (c->h_pinned[8] != 0)
     return fail(PDADMM_ENOTCONV, "the last-layer z solver did not converge on %d nodes", c->h_pinned[8]);
   if (hit_cap) return fail(PDADMM_ENOTCONV, "the tau search of a quantised p-update reached its trial cap");

@@ -181,3 +181,17 @@ def test_profile_counters_and_launch_count():
     assert prof["gemm_gradw"]["flops"] > 0
     ctx.profile(False)
     ctx.destroy()
+
+
+def test_non_finite_state_is_reported_not_propagated_silently():
+    """A NaN written into W by the caller: the next step returns ENUMERIC (the gradient norms see it)."""
+    inp = synth.make_inputs(synth.small("c1", 300, feat_dim=6, hidden=8, n_layers=3))
+    ctx = B.from_inputs(inp)
+    ctx.step(1)
+    W2 = ctx.get_tensor(B.T_W, 2)
+    W2[1, 2] = np.nan
+    ctx.set_tensor(B.T_W, 2, W2)
+    with pytest.raises(B.PdadmmError) as e:
+        ctx.step(1)
+    assert e.value.code == B.ENUMERIC
+    ctx.destroy()
