@@ -1,5 +1,5 @@
 // Thin wrappers of the sm_100a instructions used by the tensor-core products:
-// mbarrier, TMA tile loads (never multicast), tcgen05 MMA / TMEM management, proxy fences.
+// mbarrier, TMA tile loads (each block fetches its own tiles), tcgen05 MMA / TMEM management, proxy fences.
 #pragma once
 
 #include <cuda.h>
@@ -58,7 +58,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
   }
 }
 
-// ---- TMA: 2-D tile load global -> shared, completion on an mbarrier (no multicast) -------------------
+// ---- TMA: 2-D tile load global -> shared, completion on an mbarrier -------------------
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
