@@ -95,3 +95,32 @@ def test_c4_c5_full_size_parts_and_invariants(name):
         del codes, p
         assert 1 <= int(ctx.get_tensor(B.T_TRIALS, l + 1)[0]) <= 30
     ctx.destroy()
+
+
+def test_c4_full_size_level_set_variant_and_prediction():
+    """Workload c4 with the paper's level set {-1..20} for p and q: after two iterations both are on the set bit
+    for bit, and the forward pass of the trained model agrees with the oracle on sampled nodes."""
+    w = synth.get("c4")
+    inp = synth.make_inputs(w)
+    m, neg, step = 22, 1, 1.0
+    ctx = B.from_inputs(inp, flags=B.FLAG_QUANT_Q, quant_levels=m, quant_neg_levels=neg, quant_step=step)
+    ctx.step(2)
+    assert np.all(np.isfinite(ctx.objective()))
+    lev = o.level_set(step, m, -1.0).astype(np.float32)
+    for l in (1, w.n_layers // 2, w.n_layers - 1):
+        assert float(ctx.get_tensor(B.T_QSCALE, l + 1)[0]) == step
+        p, q, codes = ctx.get_tensor(B.T_P, l + 1), ctx.get_tensor(B.T_Q, l), ctx.get_tensor(B.T_CODES, l + 1)
+        assert np.array_equal(p, np.float32(-1.0) + codes.astype(np.float32) * np.float32(step))
+        assert np.all(np.isin(q, lev))
+        del p, q, codes
+    logits, pred, counts = ctx.predict()
+    assert counts[1] + counts[3] == w.n_nodes and counts[1] == int(inp.train_mask.sum())
+    assert np.array_equal(pred, np.argmax(logits, axis=1))
+    rng = np.random.default_rng(11)
+    nodes = rng.choice(w.n_nodes, size=48, replace=False)
+    X = ctx.get_tensor(B.T_X)[nodes].T.astype(np.float64)
+    Ws = [ctx.get_tensor(B.T_W, l).astype(np.float64) for l in range(1, w.n_layers + 1)]
+    bs = [ctx.get_tensor(B.T_B, l).astype(np.float64) for l in range(1, w.n_layers + 1)]
+    want = o.forward(X, Ws, bs)
+    assert U.rel_err(logits[nodes].T.astype(np.float64), want) < 1e-4
+    ctx.destroy()
