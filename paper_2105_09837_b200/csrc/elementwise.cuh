@@ -308,18 +308,20 @@ finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int 
 // half-line minimisers; a tie keeps the non-positive one; slope > 0: leaky ReLU f(x) = slope x for x <= 0, whose
 // minimiser on z <= 0 is (a + slope q + z)/(2 + slope^2)), q+ by Eq. "update q" (q_top >= 0: projected onto
 // the level set of p_{l+1}, the variant at the end of Sec. "Quantization Extension"), residual p_{l+1} - q+,
-// u+ by Eq. "update u", and the linear residual of the next iteration r = a - z+.
+// u+ by Eq. "update u", the linear residual of the next iteration r = a - z+, and t_{l+1} = u+ + rho (p_{l+1} - q+),
+// the part of the next p-gradient that does not involve a product.
 __global__ void __launch_bounds__(EW_THREADS)
 zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
            const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
-           float rho, float nu, float slope, float q_scale, float q_lo, float q_top, double *__restrict__ slots) {
+           float rho, float nu, float slope, float q_scale, float q_lo, float q_top, float *__restrict__ t_next,
+           double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_rn = 1.0f / (rho + nu), inv_neg = 1.0f / (2.0f + slope * slope);
   double ss = 0.0;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 sh = ld4(shift, i % ld4cols);
     const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i), pv = ld4(p_next, i);
-    float4 zn, qn, un, rn;
+    float4 zn, qn, un, rn, tn;
 #define PD_ZQU(f)                                                                   \
     {                                                                               \
       const float a = (rv.f - sh.f) + zv.f;                                         \
@@ -333,11 +335,12 @@ zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, 
       if (q_top >= 0.0f) { unsigned code; qq = quantize_one(qq, q_scale, q_lo, q_top, code); } \
       const float res = pv.f - qq;                                                  \
       zn.f = zz; qn.f = qq; un.f = fmaf(rho, res, uv.f); rn.f = a - zz;             \
+      tn.f = fmaf(rho, res, un.f);                                                  \
       ss += (double)res * res;                                                      \
     }
     PD_ZQU(x) PD_ZQU(y) PD_ZQU(z) PD_ZQU(w)
 #undef PD_ZQU
-    st4(z, i, zn); st4(q, i, qn); st4(u, i, un); st4(r, i, rn);
+    st4(z, i, zn); st4(q, i, qn); st4(u, i, un); st4(r, i, rn); st4(t_next, i, tn);
   }
   const double tot = block_sum<EW_THREADS>(ss, red);
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
@@ -411,6 +414,20 @@ zlast_kernel(float *__restrict__ r, float *__restrict__ z, const float *__restri
     const float zn = (float)x[c];
     zj[c] = zn;
     rj[c] = (float)(a[c] - (double)zn);
+  }
+}
+
+// t = u + rho (p - q) from the stored iterates (after the start or after the caller has set a tensor); the same
+// operations as in zqu_kernel, so both give the same bits.
+__global__ void __launch_bounds__(EW_THREADS)
+gradp_const_kernel(const float *__restrict__ u, const float *__restrict__ p, const float *__restrict__ q, float rho,
+                   float *__restrict__ t, size_t n4) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 uv = ld4(u, i), pv = ld4(p, i), qv = ld4(q, i);
+    float4 tv;
+    tv.x = fmaf(rho, pv.x - qv.x, uv.x); tv.y = fmaf(rho, pv.y - qv.y, uv.y);
+    tv.z = fmaf(rho, pv.z - qv.z, uv.z); tv.w = fmaf(rho, pv.w - qv.w, uv.w);
+    st4(t, i, tv);
   }
 }
 

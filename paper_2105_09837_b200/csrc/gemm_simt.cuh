@@ -72,34 +72,22 @@ struct EpiBiasAct {           // C = acc + b[col], then f (ReLU, leaky with `slo
   }
   __device__ __forceinline__ float4 operator()(int, int col, float4 a, double &) const { return apply(col, a, nullptr); }
 };
-struct EpiGradP {             // C = nu*acc + U + rho*(P - Q), accumulates sum(C^2)
+struct EpiGradT {             // C = nu*acc + T, accumulates sum(C^2); T = u_{l-1} + rho (p_l - q_{l-1}) is kept
+                              // up to date by the kernel that updates q and u (p-gradient of Eq. "update p")
   static constexpr bool kDirect = false, kSumsq = true;
-  static constexpr int kInputs = 3;
-  float *C; int ldc; const float *U, *P, *Q; float nu, rho;
+  static constexpr int kInputs = 1;
+  float *C; int ldc; const float *T; float nu;
   __device__ __forceinline__ void load(int row, int col, float4 *in) const {
-    const size_t o = (size_t)row * ldc + col;
-    in[0] = *reinterpret_cast<const float4 *>(U + o);
-    in[1] = *reinterpret_cast<const float4 *>(P + o);
-    in[2] = *reinterpret_cast<const float4 *>(Q + o);
+    in[0] = *reinterpret_cast<const float4 *>(T + (size_t)row * ldc + col);
   }
   __device__ __forceinline__ float4 apply(int, float4 a, const float4 *in) const {
-    return make_float4(nu * a.x + in[0].x + rho * (in[1].x - in[2].x), nu * a.y + in[0].y + rho * (in[1].y - in[2].y),
-                       nu * a.z + in[0].z + rho * (in[1].z - in[2].z), nu * a.w + in[0].w + rho * (in[1].w - in[2].w));
+    return make_float4(fmaf(nu, a.x, in[0].x), fmaf(nu, a.y, in[0].y), fmaf(nu, a.z, in[0].z), fmaf(nu, a.w, in[0].w));
   }
-  __device__ __forceinline__ void prefetch(int row, int col) const {
-    const size_t o = (size_t)row * ldc + col;
-    prefetch_l2(U + o); prefetch_l2(P + o); prefetch_l2(Q + o);
-  }
+  __device__ __forceinline__ void prefetch(int row, int col) const { prefetch_l2(T + (size_t)row * ldc + col); }
   __device__ __forceinline__ float4 operator()(int row, int col, float4 a, double &ss) const {
-    const size_t o = (size_t)row * ldc + col;
-    const float4 u = *reinterpret_cast<const float4 *>(U + o);
-    const float4 p = *reinterpret_cast<const float4 *>(P + o);
-    const float4 q = *reinterpret_cast<const float4 *>(Q + o);
-    float4 g;
-    g.x = nu * a.x + u.x + rho * (p.x - q.x);
-    g.y = nu * a.y + u.y + rho * (p.y - q.y);
-    g.z = nu * a.z + u.z + rho * (p.z - q.z);
-    g.w = nu * a.w + u.w + rho * (p.w - q.w);
+    float4 in;
+    load(row, col, &in);
+    const float4 g = apply(col, a, &in);
     ss += (double)g.x * g.x + (double)g.y * g.y + (double)g.z * g.z + (double)g.w * g.w;
     return g;
   }

@@ -400,7 +400,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       } else {
         // Inputs of the epilogue are read with the same coalesced pattern as the output is written: the warp walks
         // over its rows four at a time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.  The
-        // loads of four steps are issued together (rows past the end are clamped, their results dropped).
+        // loads of four or eight steps are issued together (rows past the end are clamped, their results dropped).
         float *C = epi.C + (size_t)z * prm.c_split_stride;
         float ssf = 0.f;
 #pragma unroll
@@ -414,16 +414,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __syncwarp();
           const int col = n0 + chalf * 64 + h * 32 + 4 * (lane & 7);
           if (col < n_pad) {
+            constexpr int BATCH = Epi::kInputs <= 1 ? 8 : 4;       // row steps whose loads are in flight together
 #pragma unroll
-            for (int s0 = 0; s0 < 8; s0 += 4) {
-              float4 in[4][Epi::kInputs > 0 ? Epi::kInputs : 1];
+            for (int s0 = 0; s0 < 8; s0 += BATCH) {
+              float4 in[BATCH][Epi::kInputs > 0 ? Epi::kInputs : 1];
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
+              for (int i = 0; i < BATCH; ++i) {
                 const int r = 4 * (s0 + i) + (lane >> 3);
                 epi.load(min(m0 + lane_base + r, prm.M - 1), col, in[i]);
               }
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
+              for (int i = 0; i < BATCH; ++i) {
                 const int r = 4 * (s0 + i) + (lane >> 3);
                 const int row = m0 + lane_base + r;
                 const float4 o = epi.apply(col, tr[r * 8 + ((lane & 7) ^ (r & 7))], in[i]);

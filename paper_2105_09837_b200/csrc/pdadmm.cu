@@ -56,6 +56,7 @@ struct Layer {
   float *b = nullptr;       // [ld_out]
   float *z = nullptr, *r = nullptr;          // [N][ld_out]
   float *q = nullptr, *u = nullptr;          // [N][ld_out], hidden layers only
+  float *t = nullptr;       // [N][ld_in], l >= 2: u_{l-1} + rho (p_l - q_{l-1}), the product-free part of grad_p phi
   float *gradW = nullptr;   // [n_out][ld_in]
   float *W_hi = nullptr, *W_lo = nullptr;   // tf32 split planes of W (tensor-core path)
   float *G_hi = nullptr, *G_lo = nullptr;   // tf32 split planes of grad_W
@@ -104,6 +105,7 @@ struct pdadmm_ctx {
   std::vector<pd::Layer> layers;
   pd::Scratch scr;
   bool r_valid = false;
+  bool t_valid = false;             // every layer's t matches the stored u, p, q
   int *d_flag = nullptr;            // device counter (z_L solver non-convergence)
   int *h_pinned = nullptr;          // pinned host words for small read-backs
   int64_t launches = 0;
@@ -347,9 +349,10 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   Scratch &s = c->scr;
   const int N = (int)c->N;
   int np = 0;
-  EpiGradP epi{s.s1, ly.ld_in, prev.u, ly.p, prev.q, c->nu, c->rho};
+  (void)prev;
+  EpiGradT epi{s.s1, ly.ld_in, ly.t, c->nu};
   PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
-                          epi, s.slots, &np, 3.0 * 4.0 * N * ly.n_in));
+                          epi, s.slots, &np, 4.0 * N * ly.n_in));
   int np2 = 0;
   double *slots_b = s.slots + s.n_slots / 2;          // second half of the slot buffer
   EpiStoreSumsq epi2{s.s2, ly.ld_out};
@@ -485,10 +488,11 @@ static void zqu_step(pdadmm_ctx *c, int l) {
     const size_t n4 = (size_t)N * ly.ld_out / 4;
     const int grid = ew_grid(n4);
     {
-      Launch k(c, KC_ZQU, s.st, 36.0 * N * ly.n_out, 0);
+      Launch k(c, KC_ZQU, s.st, 40.0 * N * ly.n_out, 0);
       const Layer &nx = c->layers[l + 1];
       zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu,
-                                               c->slope, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, s.slots);
+                                               c->slope, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, nx.t,
+                                               s.slots);
     }
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
@@ -686,6 +690,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &ly.r, e_out));
     if (l + 1 < c->L) { PD_TRY(dev_alloc(c, &ly.q, e_out)); PD_TRY(dev_alloc(c, &ly.u, e_out)); }
     if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in * c->code_bytes));
+    if (l > 0) PD_TRY(dev_alloc(c, &ly.t, (size_t)N * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.sc, 1));
     PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
     // node slices of the W-gradient product: enough blocks to fill the device twice, slices >= 256 nodes
@@ -814,6 +819,16 @@ static int ensure_residual(pdadmm_ctx *c) {
   if (!c->w_planes_valid) {
     for (auto &ly : c->layers) split_planes(c, c->scr.st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
     c->w_planes_valid = true;
+  }
+  if (!c->t_valid) {
+    for (int l = 1; l < c->L; ++l) {
+      Layer &ly = c->layers[l];
+      const Layer &pv = c->layers[l - 1];
+      const size_t n4 = (size_t)c->N * ly.ld_in / 4;
+      Launch k(c, KC_AXPY, c->scr.st, 16.0 * c->N * ly.n_in, 0);
+      gradp_const_kernel<<<ew_grid(n4), EW_THREADS, 0, c->scr.st>>>(pv.u, ly.p, pv.q, c->rho, ly.t, n4);
+    }
+    c->t_valid = true;
   }
   if (c->r_valid) return PDADMM_OK;
   for (int l = 0; l < c->L; ++l) PD_TRY(refresh_residual(c, c->layers[l], c->scr.st));
@@ -1056,6 +1071,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
   if (kind == PDADMM_T_X || kind == PDADMM_T_P || kind == PDADMM_T_W || kind == PDADMM_T_B || kind == PDADMM_T_Z)
     c->r_valid = false;
   if (kind == PDADMM_T_W) c->w_planes_valid = false;
+  if (kind == PDADMM_T_P || kind == PDADMM_T_Q || kind == PDADMM_T_U) c->t_valid = false;
   if (kind == PDADMM_T_P && c->levels && layer >= 2) {
     Layer &y = c->layers[layer - 1];
     const size_t n = (size_t)c->N * y.ld_in;

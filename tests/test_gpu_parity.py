@@ -376,3 +376,22 @@ def test_prediction_matches_the_oracle_forward_pass(case, levels, flags):
             assert np.array_equal(x, y)
     ctx.destroy()
     ref.destroy()
+
+
+@pytest.mark.parametrize("levels", [0, 16])
+def test_gradient_constant_kept_by_the_q_u_kernel_equals_the_recomputed_one(levels):
+    """t_l = u_{l-1} + rho (p_l - q_{l-1}) is written by the kernel that updates q and u and recomputed from the stored
+    iterates after the caller sets a tensor: both routes give the same bits, iteration after iteration."""
+    inp = _inputs("ba-ragged", quant_levels=levels)
+    a = B.from_inputs(inp)
+    b = B.from_inputs(inp)
+    for k in range(4):
+        a.step(1)
+        b.set_tensor(B.T_U, 1, b.get_tensor(B.T_U, 1))          # same values: only forces the recomputation
+        b.step(1)
+        sa, sb = U.read_state(a), U.read_state(b)
+        for name in ("p", "W", "b", "z", "q", "u"):
+            for x, y in zip(sa[name], sb[name]):
+                assert np.array_equal(x, y), f"{name} differs at iteration {k}"
+    a.destroy()
+    b.destroy()
