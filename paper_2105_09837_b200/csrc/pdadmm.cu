@@ -693,9 +693,20 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     if (l > 0) PD_TRY(dev_alloc(c, &ly.t, (size_t)N * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.sc, 1));
     PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
-    // node slices of the W-gradient product: enough blocks to fill the device twice, slices >= 256 nodes
+    // Node slices of the W-gradient product (slices >= 256 nodes, at most 32).  The persistent grid works through
+    // tiles x slices units in rounds of n_sms, so the count is chosen to fill its last round: the smallest number
+    // of slices within 3 % (relative) of the best fill (fewer slices = fewer partial tiles to write and add up).
     const int64_t tiles = ceil_div(ly.n_in, SG_BN) * ceil_div(ly.n_out, SG_BM);   // same tile for both kernels
-    int split = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(2 * 148, tiles), ceil_div(N, 256)));
+    const int max_split = (int)std::max<int64_t>(1, std::min<int64_t>(32, ceil_div(N, 256)));
+    auto slices_for = [&](int want) { return (int)ceil_div(N, round_up((int)ceil_div(N, want), TC_BK)); };
+    auto fill = [&](int want) {
+      const int64_t units = tiles * slices_for(want);
+      return (double)units / (double)(c->n_sms * ceil_div(units, c->n_sms));
+    };
+    double best = 0.0;
+    for (int w = 1; w <= max_split; ++w) best = std::max(best, fill(w));
+    int split = 1;
+    while (split < max_split && fill(split) < 0.97 * best) ++split;
     ly.k_chunk = round_up((int)ceil_div(N, split), TC_BK);      // multiple of both kernels' K blocks
     ly.n_split = (int)ceil_div(N, ly.k_chunk);
     max_part = std::max(max_part, (size_t)ly.n_split * ly.n_out * ly.ld_in);
