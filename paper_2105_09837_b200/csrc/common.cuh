@@ -44,6 +44,30 @@ inline int fail(int code, const char *fmt, ...) {
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// Exponent e of the scaling 2^e of a matrix whose largest magnitude has the bit pattern `amax_bits`:
+// max|x| 2^e lies in [2^14, 2^15), below the fp16 overflow threshold (the operands of the tensor-core products
+// are split into fp16 planes).  Zero, subnormal or non-finite maxima
+// take e = 0 (a NaN or Inf then travels through the product unchanged); |e| <= 100 so that 2^e is a normal float.
+__host__ __device__ __forceinline__ int tc_scale_exp(uint32_t amax_bits) {
+  const int E = (int)((amax_bits >> 23) & 0xFFu);
+  if (E == 0 || E == 255) return 0;
+  const int e = 14 - (E - 127);
+  return e < -100 ? -100 : (e > 100 ? 100 : e);
+}
+// ---- largest magnitude of an array, as a bit pattern ---------------------------------------------
+// The tensor-core products scale each operand by a power of two chosen from max|x|.  The maximum is kept as the
+// bit pattern of |x| in an unsigned word (for non-negative floats the integer order is the float order, a NaN
+// sorts above Inf), combined with atomicMax: the result does not depend on the order of the updates.
+__device__ __forceinline__ uint32_t abs_bits(float v) { return __float_as_uint(v) & 0x7FFFFFFFu; }
+__device__ __forceinline__ uint32_t abs_bits(float4 v) {
+  return max(max(abs_bits(v.x), abs_bits(v.y)), max(abs_bits(v.z), abs_bits(v.w)));
+}
+// called by the threads of a warp that are still running, each with its own maximum: one atomic per warp
+__device__ __forceinline__ void commit_amax(uint32_t m, uint32_t *__restrict__ word) {
+  const unsigned active = __activemask();
+  m = __reduce_max_sync(active, m);
+  if ((int)(threadIdx.x & 31) == __ffs(active) - 1 && m != 0u) atomicMax(word, m);
+}
 // ---- device reductions -------------------------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

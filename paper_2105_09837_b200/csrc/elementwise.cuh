@@ -7,11 +7,22 @@
 // depend on scheduling.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace pd {
 
 constexpr int EW_THREADS = 256;
+
+// ---- largest magnitude of an array (see commit_amax) ---------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+absmax_kernel(const float *__restrict__ x, size_t n4, uint32_t *__restrict__ word) {
+  uint32_t m = 0u;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x)
+    m = max(m, abs_bits(reinterpret_cast<const float4 *>(x)[i]));
+  commit_amax(m, word);
+}
 
 // Scalars of one layer that live on the device (so that an iteration needs no host round trip).
 struct LayerScalars {
@@ -68,25 +79,32 @@ __device__ __forceinline__ float quantize_one(float x, float s, float lo, float 
 // p-update  p+ = p - g/tau  (Eq. "update p") and the matching update of the linear residual,
 // r <- r - (W g)/tau, and r <- r - (grad_W p+)/theta after the W-update (Eq. "update W").
 __global__ void __launch_bounds__(EW_THREADS)
-axpy_neg_kernel(float *__restrict__ y, const float *__restrict__ x, const float *__restrict__ inv, size_t n4) {
+axpy_neg_kernel(float *__restrict__ y, const float *__restrict__ x, const float *__restrict__ inv, size_t n4,
+                uint32_t *__restrict__ amax /* receives max|y| (see commit_amax); may be null */) {
   const float a = *inv;
+  uint32_t m = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = ld4(y, i);
     const float4 w = ld4(x, i);
     v.x = fmaf(-a, w.x, v.x); v.y = fmaf(-a, w.y, v.y); v.z = fmaf(-a, w.z, v.z); v.w = fmaf(-a, w.w, v.w);
     st4(y, i, v);
+    m = max(m, abs_bits(v));
   }
+  if (amax != nullptr) commit_amax(m, amax);
 }
 
 // y += x   (r <- r + W d after an accepted quantised step)
 __global__ void __launch_bounds__(EW_THREADS)
-add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4) {
+add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4, uint32_t *__restrict__ amax) {
+  uint32_t m = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = ld4(y, i);
     const float4 w = ld4(x, i);
     v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
     st4(y, i, v);
+    m = max(m, abs_bits(v));
   }
+  if (amax != nullptr) commit_amax(m, amax);
 }
 
 // ---- quantised trial step ------------------------------------------------------------------------
@@ -94,10 +112,12 @@ add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4) {
 __global__ void __launch_bounds__(EW_THREADS)
 quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, const LayerScalars *__restrict__ sc,
                    float scale, float lo, int levels, float *__restrict__ p_new, float *__restrict__ d,
-                   void *__restrict__ codes, int wide_codes, size_t n4, double *__restrict__ slots) {
+                   void *__restrict__ codes, int wide_codes, size_t n4, double *__restrict__ slots,
+                   uint32_t *__restrict__ amax_p /* max|p_new|, may be null */, uint32_t *__restrict__ amax_d /* max|d| */) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_tau = sc->inv_tau, top = (float)(levels - 1);
   double ss = 0.0;
+  uint32_t mp = 0u, md = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 pv = ld4(p, i), gv = ld4(g, i);
     unsigned c0, c1, c2, c3;
@@ -110,11 +130,13 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
     ss += (double)dv.x * dv.x + (double)dv.y * dv.y + (double)dv.z * dv.z + (double)dv.w * dv.w;
     st4(p_new, i, nv);
     st4(d, i, dv);
+    mp = max(mp, abs_bits(nv)); md = max(md, abs_bits(dv));
     if (wide_codes)      // more than 256 levels: 16-bit codes
       reinterpret_cast<ushort4 *>(codes)[i] = make_ushort4((unsigned short)c0, (unsigned short)c1, (unsigned short)c2, (unsigned short)c3);
     else
       reinterpret_cast<uchar4 *>(codes)[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
   }
+  if (amax_p != nullptr) { commit_amax(mp, amax_p); commit_amax(md, amax_d); }
   const double tot = block_sum<EW_THREADS>(ss, red);
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
 }
@@ -153,7 +175,7 @@ __device__ __forceinline__ double block_sum_slots(const double *__restrict__ slo
 // tau = rho + nu ||W g||^2 / ||g||^2 : the smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
 __global__ void __launch_bounds__(256)
 finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots_g, int n_g, const double *slots_wg, int n_wg,
-                    int *nonfinite) {
+                    int *nonfinite, uint32_t *clear_word /* max|p| of the layer restarts with the coming p-step */) {
   __shared__ double sh[256];
   const double gg = block_sum_slots(slots_g, n_g, sh);
   const double wg = block_sum_slots(slots_wg, n_wg, sh);
@@ -166,6 +188,7 @@ finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots
     sc->inv_tau = (float)(1.0 / tau);
     sc->accepted = 0;
     sc->trials = 0;
+    if (clear_word != nullptr) *clear_word = 0u;
   }
 }
 // Stop condition of the quantised step in its quadratic form: nu||W d||^2 + rho||d||^2 <= tau||d||^2 (1 + slack).
@@ -192,7 +215,7 @@ finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack, con
 // theta = nu ||grad_W p+||^2 / ||grad_W||^2 : the smallest theta with phi(W+) <= V_l(W+; theta).
 __global__ void __launch_bounds__(256)
 finalize_theta_kernel(LayerScalars *sc, double nu, const double *slots_G, int n_G, const double *slots_Gp, int n_Gp,
-                      int *nonfinite) {
+                      int *nonfinite, uint32_t *clear_word /* max|r| of the layer restarts with the coming z-step */) {
   __shared__ double sh[256];
   const double GG = block_sum_slots(slots_G, n_G, sh);
   const double Gp = block_sum_slots(slots_Gp, n_Gp, sh);
@@ -203,27 +226,58 @@ finalize_theta_kernel(LayerScalars *sc, double nu, const double *slots_G, int n_
     const double theta = GG > 0.0 ? nu * Gp / GG : 0.0;
     sc->theta = theta;
     sc->inv_theta = theta > 0.0 ? (float)(1.0 / theta) : 0.0f;
+    if (clear_word != nullptr) *clear_word = 0u;
   }
 }
 
-// hi = value rounded to tf32 (11 significant bits), lo = value - hi (exact): the operand planes of the
-// tensor-core products for weight-sized matrices
-__device__ __forceinline__ void store_planes(float *__restrict__ hi, float *__restrict__ lo, size_t i, float4 v) {
-  float4 h;
-  h.x = __uint_as_float((__float_as_uint(v.x) + 0x1000u) & 0xFFFFE000u);
-  h.y = __uint_as_float((__float_as_uint(v.y) + 0x1000u) & 0xFFFFE000u);
-  h.z = __uint_as_float((__float_as_uint(v.z) + 0x1000u) & 0xFFFFE000u);
-  h.w = __uint_as_float((__float_as_uint(v.w) + 0x1000u) & 0xFFFFE000u);
-  st4(hi, i, h);
-  st4(lo, i, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
+// ---- fp16 operand planes of a weight-sized matrix --------------------------------------------------
+// x [rows][ld] fp32 -> hi, lo [rows][ldh] (same orientation) and, if asked for, hiT, loT [cols][ldhT] (transposed),
+// so that every tensor-core product finds its small operand contiguous along the contraction index.
+// xs = x 2^e with e from max|x| (`amax`, see tc_scale_exp); hi = xs rounded to 11 significant bits,
+// lo = (xs - hi) 2^11; e is stored in *exp_out for the products that use the planes.
+// One block of 32 x 8 threads per 32 x 32 tile.
+__global__ void __launch_bounds__(256)
+make_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, const uint32_t *__restrict__ amax,
+                   int *__restrict__ exp_out, __half *__restrict__ hi, __half *__restrict__ lo, int ldh,
+                   __half *__restrict__ hiT, __half *__restrict__ loT, int ldhT) {
+  __shared__ __half sh_hi[32][33], sh_lo[32][33];
+  const int e = tc_scale_exp(*amax);
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && threadIdx.y == 0) *exp_out = e;
+  const float scale = __uint_as_float((uint32_t)(e + 127) << 23);
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + threadIdx.y + 8 * i, c = c0 + threadIdx.x;
+    __half h = __float2half_rn(0.f), l = h;
+    if (r < rows && c < cols) {
+      const float xs = x[(size_t)r * ld + c] * scale;
+      const float hf = __uint_as_float((__float_as_uint(xs) + 0x1000u) & 0xFFFFE000u);
+      h = __float2half_rn(hf);
+      l = __float2half_rn((xs - hf) * 2048.0f);
+      if (hi != nullptr) { hi[(size_t)r * ldh + c] = h; lo[(size_t)r * ldh + c] = l; }
+    }
+    sh_hi[threadIdx.y + 8 * i][threadIdx.x] = h;
+    sh_lo[threadIdx.y + 8 * i][threadIdx.x] = l;
+  }
+  if (hiT == nullptr) return;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = c0 + threadIdx.y + 8 * i, r = r0 + threadIdx.x;
+    if (c < cols && r < rows) {
+      hiT[(size_t)c * ldhT + r] = sh_hi[threadIdx.x][threadIdx.y + 8 * i];
+      loT[(size_t)c * ldhT + r] = sh_lo[threadIdx.x][threadIdx.y + 8 * i];
+    }
+  }
 }
 
 // ---- reduction of the split partial tiles of grad_W, scaling by nu, ||grad_W||^2 ------------------
 __global__ void __launch_bounds__(EW_THREADS)
 reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, float nu, float *__restrict__ G,
-                    float *__restrict__ G_hi, float *__restrict__ G_lo, double *__restrict__ slots) {
+                    uint32_t *__restrict__ amax, double *__restrict__ slots) {
   __shared__ double red[EW_THREADS / 32];
   double ss = 0.0;
+  uint32_t m = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < n_split; ++s) {
@@ -233,8 +287,9 @@ reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, floa
     a.x *= nu; a.y *= nu; a.z *= nu; a.w *= nu;
     ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
     st4(G, i, a);
-    if (G_hi != nullptr) store_planes(G_hi, G_lo, i, a);      // tf32 planes for the tensor-core product G p+
+    m = max(m, abs_bits(a));
   }
+  if (amax != nullptr) commit_amax(m, amax);        // for the fp16 planes of the tensor-core product G p+
   const double tot = block_sum<EW_THREADS>(ss, red);
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
 }
@@ -314,10 +369,11 @@ __global__ void __launch_bounds__(EW_THREADS)
 zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
            const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
            float rho, float nu, float slope, float q_scale, float q_lo, float q_top, float *__restrict__ t_next,
-           double *__restrict__ slots) {
+           double *__restrict__ slots, uint32_t *__restrict__ amax_r /* max|r| (see commit_amax); may be null */) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_rn = 1.0f / (rho + nu), inv_neg = 1.0f / (2.0f + slope * slope);
   double ss = 0.0;
+  uint32_t mr = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 sh = ld4(shift, i % ld4cols);
     const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i), pv = ld4(p_next, i);
@@ -341,7 +397,9 @@ zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, 
     PD_ZQU(x) PD_ZQU(y) PD_ZQU(z) PD_ZQU(w)
 #undef PD_ZQU
     st4(z, i, zn); st4(q, i, qn); st4(u, i, un); st4(r, i, rn); st4(t_next, i, tn);
+    mr = max(mr, abs_bits(rn));
   }
+  if (amax_r != nullptr) commit_amax(mr, amax_r);
   const double tot = block_sum<EW_THREADS>(ss, red);
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
 }
@@ -355,7 +413,7 @@ constexpr int ZL_MAX_C = 64;
 __global__ void __launch_bounds__(128)
 zlast_kernel(float *__restrict__ r, float *__restrict__ z, const float *__restrict__ shift,
              const int *__restrict__ labels, const uint8_t *__restrict__ mask, int n_rows, int C, int ld,
-             double nu, int *__restrict__ not_converged) {
+             double nu, int *__restrict__ not_converged, uint32_t *__restrict__ amax_r /* max|r|, may be null */) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n_rows) return;
   float *rj = r + (size_t)j * ld, *zj = z + (size_t)j * ld;
@@ -410,11 +468,15 @@ zlast_kernel(float *__restrict__ r, float *__restrict__ z, const float *__restri
     }
     if (!done) atomicAdd(not_converged, 1);
   }
+  uint32_t mr = 0u;
   for (int c = 0; c < C; ++c) {
     const float zn = (float)x[c];
     zj[c] = zn;
-    rj[c] = (float)(a[c] - (double)zn);
+    const float rn = (float)(a[c] - (double)zn);
+    rj[c] = rn;
+    mr = max(mr, abs_bits(rn));
   }
+  if (amax_r != nullptr) commit_amax(mr, amax_r);
 }
 
 // t = u + rho (p - q) from the stored iterates (after the start or after the caller has set a tensor); the same
@@ -526,15 +588,17 @@ argmax_kernel(const float *__restrict__ z, const int *__restrict__ labels, const
 // W+ = W - grad_W * inv_theta  (Eq. "update W")
 __global__ void __launch_bounds__(EW_THREADS)
 wstep_kernel(float *__restrict__ W, const float *__restrict__ G, const LayerScalars *__restrict__ sc, size_t n4,
-             float *__restrict__ W_hi, float *__restrict__ W_lo) {
+             uint32_t *__restrict__ amax) {
   const float a = sc->inv_theta;
+  uint32_t m = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = ld4(W, i);
     const float4 g = ld4(G, i);
     v.x = fmaf(-a, g.x, v.x); v.y = fmaf(-a, g.y, v.y); v.z = fmaf(-a, g.z, v.z); v.w = fmaf(-a, g.w, v.w);
     st4(W, i, v);
-    if (W_hi != nullptr) store_planes(W_hi, W_lo, i, v);
+    m = max(m, abs_bits(v));
   }
+  if (amax != nullptr) commit_amax(m, amax);        // max|W+| for the fp16 planes of the tensor-core products
 }
 
 }  // namespace pd

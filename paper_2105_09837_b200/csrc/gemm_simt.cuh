@@ -22,6 +22,7 @@ __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefe
 
 // kDirect: the output is the accumulator itself (the tensor-core kernel then stores the tile by TMA);
 // kSumsq: the epilogue accumulates the sum of squares of the output.
+// `amax` (epilogues that feed a later tensor-core product): word that receives max|C| as a bit pattern; may be null.
 struct EpiStore {             // C = acc
   static constexpr bool kDirect = true, kSumsq = false;
   static constexpr int kInputs = 0;
@@ -42,7 +43,7 @@ struct EpiStoreSumsq {        // C = acc, accumulates sum(acc^2)
 struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b - z)
   static constexpr bool kDirect = false, kSumsq = false;
   static constexpr int kInputs = 1;        // float4 loads per output group: load() fetches, apply() combines
-  float *C; int ldc; const float *bias; const float *Z;
+  float *C; int ldc; const float *bias; const float *Z; uint32_t *amax;
   __device__ __forceinline__ void prefetch(int row, int col) const { prefetch_l2(Z + (size_t)row * ldc + col); }
   __device__ __forceinline__ void load(int row, int col, float4 *in) const {
     in[0] = *reinterpret_cast<const float4 *>(Z + (size_t)row * ldc + col);
@@ -60,7 +61,7 @@ struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b
 struct EpiBiasAct {           // C = acc + b[col], then f (ReLU, leaky with `slope`) if relu != 0   (z = W p + b, p' = f(z))
   static constexpr bool kDirect = false, kSumsq = false;
   static constexpr int kInputs = 0;
-  float *C; int ldc; const float *bias; int relu; float slope;
+  float *C; int ldc; const float *bias; int relu; float slope; uint32_t *amax;
   __device__ __forceinline__ float f(float x) const { return x > 0.f ? x : slope * x; }
   __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ void load(int, int, float4 *) const {}
@@ -76,7 +77,7 @@ struct EpiGradT {             // C = nu*acc + T, accumulates sum(C^2); T = u_{l-
                               // up to date by the kernel that updates q and u (p-gradient of Eq. "update p")
   static constexpr bool kDirect = false, kSumsq = true;
   static constexpr int kInputs = 1;
-  float *C; int ldc; const float *T; float nu;
+  float *C; int ldc; const float *T; float nu; uint32_t *amax;
   __device__ __forceinline__ void load(int row, int col, float4 *in) const {
     in[0] = *reinterpret_cast<const float4 *>(T + (size_t)row * ldc + col);
   }

@@ -1,17 +1,26 @@
 // fp32-accurate dense products on the sm_100a tensor cores.
 //
-// Every product C = A * B is issued as three tf32 MMAs on an error-free split of the operands,
-//     x = x_hi + x_lo,  x_hi = x rounded to tf32 (11 significant bits),  x_lo = x - x_hi (exact),
-//     A * B ~= A_hi B_hi + A_hi B_lo + A_lo B_hi            (the dropped A_lo B_lo term is below 2^-24 relative),
-// accumulated in fp32 in tensor memory.  TMA brings fp32 tiles into 128-byte-swizzled shared memory; four
-// converter warps split the streamed operand in place (hi) and into a second buffer (lo); the small operand
-// (a weight matrix) arrives as two precomputed planes.  One thread issues tcgen05.mma; completion is tracked
-// with mbarriers; four more warps read each K block's partial product from tensor memory (each warp its own
-// 32 lanes), add it to a register accumulator and finally apply the fused epilogue.
+// Every product C = A * B is issued as three fp16 MMAs on a scaled two-term split of the operands,
+//     xs = x * 2^e                      (e per matrix, from max|x|, so that max|xs| lies in [2^14, 2^15))
+//     x_hi = xs rounded to 11 significant bits      (exact in fp16 down to 2^-14)
+//     x_lo = (xs - x_hi) * 2^11, rounded to fp16    (xs - x_hi is exact in fp32; the factor keeps it out of the
+//                                                    fp16 subnormals, so the pair carries 22 bits down to 2^-14
+//                                                    and at least 11 bits down to 2^-25 of the scaled range)
+//     A * B ~= 2^-(eA+eB) [ A_hi B_hi + 2^-11 (A_hi B_lo + A_lo B_hi) ]      (the dropped lo*lo term is 2^-24 relative)
+// Products of two 11-bit numbers are exact in the fp32 accumulator, so the split is as accurate as the same
+// split on tf32 operands at twice the tensor-core rate and half the shared-memory footprint per operand.
 //
-// Tile: 128 x 128 outputs per CTA, 32-float K blocks, 3 stages of 64 KB, two accumulator tiles in tensor memory.
+// TMA brings fp32 tiles of the node-sized operand into shared memory; converter warps turn them, in place,
+// into the two fp16 planes (K-major, 128-byte swizzle); the small operand (a weight matrix) arrives as two
+// precomputed fp16 planes.  One thread issues tcgen05.mma; completion is tracked with mbarriers; eight more
+// warps read each K block's main term from tensor memory, add it to a register accumulator and finally apply
+// the scaling and the fused epilogue.
+//
+// Tile: 128 x 128 outputs per CTA, 64-deep K blocks, 3 stages of 64 KB, four accumulator tiles in tensor memory.
 // Every wait is bounded; a wait that expires raises an error word in global memory and the CTA drains and exits.
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 #include "gemm_simt.cuh"   // epilogue functors
@@ -19,27 +28,41 @@
 
 namespace pd {
 
-constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 32, TC_STAGES = 3;
+constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64, TC_STAGES = 3;
+constexpr int TC_KSTEPS = TC_BK / 16;                          // MMAs (K = 16) per pair of planes and K block
 constexpr int TC_FLUSH = 1;                                    // K blocks per read-out of the main accumulator
-constexpr int TC_TILE_BYTES = 128 * TC_BK * 4;                 // 16 KB: one 128 x 32 fp32 operand tile
-constexpr int TC_MN_CHUNK = TC_BK * 128;                       // MN-major tiles: 32 output indices x TC_BK rows
-constexpr int TC_STAGE_BYTES = 4 * TC_TILE_BYTES;              // A_hi, A_lo, B_hi, B_lo
-// warp 0: TMA, warp 1: MMA, then 4 (8) operand-split warps, then 8 accumulate + epilogue warps
-// (two warps per 32-lane quarter of tensor memory, 64 columns each)
-constexpr int TC_THREADS = 448;                                // 576 when both operands are split in the kernel
-// number of operand-split warps: twice as many when both operands are split in shared memory (the contraction over
-// nodes), where the split and not the MMA issue sets the pace
-__host__ __device__ constexpr int tc_conv_warps(bool b_split) { return b_split ? 8 : 4; }
-__host__ __device__ constexpr int tc_threads(bool b_split) { return 32 * (2 + tc_conv_warps(b_split) + 8); }
+constexpr int TC_PLANE_BYTES = 128 * TC_BK * 2;                // 16 KB: one 128 x 64 fp16 operand plane
+constexpr int TC_STAGE_BYTES = 4 * TC_PLANE_BYTES;             // A_hi, A_lo, B_hi, B_lo (= two fp32 tiles of 128 x 64)
+// warp 0: TMA, warp 1: MMA, then 8 converter warps (all on A, or four on each of A and B), then 8 accumulate +
+// epilogue warps (two warps per 32-lane quarter of tensor memory, 64 columns each)
+constexpr int TC_CONV_WARPS = 8;
+constexpr int TC_THREADS = 32 * (2 + TC_CONV_WARPS + 8);      // 576
 constexpr int TC_ACC_THREADS = 256;
 constexpr int TC_ACC_BUFS = 3;                                 // main-term accumulator tiles in tensor memory
 constexpr int TC_TMEM_COLS = 512;                              // 3 main tiles + 1 correction tile
 constexpr int TC_TR_BYTES = 8 * 32 * 32 * 4;                   // epilogue transpose: 8 warps x 32 rows x 32 columns
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + TC_TR_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 
-// x_hi: x rounded to the nearest tf32 number (11 significant bits).  x_lo = x - x_hi is then exact in fp32,
-// at most 2^-12 |x| and of either sign, so what the MMA drops of it (its last bit) has no preferred direction.
-__host__ __device__ __forceinline__ uint32_t tf32_hi(uint32_t bits) { return (bits + 0x1000u) & 0xFFFFE000u; }
+__device__ __forceinline__ float tc_pow2(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
+
+// One scaled value -> its two planes (as floats that fp16 holds exactly inside the normal range).
+__device__ __forceinline__ void tc_split(float x, float scale, float &hi, float &lo) {
+  const float xs = x * scale;
+  hi = __uint_as_float((__float_as_uint(xs) + 0x1000u) & 0xFFFFE000u);     // 11 significant bits, nearest
+  lo = (xs - hi) * 2048.0f;
+}
+// Eight consecutive values -> 16 bytes of the hi plane and 16 bytes of the lo plane.
+__device__ __forceinline__ void tc_split8(const float (&x)[8], float scale, uint4 &h, uint4 &l) {
+  float hi[8], lo[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tc_split(x[i], scale, hi[i], lo[i]);
+  auto pack = [](float a, float b) {
+    const __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<const uint32_t *>(&v);
+  };
+  h = make_uint4(pack(hi[0], hi[1]), pack(hi[2], hi[3]), pack(hi[4], hi[5]), pack(hi[6], hi[7]));
+  l = make_uint4(pack(lo[0], lo[1]), pack(lo[2], lo[3]), pack(lo[4], lo[5]), pack(lo[6], lo[7]));
+}
 
 struct TcParams {
   int M, N, K;            // output rows, output columns, contraction length
@@ -47,6 +70,9 @@ struct TcParams {
   int n_split;            // number of contraction slices; slice z writes its own partial output
   size_t c_split_stride;  // elements between the partial outputs of consecutive slices
   int *error;             // set to 1 if a bounded wait expired
+  const uint32_t *amax_a; // bit pattern of max|A| (device word); nullptr = no scaling
+  const uint32_t *amax_b; // the same for B when B is converted in the kernel
+  const int *exp_b;       // scaling exponent stored with the precomputed planes of B
   // Tail balancing (n_split == 1 only): output tiles from tail_begin on are cut into tail_split contraction
   // slices, one work unit each, so that the last, partly filled round of the persistent grid is shorter.
   // A slice leaves its accumulators in tail_ws; the warp that finds itself last (tail_count) adds the slices
@@ -56,9 +82,10 @@ struct TcParams {
   int *tail_count;        // [tiles from tail_begin][8 warps], zero before and after every launch
 };
 
-// A_MN / B_MN: operand is stored contiguous along its output index (rows of the tile are K slices);
-//              otherwise contiguous along K.
-// B_SPLIT: B is one fp32 tensor split in shared memory like A; otherwise it arrives as two planes (map_b, map_blo).
+// MN = false: A is [M][K] fp32, contiguous along K (a node-major matrix, rows = nodes); B arrives as two fp16
+//              planes [N][K] (map_b = hi, map_blo = lo), contiguous along K.
+// MN = true:  both operands are fp32 and contiguous along their output index, A = [K][M], B = [K][N] (the
+//              contraction over nodes of the W-gradient); the converter warps transpose while they split.
 //
 // Persistent: the grid has at most one block per SM and block i works on output tiles i, i + gridDim.x, ...
 // (column tile fastest, so that neighbouring blocks share the streamed operand in L2).  All roles keep running
@@ -68,10 +95,10 @@ struct TcParams {
 // accumulator per MMA and always in the same direction.  To keep fp32-class accuracy the main term
 // A_hi B_hi is accumulated in tensor memory for ONE K block only (4 MMAs): after each block the accumulate
 // warps read it out and add it to a register accumulator with round-to-nearest, while the MMAs of the next
-// block fill the other buffer.  The two correction terms are 2^-12 of the main term, so they are summed over
-// the whole contraction in a third tensor-memory tile and added once at the end.
-template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
-__global__ void __launch_bounds__(tc_threads(B_SPLIT), 1)
+// block fill the other buffer.  The two correction terms are 2^-11 of the main term, so they are summed over
+// the whole contraction in a fourth tensor-memory tile and added once at the end.
+template <bool MN, class Epi>
+__global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_blo, const __grid_constant__ CUtensorMap map_c,
                const TcParams prm, Epi epi, double *__restrict__ partials) {
@@ -87,8 +114,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int ACC0 = 2 + tc_conv_warps(B_SPLIT);              // first accumulate warp
-  constexpr int CONV_T = 32 * tc_conv_warps(B_SPLIT);           // operand-split threads
+  constexpr int ACC0 = 2 + TC_CONV_WARPS;              // first accumulate warp
   const int tiles_n = (prm.N + TC_BN - 1) / TC_BN, tiles_m = (prm.M + TC_BM - 1) / TC_BM;
   const int n_out_tiles = tiles_n * tiles_m * prm.n_split;
   const bool tail_on = prm.tail_split > 1;
@@ -98,7 +124,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
-      ptx::mbar_init(&conv_bar[s], 32 * tc_conv_warps(B_SPLIT));
+      ptx::mbar_init(&conv_bar[s], 32 * TC_CONV_WARPS);
       ptx::mbar_init(&empty_bar[s], 1);
     }
     for (int b = 0; b < TC_ACC_BUFS; ++b) {
@@ -111,7 +137,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&map_a);
     ptx::prefetch_tmap(&map_b);
-    if (!B_SPLIT) ptx::prefetch_tmap(&map_blo);
+    if (!MN) ptx::prefetch_tmap(&map_blo);
     if (Epi::kDirect) ptx::prefetch_tmap(&map_c);
   }
   if (warp == 1) {
@@ -122,6 +148,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // scaling exponents of the two operands (written by earlier kernels of the stream)
+  const int exp_a = prm.amax_a ? tc_scale_exp(*prm.amax_a) : 0;
+  const int exp_b = MN ? (prm.amax_b ? tc_scale_exp(*prm.amax_b) : 0) : (prm.exp_b ? *prm.exp_b : 0);
 
   // work unit -> (row tile origin, column tile origin, first and number of K blocks); a unit is an output tile or,
   // in the tail, one contraction slice of an output tile
@@ -158,19 +187,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (use > 0 && !ptx::mbar_wait(&empty_bar[s], (use - 1) & 1, abort_flag)) { ok = false; break; }
           uint8_t *st = smem + s * TC_STAGE_BYTES;
           const int k0 = k_begin + kb * TC_BK;
-          ptx::mbar_expect_tx(&full_bar[s], (B_SPLIT ? 2 : 3) * TC_TILE_BYTES);
-          if (A_MN) {
-            ptx::tma_load_3d(st, &map_a, 0, k0, m0 / 32, &full_bar[s]);
+          ptx::mbar_expect_tx(&full_bar[s], TC_STAGE_BYTES);
+          if (MN) {
+            // fp32 [64 contraction rows][128 output indices], 512-byte rows, no swizzle (only the converters read it)
+            ptx::tma_load_2d(st, &map_a, m0, k0, &full_bar[s]);
+            ptx::tma_load_2d(st + 2 * TC_PLANE_BYTES, &map_b, n0, k0, &full_bar[s]);
           } else {
+            // fp32 [128 rows][64 floats] as two 128-byte-swizzled boxes of 32 floats; fp16 planes of B as they are used
             ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
-          }
-          uint8_t *bh = st + 2 * TC_TILE_BYTES, *bl = st + 3 * TC_TILE_BYTES;
-          if (B_MN) {
-            ptx::tma_load_3d(bh, &map_b, 0, k0, n0 / 32, &full_bar[s]);
-            if (!B_SPLIT) ptx::tma_load_3d(bl, &map_blo, 0, k0, n0 / 32, &full_bar[s]);
-          } else {
-            ptx::tma_load_2d(bh, &map_b, k0, n0, &full_bar[s]);
-            if (!B_SPLIT) ptx::tma_load_2d(bl, &map_blo, k0, n0, &full_bar[s]);
+            ptx::tma_load_2d(st + TC_PLANE_BYTES, &map_a, k0 + 32, m0, &full_bar[s]);
+            ptx::tma_load_2d(st + 2 * TC_PLANE_BYTES, &map_b, k0, n0, &full_bar[s]);
+            ptx::tma_load_2d(st + 3 * TC_PLANE_BYTES, &map_blo, k0, n0, &full_bar[s]);
           }
         }
       }
@@ -183,13 +210,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (one lane)
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_tf32(TC_BM, TC_BN, A_MN, B_MN);
+      constexpr uint32_t idesc = ptx::idesc_f16(TC_BM, TC_BN);
       const uint32_t d_corr = tmem_base + (uint32_t)(TC_ACC_BUFS * TC_BN);
       // descriptors: constant high words; the low word of stage 0 advances by whole stages / K steps
-      const uint32_t hi_a = ptx::smem_desc_hi(A_MN, TC_BK * 4), hi_b = ptx::smem_desc_hi(B_MN, TC_BK * 4);
-      const uint32_t lo_a0 = ptx::smem_desc_lo(ptx::smem_u32(smem), A_MN, TC_MN_CHUNK);
-      const uint32_t lo_b0 = ptx::smem_desc_lo(ptx::smem_u32(smem) + 2 * TC_TILE_BYTES, B_MN, TC_MN_CHUNK);
-      constexpr uint32_t step_a = (A_MN ? 1024u : 32u) >> 4, step_b = (B_MN ? 1024u : 32u) >> 4;
+      // (all four planes are K-major with 128-byte rows; 16 fp16 of K are 32 bytes)
+      const uint32_t hi_a = ptx::smem_desc_hi(false, TC_BK * 2), hi_b = hi_a;
+      const uint32_t lo_a0 = ptx::smem_desc_lo(ptx::smem_u32(smem), false, 0);
+      const uint32_t lo_b0 = ptx::smem_desc_lo(ptx::smem_u32(smem) + 2 * TC_PLANE_BYTES, false, 0);
+      constexpr uint32_t step_a = 32u >> 4, step_b = 32u >> 4;
       bool ok = true;
       // running state: stage s with phase bit sp, accumulator buffer b with phase bit bp (of its *previous* use),
       // and whether the barriers of the coming K block were already seen complete by the probe below
@@ -216,15 +244,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t bp_next = b + 1 == TC_ACC_BUFS ? bp ^ 1u : bp;
           const bool round_next = first_round && b + 1 != TC_ACC_BUFS;
 #pragma unroll
-          for (int kk = 0; kk < TC_BK / 8; ++kk) {
+          for (int kk = 0; kk < TC_KSTEPS; ++kk) {
             const uint64_t dah = ptx::smem_desc(hi_a, la + kk * step_a);
-            const uint64_t dal = ptx::smem_desc(hi_a, la + (TC_TILE_BYTES >> 4) + kk * step_a);
+            const uint64_t dal = ptx::smem_desc(hi_a, la + (TC_PLANE_BYTES >> 4) + kk * step_a);
             const uint64_t dbh = ptx::smem_desc(hi_b, lb + kk * step_b);
-            const uint64_t dbl = ptx::smem_desc(hi_b, lb + (TC_TILE_BYTES >> 4) + kk * step_b);
-            ptx::mma_tf32(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
-            ptx::mma_tf32(d_corr, dah, dbl, idesc, true);
-            ptx::mma_tf32(d, dah, dbh, idesc, !first || kk > 0);
-            if (kk == TC_BK / 8 - 2) {
+            const uint64_t dbl = ptx::smem_desc(hi_b, lb + (TC_PLANE_BYTES >> 4) + kk * step_b);
+            ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
+            ptx::mma_f16(d_corr, dah, dbl, idesc, true);
+            ptx::mma_f16(d, dah, dbh, idesc, !first || kk > 0);
+            if (kk == TC_KSTEPS - 2) {
               // probe the coming block's barriers while the tensor pipe still has work queued
               seen_conv = ptx::mbar_test_wait(&conv_bar[s_next], sp_next);
               seen_acc = last ? (round_next ? true : ptx::mbar_test_wait(&acc_empty[b_next], bp_next)) : true;
@@ -246,8 +274,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp < ACC0) {
-    // ---------------------------------------------------------------- operand split (128 or 256 threads)
-    const int t = threadIdx.x - 64;                       // 0 .. CONV_T-1
+    // ---------------------------------------------------------------- converters (256 threads)
+    // MN = false: all eight warps work on A; thread (row t, half h) reads the 32 fp32 values h*32 .. h*32+31 of
+    // row t.  MN = true: four warps per operand; thread t reads the 64 values of output index t (a column of the
+    // fp32 tile).  The group then waits until all of it has read (the planes overwrite the fp32 tile) and each
+    // thread writes its part of row t of the hi plane and of the lo plane, 16-byte chunk j at position
+    // j ^ (t mod 8) (the 128-byte swizzle).
+    constexpr int NV = MN ? TC_BK : TC_BK / 2;             // values per thread
+    const int ct = threadIdx.x - 64;                       // 0 .. 255
+    const int op = MN ? ct >> 7 : 0;                       // 0: A, 1: B
+    const int half = MN ? 0 : ct >> 7;
+    const int t = ct & 127;
+    const float scale = tc_pow2(op == 0 ? exp_a : exp_b);
+    const uint32_t sw = (uint32_t)(t & 7);
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -256,25 +295,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
         const int s = it % TC_STAGES, use = it / TC_STAGES;
         ok = ptx::mbar_wait(&full_bar[s], use & 1, abort_flag);
-        if (!ok) break;
-        uint8_t *st = smem + s * TC_STAGE_BYTES;
-        auto split = [&](uint8_t *hi_buf, uint8_t *lo_buf) {
-          uint4 *hi = reinterpret_cast<uint4 *>(hi_buf), *lo = reinterpret_cast<uint4 *>(lo_buf);
+        uint8_t *region = smem + s * TC_STAGE_BYTES + op * 2 * TC_PLANE_BYTES;
+        float v[NV];
+        if (!ok) {
+          // abandoned wait: still meet the group at its barrier below, which tells everyone to stop
+        } else if (MN) {
+          const float *raw = reinterpret_cast<const float *>(region);      // [64][128]
 #pragma unroll
-          for (int i = 0; i < TC_TILE_BYTES / 16 / CONV_T; ++i) {
-            const uint4 v = hi[t + CONV_T * i];
-            uint4 h, l;
-            h.x = tf32_hi(v.x); h.y = tf32_hi(v.y); h.z = tf32_hi(v.z); h.w = tf32_hi(v.w);
-            l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
-            l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
-            l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
-            l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
-            hi[t + CONV_T * i] = h;
-            lo[t + CONV_T * i] = l;
+          for (int k = 0; k < NV; ++k) v[k] = raw[k * 128 + t];
+        } else {
+#pragma unroll
+          for (int c = 0; c < NV / 4; ++c) {
+            const float4 q = *reinterpret_cast<const float4 *>(region + half * TC_PLANE_BYTES + t * 128 +
+                                                               (((uint32_t)c ^ sw) << 4));
+            v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
           }
-        };
-        split(st, st + TC_TILE_BYTES);
-        if (B_SPLIT) split(st + 2 * TC_TILE_BYTES, st + 3 * TC_TILE_BYTES);
+        }
+        // every thread of the group has read its values (or given up: then the whole group stops here)
+        if (ptx::named_barrier_or(1 + op, MN ? 128 : 256, !ok)) { ok = false; break; }
+#pragma unroll
+        for (int j = 0; j < NV / 8; ++j) {
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
+          uint4 h, l;
+          tc_split8(x, scale, h, l);
+          const uint32_t off = (uint32_t)t * 128u + (((uint32_t)(j + half * (NV / 8)) ^ sw) << 4);
+          *reinterpret_cast<uint4 *>(region + off) = h;
+          *reinterpret_cast<uint4 *>(region + TC_PLANE_BYTES + off) = l;
+        }
         ptx::fence_proxy_async_smem();
         ptx::mbar_arrive(&conv_bar[s]);
       }
@@ -302,25 +351,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       float acc[64];
 #pragma unroll
       for (int j = 0; j < 64; ++j) acc[j] = 0.f;
-      auto add_tile = [&](uint32_t col_base) {
+      auto add_tile = [&](uint32_t col_base, float w) {       // acc += w * tile (w = 1: plain add)
         const uint32_t src = tmem_base + ((uint32_t)lane_base << 16) + col_base + (uint32_t)(chalf * 64);
-        if constexpr (B_SPLIT) {
-          // 576 threads leave 96 registers per thread: 16 columns at a time
+        // 576 threads leave about 100 registers per thread: 16 columns at a time
 #pragma unroll
-          for (int h = 0; h < 4; ++h) {
-            uint32_t v[16];
-            ptx::tmem_ld16(src + 16u * h, v);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 16; ++j) acc[16 * h + j] += __uint_as_float(v[j]);
-          }
-        } else {
-          uint32_t v0[32], v1[32];
-          ptx::tmem_ld32(src, v0);
-          ptx::tmem_ld32(src + 32u, v1);
+        for (int h = 0; h < 4; ++h) {
+          uint32_t v[16];
+          ptx::tmem_ld16(src + 16u * h, v);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) { acc[j] += __uint_as_float(v0[j]); acc[32 + j] += __uint_as_float(v1[j]); }
+          for (int j = 0; j < 16; ++j) acc[16 * h + j] = fmaf(w, __uint_as_float(v[j]), acc[16 * h + j]);
         }
       };
       const int n_grp = (n_kb + TC_FLUSH - 1) / TC_FLUSH;
@@ -329,16 +369,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ok = ptx::mbar_wait(&acc_full[b], buse & 1, abort_flag);
         if (!ok) break;
         ptx::tc_fence_after_sync();
-        add_tile((uint32_t)(b * TC_BN));
+        add_tile((uint32_t)(b * TC_BN), 1.0f);
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(&acc_empty[b]);
       }
       if (!ok) break;
       if (n_kb > 0) {
         // correction terms: complete once the last block's commit has arrived (it covers every earlier MMA)
-        add_tile((uint32_t)(TC_ACC_BUFS * TC_BN));
+        add_tile((uint32_t)(TC_ACC_BUFS * TC_BN), 1.0f / 2048.0f);
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(corr_empty);
+        // undo the operand scalings (two exact factors, so that neither leaves the range on its own)
+        const int e1 = (exp_a + exp_b) / 2, e2 = exp_a + exp_b - e1;
+        const float u1 = tc_pow2(-e1), u2 = tc_pow2(-e2);
+#pragma unroll
+        for (int j = 0; j < 64; ++j) acc[j] = (acc[j] * u1) * u2;
       }
       int out_tile = tile;
       if (tile >= tail_begin) {
@@ -403,6 +448,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // loads of four or eight steps are issued together (rows past the end are clamped, their results dropped).
         float *C = epi.C + (size_t)z * prm.c_split_stride;
         float ssf = 0.f;
+        uint32_t mx = 0u;                  // largest magnitude stored by this thread
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           __syncwarp();
@@ -431,12 +477,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (row < prm.M) {
                   if (Epi::kSumsq) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
                   *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
+                  mx = max(mx, abs_bits(o));
                 }
               }
             }
           }
         }
         ss = (double)ssf;
+        if (epi.amax != nullptr) commit_amax(mx, epi.amax);      // the output is an operand of a later product
       }
       if (partials != nullptr) {          // one slot per tile and warp; the host adds the slots in index order
         ss = warp_sum(ss);
@@ -452,17 +500,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::tmem_dealloc(tmem_base, TC_TMEM_COLS);
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(prm.error, 1);
-}
-
-// x -> (x_hi, x_lo) planes of a small matrix (weights): x_hi = x rounded to tf32, x_lo = x - x_hi.
-__global__ void __launch_bounds__(256)
-split_planes_kernel(const float *__restrict__ x, float *__restrict__ hi, float *__restrict__ lo, size_t n) {
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    const float v = x[i];
-    const float h = __uint_as_float(tf32_hi(__float_as_uint(v)));
-    hi[i] = h;
-    lo[i] = v - h;
-  }
 }
 
 }  // namespace pd

@@ -43,11 +43,24 @@ enum KClass {
   KC_ZLAST,           // z update of the last layer
   KC_WSTEP,           // W -= G/theta
   KC_SMALL,           // single-block finalisers
+  KC_AMAX,            // largest magnitude of a product's node-sized operand (for its power-of-two scaling)
+  KC_PLANES,          // fp16 planes of a weight-sized operand
   KC_COUNT
 };
 static const char *kclass_names[KC_COUNT] = {
     "gemm_resid", "gemm_gradp", "gemm_wg", "gemm_gradw", "gradw_reduce", "gemm_gp", "axpy",
-    "quant_trial", "resid_colsum", "zqu", "zlast", "wstep", "finalize"};
+    "quant_trial", "resid_colsum", "zqu", "zlast", "wstep", "finalize", "absmax", "make_planes"};
+
+// fp16 hi/lo planes of a weight-sized matrix [rows][cols] for the tensor-core products, in the orientation(s)
+// in which it is contracted, and the exponent of the power-of-two scaling they were made with.
+struct Planes {
+  __half *hi = nullptr, *lo = nullptr;     // [rows][ldh], ldh = cols rounded up to 8
+  __half *hiT = nullptr, *loT = nullptr;   // [cols][ldhT], ldhT = rows rounded up to 8 (only where needed)
+  int ldh = 0, ldhT = 0;
+  int *exp = nullptr;                      // device word
+};
+// one operand of a tensor-core product as two fp16 planes [n][ld], contiguous along the contraction index
+struct PlaneRef { const __half *hi, *lo; int ld; const int *exp; };
 
 struct Layer {
   int n_in = 0, n_out = 0, ld_in = 0, ld_out = 0;
@@ -58,13 +71,17 @@ struct Layer {
   float *q = nullptr, *u = nullptr;          // [N][ld_out], hidden layers only
   float *t = nullptr;       // [N][ld_in], l >= 2: u_{l-1} + rho (p_l - q_{l-1}), the product-free part of grad_p phi
   float *gradW = nullptr;   // [n_out][ld_in]
-  float *W_hi = nullptr, *W_lo = nullptr;   // tf32 split planes of W (tensor-core path)
-  float *G_hi = nullptr, *G_lo = nullptr;   // tf32 split planes of grad_W
+  Planes Wp;                // fp16 planes of W: [n_out][ldh_in], and of W^T: [n_in][ldh_out] (tensor-core path)
+  Planes Gp;                // fp16 planes of grad_W: [n_out][ldh_in]
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in] codes of 1 byte (up to 256 levels) or 2 bytes, quantised mode, l >= 2
   float scale = 1.0f;       // level spacing s_l of p_l
   float lo = 0.0f;          // smallest level of p_l: -(levels below zero) * s_l
   LayerScalars *sc = nullptr;
+  // Largest magnitudes (bit patterns) of the two node-sized operands of this layer's products, kept by the kernels
+  // that write them: amax_p covers every p_l written since the last tau of the layer, amax_r every r_l written
+  // since its last theta -- upper bounds of the current maxima, which is all the power-of-two scaling needs.
+  uint32_t *amax_p = nullptr, *amax_r = nullptr;
   int n_split = 1, k_chunk = 0;
 };
 
@@ -80,6 +97,8 @@ struct Scratch {
   size_t n_slots = 0;
   float *tail_ws = nullptr; // accumulators of the contraction slices of tail tiles (one tile per SM at most)
   int *tail_count = nullptr;
+  uint32_t *amax_pool = nullptr;   // words for the largest magnitudes of product operands, handed out in stream order
+  int amax_next = 0;
 };
 
 struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
@@ -123,6 +142,7 @@ struct pdadmm_ctx {
   bool graph_failed = false;
   int n_sms = 148;
   bool w_planes_valid = false;
+  bool amax_p_valid = false;        // every layer's amax_p covers the stored p
   std::map<std::tuple<const void *, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t>, CUtensorMap> tmaps;
 };
 
@@ -198,39 +218,30 @@ static EncodeTiledFn encode_tiled_fn() {
   }();
   return fn;
 }
-// fp32 matrix with `inner` contiguous elements per row, `outer` rows, row stride `ld` elements; tiles of
-// box_inner x box_outer elements land in shared memory with the 128-byte swizzle; out-of-range elements read 0.
-// mn_major = the rows of the tile are K slices (tensor-core "MN-major" operand): 128-byte swizzle with 32-byte
-// atoms, the only shared-memory layout the tf32 MMA accepts for such operands; otherwise 16-byte atoms.
-static int get_tmap(pdadmm_ctx *c, const float *base, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_inner,
-                    uint32_t box_outer, bool mn_major, CUtensorMap *out) {
-  auto key = std::make_tuple((const void *)base, inner, outer, ld, box_inner, box_outer + (mn_major ? 1u << 16 : 0u));
+// Operand tiles of the tensor-core products; elements outside the matrix read as zero.
+//   TM_RAW_K:  fp32 [outer][inner], tile = box of 32 floats x 128 rows, 128-byte swizzle (the contraction index is the
+//              inner one; a 64-deep K block is two such boxes)
+//   TM_RAW_MN: fp32 [outer][inner], tile = 128 floats x 64 rows, no swizzle (the contraction index is the outer one;
+//              only the converter warps read it)
+//   TM_PLANE:  fp16 [outer][inner], tile = 64 halves x 128 rows, 128-byte swizzle (what the MMA reads)
+enum TmapKind { TM_RAW_K = 0, TM_RAW_MN = 1, TM_PLANE = 2 };
+static int get_tmap(pdadmm_ctx *c, const void *base, uint64_t inner, uint64_t outer, uint64_t ld, TmapKind kind,
+                    CUtensorMap *out) {
+  auto key = std::make_tuple(base, inner, outer, ld, (uint32_t)kind, 0u);
   auto it = c->tmaps.find(key);
   if (it != c->tmaps.end()) { *out = it->second; return PDADMM_OK; }
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled is not available in this driver");
+  const uint64_t esize = kind == TM_PLANE ? 2 : 4;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * esize};
+  cuuint32_t box[2] = {kind == TM_RAW_K ? 32u : (kind == TM_RAW_MN ? 128u : 64u), kind == TM_RAW_MN ? 64u : 128u};
+  cuuint32_t estr[2] = {1, 1};
   CUtensorMap m;
-  CUresult r;
-  if (mn_major) {
-    // rows = contraction index, `inner` output indices per row.  Seen as [inner / 32][outer][32] so that one copy
-    // brings four 32-wide column chunks, each as consecutive 128-byte rows (the layout of an MN-major operand).
-    // The last chunk may reach past the row end into the next row (or the slack after the allocation): those
-    // columns only feed output elements outside the matrix, which are never stored.
-    cuuint64_t dims[3] = {32, outer, (inner + 31) / 32};
-    cuuint64_t strides[2] = {ld * 4, 128};
-    cuuint32_t box[3] = {32, box_outer, 4};
-    cuuint32_t estr[3] = {1, 1, 1};
-    r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-           CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  } else {
-    cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {ld * 4};
-    cuuint32_t box[2] = {box_inner, box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-           box_inner * 4 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  }
+  const CUresult r = fn(&m, kind == TM_PLANE ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                        const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        kind == TM_RAW_MN ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
   if (c->tmaps.size() > 4096) c->tmaps.clear();
   c->tmaps[key] = m;
@@ -262,30 +273,85 @@ static int get_tmap_out(pdadmm_ctx *c, const float *base, uint64_t ld, uint64_t 
   return PDADMM_OK;
 }
 
-template <bool A_MN, bool B_MN, bool B_SPLIT, class Epi>
+template <bool MN, class Epi>
 static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mbl,
                      const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
   CUtensorMap mc = ma;                 // not used unless the epilogue stores the accumulator itself
   if (Epi::kDirect)
     PD_TRY(get_tmap_out(c, epi.C, (uint64_t)epi.ldc, (uint64_t)prm.M, (uint64_t)prm.n_split, prm.c_split_stride, &mc));
-  auto kern = gemm_tc_kernel<A_MN, B_MN, B_SPLIT, Epi>;
+  auto kern = gemm_tc_kernel<MN, Epi>;
   const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
   static bool configured = false;
   if (!configured) {
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     configured = true;
   }
-  kern<<<grid, tc_threads(B_SPLIT), TC_SMEM_BYTES, st>>>(ma, mb, mbl, mc, prm, epi, partials);
+  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, mc, prm, epi, partials);
+  return PDADMM_OK;
+}
+
+// ---- largest magnitudes of product operands ------------------------------------------------------------------
+// Each tensor-core product scales its operands by powers of two taken from their largest magnitudes.  The words
+// that receive them come from a pool that is cleared in stream order: at the start of every iteration (so that a
+// captured iteration always uses the same words) and whenever it runs out.
+constexpr int AMAX_POOL = 4096;
+static int amax_reset(pdadmm_ctx *c, cudaStream_t st) {
+  PD_CUDA(cudaMemsetAsync(c->scr.amax_pool, 0, AMAX_POOL * sizeof(uint32_t), st));
+  c->scr.amax_next = 0;
+  return PDADMM_OK;
+}
+// room for n more words that must stay valid together
+static int amax_reserve(pdadmm_ctx *c, cudaStream_t st, int n) {
+  if (c->scr.amax_next + n > AMAX_POOL) PD_TRY(amax_reset(c, st));
+  return PDADMM_OK;
+}
+static uint32_t *amax_take(pdadmm_ctx *c) { return c->scr.amax_pool + c->scr.amax_next++; }
+// max|x| of a matrix stored as n4 float4 values -> a fresh word
+static uint32_t *amax_of(pdadmm_ctx *c, cudaStream_t st, const float *x, size_t n4) {
+  uint32_t *w = amax_take(c);
+  Launch l(c, KC_AMAX, st, 16.0 * (double)n4, 0);
+  absmax_kernel<<<ew_grid(n4), EW_THREADS, 0, st>>>(x, n4, w);
+  return w;
+}
+
+// fp16 planes of x [rows][ld] (cols valid columns) from the largest magnitude in *amax
+static void make_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, int rows, int cols, int ld, const uint32_t *amax,
+                        Planes &pl) {
+  Launch l(c, KC_PLANES, st, (4.0 + 4.0 + (pl.hiT ? 4.0 : 0.0)) * rows * cols, 0);
+  const dim3 grid((unsigned)ceil_div(cols, 32), (unsigned)ceil_div(rows, 32));
+  make_planes_kernel<<<grid, dim3(32, 8), 0, st>>>(x, rows, cols, ld, amax, pl.exp, pl.hi, pl.lo, pl.ldh, pl.hiT, pl.loT,
+                                                   pl.ldhT);
+}
+// the same for a matrix whose largest magnitude is not known yet
+static int split_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, int rows, int cols, int ld, Planes &pl) {
+  if (!c->use_tc) return PDADMM_OK;
+  PD_TRY(amax_reserve(c, st, 1));
+  const uint32_t *w = amax_of(c, st, x, (size_t)rows * ld / 4);
+  make_planes(c, st, x, rows, cols, ld, w, pl);
+  return PDADMM_OK;
+}
+static int alloc_planes(pdadmm_ctx *c, int rows, int cols, bool transposed_too, bool natural, Planes *pl) {
+  pl->ldh = round_up(cols, 8); pl->ldhT = round_up(rows, 8);
+  if (natural) {
+    PD_TRY(dev_alloc(c, &pl->hi, (size_t)rows * pl->ldh));
+    PD_TRY(dev_alloc(c, &pl->lo, (size_t)rows * pl->ldh));
+  }
+  if (transposed_too) {
+    PD_TRY(dev_alloc(c, &pl->hiT, (size_t)cols * pl->ldhT));
+    PD_TRY(dev_alloc(c, &pl->loT, (size_t)cols * pl->ldhT));
+  }
+  PD_TRY(dev_alloc(c, &pl->exp, 1));
   return PDADMM_OK;
 }
 
 // ---- dense products --------------------------------------------------------------------------------------
 // C[M][N] = A[M][K] * op(B), fused epilogue; per-block sums of squares go to `partials` (or nullptr).
-// B is given by its fp32 matrix (CUDA-core path) and by its two tf32 planes (tensor-core path).
+// B is given by its fp32 matrix (CUDA-core path; B_NMAJOR tells its orientation) and by its two fp16 planes
+// [N][K] (tensor-core path).  `amax_a`: the largest magnitude of A if the caller has it, else it is computed here.
 template <bool B_NMAJOR, class Epi>
 static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
-                      const float *B, const float *B_hi, const float *B_lo, int ldb, const Epi &epi, double *partials,
-                      int *n_partials, double extra_bytes) {
+                      const float *B, int ldb, const PlaneRef &Bp, const Epi &epi, double *partials,
+                      int *n_partials, double extra_bytes, const uint32_t *amax_a = nullptr) {
   const double bytes = 4.0 * ((double)M * K + (double)N * K + (double)M * N) + extra_bytes;
   if (!c->use_tc) {
     dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM));
@@ -296,22 +362,21 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
   }
   const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM));
   if (n_partials) *n_partials = 8 * n_tiles;        // one slot per tile and epilogue warp
-  CUtensorMap ma, mb, mbl;
-  PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TC_BK, TC_BM, false, &ma));
-  if (B_NMAJOR) {
-    PD_TRY(get_tmap(c, B_hi, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mb));
-    PD_TRY(get_tmap(c, B_lo, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mbl));
-  } else {
-    PD_TRY(get_tmap(c, B_hi, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mb));
-    PD_TRY(get_tmap(c, B_lo, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, TC_BK, TC_BN, false, &mbl));
+  if (amax_a == nullptr) {
+    PD_TRY(amax_reserve(c, st, 1));
+    amax_a = amax_of(c, st, A, (size_t)M * lda / 4);
   }
-  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1};
+  CUtensorMap ma, mb, mbl;
+  PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TM_RAW_K, &ma));
+  PD_TRY(get_tmap(c, Bp.hi, (uint64_t)K, (uint64_t)N, (uint64_t)Bp.ld, TM_PLANE, &mb));
+  PD_TRY(get_tmap(c, Bp.lo, (uint64_t)K, (uint64_t)N, (uint64_t)Bp.ld, TM_PLANE, &mbl));
+  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1, amax_a, nullptr, Bp.exp};
   // The persistent grid works through the tiles in rounds of n_sms; a last round that fills only part of the
   // SMs costs as much as a full one, so its tiles are cut along the contraction into as many slices as fit.
   int n_units = n_tiles;
   const int tail = n_tiles % c->n_sms, n_kb = (int)ceil_div(K, TC_BK);
   if (tail > 0 && c->scr.tail_ws != nullptr) {
-    const int split = std::min(std::min(c->n_sms / tail, n_kb / 4), 8);     // at least 4 K blocks per slice
+    const int split = std::min(std::min(c->n_sms / tail, n_kb / 2), 8);     // at least 2 K blocks per slice
     if (split > 1) {
       prm.tail_begin = n_tiles - tail; prm.tail_split = split;
       prm.tail_ws = c->scr.tail_ws; prm.tail_count = c->scr.tail_count;
@@ -319,14 +384,24 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     }
   }
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
-  return launch_tc<false, B_NMAJOR, false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, n_units);
+  return launch_tc<false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, n_units);
 }
 
-// hi/lo planes of a weight-sized matrix for the tensor-core path
-static void split_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, float *hi, float *lo, size_t n) {
-  if (!c->use_tc) return;
-  Launch l(c, KC_SMALL, st, 12.0 * n, 0);
-  split_planes_kernel<<<(int)std::min<size_t>(ceil_div((int64_t)n, 256), 1024), 256, 0, st>>>(x, hi, lo, n);
+// C parts [n_split][M][ldc] = A^T B over node slices: A = [K][lda] (M valid columns), B = [K][ldb] (N valid columns)
+static int gemm_over_nodes_tc(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
+                              const float *B, int ldb, float *part, int ldc, int k_chunk, int n_split,
+                              const uint32_t *wa = nullptr, const uint32_t *wb = nullptr) {
+  const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM)) * n_split;
+  PD_TRY(amax_reserve(c, st, 2));
+  if (wa == nullptr) wa = amax_of(c, st, A, (size_t)K * lda / 4);
+  if (wb == nullptr) wb = amax_of(c, st, B, (size_t)K * ldb / 4);
+  CUtensorMap ma, mb;
+  PD_TRY(get_tmap(c, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, TM_RAW_MN, &ma));
+  PD_TRY(get_tmap(c, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, TM_RAW_MN, &mb));
+  TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1, wa, wb, nullptr};
+  EpiStore epi{part, ldc};
+  Launch k(c, cls, st, 4.0 * ((double)K * N + (double)K * M), 2.0 * K * N * M);
+  return launch_tc<true, EpiStore>(c, st, ma, mb, mb, prm, epi, nullptr, n_tiles);
 }
 
 }  // namespace pd
@@ -335,11 +410,23 @@ namespace pd {
 
 // ---- pieces of one iteration -------------------------------------------------------------------------------
 
+// planes of W_l as the operand of a product with rows n_out contracted over n_in (P W^T, g W^T) ...
+static PlaneRef planes_W(const Layer &ly) { return PlaneRef{ly.Wp.hi, ly.Wp.lo, ly.Wp.ldh, ly.Wp.exp}; }
+// ... and of W_l^T, rows n_in contracted over n_out (r W)
+static PlaneRef planes_WT(const Layer &ly) { return PlaneRef{ly.Wp.hiT, ly.Wp.loT, ly.Wp.ldhT, ly.Wp.exp}; }
+static PlaneRef planes_G(const Layer &ly) { return PlaneRef{ly.Gp.hi, ly.Gp.lo, ly.Gp.ldh, ly.Gp.exp}; }
+
 // r_l = P_l W_l^T + b_l - z_l from scratch (only when the cached residual is not valid).
 static int refresh_residual(pdadmm_ctx *c, Layer &ly, cudaStream_t st) {
-  EpiLinearResidual epi{ly.r, ly.ld_out, ly.b, ly.z};
-  return gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)c->N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.W_hi, ly.W_lo,
-                           ly.ld_in, epi, nullptr, nullptr, 4.0 * c->N * ly.n_out);
+  PD_CUDA(cudaMemsetAsync(ly.amax_r, 0, sizeof(uint32_t), st));
+  EpiLinearResidual epi{ly.r, ly.ld_out, ly.b, ly.z, ly.amax_r};
+  PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)c->N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in,
+                           planes_W(ly), epi, nullptr, nullptr, 4.0 * c->N * ly.n_out, ly.amax_p));
+  if (!c->use_tc) {       // the CUDA-core product does not track the maximum of what it stores
+    Launch l(c, KC_AMAX, st, 4.0 * c->N * ly.ld_out, 0);
+    absmax_kernel<<<ew_grid((size_t)c->N * ly.ld_out / 4), EW_THREADS, 0, st>>>(ly.r, (size_t)c->N * ly.ld_out / 4, ly.amax_r);
+  }
+  return PDADMM_OK;
 }
 
 // g = nu r W + u_{l-1} + rho (p - q_{l-1}) -> s1, ||g||^2 ; W g -> s2, ||W g||^2 ; tau.
@@ -350,17 +437,20 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   const int N = (int)c->N;
   int np = 0;
   (void)prev;
-  EpiGradT epi{s.s1, ly.ld_in, ly.t, c->nu};
-  PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
-                          epi, s.slots, &np, 4.0 * N * ly.n_in));
+  uint32_t *w_g = nullptr;                 // max|g|, kept by the epilogue that writes g
+  if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_g = amax_take(c); }
+  EpiGradT epi{s.s1, ly.ld_in, ly.t, c->nu, w_g};
+  PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.ld_in, planes_WT(ly),
+                          epi, s.slots, &np, 4.0 * N * ly.n_in, ly.amax_r));
   int np2 = 0;
   double *slots_b = s.slots + s.n_slots / 2;          // second half of the slot buffer
   EpiStoreSumsq epi2{s.s2, ly.ld_out};
-  PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
-                           epi2, slots_b, &np2, 0));
+  PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
+                           epi2, slots_b, &np2, 0, w_g));
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
-    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2);
+    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2,
+                                             ly.amax_p);
   }
   return PDADMM_OK;
 }
@@ -372,11 +462,11 @@ static void p_step_plain(pdadmm_ctx *c, int l) {
   const size_t n4p = (size_t)c->N * ly.ld_in / 4, n4r = (size_t)c->N * ly.ld_out / 4;
   {
     Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_in, 0);
-    axpy_neg_kernel<<<ew_grid(n4p), EW_THREADS, 0, s.st>>>(ly.p, s.s1, &ly.sc->inv_tau, n4p);
+    axpy_neg_kernel<<<ew_grid(n4p), EW_THREADS, 0, s.st>>>(ly.p, s.s1, &ly.sc->inv_tau, n4p, ly.amax_p);
   }
   {
     Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_out, 0);
-    axpy_neg_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, &ly.sc->inv_tau, n4r);
+    axpy_neg_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, &ly.sc->inv_tau, n4r, ly.amax_r);
   }
 }
 
@@ -390,16 +480,19 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
   const int max_trials = 30;
   for (int trial = 0;; ++trial) {
     const int grid = ew_grid(n4p);
+    uint32_t *w_d = nullptr;               // max|d| of this trial
+    if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_d = amax_take(c); }
     {
       Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
       quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
-                                                       s.codes_new, c->code_bytes == 2, n4p, s.slots);
+                                                       s.codes_new, c->code_bytes == 2, n4p, s.slots,
+                                                       c->use_tc ? ly.amax_p : nullptr, w_d);
     }
     int np = 0;
     double *slots_b = s.slots + s.n_slots / 2;
     EpiStoreSumsq epi{s.s2, ly.ld_out};
-    PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in, epi,
-                             slots_b, &np, 0));
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, planes_W(ly), epi,
+                             slots_b, &np, 0, w_d));
     {
       Launch k(c, KC_SMALL, s.st, 8.0 * (grid + np), 0);
       finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
@@ -415,7 +508,7 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
   std::swap(ly.codes, s.codes_new);
   {
     Launch k(c, KC_AXPY, s.st, 12.0 * N * ly.n_out, 0);
-    add_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, n4r);
+    add_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, n4r, ly.amax_r);
   }
   return PDADMM_OK;
 }
@@ -433,33 +526,33 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
                                                  s.part, ly.ld_in);
   } else {
     // both operands are node-major, i.e. contiguous along their output index: r is [nodes][n_out], p+ is [nodes][n_in]
-    const int n_tiles = (int)(ceil_div(ly.n_in, TC_BN) * ceil_div(ly.n_out, TC_BM)) * ly.n_split;
-    CUtensorMap ma, mb;
-    PD_TRY(get_tmap(c, ly.r, (uint64_t)ly.n_out, (uint64_t)N, (uint64_t)ly.ld_out, 32, TC_BK, true, &ma));
-    PD_TRY(get_tmap(c, ly.p, (uint64_t)ly.n_in, (uint64_t)N, (uint64_t)ly.ld_in, 32, TC_BK, true, &mb));
-    TcParams prm{ly.n_out, ly.n_in, N, ly.k_chunk, ly.n_split, (size_t)ly.n_out * ly.ld_in, c->d_flag + 1};
-    EpiStore epi{s.part, ly.ld_in};
-    Launch k(c, KC_GEMM_GRADW, s.st, 4.0 * ((double)N * ly.n_in + (double)N * ly.n_out), 2.0 * N * ly.n_in * ly.n_out);
-    PD_TRY((launch_tc<true, true, true, EpiStore>(c, s.st, ma, mb, mb, prm, epi, nullptr, n_tiles)));
+    PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, s.st, ly.n_out, ly.n_in, N, ly.r, ly.ld_out, ly.p, ly.ld_in, s.part,
+                              ly.ld_in, ly.k_chunk, ly.n_split, ly.amax_r, ly.amax_p));
   }
   const size_t n4w = (size_t)ly.n_out * ly.ld_in / 4;
   const int gw = ew_grid(n4w);
   {
     Launch k(c, KC_GRADW_REDUCE, s.st, 4.0 * (ly.n_split + 1.0) * ly.n_out * ly.n_in, 0);
-    reduce_gradW_kernel<<<gw, EW_THREADS, 0, s.st>>>(s.part, ly.n_split, n4w, c->nu, ly.gradW, ly.G_hi, ly.G_lo, s.slots);
+    uint32_t *w = nullptr;
+    if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w = amax_take(c); }
+    reduce_gradW_kernel<<<gw, EW_THREADS, 0, s.st>>>(s.part, ly.n_split, n4w, c->nu, ly.gradW, w, s.slots);
+    if (c->use_tc) make_planes(c, s.st, ly.gradW, ly.n_out, ly.n_in, ly.ld_in, w, ly.Gp);
   }
   int np = 0;
   double *slots_b = s.slots + s.n_slots / 2;
   EpiStoreSumsq epi{s.s1, ly.ld_out};
-  PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.G_hi, ly.G_lo, ly.ld_in,
-                           epi, slots_b, &np, 0));
+  PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.ld_in, planes_G(ly),
+                           epi, slots_b, &np, 0, ly.amax_p));
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (gw + np), 0);
-    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2);
+    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2, ly.amax_r);
   }
   {
     Launch k(c, KC_WSTEP, s.st, 20.0 * ly.n_out * ly.n_in, 0);
-    wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w, ly.W_hi, ly.W_lo);
+    uint32_t *w = nullptr;
+    if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w = amax_take(c); }
+    wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w, w);
+    if (c->use_tc) make_planes(c, s.st, ly.W, ly.n_out, ly.n_in, ly.ld_in, w, ly.Wp);
   }
   const int n_blocks = (int)std::min<int64_t>(c->n_sms * 2, ceil_div(N, 16));
   const int rows_per_block = (int)ceil_div(N, n_blocks);
@@ -492,16 +585,17 @@ static void zqu_step(pdadmm_ctx *c, int l) {
       const Layer &nx = c->layers[l + 1];
       zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu,
                                                c->slope, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, nx.t,
-                                               s.slots);
+                                               s.slots, ly.amax_r);
     }
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
     zlast_kernel<<<(int)ceil_div(N, 128), 128, 0, s.st>>>(ly.r, ly.z, ly.shift, c->labels, c->mask, N, ly.n_out,
-                                                          ly.ld_out, (double)c->nu, c->d_flag);
+                                                          ly.ld_out, (double)c->nu, c->d_flag, ly.amax_r);
   }
 }
 
 static int iterate_once(pdadmm_ctx *c, bool *hit_cap) {
+  if (c->use_tc) PD_TRY(amax_reset(c, c->scr.st));
   // p-update of layers 2..L from the iterates of the previous iteration
   for (int l = 1; l < c->L; ++l) {
     PD_TRY(p_gradient_and_tau(c, l));
@@ -529,6 +623,7 @@ static int check_config(const pdadmm_config *cfg) {
   if (cfg->feat_dim < 1 || !cfg->features) return fail(PDADMM_EINVAL, "features missing");
   if (cfg->n_hops < 0 || cfg->n_hops > 16) return fail(PDADMM_EINVAL, "n_hops must be in [0, 16]");
   if (cfg->n_layers < 1 || !cfg->layer_widths || !cfg->init_W) return fail(PDADMM_EINVAL, "layers missing");
+  if (cfg->n_layers > 1024) return fail(PDADMM_EINVAL, "at most 1024 layers");
   if (cfg->n_classes < 2 || cfg->n_classes > ZL_MAX_C)
     return fail(PDADMM_EINVAL, "n_classes must be in [2, %d]", ZL_MAX_C);
   if (cfg->layer_widths[cfg->n_layers - 1] != cfg->n_classes)
@@ -679,10 +774,8 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &ly.W, (size_t)ly.n_out * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.gradW, (size_t)ly.n_out * ly.ld_in));
     if (c->use_tc) {
-      PD_TRY(dev_alloc(c, &ly.W_hi, (size_t)ly.n_out * ly.ld_in));
-      PD_TRY(dev_alloc(c, &ly.W_lo, (size_t)ly.n_out * ly.ld_in));
-      PD_TRY(dev_alloc(c, &ly.G_hi, (size_t)ly.n_out * ly.ld_in));
-      PD_TRY(dev_alloc(c, &ly.G_lo, (size_t)ly.n_out * ly.ld_in));
+      PD_TRY(alloc_planes(c, ly.n_out, ly.n_in, l > 0, true, &ly.Wp));     // W^T only where a p-gradient is taken
+      PD_TRY(alloc_planes(c, ly.n_out, ly.n_in, false, true, &ly.Gp));
     }
     PD_TRY(dev_alloc(c, &ly.b, (size_t)ly.ld_out));
     PD_TRY(dev_alloc(c, &ly.shift, (size_t)ly.ld_out));
@@ -692,6 +785,8 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in * c->code_bytes));
     if (l > 0) PD_TRY(dev_alloc(c, &ly.t, (size_t)N * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.sc, 1));
+    PD_TRY(dev_alloc(c, &ly.amax_p, 1));
+    PD_TRY(dev_alloc(c, &ly.amax_r, 1));
     PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
     // Node slices of the W-gradient product (slices >= 256 nodes, at most 32).  The persistent grid works through
     // tiles x slices units in rounds of n_sms, so the count is chosen to fill its last round: the smallest number
@@ -728,6 +823,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   if (c->use_tc) {
     PD_TRY(dev_alloc(c, &s.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
     PD_TRY(dev_alloc(c, &s.tail_count, (size_t)c->n_sms * 8));
+    PD_TRY(dev_alloc(c, &s.amax_pool, (size_t)AMAX_POOL));
   }
 
   // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
@@ -741,9 +837,10 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   for (int l = 0; l < c->L; ++l) {
     Layer &ly = c->layers[l];
     EpiStore epi{ly.z, ly.ld_out};
-    split_planes(c, st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
-    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.W_hi, ly.W_lo,
-                             ly.ld_in, epi, nullptr, nullptr, 0));
+    PD_TRY(split_planes(c, st, ly.W, ly.n_out, ly.n_in, ly.ld_in, ly.Wp));
+    absmax_kernel<<<ew_grid((size_t)N * ly.ld_in / 4), EW_THREADS, 0, st>>>(ly.p, (size_t)N * ly.ld_in / 4, ly.amax_p);
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
+                             epi, nullptr, nullptr, 0, ly.amax_p));
     if (l + 1 == c->L) break;
     Layer &nx = c->layers[l + 1];
     const size_t n4 = (size_t)N * ly.ld_out / 4;
@@ -770,6 +867,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   PD_CUDA(cudaGetLastError());
   c->r_valid = true;                        // z = W p + b exactly by construction, r = 0 (allocated as zero)
   c->w_planes_valid = true;
+  c->amax_p_valid = true;
   c->launches = 0;
   return PDADMM_OK;
 }
@@ -828,8 +926,17 @@ extern "C" int pdadmm_destroy(pdadmm_ctx *c) {
 
 static int ensure_residual(pdadmm_ctx *c) {
   if (!c->w_planes_valid) {
-    for (auto &ly : c->layers) split_planes(c, c->scr.st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
+    for (auto &ly : c->layers) PD_TRY(split_planes(c, c->scr.st, ly.W, ly.n_out, ly.n_in, ly.ld_in, ly.Wp));
     c->w_planes_valid = true;
+  }
+  if (!c->amax_p_valid) {
+    for (auto &ly : c->layers) {
+      const size_t n4 = (size_t)c->N * ly.ld_in / 4;
+      PD_CUDA(cudaMemsetAsync(ly.amax_p, 0, sizeof(uint32_t), c->scr.st));
+      Launch k(c, KC_AMAX, c->scr.st, 16.0 * n4, 0);
+      absmax_kernel<<<ew_grid(n4), EW_THREADS, 0, c->scr.st>>>(ly.p, n4, ly.amax_p);
+    }
+    c->amax_p_valid = true;
   }
   if (!c->t_valid) {
     for (int l = 1; l < c->L; ++l) {
@@ -949,7 +1056,7 @@ extern "C" int pdadmm_predict(pdadmm_ctx *c, float *logits_out, int32_t *pred_ou
   PD_CUDA(cudaSetDevice(c->device));
   cudaStream_t st = c->scr.st;
   if (!c->w_planes_valid) {
-    for (auto &ly : c->layers) split_planes(c, st, ly.W, ly.W_hi, ly.W_lo, (size_t)ly.n_out * ly.ld_in);
+    for (auto &ly : c->layers) PD_TRY(split_planes(c, st, ly.W, ly.n_out, ly.n_in, ly.ld_in, ly.Wp));
     c->w_planes_valid = true;
   }
   // forward pass with the constraints enforced: activations alternate between the two scratch matrices
@@ -957,12 +1064,20 @@ extern "C" int pdadmm_predict(pdadmm_ctx *c, float *logits_out, int32_t *pred_ou
   const float *in = c->layers[0].p;
   float *bufs[2] = {c->scr.s1, c->scr.s2};
   float *out = nullptr;
+  const uint32_t *w_in = nullptr;            // max|activations| of the layer's input
+  if (c->use_tc) {
+    PD_TRY(amax_reset(c, st));               // one word per layer output, all from one pass through the pool
+    w_in = amax_of(c, st, in, (size_t)N * c->layers[0].ld_in / 4);
+  }
   for (int l = 0; l < c->L; ++l) {
     Layer &ly = c->layers[l];
     out = bufs[l & 1];
-    EpiBiasAct epi{out, ly.ld_out, ly.b, l + 1 < c->L ? 1 : 0, c->slope};
-    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, N, ly.n_out, ly.n_in, in, ly.ld_in, ly.W, ly.W_hi, ly.W_lo, ly.ld_in,
-                             epi, nullptr, nullptr, 0));
+    uint32_t *w_out = nullptr;
+    if (c->use_tc) w_out = amax_take(c);
+    EpiBiasAct epi{out, ly.ld_out, ly.b, l + 1 < c->L ? 1 : 0, c->slope, w_out};
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, N, ly.n_out, ly.n_in, in, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
+                             epi, nullptr, nullptr, 0, w_in));
+    w_in = w_out;
     in = out;
   }
   const Layer &last = c->layers[c->L - 1];
@@ -1082,6 +1197,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
   if (kind == PDADMM_T_X || kind == PDADMM_T_P || kind == PDADMM_T_W || kind == PDADMM_T_B || kind == PDADMM_T_Z)
     c->r_valid = false;
   if (kind == PDADMM_T_W) c->w_planes_valid = false;
+  if (kind == PDADMM_T_X || kind == PDADMM_T_P) c->amax_p_valid = false;
   if (kind == PDADMM_T_P || kind == PDADMM_T_Q || kind == PDADMM_T_U) c->t_valid = false;
   if (kind == PDADMM_T_P && c->levels && layer >= 2) {
     Layer &y = c->layers[layer - 1];
@@ -1180,25 +1296,31 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
     const int a_rows = mode == 2 ? K : M, a_cols = mode == 2 ? M : K;
     const int b_rows = mode == 0 ? N : K, b_cols = mode == 0 ? K : N;
     const int lda = round_up(a_cols, 4), ldb = round_up(b_cols, 4), ldc = round_up(N, 4);
-    float *dA, *dB, *dBh, *dBl, *dC, *part = nullptr;
+    float *dA, *dB, *dC, *part = nullptr;
     double *slots;
+    Planes Bp;
     PD_TRY(dev_alloc(c, &dA, (size_t)a_rows * lda));
     PD_TRY(dev_alloc(c, &dB, (size_t)b_rows * ldb));
-    PD_TRY(dev_alloc(c, &dBh, (size_t)b_rows * ldb));
-    PD_TRY(dev_alloc(c, &dBl, (size_t)b_rows * ldb));
     PD_TRY(dev_alloc(c, &dC, (size_t)M * ldc));
     const int n_slots = 8 * (int)(ceil_div(M, 128) * ceil_div(N, 128)) + 2048;
     PD_TRY(dev_alloc(c, &slots, (size_t)n_slots));
     PD_TRY(upload_rows(st, dA, lda, A, a_cols, a_rows));
     PD_TRY(upload_rows(st, dB, ldb, B, b_cols, b_rows));
-    split_planes(c, st, dB, dBh, dBl, (size_t)b_rows * ldb);
+    if (c->use_tc) {
+      PD_TRY(dev_alloc(c, &c->scr.amax_pool, (size_t)AMAX_POOL));
+      // planes of B as [N][K]: B itself in mode 0, its transpose in mode 1
+      if (mode != 2) PD_TRY(alloc_planes(c, b_rows, b_cols, mode == 1, mode == 0, &Bp));
+      if (mode != 2) PD_TRY(split_planes(c, st, dB, b_rows, b_cols, ldb, Bp));
+    }
     int np = 0;
     if (mode == 0) {
       EpiStoreSumsq epi{dC, ldc};
-      PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, st, M, N, K, dA, lda, dB, dBh, dBl, ldb, epi, slots, &np, 0));
+      PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, st, M, N, K, dA, lda, dB, ldb, PlaneRef{Bp.hi, Bp.lo, Bp.ldh, Bp.exp}, epi,
+                               slots, &np, 0));
     } else if (mode == 1) {
       EpiStoreSumsq epi{dC, ldc};
-      PD_TRY(gemm_nodes<true>(c, KC_GEMM_WG, st, M, N, K, dA, lda, dB, dBh, dBl, ldb, epi, slots, &np, 0));
+      PD_TRY(gemm_nodes<true>(c, KC_GEMM_WG, st, M, N, K, dA, lda, dB, ldb, PlaneRef{Bp.hiT, Bp.loT, Bp.ldhT, Bp.exp}, epi,
+                              slots, &np, 0));
     } else {
       const int split = (int)std::max<int64_t>(1, std::min<int64_t>(8, ceil_div(K, 64)));
       const int k_chunk = round_up((int)ceil_div(K, split), TC_BK);
@@ -1208,17 +1330,11 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
         dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM), (unsigned)n_split);
         gemm_tn_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, k_chunk, dA, lda, dB, ldb, part, ldc);
       } else {
-        const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM)) * n_split;
-        CUtensorMap ma, mb;
-        PD_TRY(get_tmap(c, dA, (uint64_t)M, (uint64_t)K, (uint64_t)lda, 32, TC_BK, true, &ma));
-        PD_TRY(get_tmap(c, dB, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, TC_BK, true, &mb));
-        TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1};
-        EpiStore epi{part, ldc};
-        PD_TRY((launch_tc<true, true, true, EpiStore>(c, st, ma, mb, mb, prm, epi, nullptr, n_tiles)));
+        PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, st, M, N, K, dA, lda, dB, ldb, part, ldc, k_chunk, n_split));
       }
       const size_t n4 = (size_t)M * ldc / 4;
       np = ew_grid(n4);
-      reduce_gradW_kernel<<<np, EW_THREADS, 0, st>>>(part, n_split, n4, 1.0f, dC, nullptr, nullptr, slots);
+      reduce_gradW_kernel<<<np, EW_THREADS, 0, st>>>(part, n_split, n4, 1.0f, dC, nullptr, slots);
     }
     double *res = slots + n_slots - 1;
     reduce_slots_kernel<<<1, 256, 0, st>>>(slots, np, 1, 1, res);
