@@ -38,8 +38,11 @@ constexpr int TC_STAGE_BYTES = 4 * TC_PLANE_BYTES;             // A_hi, A_lo, B_
 constexpr int TC_CONV_WARPS = 8;
 constexpr int TC_THREADS = 32 * (2 + TC_CONV_WARPS + 8);      // 576
 constexpr int TC_ACC_THREADS = 256;
-constexpr int TC_ACC_BUFS = 3;                                 // main-term accumulator tiles in tensor memory
-constexpr int TC_TMEM_COLS = 512;                              // 3 main tiles + 1 correction tile
+constexpr int TC_ACC_BUFS = 2;                                 // main-term accumulator tiles in tensor memory
+constexpr int TC_A_SLOTS = 2;                                  // K blocks of A planes in tensor memory
+constexpr int TC_TMEM_COLS = 512;                              // 2 main tiles, 1 correction tile, 2 x (A_hi, A_lo)
+constexpr uint32_t TC_COL_CORR = TC_ACC_BUFS * TC_BN;          // first column of the correction tile
+constexpr uint32_t TC_COL_A = TC_COL_CORR + TC_BN;             // A slot a: columns + 64 a (hi), + 64 a + 32 (lo)
 constexpr int TC_TR_BYTES = 8 * 32 * 32 * 4;                   // epilogue transpose: 8 warps x 32 rows x 32 columns
 constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + TC_TR_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 
@@ -100,8 +103,7 @@ struct TcParams {
 template <bool MN, class Epi>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_blo, const __grid_constant__ CUtensorMap map_c,
-               const TcParams prm, Epi epi, double *__restrict__ partials) {
+               const __grid_constant__ CUtensorMap map_blo, const TcParams prm, Epi epi, double *__restrict__ partials) {
   if (*reinterpret_cast<volatile int *>(prm.error) != 0) return;   // an earlier block gave up: do not queue behind it
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -109,8 +111,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint64_t *bars = reinterpret_cast<uint64_t *>(tr_base + TC_TR_BYTES);
   uint64_t *full_bar = bars, *conv_bar = bars + TC_STAGES, *empty_bar = bars + 2 * TC_STAGES;
   uint64_t *acc_full = bars + 3 * TC_STAGES, *acc_empty = acc_full + TC_ACC_BUFS;
-  uint64_t *corr_empty = acc_empty + TC_ACC_BUFS, *drain_bar = corr_empty + 1;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(drain_bar + 1);
+  uint64_t *corr_empty = acc_empty + TC_ACC_BUFS, *drain_bar = corr_empty + 1, *a_empty = drain_bar + 1;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(a_empty + TC_A_SLOTS);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -133,12 +135,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     ptx::mbar_init(corr_empty, TC_ACC_THREADS);
     ptx::mbar_init(drain_bar, 1);
+    for (int a = 0; a < TC_A_SLOTS; ++a) ptx::mbar_init(&a_empty[a], 1);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&map_a);
     ptx::prefetch_tmap(&map_b);
     if (!MN) ptx::prefetch_tmap(&map_blo);
-    if (Epi::kDirect) ptx::prefetch_tmap(&map_c);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, TC_TMEM_COLS);
@@ -211,18 +213,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ---------------------------------------------------------------- MMA issuer (one lane)
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::idesc_f16(TC_BM, TC_BN);
-      const uint32_t d_corr = tmem_base + (uint32_t)(TC_ACC_BUFS * TC_BN);
-      // descriptors: constant high words; the low word of stage 0 advances by whole stages / K steps
-      // (all four planes are K-major with 128-byte rows; 16 fp16 of K are 32 bytes)
-      const uint32_t hi_a = ptx::smem_desc_hi(false, TC_BK * 2), hi_b = hi_a;
-      const uint32_t lo_a0 = ptx::smem_desc_lo(ptx::smem_u32(smem), false, 0);
+      const uint32_t d_corr = tmem_base + TC_COL_CORR;
+      // A: tensor memory, 8 columns per K step.  B: shared-memory descriptors with a constant high word; the low
+      // word of stage 0 advances by whole stages / K steps (K-major planes with 128-byte rows; 16 fp16 are 32 bytes)
+      const uint32_t hi_b = ptx::smem_desc_hi(false, TC_BK * 2);
       const uint32_t lo_b0 = ptx::smem_desc_lo(ptx::smem_u32(smem) + 2 * TC_PLANE_BYTES, false, 0);
-      constexpr uint32_t step_a = 32u >> 4, step_b = 32u >> 4;
+      constexpr uint32_t step_b = 32u >> 4;
       bool ok = true;
       // running state: stage s with phase bit sp, accumulator buffer b with phase bit bp (of its *previous* use),
       // and whether the barriers of the coming K block were already seen complete by the probe below
       int s = 0, b = 0, ti = 0;
-      uint32_t sp = 0, bp = 1;
+      uint32_t sp = 0, bp = 1, aslot = 0;
       bool first_round = true, seen_conv = false, seen_acc = false;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++ti) {
         int m0, n0, k_begin, n_kb, z;
@@ -235,7 +236,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (ok && first && !first_round && !seen_acc) ok = ptx::mbar_wait(&acc_empty[b], bp, abort_flag);
           if (!ok) break;
           ptx::tc_fence_after_sync();
-          const uint32_t la = lo_a0 + (uint32_t)s * (TC_STAGE_BYTES >> 4), lb = lo_b0 + (uint32_t)s * (TC_STAGE_BYTES >> 4);
+          const uint32_t ta = tmem_base + TC_COL_A + aslot * 64u, lb = lo_b0 + (uint32_t)s * (TC_STAGE_BYTES >> 4);
           const uint32_t d = tmem_base + (uint32_t)(b * TC_BN);
           // next K block's stage and, if it starts a new group, its accumulator buffer
           const int s_next = s + 1 == TC_STAGES ? 0 : s + 1;
@@ -245,13 +246,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const bool round_next = first_round && b + 1 != TC_ACC_BUFS;
 #pragma unroll
           for (int kk = 0; kk < TC_KSTEPS; ++kk) {
-            const uint64_t dah = ptx::smem_desc(hi_a, la + kk * step_a);
-            const uint64_t dal = ptx::smem_desc(hi_a, la + (TC_PLANE_BYTES >> 4) + kk * step_a);
+            const uint32_t ah = ta + 8u * kk, al = ah + 32u;
             const uint64_t dbh = ptx::smem_desc(hi_b, lb + kk * step_b);
             const uint64_t dbl = ptx::smem_desc(hi_b, lb + (TC_PLANE_BYTES >> 4) + kk * step_b);
-            ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
-            ptx::mma_f16(d_corr, dah, dbl, idesc, true);
-            ptx::mma_f16(d, dah, dbh, idesc, !first || kk > 0);
+            ptx::mma_f16_ts(d_corr, al, dbh, idesc, kb > 0 || kk > 0);
+            ptx::mma_f16_ts(d_corr, ah, dbl, idesc, true);
+            ptx::mma_f16_ts(d, ah, dbh, idesc, !first || kk > 0);
             if (kk == TC_KSTEPS - 2) {
               // probe the coming block's barriers while the tensor pipe still has work queued
               seen_conv = ptx::mbar_test_wait(&conv_bar[s_next], sp_next);
@@ -259,6 +259,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           }
           ptx::mma_commit(&empty_bar[s]);          // stage can be refilled once these MMAs have read it
+          ptx::mma_commit(&a_empty[aslot]);        // and so can the A planes' slot in tensor memory
+          aslot ^= 1u;
           if (last) {
             ptx::mma_commit(&acc_full[b]);         // this group's partial product is complete
             if (b + 1 == TC_ACC_BUFS) first_round = false;
@@ -275,18 +277,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else if (warp < ACC0) {
     // ---------------------------------------------------------------- converters (256 threads)
-    // MN = false: all eight warps work on A; thread (row t, half h) reads the 32 fp32 values h*32 .. h*32+31 of
-    // row t.  MN = true: four warps per operand; thread t reads the 64 values of output index t (a column of the
-    // fp32 tile).  The group then waits until all of it has read (the planes overwrite the fp32 tile) and each
-    // thread writes its part of row t of the hi plane and of the lo plane, 16-byte chunk j at position
-    // j ^ (t mod 8) (the 128-byte swizzle).
-    constexpr int NV = MN ? TC_BK : TC_BK / 2;             // values per thread
-    const int ct = threadIdx.x - 64;                       // 0 .. 255
-    const int op = MN ? ct >> 7 : 0;                       // 0: A, 1: B
-    const int half = MN ? 0 : ct >> 7;
-    const int t = ct & 127;
-    const float scale = tc_pow2(op == 0 ? exp_a : exp_b);
-    const uint32_t sw = (uint32_t)(t & 7);
+    // The planes of A go to tensor memory, where the MMA reads them without touching shared memory: row i of the
+    // tile lives in lane i, and a warp can only write the 32 lanes of its own quarter (warp index mod 4).  So two
+    // warps share a quarter: thread (row t = 32 (warp mod 4) + lane, half h) converts the 32 values h*32 .. h*32+31
+    // of the K block of row t and writes 16 + 16 columns.
+    // MN = false: the values come from the swizzled [128][64] fp32 tile (row t, 16-byte chunks).
+    // MN = true:  the tile is [64][128] (contraction index first), so the thread reads a column; and B is converted
+    //             too, in place in shared memory: thread (output index tb, half hb) reads its 32 values, all 256
+    //             threads wait until everyone has read (the planes overwrite the fp32 tile), then the thread writes
+    //             four 16-byte chunks of row tb of the hi and of the lo plane, chunk j at position j ^ (tb mod 8)
+    //             (the 128-byte swizzle).
+    const int cw = warp - 2;                               // 0 .. 7
+    const int quarter = warp & 3, half = cw >> 2;
+    const int t = quarter * 32 + lane;
+    const int ct = threadIdx.x - 64, tb = ct & 127, hb = ct >> 7;
+    const float scale_a = tc_pow2(exp_a), scale_b = tc_pow2(exp_b);
+    const uint32_t sw = (uint32_t)((MN ? tb : t) & 7);
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -295,36 +301,68 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
         const int s = it % TC_STAGES, use = it / TC_STAGES;
         ok = ptx::mbar_wait(&full_bar[s], use & 1, abort_flag);
-        uint8_t *region = smem + s * TC_STAGE_BYTES + op * 2 * TC_PLANE_BYTES;
-        float v[NV];
-        if (!ok) {
-          // abandoned wait: still meet the group at its barrier below, which tells everyone to stop
-        } else if (MN) {
-          const float *raw = reinterpret_cast<const float *>(region);      // [64][128]
+        uint8_t *stage = smem + s * TC_STAGE_BYTES;
+        const int aslot = it % TC_A_SLOTS, ause = it / TC_A_SLOTS;
+        if (ok && ause > 0) ok = ptx::mbar_wait(&a_empty[aslot], (ause - 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);                  // the tensor-memory stores below are warp-wide
+        if (ok) {
+          ptx::tc_fence_after_sync();
+          float v[32];
+          if (MN) {
+            const float *raw = reinterpret_cast<const float *>(stage);     // [64][128]
 #pragma unroll
-          for (int k = 0; k < NV; ++k) v[k] = raw[k * 128 + t];
-        } else {
+            for (int k = 0; k < 32; ++k) v[k] = raw[(32 * half + k) * 128 + t];
+          } else {
 #pragma unroll
-          for (int c = 0; c < NV / 4; ++c) {
-            const float4 q = *reinterpret_cast<const float4 *>(region + half * TC_PLANE_BYTES + t * 128 +
-                                                               (((uint32_t)c ^ sw) << 4));
-            v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
+            for (int c = 0; c < 8; ++c) {
+              const float4 q = *reinterpret_cast<const float4 *>(stage + half * TC_PLANE_BYTES + t * 128 +
+                                                                 (((uint32_t)c ^ sw) << 4));
+              v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
+            }
           }
-        }
-        // every thread of the group has read its values (or given up: then the whole group stops here)
-        if (ptx::named_barrier_or(1 + op, MN ? 128 : 256, !ok)) { ok = false; break; }
+          uint32_t hreg[16], lreg[16];
 #pragma unroll
-        for (int j = 0; j < NV / 8; ++j) {
-          float x[8];
+          for (int j = 0; j < 4; ++j) {
+            float x[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
-          uint4 h, l;
-          tc_split8(x, scale, h, l);
-          const uint32_t off = (uint32_t)t * 128u + (((uint32_t)(j + half * (NV / 8)) ^ sw) << 4);
-          *reinterpret_cast<uint4 *>(region + off) = h;
-          *reinterpret_cast<uint4 *>(region + TC_PLANE_BYTES + off) = l;
+            for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
+            uint4 h, l;
+            tc_split8(x, scale_a, h, l);
+            hreg[4 * j] = h.x; hreg[4 * j + 1] = h.y; hreg[4 * j + 2] = h.z; hreg[4 * j + 3] = h.w;
+            lreg[4 * j] = l.x; lreg[4 * j + 1] = l.y; lreg[4 * j + 2] = l.z; lreg[4 * j + 3] = l.w;
+          }
+          const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + TC_COL_A + (uint32_t)aslot * 64u +
+                               16u * (uint32_t)half;
+          ptx::tmem_st16(col, hreg);
+          ptx::tmem_st16(col + 32u, lreg);
         }
-        ptx::fence_proxy_async_smem();
+        if constexpr (MN) {
+          uint8_t *region = stage + 2 * TC_PLANE_BYTES;
+          const float *raw = reinterpret_cast<const float *>(region);      // [64][128]
+          float v[32];
+          if (ok) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) v[k] = raw[(32 * hb + k) * 128 + tb];
+          }
+          // everyone has read its values of B (or someone gave up: then all stop here)
+          if (ptx::named_barrier_or(1, 256, !ok)) { ok = false; break; }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
+            uint4 h, l;
+            tc_split8(x, scale_b, h, l);
+            const uint32_t off = (uint32_t)tb * 128u + (((uint32_t)(4 * hb + j) ^ sw) << 4);
+            *reinterpret_cast<uint4 *>(region + off) = h;
+            *reinterpret_cast<uint4 *>(region + TC_PLANE_BYTES + off) = l;
+          }
+          ptx::fence_proxy_async_smem();
+        } else if (!ok) {
+          break;
+        }
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before_sync();
         ptx::mbar_arrive(&conv_bar[s]);
       }
     }
@@ -376,7 +414,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!ok) break;
       if (n_kb > 0) {
         // correction terms: complete once the last block's commit has arrived (it covers every earlier MMA)
-        add_tile((uint32_t)(TC_ACC_BUFS * TC_BN), 1.0f / 2048.0f);
+        add_tile(TC_COL_CORR, 1.0f / 2048.0f);
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(corr_empty);
         // undo the operand scalings (two exact factors, so that neither leaves the range on its own)
@@ -411,41 +449,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       // Epilogue.  Thread i of the warp holds row (lane_base + i), 64 columns.  The warp's piece goes through shared
       // memory 32 columns at a time: thread i writes its 8 float4 groups with the group index XOR-ed by (i mod 8)
-      // (conflict-free 128-bit stores; this is also the 128-byte swizzle of the output tensor map).
+      // (conflict-free 128-bit stores), then the warp reads the piece back transposed, so that the output is written,
+      // and the inputs of the epilogue are read, in a coalesced pattern: the warp walks over its rows four at a
+      // time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.  The loads of four or eight steps
+      // are issued together (rows past the end are clamped, their results dropped).
       double ss = 0.0;
-      if constexpr (Epi::kDirect) {
-        // The output is the accumulator: sum of squares straight from the registers (four fp32 partial sums of 16
-        // squares each, added in double), and the 32 x 32 pieces leave shared memory as TMA stores, which clip at the
-        // matrix edges.  Rows and columns outside the matrix hold exact zeros (zero-filled operand tiles).
-        if constexpr (Epi::kSumsq) {
-          float s4[4] = {0.f, 0.f, 0.f, 0.f};
-          const int n_valid = prm.N - (n0 + chalf * 64);      // columns of this thread inside the matrix
-#pragma unroll
-          for (int j = 0; j < 64; ++j)
-            if (j < n_valid) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
-          ss = ((double)s4[0] + (double)s4[1]) + ((double)s4[2] + (double)s4[3]);
-        }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (lane == 0) ptx::bulk_wait_read();       // the previous store has read the staging buffer
-          __syncwarp();
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int jj = h * 8 + j;
-            tr[lane * 8 + (j ^ (lane & 7))] = make_float4(acc[4 * jj], acc[4 * jj + 1], acc[4 * jj + 2], acc[4 * jj + 3]);
-          }
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            const int x = n0 + chalf * 64 + h * 32, y = m0 + lane_base;
-            if (x < epi.ldc && y < prm.M) ptx::tma_store_3d(&map_c, tr, x, y, z);
-            ptx::bulk_commit();
-          }
-        }
-      } else {
-        // Inputs of the epilogue are read with the same coalesced pattern as the output is written: the warp walks
-        // over its rows four at a time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.  The
-        // loads of four or eight steps are issued together (rows past the end are clamped, their results dropped).
+      {
         float *C = epi.C + (size_t)z * prm.c_split_stride;
         float ssf = 0.f;
         uint32_t mx = 0u;                  // largest magnitude stored by this thread
@@ -467,31 +476,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
               for (int i = 0; i < BATCH; ++i) {
                 const int r = 4 * (s0 + i) + (lane >> 3);
-                epi.load(min(m0 + lane_base + r, prm.M - 1), col, in[i]);
+                if constexpr (!Epi::kDirect) epi.load(min(m0 + lane_base + r, prm.M - 1), col, in[i]);
               }
 #pragma unroll
               for (int i = 0; i < BATCH; ++i) {
                 const int r = 4 * (s0 + i) + (lane >> 3);
                 const int row = m0 + lane_base + r;
-                const float4 o = epi.apply(col, tr[r * 8 + ((lane & 7) ^ (r & 7))], in[i]);
+                float4 o = tr[r * 8 + ((lane & 7) ^ (r & 7))];
+                if constexpr (!Epi::kDirect) o = epi.apply(col, o, in[i]);
                 if (row < prm.M) {
                   if (Epi::kSumsq) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
                   *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
-                  mx = max(mx, abs_bits(o));
+                  if constexpr (!Epi::kDirect) mx = max(mx, abs_bits(o));
                 }
               }
             }
           }
         }
         ss = (double)ssf;
-        if (epi.amax != nullptr) commit_amax(mx, epi.amax);      // the output is an operand of a later product
+        if constexpr (!Epi::kDirect) {
+          if (epi.amax != nullptr) commit_amax(mx, epi.amax);      // the output is an operand of a later product
+        }
       }
       if (partials != nullptr) {          // one slot per tile and warp; the host adds the slots in index order
         ss = warp_sum(ss);
         if (lane == 0) partials[(size_t)out_tile * 8 + (warp - ACC0)] = ss;
       }
     }
-    if (Epi::kDirect && lane == 0) ptx::bulk_wait_all();
   }
   ptx::tc_fence_before_sync();
   __syncthreads();

@@ -249,36 +249,9 @@ static int get_tmap(pdadmm_ctx *c, const void *base, uint64_t inner, uint64_t ou
   return PDADMM_OK;
 }
 
-// Output of a product as a 3-D tensor [n_split][rows][ld] for the TMA stores of the epilogue: 32 x 32 boxes,
-// 128-byte swizzle (the layout the epilogue leaves in shared memory).
-static int get_tmap_out(pdadmm_ctx *c, const float *base, uint64_t ld, uint64_t rows, uint64_t n_split,
-                        uint64_t split_stride, CUtensorMap *out) {
-  auto key = std::make_tuple((const void *)base, ld, rows, n_split, 0xC0000000u, (uint32_t)(split_stride & 0xffffffffu));
-  auto it = c->tmaps.find(key);
-  if (it != c->tmaps.end()) { *out = it->second; return PDADMM_OK; }
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled is not available in this driver");
-  cuuint64_t dims[3] = {ld, rows, n_split};
-  cuuint64_t strides[2] = {ld * 4, (n_split > 1 ? split_stride : rows * ld) * 4};
-  cuuint32_t box[3] = {32, 32, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUtensorMap m;
-  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void *)base, dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return fail(PDADMM_ECUDA, "cuTensorMapEncodeTiled (output) failed with code %d", (int)r);
-  if (c->tmaps.size() > 4096) c->tmaps.clear();
-  c->tmaps[key] = m;
-  *out = m;
-  return PDADMM_OK;
-}
-
 template <bool MN, class Epi>
 static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mbl,
                      const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
-  CUtensorMap mc = ma;                 // not used unless the epilogue stores the accumulator itself
-  if (Epi::kDirect)
-    PD_TRY(get_tmap_out(c, epi.C, (uint64_t)epi.ldc, (uint64_t)prm.M, (uint64_t)prm.n_split, prm.c_split_stride, &mc));
   auto kern = gemm_tc_kernel<MN, Epi>;
   const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
   static bool configured = false;
@@ -286,7 +259,7 @@ static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, cons
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     configured = true;
   }
-  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, mc, prm, epi, partials);
+  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, prm, epi, partials);
   return PDADMM_OK;
 }
 
