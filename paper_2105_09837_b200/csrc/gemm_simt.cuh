@@ -179,7 +179,7 @@ gemm_nt_kernel(int M, int N, int K, const float *__restrict__ A, int lda, const 
   }
 
   double ss = 0.0;
-  const int n_pad = (N + 3) & ~3;
+  const int n_pad = epi.ldc;        // padding columns are written too: they come out as exact zeros
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int row = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
@@ -263,7 +263,7 @@ gemm_tn_kernel(int M, int N, int K, int k_chunk, const float *__restrict__ A, in
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int col = n0 + h * 64 + tx * 4;
-      if (col >= na) continue;
+      if (col >= ldc) continue;      // padding columns are written too (exact zeros)
       *reinterpret_cast<float4 *>(out + (size_t)row * ldc + col) =
           make_float4(acc[i][h * 4 + 0], acc[i][h * 4 + 1], acc[i][h * 4 + 2], acc[i][h * 4 + 3]);
     }

@@ -373,7 +373,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int lane_base = (warp & 3) * 32;
     const int chalf = (warp - ACC0) >> 2;
     float4 *tr = reinterpret_cast<float4 *>(tr_base) + (size_t)(warp - ACC0) * 32 * 8;    // 32 rows x 8 float4 per warp
-    const int n_pad = (prm.N + 3) & ~3;
+    // columns up to the leading dimension are written: those from N on come out as exact zeros (zero-filled
+    // operand rows, zero padding of the epilogue inputs), which keeps the padding of every matrix zero
+    const int n_pad = epi.ldc;
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {

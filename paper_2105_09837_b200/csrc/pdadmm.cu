@@ -1,7 +1,7 @@
 // pdADMM-G / pdADMM-G-Q on one B200: context, host orchestration of one iteration, C ABI.
 //
 // Data layout (device): every N x width matrix is node-major with its leading dimension padded to a
-// multiple of 4 floats and zero padding columns.  Per layer l the context keeps p_l, z_l, q_l, u_l,
+// multiple of 32 floats (128-byte rows) and zero padding columns.  Per layer l the context keeps p_l, z_l, q_l, u_l,
 // W_l, b_l and the linear residual r_l = W_l p_l + b_l - z_l, which every step of the iteration
 // updates in place instead of recomputing the product:
 //     p+ = p - g/tau        =>  r <- r - (W g)/tau            (pdADMM-G-Q: r <- r + W (p+ - p))
@@ -61,6 +61,10 @@ struct Planes {
 };
 // one operand of a tensor-core product as two fp16 planes [n][ld], contiguous along the contraction index
 struct PlaneRef { const __half *hi, *lo; int ld; const int *exp; };
+
+// Rows of every node-major matrix start on a 128-byte boundary (leading dimensions are multiples of 32 floats):
+// tile copies and the coalesced stores of the epilogues then move whole 32-byte sectors.
+constexpr int LD_ALIGN = 32;
 
 struct Layer {
   int n_in = 0, n_out = 0, ld_in = 0, ld_out = 0;
@@ -704,7 +708,7 @@ static int build_csr(pdadmm_ctx *c, const pdadmm_config *cfg) {
 static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   const int64_t N = cfg->n_nodes;
   c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
-  c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, 4); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
+  c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, LD_ALIGN); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
   c->neg_levels = cfg->quant_neg_levels; c->fixed_step = cfg->quant_step;
   c->code_bytes = cfg->quant_levels > 256 ? 2 : 1;
   c->quant_q = (cfg->flags & PDADMM_FLAG_QUANT_Q) != 0;
@@ -733,12 +737,12 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->layers.resize(c->L);
   int max_in = 0, max_out = 0;
   size_t max_part = 0;
-  for (int l = 1; l < c->L; ++l) max_in = std::max(max_in, round_up(cfg->layer_widths[l - 1], 4));
+  for (int l = 1; l < c->L; ++l) max_in = std::max(max_in, round_up(cfg->layer_widths[l - 1], LD_ALIGN));
   for (int l = 0; l < c->L; ++l) {
     Layer &ly = c->layers[l];
     ly.n_in = l == 0 ? c->n0 : cfg->layer_widths[l - 1];
     ly.n_out = cfg->layer_widths[l];
-    ly.ld_in = round_up(ly.n_in, 4); ly.ld_out = round_up(ly.n_out, 4);
+    ly.ld_in = round_up(ly.n_in, LD_ALIGN); ly.ld_out = round_up(ly.n_out, LD_ALIGN);
     max_out = std::max(max_out, ly.ld_out);
     const size_t e_out = (size_t)N * ly.ld_out;
     // quantised mode: p_l and its codes trade places with the trial buffers, so all share one size
