@@ -175,6 +175,7 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--simt", action="store_true", help="run the dense products on CUDA cores")
+    ap.add_argument("--one-lane", action="store_true", help="queue all layers on one stream (no concurrency across layers)")
     ap.add_argument("--quant-q", action="store_true",
                     help="pdADMM-G-Q workloads: keep q on the level set as well (variant of Sec. Quantization Extension)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -229,6 +230,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     device = replicas.device_for(local_rank, world)
     flags = (B.FLAG_SIMT_GEMM if args.simt else 0) | (B.FLAG_QUANT_Q if args.quant_q else 0)
+    flags |= B.FLAG_ONE_LANE if args.one_lane else 0
 
     inp = synth.make_inputs(w)
     ctx = B.from_inputs(inp, device=device, flags=flags)

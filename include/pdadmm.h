@@ -66,6 +66,7 @@ typedef enum {
 #define PDADMM_FLAG_SIMT_GEMM 1u     /* run the dense products on CUDA cores (fp32 FMA) instead of tensor cores */
 #define PDADMM_FLAG_QUANT_Q 2u       /* pdADMM-G-Q variant that keeps q_l on the level set of p_{l+1} as well   */
 #define PDADMM_FLAG_NO_GRAPH 4u      /* launch every kernel of an iteration directly instead of replaying a CUDA graph */
+#define PDADMM_FLAG_ONE_LANE 8u      /* queue all layers on one stream instead of spreading them over concurrent lanes */
 
 /*
  * Problem statement (paper: Problem 2 / Problem 3, Algorithm 1 "Require", and the experimental

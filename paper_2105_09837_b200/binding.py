@@ -21,6 +21,7 @@ T_X, T_P, T_W, T_B, T_Z, T_Q, T_U, T_CODES, T_TAU, T_THETA, T_QSCALE, T_CSR_ROWP
 FLAG_SIMT_GEMM = 1
 FLAG_QUANT_Q = 2
 FLAG_NO_GRAPH = 4
+FLAG_ONE_LANE = 8
 
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 

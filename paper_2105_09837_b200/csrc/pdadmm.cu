@@ -126,7 +126,16 @@ struct pdadmm_ctx {
   int *labels = nullptr;
   uint8_t *mask = nullptr;
   std::vector<pd::Layer> layers;
-  pd::Scratch scr;
+  pd::Scratch scr;                  // lane 0: the context's main stream and its scratch
+  // Layer concurrency: the updates of different layers are independent inside each phase of an iteration, so
+  // layer l's chain of kernels is queued on lane l mod n_lanes.  Every lane has its own stream and its own scratch
+  // (product outputs, partial tiles, reduction slots), so that chains of different layers can overlap: the next
+  // product starts on the SMs that the previous one has already left, and bandwidth-bound kernels run beside
+  // tensor-bound ones.  `cur` is the lane that the host code is queueing on.
+  std::vector<std::unique_ptr<pd::Scratch>> more_lanes;
+  pd::Scratch *cur = &scr;
+  std::vector<cudaEvent_t> ev_p;    // [L]: p_l of this iteration is complete
+  std::vector<cudaEvent_t> ev_lane; // [n_lanes]: fork / join
   bool r_valid = false;
   bool t_valid = false;             // every layer's t matches the stored u, p, q
   int *d_flag = nullptr;            // device counter (z_L solver non-convergence)
@@ -273,16 +282,16 @@ static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, cons
 // captured iteration always uses the same words) and whenever it runs out.
 constexpr int AMAX_POOL = 4096;
 static int amax_reset(pdadmm_ctx *c, cudaStream_t st) {
-  PD_CUDA(cudaMemsetAsync(c->scr.amax_pool, 0, AMAX_POOL * sizeof(uint32_t), st));
-  c->scr.amax_next = 0;
+  PD_CUDA(cudaMemsetAsync(c->cur->amax_pool, 0, AMAX_POOL * sizeof(uint32_t), st));
+  c->cur->amax_next = 0;
   return PDADMM_OK;
 }
 // room for n more words that must stay valid together
 static int amax_reserve(pdadmm_ctx *c, cudaStream_t st, int n) {
-  if (c->scr.amax_next + n > AMAX_POOL) PD_TRY(amax_reset(c, st));
+  if (c->cur->amax_next + n > AMAX_POOL) PD_TRY(amax_reset(c, st));
   return PDADMM_OK;
 }
-static uint32_t *amax_take(pdadmm_ctx *c) { return c->scr.amax_pool + c->scr.amax_next++; }
+static uint32_t *amax_take(pdadmm_ctx *c) { return c->cur->amax_pool + c->cur->amax_next++; }
 // max|x| of a matrix stored as n4 float4 values -> a fresh word
 static uint32_t *amax_of(pdadmm_ctx *c, cudaStream_t st, const float *x, size_t n4) {
   uint32_t *w = amax_take(c);
@@ -352,11 +361,11 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
   // SMs costs as much as a full one, so its tiles are cut along the contraction into as many slices as fit.
   int n_units = n_tiles;
   const int tail = n_tiles % c->n_sms, n_kb = (int)ceil_div(K, TC_BK);
-  if (tail > 0 && c->scr.tail_ws != nullptr) {
+  if (tail > 0 && c->cur->tail_ws != nullptr) {
     const int split = std::min(std::min(c->n_sms / tail, n_kb / 2), 8);     // at least 2 K blocks per slice
     if (split > 1) {
       prm.tail_begin = n_tiles - tail; prm.tail_split = split;
-      prm.tail_ws = c->scr.tail_ws; prm.tail_count = c->scr.tail_count;
+      prm.tail_ws = c->cur->tail_ws; prm.tail_count = c->cur->tail_count;
       n_units = prm.tail_begin + tail * split;
     }
   }
@@ -410,7 +419,7 @@ static int refresh_residual(pdadmm_ctx *c, Layer &ly, cudaStream_t st) {
 static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   Layer &ly = c->layers[l];
   Layer &prev = c->layers[l - 1];
-  Scratch &s = c->scr;
+  Scratch &s = *c->cur;
   const int N = (int)c->N;
   int np = 0;
   (void)prev;
@@ -435,7 +444,7 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
 // pdADMM-G: p <- p - g/tau, r <- r - (W g)/tau.
 static void p_step_plain(pdadmm_ctx *c, int l) {
   Layer &ly = c->layers[l];
-  Scratch &s = c->scr;
+  Scratch &s = *c->cur;
   const size_t n4p = (size_t)c->N * ly.ld_in / 4, n4r = (size_t)c->N * ly.ld_out / 4;
   {
     Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_in, 0);
@@ -451,7 +460,7 @@ static void p_step_plain(pdadmm_ctx *c, int l) {
 // Each trial ends with a read-back of the accept flag (the only host round trip of an iteration).
 static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
   Layer &ly = c->layers[l];
-  Scratch &s = c->scr;
+  Scratch &s = *c->cur;
   const int N = (int)c->N;
   const size_t n4p = (size_t)N * ly.ld_in / 4, n4r = (size_t)N * ly.ld_out / 4;
   const int max_trials = 30;
@@ -494,7 +503,7 @@ static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
 // b <- b - mean_j r, shift = mean_j r.
 static int w_and_b_step(pdadmm_ctx *c, int l) {
   Layer &ly = c->layers[l];
-  Scratch &s = c->scr;
+  Scratch &s = *c->cur;
   const int N = (int)c->N;
   if (!c->use_tc) {
     dim3 grid((unsigned)ceil_div(ly.n_in, SG_BN), (unsigned)ceil_div(ly.n_out, SG_BM), (unsigned)ly.n_split);
@@ -552,7 +561,7 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
 // z (and q, u for hidden layers) of layer l; needs p_{l+1} of this iteration.
 static void zqu_step(pdadmm_ctx *c, int l) {
   Layer &ly = c->layers[l];
-  Scratch &s = c->scr;
+  Scratch &s = *c->cur;
   const int N = (int)c->N;
   if (l + 1 < c->L) {
     const size_t n4 = (size_t)N * ly.ld_out / 4;
@@ -571,18 +580,46 @@ static void zqu_step(pdadmm_ctx *c, int l) {
   }
 }
 
+static Scratch &lane(pdadmm_ctx *c, int i) { return i == 0 ? c->scr : *c->more_lanes[i - 1]; }
+
 static int iterate_once(pdadmm_ctx *c, bool *hit_cap) {
-  if (c->use_tc) PD_TRY(amax_reset(c, c->scr.st));
-  // p-update of layers 2..L from the iterates of the previous iteration
+  // per-kernel timing wants one kernel at a time: a single lane then
+  const int S = c->profiling ? 1 : 1 + (int)c->more_lanes.size();
+  auto lane_of = [&](int l) -> Scratch & { return lane(c, l % S); };
+  struct Restore { pdadmm_ctx *c; ~Restore() { c->cur = &c->scr; } } restore{c};
+  // the other lanes start after everything queued on the main stream so far
+  if (S > 1) {
+    PD_CUDA(cudaEventRecord(c->ev_lane[0], c->scr.st));
+    for (int i = 1; i < S; ++i) PD_CUDA(cudaStreamWaitEvent(lane(c, i).st, c->ev_lane[0], 0));
+  }
+  if (c->use_tc)
+    for (int i = 0; i < S; ++i) { c->cur = &lane(c, i); PD_TRY(amax_reset(c, c->cur->st)); }
+  // p-update of layers 2..L from the iterates of the previous iteration.  The quantised update reads an accept
+  // flag on the host after every trial, so it stays on the main stream.
   for (int l = 1; l < c->L; ++l) {
+    c->cur = c->levels ? &c->scr : &lane_of(l);
     PD_TRY(p_gradient_and_tau(c, l));
     if (c->levels) PD_TRY(p_step_quantised(c, l, hit_cap));
     else p_step_plain(c, l);
+    if (S > 1) PD_CUDA(cudaEventRecord(c->ev_p[l], c->cur->st));
   }
   // W- and b-update of every layer with the new p
-  for (int l = 0; l < c->L; ++l) PD_TRY(w_and_b_step(c, l));
-  // z-, q-, u-update (q_l and u_l need p_{l+1} of this iteration)
-  for (int l = 0; l < c->L; ++l) zqu_step(c, l);
+  for (int l = 0; l < c->L; ++l) {
+    c->cur = &lane_of(l);
+    if (S > 1 && l >= 1 && c->levels && c->cur != &c->scr) PD_CUDA(cudaStreamWaitEvent(c->cur->st, c->ev_p[l], 0));
+    PD_TRY(w_and_b_step(c, l));
+  }
+  // z-, q-, u-update (q_l and u_l need p_{l+1} of this iteration, which another lane may have written)
+  for (int l = 0; l < c->L; ++l) {
+    c->cur = &lane_of(l);
+    if (S > 1 && l + 1 < c->L) PD_CUDA(cudaStreamWaitEvent(c->cur->st, c->ev_p[l + 1], 0));
+    zqu_step(c, l);
+  }
+  // join: the main stream continues after every lane
+  for (int i = 1; i < S; ++i) {
+    PD_CUDA(cudaEventRecord(c->ev_lane[i], lane(c, i).st));
+    PD_CUDA(cudaStreamWaitEvent(c->scr.st, c->ev_lane[i], 0));
+  }
   return PDADMM_OK;
 }
 
@@ -803,6 +840,28 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &s.amax_pool, (size_t)AMAX_POOL));
   }
 
+  // further lanes for the concurrency across layers: own stream, product outputs, partial tiles, slots
+  const int n_lanes = (cfg->flags & PDADMM_FLAG_ONE_LANE) ? 1 : std::min(c->L, 2);
+  for (int i = 1; i < n_lanes; ++i) {
+    c->more_lanes.emplace_back(new Scratch());
+    Scratch &x = *c->more_lanes.back();
+    PD_CUDA(cudaStreamCreateWithFlags(&x.st, cudaStreamNonBlocking));
+    PD_TRY(dev_alloc(c, &x.s1, e_max));
+    PD_TRY(dev_alloc(c, &x.s2, (size_t)N * max_out));
+    PD_TRY(dev_alloc(c, &x.part, max_part));
+    x.n_slots = s.n_slots;
+    PD_TRY(dev_alloc(c, &x.slots, x.n_slots));
+    if (c->use_tc) {
+      PD_TRY(dev_alloc(c, &x.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
+      PD_TRY(dev_alloc(c, &x.tail_count, (size_t)c->n_sms * 8));
+      PD_TRY(dev_alloc(c, &x.amax_pool, (size_t)AMAX_POOL));
+    }
+  }
+  c->ev_p.resize(c->L);
+  for (auto &e : c->ev_p) PD_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  c->ev_lane.resize(n_lanes);
+  for (auto &e : c->ev_lane) PD_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+
   // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
   Layer &l0 = c->layers[0];
   PD_TRY(upload_rows(st, l0.p, l0.ld_in, cfg->features, c->d, N));
@@ -860,6 +919,9 @@ static void destroy(pdadmm_ctx *c) {
   if (c->ev_begin) cudaEventDestroy(c->ev_begin);
   if (c->ev_end) cudaEventDestroy(c->ev_end);
   if (c->iter_graph) cudaGraphExecDestroy(c->iter_graph);
+  for (auto e : c->ev_p) cudaEventDestroy(e);
+  for (auto e : c->ev_lane) cudaEventDestroy(e);
+  for (auto &x : c->more_lanes) if (x->st) cudaStreamDestroy(x->st);
   if (c->scr.st) cudaStreamDestroy(c->scr.st);
   delete c;
 }
