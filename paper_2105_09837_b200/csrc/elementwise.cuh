@@ -160,8 +160,12 @@ quantize_kernel(const float *__restrict__ x, size_t n, float scale, float lo, in
 // ---- finalisers of the step parameters (one block of 256 threads) ---------------------------------
 // Fixed-order sum of n slots by one block: thread t adds slots t, t+256, ..., then a fixed tree.  Result in thread 0.
 __device__ __forceinline__ double block_sum_slots(const double *__restrict__ slots, int n, double *sh /* 256 */) {
-  double s = 0.0;
-  for (int i = threadIdx.x; i < n; i += 256) s += slots[i];
+  // four independent partial sums per thread keep four loads in flight; the order of the additions is fixed
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  int i = threadIdx.x;
+  for (; i + 768 < n; i += 1024) { s0 += slots[i]; s1 += slots[i + 256]; s2 += slots[i + 512]; s3 += slots[i + 768]; }
+  for (; i < n; i += 256) s0 += slots[i];
+  const double s = (s0 + s1) + (s2 + s3);
   __syncthreads();
   sh[threadIdx.x] = s;
   __syncthreads();

@@ -63,6 +63,39 @@ def test_spmm_against_sparse_library(width):
     assert np.all(B.spmm(E.indptr, E.indices, E.data, np.ones((5, 3), np.float32)) == 0)
 
 
+@pytest.mark.parametrize("mode,M,N,K", [(0, 300, 200, 100), (1, 300, 200, 100), (2, 300, 200, 1000), (0, 1000, 500, 500),
+                                        (1, 1000, 500, 500), (2, 500, 500, 5000), (0, 129, 7, 65), (1, 5, 131, 3),
+                                        (2, 7, 100, 129)])
+@pytest.mark.parametrize("kind", ["normal", "positive", "tiny", "huge", "mixed"])
+def test_dense_products_keep_single_precision_accuracy_at_any_scale(mode, M, N, K, kind):
+    """The tensor-core products split each operand into two half-precision planes after scaling it by a power of two
+    taken from its largest magnitude: the result must be as accurate as a single-precision product (relative
+    Frobenius error below 4e-7 against the product in double precision) whatever the magnitude of the operands,
+    also when the entries of one operand span many orders of magnitude, for all three operand layouts, with ragged
+    tiles and with contraction lengths that are not a multiple of the K block."""
+    rng = np.random.default_rng(1000 * mode + M + N + K)
+    a = rng.standard_normal((K, M) if mode == 2 else (M, K))
+    b = rng.standard_normal((N, K) if mode == 0 else (K, N))
+    if kind == "positive":
+        a, b = np.abs(a), np.abs(b)
+    elif kind == "tiny":
+        a, b = a * 1e-20, b * 1e-9
+    elif kind == "huge":
+        a, b = a * 1e12, b * 3e7
+    elif kind == "mixed":
+        a = a * np.exp(rng.uniform(-12, 12, size=a.shape))
+        b = b * np.exp(rng.uniform(-8, 8, size=b.shape))
+    a, b = a.astype(np.float32), b.astype(np.float32)
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    want = a64 @ b64.T if mode == 0 else (a64 @ b64 if mode == 1 else a64.T @ b64)
+    got, ss = B.matmul(mode, a, b)
+    assert U.rel_err(got.astype(np.float64), want) < 4e-7
+    if kind in ("normal", "positive", "mixed"):          # the squares of the other two leave the single-precision range
+        assert abs(ss - np.sum(want ** 2)) <= 2e-6 * np.sum(want ** 2)
+    ref, _ = B.matmul(mode, a, b, flags=B.FLAG_SIMT_GEMM)             # the CUDA-core product of the same library
+    assert U.rel_err(ref.astype(np.float64), want) < 1e-6
+
+
 def test_single_layer_model_and_zero_hops():
     inp = synth.make_inputs(synth.small("c1", 333, feat_dim=9, hidden=5, n_layers=1, n_hops=0))
     prm, s, _ = U.oracle_problem(inp)
