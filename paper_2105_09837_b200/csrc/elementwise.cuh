@@ -275,6 +275,52 @@ make_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, cons
   }
 }
 
+// ---- fp16 planes of a node-major matrix, transposed -------------------------------------------------
+// x [rows = nodes][ld] fp32 -> hiT, loT [cols][ldT] with the node index contiguous: operands of the product that
+// contracts over the nodes (the W-gradient r^T p+), for layers where splitting them once here is cheaper than
+// splitting them once per output tile inside that product.  Scaling and split as in make_planes_kernel; the
+// exponent goes to *exp_out.
+// A warp handles 32 nodes x 16 columns: lane (q, g) loads the 4 x 4 block of nodes 4q..4q+3, columns 4g..4g+3
+// (four 16-byte loads, 64 contiguous bytes per row and warp), transposes it in registers and stores, per column,
+// the four nodes as 8 bytes of each plane (64 contiguous bytes per column and warp): whole sectors both ways, no
+// shared memory.  Tiles are numbered with the node index fastest.
+__global__ void __launch_bounds__(256)
+transpose_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, const uint32_t *__restrict__ amax,
+                        int *__restrict__ exp_out, __half *__restrict__ hiT, __half *__restrict__ loT, int ldT) {
+  const int e = tc_scale_exp(*amax);
+  if (blockIdx.x == 0 && threadIdx.x == 0) *exp_out = e;
+  const float scale = __uint_as_float((uint32_t)(e + 127) << 23);
+  const int lane = threadIdx.x & 31, q = lane & 7, g = lane >> 3;
+  const long long row_tiles = (rows + 31) / 32, n_tiles = row_tiles * ((cols + 15) / 16);
+  for (long long wt = blockIdx.x * 8ll + (threadIdx.x >> 5); wt < n_tiles; wt += gridDim.x * 8ll) {
+    const int node0 = (int)(wt % row_tiles) * 32 + 4 * q, col = (int)(wt / row_tiles) * 16 + 4 * g;
+    if (node0 >= rows || col >= cols) continue;
+    float v[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (node0 + i < rows) t = *reinterpret_cast<const float4 *>(x + (size_t)(node0 + i) * ld + col);   // col + 3 < ld
+      v[i][0] = t.x; v[i][1] = t.y; v[i][2] = t.z; v[i][3] = t.w;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (col + j >= cols) break;
+      float h[4], l[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float xs = v[i][j] * scale;
+        h[i] = __uint_as_float((__float_as_uint(xs) + 0x1000u) & 0xFFFFE000u);
+        l[i] = (xs - h[i]) * 2048.0f;
+      }
+      const __half2 h0 = __floats2half2_rn(h[0], h[1]), h1 = __floats2half2_rn(h[2], h[3]);
+      const __half2 l0 = __floats2half2_rn(l[0], l[1]), l1 = __floats2half2_rn(l[2], l[3]);
+      const size_t o = (size_t)(col + j) * ldT + node0;
+      *reinterpret_cast<uint2 *>(hiT + o) = make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
+      *reinterpret_cast<uint2 *>(loT + o) = make_uint2(*reinterpret_cast<const uint32_t *>(&l0), *reinterpret_cast<const uint32_t *>(&l1));
+    }
+  }
+}
+
 // ---- reduction of the split partial tiles of grad_W, scaling by nu, ||grad_W||^2 ------------------
 __global__ void __launch_bounds__(EW_THREADS)
 reduce_gradW_kernel(const float *__restrict__ part, int n_split, size_t n4, float nu, float *__restrict__ G,

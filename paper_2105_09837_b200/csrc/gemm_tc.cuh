@@ -10,9 +10,9 @@
 // Products of two 11-bit numbers are exact in the fp32 accumulator, so the split is as accurate as the same
 // split on tf32 operands at twice the tensor-core rate and half the shared-memory footprint per operand.
 //
-// TMA brings fp32 tiles of the node-sized operand into shared memory; converter warps turn them, in place,
-// into the two fp16 planes (K-major, 128-byte swizzle); the small operand (a weight matrix) arrives as two
-// precomputed fp16 planes.  One thread issues tcgen05.mma; completion is tracked with mbarriers; eight more
+// TMA brings fp32 tiles of the node-sized operand into shared memory; converter warps turn them into the two
+// fp16 planes, which they write to tensor memory; the small operand (a weight matrix) arrives as two precomputed
+// fp16 planes (K-major, 128-byte swizzle).  One thread issues tcgen05.mma; completion is tracked with mbarriers; eight more
 // warps read each K block's main term from tensor memory, add it to a register accumulator and finally apply
 // the scaling and the fused epilogue.
 //
@@ -33,8 +33,8 @@ constexpr int TC_KSTEPS = TC_BK / 16;                          // MMAs (K = 16) 
 constexpr int TC_FLUSH = 1;                                    // K blocks per read-out of the main accumulator
 constexpr int TC_PLANE_BYTES = 128 * TC_BK * 2;                // 16 KB: one 128 x 64 fp16 operand plane
 constexpr int TC_STAGE_BYTES = 4 * TC_PLANE_BYTES;             // A_hi, A_lo, B_hi, B_lo (= two fp32 tiles of 128 x 64)
-// warp 0: TMA, warp 1: MMA, then 8 converter warps (all on A, or four on each of A and B), then 8 accumulate +
-// epilogue warps (two warps per 32-lane quarter of tensor memory, 64 columns each)
+// warp 0: TMA, warp 1: MMA, then 8 converter warps, then 8 accumulate + epilogue warps (two warps per 32-lane
+// quarter of tensor memory, 64 columns each)
 constexpr int TC_CONV_WARPS = 8;
 constexpr int TC_THREADS = 32 * (2 + TC_CONV_WARPS + 8);      // 576
 constexpr int TC_ACC_THREADS = 256;
@@ -73,8 +73,9 @@ struct TcParams {
   int n_split;            // number of contraction slices; slice z writes its own partial output
   size_t c_split_stride;  // elements between the partial outputs of consecutive slices
   int *error;             // set to 1 if a bounded wait expired
-  const uint32_t *amax_a; // bit pattern of max|A| (device word); nullptr = no scaling
-  const uint32_t *amax_b; // the same for B when B is converted in the kernel
+  const uint32_t *amax_a; // bit pattern of max|A| (device word) when A is converted in the kernel; nullptr = no scaling
+  const uint32_t *amax_b; // the same for B when B is converted in the kernel (TC_RAW_MN)
+  const int *exp_a;       // scaling exponent stored with the precomputed planes of A (TC_PLANES)
   const int *exp_b;       // scaling exponent stored with the precomputed planes of B
   // Tail balancing (n_split == 1 only): output tiles from tail_begin on are cut into tail_split contraction
   // slices, one work unit each, so that the last, partly filled round of the persistent grid is shorter.
@@ -85,10 +86,15 @@ struct TcParams {
   int *tail_count;        // [tiles from tail_begin][8 warps], zero before and after every launch
 };
 
-// MN = false: A is [M][K] fp32, contiguous along K (a node-major matrix, rows = nodes); B arrives as two fp16
-//              planes [N][K] (map_b = hi, map_blo = lo), contiguous along K.
-// MN = true:  both operands are fp32 and contiguous along their output index, A = [K][M], B = [K][N] (the
-//              contraction over nodes of the W-gradient); the converter warps transpose while they split.
+// MODE TC_RAW_K:  A is [M][K] fp32, contiguous along K (a node-major matrix, rows = nodes), converted in the kernel;
+//                  B arrives as two fp16 planes [N][K] (map_b = hi, map_blo = lo), contiguous along K.
+// The contraction over nodes of the W-gradient has both operands node-major, i.e. contiguous along their output
+// index, A = [K][M], B = [K][N], and comes in two forms:
+// MODE TC_RAW_MN:  both arrive as fp32 tiles and the converter warps transpose while they split (A to tensor
+//                  memory, B in place in shared memory).  Every output tile converts its operand tiles again, so
+//                  this form suits outputs with few tiles.
+// MODE TC_PLANES:  both arrive as fp16 planes [M][K], [N][K] (map_a / map_alo, map_b / map_blo), transposed and
+//                  split once by transpose_planes_kernel; the converter warps have nothing to do.
 //
 // Persistent: the grid has at most one block per SM and block i works on output tiles i, i + gridDim.x, ...
 // (column tile fastest, so that neighbouring blocks share the streamed operand in L2).  All roles keep running
@@ -100,10 +106,13 @@ struct TcParams {
 // warps read it out and add it to a register accumulator with round-to-nearest, while the MMAs of the next
 // block fill the other buffer.  The two correction terms are 2^-11 of the main term, so they are summed over
 // the whole contraction in a fourth tensor-memory tile and added once at the end.
-template <bool MN, class Epi>
+enum : int { TC_RAW_K = 0, TC_RAW_MN = 1, TC_PLANES = 2 };
+template <int MODE, class Epi>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_blo, const TcParams prm, Epi epi, double *__restrict__ partials) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_alo,
+               const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_blo,
+               const TcParams prm, Epi epi, double *__restrict__ partials) {
+  constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN;
   if (*reinterpret_cast<volatile int *>(prm.error) != 0) return;   // an earlier block gave up: do not queue behind it
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -140,7 +149,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&map_a);
     ptx::prefetch_tmap(&map_b);
-    if (!MN) ptx::prefetch_tmap(&map_blo);
+    ptx::prefetch_tmap(&map_blo);
+    if (PP) ptx::prefetch_tmap(&map_alo);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, TC_TMEM_COLS);
@@ -151,7 +161,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   // scaling exponents of the two operands (written by earlier kernels of the stream)
-  const int exp_a = prm.amax_a ? tc_scale_exp(*prm.amax_a) : 0;
+  const int exp_a = PP ? (prm.exp_a ? *prm.exp_a : 0) : (prm.amax_a ? tc_scale_exp(*prm.amax_a) : 0);
   const int exp_b = MN ? (prm.amax_b ? tc_scale_exp(*prm.amax_b) : 0) : (prm.exp_b ? *prm.exp_b : 0);
 
   // work unit -> (row tile origin, column tile origin, first and number of K blocks); a unit is an output tile or,
@@ -195,9 +205,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             ptx::tma_load_2d(st, &map_a, m0, k0, &full_bar[s]);
             ptx::tma_load_2d(st + 2 * TC_PLANE_BYTES, &map_b, n0, k0, &full_bar[s]);
           } else {
-            // fp32 [128 rows][64 floats] as two 128-byte-swizzled boxes of 32 floats; fp16 planes of B as they are used
-            ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
-            ptx::tma_load_2d(st + TC_PLANE_BYTES, &map_a, k0 + 32, m0, &full_bar[s]);
+            if (PP) {
+              ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
+              ptx::tma_load_2d(st + TC_PLANE_BYTES, &map_alo, k0, m0, &full_bar[s]);
+            } else {
+              // fp32 [128 rows][64 floats] as two 128-byte-swizzled boxes of 32 floats
+              ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
+              ptx::tma_load_2d(st + TC_PLANE_BYTES, &map_a, k0 + 32, m0, &full_bar[s]);
+            }
+            // fp16 planes of B as the MMA reads them
             ptx::tma_load_2d(st + 2 * TC_PLANE_BYTES, &map_b, k0, n0, &full_bar[s]);
             ptx::tma_load_2d(st + 3 * TC_PLANE_BYTES, &map_blo, k0, n0, &full_bar[s]);
           }
@@ -217,7 +233,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // A: tensor memory, 8 columns per K step.  B: shared-memory descriptors with a constant high word; the low
       // word of stage 0 advances by whole stages / K steps (K-major planes with 128-byte rows; 16 fp16 are 32 bytes)
       const uint32_t hi_b = ptx::smem_desc_hi(false, TC_BK * 2);
+      const uint32_t lo_a0 = ptx::smem_desc_lo(ptx::smem_u32(smem), false, 0);       // PP: A planes in shared memory too
       const uint32_t lo_b0 = ptx::smem_desc_lo(ptx::smem_u32(smem) + 2 * TC_PLANE_BYTES, false, 0);
+      uint64_t *const ready_bar = PP ? full_bar : conv_bar;      // what tells that a stage's operands are in place
       constexpr uint32_t step_b = 32u >> 4;
       bool ok = true;
       // running state: stage s with phase bit sp, accumulator buffer b with phase bit bp (of its *previous* use),
@@ -232,11 +250,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (ti > 0 && n_kb > 0) ok = ptx::mbar_wait(corr_empty, (ti - 1) & 1, abort_flag);
         for (int kb = 0; kb < n_kb && ok; ++kb) {
           const bool first = kb % TC_FLUSH == 0, last = kb % TC_FLUSH == TC_FLUSH - 1 || kb == n_kb - 1;
-          if (!seen_conv) ok = ptx::mbar_wait(&conv_bar[s], sp, abort_flag);
+          if (!seen_conv) ok = ptx::mbar_wait(&ready_bar[s], sp, abort_flag);
           if (ok && first && !first_round && !seen_acc) ok = ptx::mbar_wait(&acc_empty[b], bp, abort_flag);
           if (!ok) break;
           ptx::tc_fence_after_sync();
           const uint32_t ta = tmem_base + TC_COL_A + aslot * 64u, lb = lo_b0 + (uint32_t)s * (TC_STAGE_BYTES >> 4);
+          const uint32_t la = lo_a0 + (uint32_t)s * (TC_STAGE_BYTES >> 4);
           const uint32_t d = tmem_base + (uint32_t)(b * TC_BN);
           // next K block's stage and, if it starts a new group, its accumulator buffer
           const int s_next = s + 1 == TC_STAGES ? 0 : s + 1;
@@ -249,18 +268,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t ah = ta + 8u * kk, al = ah + 32u;
             const uint64_t dbh = ptx::smem_desc(hi_b, lb + kk * step_b);
             const uint64_t dbl = ptx::smem_desc(hi_b, lb + (TC_PLANE_BYTES >> 4) + kk * step_b);
-            ptx::mma_f16_ts(d_corr, al, dbh, idesc, kb > 0 || kk > 0);
-            ptx::mma_f16_ts(d_corr, ah, dbl, idesc, true);
-            ptx::mma_f16_ts(d, ah, dbh, idesc, !first || kk > 0);
+            if constexpr (PP) {
+              const uint64_t dah = ptx::smem_desc(hi_b, la + kk * step_b);
+              const uint64_t dal = ptx::smem_desc(hi_b, la + (TC_PLANE_BYTES >> 4) + kk * step_b);
+              ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
+              ptx::mma_f16(d_corr, dah, dbl, idesc, true);
+              ptx::mma_f16(d, dah, dbh, idesc, !first || kk > 0);
+            } else {
+              ptx::mma_f16_ts(d_corr, al, dbh, idesc, kb > 0 || kk > 0);
+              ptx::mma_f16_ts(d_corr, ah, dbl, idesc, true);
+              ptx::mma_f16_ts(d, ah, dbh, idesc, !first || kk > 0);
+            }
             if (kk == TC_KSTEPS - 2) {
               // probe the coming block's barriers while the tensor pipe still has work queued
-              seen_conv = ptx::mbar_test_wait(&conv_bar[s_next], sp_next);
+              seen_conv = ptx::mbar_test_wait(&ready_bar[s_next], sp_next);
               seen_acc = last ? (round_next ? true : ptx::mbar_test_wait(&acc_empty[b_next], bp_next)) : true;
             }
           }
           ptx::mma_commit(&empty_bar[s]);          // stage can be refilled once these MMAs have read it
-          ptx::mma_commit(&a_empty[aslot]);        // and so can the A planes' slot in tensor memory
-          aslot ^= 1u;
+          if (!PP) {
+            ptx::mma_commit(&a_empty[aslot]);      // and so can the A planes' slot in tensor memory
+            aslot ^= 1u;
+          }
           if (last) {
             ptx::mma_commit(&acc_full[b]);         // this group's partial product is complete
             if (b + 1 == TC_ACC_BUFS) first_round = false;
@@ -276,94 +305,96 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp < ACC0) {
-    // ---------------------------------------------------------------- converters (256 threads)
+    // ---------------------------------------------------------------- converters (256 threads; idle with TC_PLANES)
     // The planes of A go to tensor memory, where the MMA reads them without touching shared memory: row i of the
     // tile lives in lane i, and a warp can only write the 32 lanes of its own quarter (warp index mod 4).  So two
     // warps share a quarter: thread (row t = 32 (warp mod 4) + lane, half h) converts the 32 values h*32 .. h*32+31
     // of the K block of row t and writes 16 + 16 columns.
-    // MN = false: the values come from the swizzled [128][64] fp32 tile (row t, 16-byte chunks).
-    // MN = true:  the tile is [64][128] (contraction index first), so the thread reads a column; and B is converted
+    // TC_RAW_K:  the values come from the swizzled [128][64] fp32 tile (row t, 16-byte chunks).
+    // TC_RAW_MN: the tile is [64][128] (contraction index first), so the thread reads a column; and B is converted
     //             too, in place in shared memory: thread (output index tb, half hb) reads its 32 values, all 256
     //             threads wait until everyone has read (the planes overwrite the fp32 tile), then the thread writes
     //             four 16-byte chunks of row tb of the hi and of the lo plane, chunk j at position j ^ (tb mod 8)
     //             (the 128-byte swizzle).
-    const int cw = warp - 2;                               // 0 .. 7
-    const int quarter = warp & 3, half = cw >> 2;
-    const int t = quarter * 32 + lane;
-    const int ct = threadIdx.x - 64, tb = ct & 127, hb = ct >> 7;
-    const float scale_a = tc_pow2(exp_a), scale_b = tc_pow2(exp_b);
-    const uint32_t sw = (uint32_t)((MN ? tb : t) & 7);
-    bool ok = true;
-    int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      int m0, n0, k_begin, n_kb, z;
-      tile_coords(tile, m0, n0, k_begin, n_kb, z);
-      for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
-        const int s = it % TC_STAGES, use = it / TC_STAGES;
-        ok = ptx::mbar_wait(&full_bar[s], use & 1, abort_flag);
-        uint8_t *stage = smem + s * TC_STAGE_BYTES;
-        const int aslot = it % TC_A_SLOTS, ause = it / TC_A_SLOTS;
-        if (ok && ause > 0) ok = ptx::mbar_wait(&a_empty[aslot], (ause - 1) & 1, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);                  // the tensor-memory stores below are warp-wide
-        if (ok) {
-          ptx::tc_fence_after_sync();
-          float v[32];
-          if (MN) {
-            const float *raw = reinterpret_cast<const float *>(stage);     // [64][128]
-#pragma unroll
-            for (int k = 0; k < 32; ++k) v[k] = raw[(32 * half + k) * 128 + t];
-          } else {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              const float4 q = *reinterpret_cast<const float4 *>(stage + half * TC_PLANE_BYTES + t * 128 +
-                                                                 (((uint32_t)c ^ sw) << 4));
-              v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
-            }
-          }
-          uint32_t hreg[16], lreg[16];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float x[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
-            uint4 h, l;
-            tc_split8(x, scale_a, h, l);
-            hreg[4 * j] = h.x; hreg[4 * j + 1] = h.y; hreg[4 * j + 2] = h.z; hreg[4 * j + 3] = h.w;
-            lreg[4 * j] = l.x; lreg[4 * j + 1] = l.y; lreg[4 * j + 2] = l.z; lreg[4 * j + 3] = l.w;
-          }
-          const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + TC_COL_A + (uint32_t)aslot * 64u +
-                               16u * (uint32_t)half;
-          ptx::tmem_st16(col, hreg);
-          ptx::tmem_st16(col + 32u, lreg);
-        }
-        if constexpr (MN) {
-          uint8_t *region = stage + 2 * TC_PLANE_BYTES;
-          const float *raw = reinterpret_cast<const float *>(region);      // [64][128]
-          float v[32];
+    if constexpr (!PP) {
+      const int cw = warp - 2;                               // 0 .. 7
+      const int quarter = warp & 3, half = cw >> 2;
+      const int t = quarter * 32 + lane;
+      const int ct = threadIdx.x - 64, tb = ct & 127, hb = ct >> 7;
+      const float scale_a = tc_pow2(exp_a), scale_b = tc_pow2(exp_b);
+      const uint32_t sw = (uint32_t)((MN ? tb : t) & 7);
+      bool ok = true;
+      int it = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        int m0, n0, k_begin, n_kb, z;
+        tile_coords(tile, m0, n0, k_begin, n_kb, z);
+        for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+          const int s = it % TC_STAGES, use = it / TC_STAGES;
+          ok = ptx::mbar_wait(&full_bar[s], use & 1, abort_flag);
+          uint8_t *stage = smem + s * TC_STAGE_BYTES;
+          const int aslot = it % TC_A_SLOTS, ause = it / TC_A_SLOTS;
+          if (ok && ause > 0) ok = ptx::mbar_wait(&a_empty[aslot], (ause - 1) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);                  // the tensor-memory stores below are warp-wide
           if (ok) {
+            ptx::tc_fence_after_sync();
+            float v[32];
+            if (MN) {
+              const float *raw = reinterpret_cast<const float *>(stage);     // [64][128]
 #pragma unroll
-            for (int k = 0; k < 32; ++k) v[k] = raw[(32 * hb + k) * 128 + tb];
+              for (int k = 0; k < 32; ++k) v[k] = raw[(32 * half + k) * 128 + t];
+            } else {
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                const float4 q = *reinterpret_cast<const float4 *>(stage + half * TC_PLANE_BYTES + t * 128 +
+                                                                   (((uint32_t)c ^ sw) << 4));
+                v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
+              }
+            }
+            uint32_t hreg[16], lreg[16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              float x[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
+              uint4 h, l;
+              tc_split8(x, scale_a, h, l);
+              hreg[4 * j] = h.x; hreg[4 * j + 1] = h.y; hreg[4 * j + 2] = h.z; hreg[4 * j + 3] = h.w;
+              lreg[4 * j] = l.x; lreg[4 * j + 1] = l.y; lreg[4 * j + 2] = l.z; lreg[4 * j + 3] = l.w;
+            }
+            const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + TC_COL_A + (uint32_t)aslot * 64u +
+                                 16u * (uint32_t)half;
+            ptx::tmem_st16(col, hreg);
+            ptx::tmem_st16(col + 32u, lreg);
           }
-          // everyone has read its values of B (or someone gave up: then all stop here)
-          if (ptx::named_barrier_or(1, 256, !ok)) { ok = false; break; }
+          if constexpr (MN) {
+            uint8_t *region = stage + 2 * TC_PLANE_BYTES;
+            const float *raw = reinterpret_cast<const float *>(region);      // [64][128]
+            float v[32];
+            if (ok) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float x[8];
+              for (int k = 0; k < 32; ++k) v[k] = raw[(32 * hb + k) * 128 + tb];
+            }
+            // everyone has read its values of B (or someone gave up: then all stop here)
+            if (ptx::named_barrier_or(1, 256, !ok)) { ok = false; break; }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
-            uint4 h, l;
-            tc_split8(x, scale_b, h, l);
-            const uint32_t off = (uint32_t)tb * 128u + (((uint32_t)(4 * hb + j) ^ sw) << 4);
-            *reinterpret_cast<uint4 *>(region + off) = h;
-            *reinterpret_cast<uint4 *>(region + TC_PLANE_BYTES + off) = l;
+            for (int j = 0; j < 4; ++j) {
+              float x[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
+              uint4 h, l;
+              tc_split8(x, scale_b, h, l);
+              const uint32_t off = (uint32_t)tb * 128u + (((uint32_t)(4 * hb + j) ^ sw) << 4);
+              *reinterpret_cast<uint4 *>(region + off) = h;
+              *reinterpret_cast<uint4 *>(region + TC_PLANE_BYTES + off) = l;
+            }
+            ptx::fence_proxy_async_smem();
+          } else if (!ok) {
+            break;
           }
-          ptx::fence_proxy_async_smem();
-        } else if (!ok) {
-          break;
+          ptx::tmem_st_wait();
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(&conv_bar[s]);
         }
-        ptx::tmem_st_wait();
-        ptx::tc_fence_before_sync();
-        ptx::mbar_arrive(&conv_bar[s]);
       }
     }
   } else {

@@ -81,6 +81,8 @@ struct Layer {
   float *gradW = nullptr;   // [n_out][ld_in]
   Planes Wp;                // fp16 planes of W: [n_out][ldh_in], and of W^T: [n_in][ldh_out] (tensor-core path)
   Planes Gp;                // fp16 planes of grad_W: [n_out][ldh_in]
+  __half *xT_hi = nullptr, *xT_lo = nullptr;   // layer 1 only: transposed planes of p_1 = X, which never changes
+  int *xT_exp = nullptr;
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in] codes of 1 byte (up to 256 levels) or 2 bytes, quantised mode, l >= 2
   float scale = 1.0f;       // level spacing s_l of p_l
@@ -107,6 +109,9 @@ struct Scratch {
   int *tail_count = nullptr;
   uint32_t *amax_pool = nullptr;   // words for the largest magnitudes of product operands, handed out in stream order
   int amax_next = 0;
+  // transposed fp16 planes ([width][ldT], node index contiguous) of r_l and p_l for the product over the nodes
+  __half *rT_hi = nullptr, *rT_lo = nullptr, *pT_hi = nullptr, *pT_lo = nullptr;
+  int *rT_exp = nullptr, *pT_exp = nullptr;
 };
 
 struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
@@ -160,6 +165,8 @@ struct pdadmm_ctx {
   int n_sms = 148;
   bool w_planes_valid = false;
   bool amax_p_valid = false;        // every layer's amax_p covers the stored p
+  bool xT_valid = false;            // the transposed planes of X match the stored X
+  int ldT = 0;                      // leading dimension of transposed planes: N rounded up to 8
   std::map<std::tuple<const void *, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t>, CUtensorMap> tmaps;
 };
 
@@ -266,17 +273,17 @@ static int get_tmap(pdadmm_ctx *c, const void *base, uint64_t inner, uint64_t ou
   return PDADMM_OK;
 }
 
-template <bool MN, class Epi>
-static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mbl,
-                     const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
-  auto kern = gemm_tc_kernel<MN, Epi>;
+template <int MODE, class Epi>
+static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mal, const CUtensorMap &mb,
+                     const CUtensorMap &mbl, const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
+  auto kern = gemm_tc_kernel<MODE, Epi>;
   const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
   static bool configured = false;
   if (!configured) {
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     configured = true;
   }
-  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mb, mbl, prm, epi, partials);
+  kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mal, mb, mbl, prm, epi, partials);
   return PDADMM_OK;
 }
 
@@ -360,7 +367,7 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
   PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TM_RAW_K, &ma));
   PD_TRY(get_tmap(c, Bp.hi, (uint64_t)K, (uint64_t)N, (uint64_t)Bp.ld, TM_PLANE, &mb));
   PD_TRY(get_tmap(c, Bp.lo, (uint64_t)K, (uint64_t)N, (uint64_t)Bp.ld, TM_PLANE, &mbl));
-  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1, amax_a, nullptr, Bp.exp};
+  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1, amax_a, nullptr, nullptr, Bp.exp};
   // The persistent grid works through the tiles in rounds of n_sms; a last round that fills only part of the
   // SMs costs as much as a full one, so its tiles are cut along the contraction into as many slices as fit.
   int n_units = n_tiles;
@@ -374,24 +381,58 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     }
   }
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
-  return launch_tc<false, Epi>(c, st, ma, mb, mbl, prm, epi, partials, n_units);
+  return launch_tc<TC_RAW_K, Epi>(c, st, ma, ma, mb, mbl, prm, epi, partials, n_units);
 }
 
-// C parts [n_split][M][ldc] = A^T B over node slices: A = [K][lda] (M valid columns), B = [K][ldb] (N valid columns)
-static int gemm_over_nodes_tc(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
-                              const float *B, int ldb, float *part, int ldc, int k_chunk, int n_split,
-                              const uint32_t *wa = nullptr, const uint32_t *wb = nullptr) {
+// transposed fp16 planes [cols][ldT] of a node-major matrix x [rows][ld] whose largest magnitude is in *amax
+static void transpose_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, int rows, int cols, int ld,
+                             const uint32_t *amax, __half *hiT, __half *loT, int ldT, int *exp_out) {
+  Launch l(c, KC_PLANES, st, 8.0 * rows * cols, 0);
+  const int64_t warp_tiles = ceil_div(rows, 32) * ceil_div(cols, 16);
+  const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(warp_tiles, 8), 148 * 16));
+  transpose_planes_kernel<<<grid, 256, 0, st>>>(x, rows, cols, ld, amax, exp_out, hiT, loT, ldT);
+}
+
+// C parts [n_split][M][ldc] = A^T B over node slices, both operands given by their transposed planes:
+// A^T = [M][K nodes], B^T = [N][K nodes]
+static int gemm_over_nodes_tc(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const PlaneRef &At,
+                              const PlaneRef &Bt, float *part, int ldc, int k_chunk, int n_split) {
   const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM)) * n_split;
-  PD_TRY(amax_reserve(c, st, 2));
-  if (wa == nullptr) wa = amax_of(c, st, A, (size_t)K * lda / 4);
-  if (wb == nullptr) wb = amax_of(c, st, B, (size_t)K * ldb / 4);
+  CUtensorMap ma, mal, mb, mbl;
+  PD_TRY(get_tmap(c, At.hi, (uint64_t)K, (uint64_t)M, (uint64_t)At.ld, TM_PLANE, &ma));
+  PD_TRY(get_tmap(c, At.lo, (uint64_t)K, (uint64_t)M, (uint64_t)At.ld, TM_PLANE, &mal));
+  PD_TRY(get_tmap(c, Bt.hi, (uint64_t)K, (uint64_t)N, (uint64_t)Bt.ld, TM_PLANE, &mb));
+  PD_TRY(get_tmap(c, Bt.lo, (uint64_t)K, (uint64_t)N, (uint64_t)Bt.ld, TM_PLANE, &mbl));
+  TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1, nullptr, nullptr, At.exp, Bt.exp};
+  EpiStore epi{part, ldc};
+  Launch k(c, cls, st, 4.0 * ((double)K * N + (double)K * M), 2.0 * K * N * M);
+  return launch_tc<TC_PLANES, EpiStore>(c, st, ma, mal, mb, mbl, prm, epi, nullptr, n_tiles);
+}
+
+// The same from the fp32 operands themselves, A = [K][lda] (M valid columns), B = [K][ldb] (N valid columns), which
+// the product transposes and splits tile by tile; wa, wb: their largest magnitudes.
+static int gemm_over_nodes_raw(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
+                               const float *B, int ldb, float *part, int ldc, int k_chunk, int n_split,
+                               const uint32_t *wa, const uint32_t *wb) {
+  const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM)) * n_split;
   CUtensorMap ma, mb;
   PD_TRY(get_tmap(c, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, TM_RAW_MN, &ma));
   PD_TRY(get_tmap(c, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, TM_RAW_MN, &mb));
-  TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1, wa, wb, nullptr};
+  TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1, wa, wb, nullptr, nullptr};
   EpiStore epi{part, ldc};
   Launch k(c, cls, st, 4.0 * ((double)K * N + (double)K * M), 2.0 * K * N * M);
-  return launch_tc<true, EpiStore>(c, st, ma, mb, mb, prm, epi, nullptr, n_tiles);
+  return launch_tc<TC_RAW_MN, EpiStore>(c, st, ma, ma, mb, mb, prm, epi, nullptr, n_tiles);
+}
+
+// Which form the product over the nodes takes for an M x N output.  Splitting the operands inside the product
+// costs every output tile its own conversion of the operand tiles (the converter warps then set the pace, about
+// twice the time of the MMAs); splitting them beforehand costs one bandwidth-bound pass per operand.  Measured on
+// the B200: 16 output tiles (500 x 500) 88 us inside against 53 + 2 x 21 us beforehand; 64 tiles and more are
+// faster beforehand (workloads c4, c5: +2 % and +6 % per iteration), and so is layer 1, whose second operand X
+// never changes and keeps its planes.
+static bool planes_beforehand(int M, int N, bool second_operand_cached) {
+  const int64_t tiles = ceil_div(M, TC_BM) * ceil_div(N, TC_BN);
+  return tiles >= 32 || (second_operand_cached && tiles >= 8);
 }
 
 }  // namespace pd
@@ -515,9 +556,21 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
     gemm_tn_kernel<<<grid, SG_THREADS, 0, s.st>>>(ly.n_out, ly.n_in, N, ly.k_chunk, ly.r, ly.ld_out, ly.p, ly.ld_in,
                                                  s.part, ly.ld_in);
   } else {
-    // both operands are node-major, i.e. contiguous along their output index: r is [nodes][n_out], p+ is [nodes][n_in]
-    PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, s.st, ly.n_out, ly.n_in, N, ly.r, ly.ld_out, ly.p, ly.ld_in, s.part,
-                              ly.ld_in, ly.k_chunk, ly.n_split, ly.amax_r, ly.amax_p));
+    // both operands are node-major, i.e. contiguous along their output index (r is [nodes][n_out], p+ is
+    // [nodes][n_in]): transposed and split into planes beforehand, or tile by tile inside the product
+    if (planes_beforehand(ly.n_out, ly.n_in, l == 0)) {
+      transpose_planes(c, s.st, ly.r, N, ly.n_out, ly.ld_out, ly.amax_r, s.rT_hi, s.rT_lo, c->ldT, s.rT_exp);
+      PlaneRef Bt{s.pT_hi, s.pT_lo, c->ldT, s.pT_exp};
+      if (l == 0)          // p_1 = X never changes: its planes are kept (made before the first iteration)
+        Bt = PlaneRef{ly.xT_hi, ly.xT_lo, c->ldT, ly.xT_exp};
+      else
+        transpose_planes(c, s.st, ly.p, N, ly.n_in, ly.ld_in, ly.amax_p, s.pT_hi, s.pT_lo, c->ldT, s.pT_exp);
+      PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, s.st, ly.n_out, ly.n_in, N,
+                                PlaneRef{s.rT_hi, s.rT_lo, c->ldT, s.rT_exp}, Bt, s.part, ly.ld_in, ly.k_chunk, ly.n_split));
+    } else {
+      PD_TRY(gemm_over_nodes_raw(c, KC_GEMM_GRADW, s.st, ly.n_out, ly.n_in, N, ly.r, ly.ld_out, ly.p, ly.ld_in, s.part,
+                                 ly.ld_in, ly.k_chunk, ly.n_split, ly.amax_r, ly.amax_p));
+    }
   }
   const size_t n4w = (size_t)ly.n_out * ly.ld_in / 4;
   const int gw = ew_grid(n4w);
@@ -746,6 +799,21 @@ static int build_csr(pdadmm_ctx *c, const pdadmm_config *cfg) {
   return PDADMM_OK;
 }
 
+// transposed planes of r_l (up to max_out columns) and of p_l, l >= 2 (up to max_in columns) of one lane
+static int alloc_transposed(pdadmm_ctx *c, Scratch &s, int max_out, int max_in) {
+  if (max_out > 0) {
+    PD_TRY(dev_alloc(c, &s.rT_hi, (size_t)max_out * c->ldT));
+    PD_TRY(dev_alloc(c, &s.rT_lo, (size_t)max_out * c->ldT));
+  }
+  PD_TRY(dev_alloc(c, &s.rT_exp, 1));
+  if (max_in > 0) {
+    PD_TRY(dev_alloc(c, &s.pT_hi, (size_t)max_in * c->ldT));
+    PD_TRY(dev_alloc(c, &s.pT_lo, (size_t)max_in * c->ldT));
+  }
+  PD_TRY(dev_alloc(c, &s.pT_exp, 1));
+  return PDADMM_OK;
+}
+
 static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   const int64_t N = cfg->n_nodes;
   c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
@@ -826,6 +894,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   }
   // scratch
   Scratch &s = c->scr;
+  int tr_out = 0, tr_in = 0;
   const size_t e_max = (size_t)N * std::max(max_in, max_out);
   PD_TRY(dev_alloc(c, &s.s1, e_max));
   PD_TRY(dev_alloc(c, &s.s2, (size_t)N * max_out));
@@ -842,6 +911,21 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &s.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
     PD_TRY(dev_alloc(c, &s.tail_count, (size_t)c->n_sms * 8));
     PD_TRY(dev_alloc(c, &s.amax_pool, (size_t)AMAX_POOL));
+    c->ldT = round_up((int)N, 8);
+    // widest r_l and p_l (l >= 2) among the layers whose product over the nodes takes its operands as planes
+    for (int l = 0; l < c->L; ++l) {
+      const Layer &ly = c->layers[l];
+      if (!planes_beforehand(ly.n_out, ly.n_in, l == 0)) continue;
+      tr_out = std::max(tr_out, ly.n_out);
+      if (l > 0) tr_in = std::max(tr_in, ly.n_in);
+    }
+    PD_TRY(alloc_transposed(c, s, tr_out, tr_in));
+    Layer &l0 = c->layers[0];
+    if (planes_beforehand(l0.n_out, l0.n_in, true)) {
+      PD_TRY(dev_alloc(c, &l0.xT_hi, (size_t)l0.n_in * c->ldT));
+      PD_TRY(dev_alloc(c, &l0.xT_lo, (size_t)l0.n_in * c->ldT));
+    }
+    PD_TRY(dev_alloc(c, &l0.xT_exp, 1));
   }
 
   // further lanes for the concurrency across layers: own stream, product outputs, partial tiles, slots
@@ -859,6 +943,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
       PD_TRY(dev_alloc(c, &x.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
       PD_TRY(dev_alloc(c, &x.tail_count, (size_t)c->n_sms * 8));
       PD_TRY(dev_alloc(c, &x.amax_pool, (size_t)AMAX_POOL));
+      PD_TRY(alloc_transposed(c, x, tr_out, tr_in));
     }
   }
   c->ev_p.resize(c->L);
@@ -980,6 +1065,11 @@ static int ensure_residual(pdadmm_ctx *c) {
       absmax_kernel<<<ew_grid(n4), EW_THREADS, 0, c->scr.st>>>(ly.p, n4, ly.amax_p);
     }
     c->amax_p_valid = true;
+  }
+  if (!c->xT_valid && c->use_tc && planes_beforehand(c->layers[0].n_out, c->layers[0].n_in, true)) {
+    Layer &l0 = c->layers[0];
+    transpose_planes(c, c->scr.st, l0.p, (int)c->N, l0.n_in, l0.ld_in, l0.amax_p, l0.xT_hi, l0.xT_lo, c->ldT, l0.xT_exp);
+    c->xT_valid = true;
   }
   if (!c->t_valid) {
     for (int l = 1; l < c->L; ++l) {
@@ -1241,6 +1331,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
     c->r_valid = false;
   if (kind == PDADMM_T_W) c->w_planes_valid = false;
   if (kind == PDADMM_T_X || kind == PDADMM_T_P) c->amax_p_valid = false;
+  if (kind == PDADMM_T_X || (kind == PDADMM_T_P && layer == 1)) c->xT_valid = false;
   if (kind == PDADMM_T_P || kind == PDADMM_T_Q || kind == PDADMM_T_U) c->t_valid = false;
   if (kind == PDADMM_T_P && c->levels && layer >= 2) {
     Layer &y = c->layers[layer - 1];
@@ -1373,7 +1464,25 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
         dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM), (unsigned)n_split);
         gemm_tn_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, k_chunk, dA, lda, dB, ldb, part, ldc);
       } else {
-        PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, st, M, N, K, dA, lda, dB, ldb, part, ldc, k_chunk, n_split));
+        if (!planes_beforehand(M, N, false)) {
+          PD_TRY(amax_reserve(c, st, 2));
+          const uint32_t *wa = amax_of(c, st, dA, (size_t)K * lda / 4), *wb = amax_of(c, st, dB, (size_t)K * ldb / 4);
+          PD_TRY(gemm_over_nodes_raw(c, KC_GEMM_GRADW, st, M, N, K, dA, lda, dB, ldb, part, ldc, k_chunk, n_split, wa, wb));
+        } else {
+        // transposed planes of both operands, then the contraction over their rows
+        const int ldT = round_up(K, 8);
+        __half *ah, *al, *bh, *bl;
+        int *ea, *eb;
+        PD_TRY(dev_alloc(c, &ah, (size_t)M * ldT)); PD_TRY(dev_alloc(c, &al, (size_t)M * ldT));
+        PD_TRY(dev_alloc(c, &bh, (size_t)N * ldT)); PD_TRY(dev_alloc(c, &bl, (size_t)N * ldT));
+        PD_TRY(dev_alloc(c, &ea, 1)); PD_TRY(dev_alloc(c, &eb, 1));
+        PD_TRY(amax_reserve(c, st, 2));
+        const uint32_t *wa = amax_of(c, st, dA, (size_t)K * lda / 4), *wb = amax_of(c, st, dB, (size_t)K * ldb / 4);
+        transpose_planes(c, st, dA, K, M, lda, wa, ah, al, ldT, ea);
+        transpose_planes(c, st, dB, K, N, ldb, wb, bh, bl, ldT, eb);
+        PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, st, M, N, K, PlaneRef{ah, al, ldT, ea}, PlaneRef{bh, bl, ldT, eb}, part,
+                                  ldc, k_chunk, n_split));
+        }
       }
       const size_t n4 = (size_t)M * ldc / 4;
       np = ew_grid(n4);

@@ -65,14 +65,16 @@ def test_spmm_against_sparse_library(width):
 
 @pytest.mark.parametrize("mode,M,N,K", [(0, 300, 200, 100), (1, 300, 200, 100), (2, 300, 200, 1000), (0, 1000, 500, 500),
                                         (1, 1000, 500, 500), (2, 500, 500, 5000), (0, 129, 7, 65), (1, 5, 131, 3),
-                                        (2, 7, 100, 129)])
+                                        (2, 7, 100, 129), (2, 1000, 600, 333)])
 @pytest.mark.parametrize("kind", ["normal", "positive", "tiny", "huge", "mixed"])
 def test_dense_products_keep_single_precision_accuracy_at_any_scale(mode, M, N, K, kind):
     """The tensor-core products split each operand into two half-precision planes after scaling it by a power of two
     taken from its largest magnitude: the result must be as accurate as a single-precision product (relative
     Frobenius error below 4e-7 against the product in double precision) whatever the magnitude of the operands,
     also when the entries of one operand span many orders of magnitude, for all three operand layouts, with ragged
-    tiles and with contraction lengths that are not a multiple of the K block."""
+    tiles and with contraction lengths that are not a multiple of the K block.  The last shape has enough output
+    tiles (40) for the contraction over rows to take its operands as planes split beforehand; the smaller ones
+    split them inside the product."""
     rng = np.random.default_rng(1000 * mode + M + N + K)
     a = rng.standard_normal((K, M) if mode == 2 else (M, K))
     b = rng.standard_normal((N, K) if mode == 0 else (K, N))
