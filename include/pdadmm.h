@@ -193,7 +193,9 @@ int pdadmm_spmm(int device, int64_t n_rows, const int32_t *row_ptr, const int32_
  *   mode 0: C[M][N] = A[M][K] * B[N][K]^T      mode 1: C[M][N] = A[M][K] * B[K][N]
  *   mode 2: C[M][N] = A[K][M]^T * B[K][N]      (contraction over the leading index, split over node slices)
  * flags: PDADMM_FLAG_SIMT_GEMM selects the CUDA-core kernels, 0 the tensor-core kernels.
- * sumsq (may be null) receives sum(C^2) accumulated by the fused epilogue (modes 0 and 1).
+ * sumsq (may be null) receives sum(C^2) accumulated by the fused epilogue (modes 0 and 1); the tensor-core
+ * kernels square in single precision, so it is meaningful for 1e-19 < |C| < 1e19 (C itself has no such limit:
+ * every operand is scaled by a power of two taken from its largest magnitude before it is split into fp16 planes).
  */
 int pdadmm_matmul(int device, int mode, int M, int N, int K, const float *A, const float *B, float *C,
                   double *sumsq, uint32_t flags);

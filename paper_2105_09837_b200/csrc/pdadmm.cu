@@ -597,7 +597,7 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
     wstep_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.W, ly.gradW, ly.sc, n4w, w);
     if (c->use_tc) make_planes(c, s.st, ly.W, ly.n_out, ly.n_in, ly.ld_in, w, ly.Wp);
   }
-  const int n_blocks = (int)std::min<int64_t>(c->n_sms * 2, ceil_div(N, 16));
+  const int n_blocks = (int)std::min<int64_t>(c->n_sms * 4, ceil_div(N, 16));
   const int rows_per_block = (int)ceil_div(N, n_blocks);
   const int used_blocks = (int)ceil_div(N, rows_per_block);
   {
@@ -904,7 +904,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &s.codes_new, (size_t)N * max_in * c->code_bytes));
   }
   PD_TRY(dev_alloc(c, &s.part, max_part));
-  s.n_slots = std::max<size_t>((size_t)148 * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
+  s.n_slots = std::max<size_t>((size_t)c->n_sms * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
   s.n_slots *= 2;                       // two halves: consecutive reductions of one layer use different halves
   PD_TRY(dev_alloc(c, &s.slots, s.n_slots));
   if (c->use_tc) {

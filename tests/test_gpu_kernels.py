@@ -92,7 +92,8 @@ def test_dense_products_keep_single_precision_accuracy_at_any_scale(mode, M, N, 
     want = a64 @ b64.T if mode == 0 else (a64 @ b64 if mode == 1 else a64.T @ b64)
     got, ss = B.matmul(mode, a, b)
     assert U.rel_err(got.astype(np.float64), want) < 4e-7
-    if kind in ("normal", "positive", "mixed"):          # the squares of the other two leave the single-precision range
+    if kind in ("normal", "positive", "mixed"):          # the sum of squares is taken in single precision per thread
+                                                         # (1e-19 < |C| < 1e19), which the other two kinds leave
         assert abs(ss - np.sum(want ** 2)) <= 2e-6 * np.sum(want ** 2)
     ref, _ = B.matmul(mode, a, b, flags=B.FLAG_SIMT_GEMM)             # the CUDA-core product of the same library
     assert U.rel_err(ref.astype(np.float64), want) < 1e-6
