@@ -112,6 +112,8 @@ struct Scratch {
   // transposed fp16 planes ([width][ldT], node index contiguous) of r_l and p_l for the product over the nodes
   __half *rT_hi = nullptr, *rT_lo = nullptr, *pT_hi = nullptr, *pT_lo = nullptr;
   int *rT_exp = nullptr, *pT_exp = nullptr;
+  int *h_flag = nullptr;           // pinned word that receives the accept flag of the lane's quantised trial
+  cudaEvent_t ev_flag = nullptr;   // recorded after the copy of that flag
 };
 
 struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
@@ -501,44 +503,57 @@ static void p_step_plain(pdadmm_ctx *c, int l) {
   }
 }
 
-// pdADMM-G-Q: project p - g/tau on the level set, doubling tau until the stop condition holds.
-// Each trial ends with a read-back of the accept flag (the only host round trip of an iteration).
-static int p_step_quantised(pdadmm_ctx *c, int l, bool *hit_cap) {
+// pdADMM-G-Q: project p - g/tau on the level set, doubling tau until the stop condition holds.  Each trial ends
+// with a copy of the accept flag to the host, which decides whether another trial is needed (the only host round
+// trips of an iteration).  The two halves below let the caller queue another layer's work on the other lane before
+// it waits for the flag.
+// One trial: trial p, d = trial p - p and its codes, W d with its squared norm, the accept test, the flag's copy.
+static int q_trial(pdadmm_ctx *c, int l) {
   Layer &ly = c->layers[l];
   Scratch &s = *c->cur;
   const int N = (int)c->N;
-  const size_t n4p = (size_t)N * ly.ld_in / 4, n4r = (size_t)N * ly.ld_out / 4;
+  const size_t n4p = (size_t)N * ly.ld_in / 4;
+  const int grid = ew_grid(n4p);
+  uint32_t *w_d = nullptr;               // max|d| of this trial
+  if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_d = amax_take(c); }
+  {
+    Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
+    quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
+                                                     s.codes_new, c->code_bytes == 2, n4p, s.slots,
+                                                     c->use_tc ? ly.amax_p : nullptr, w_d);
+  }
+  int np = 0;
+  double *slots_b = s.slots + s.n_slots / 2;
+  EpiStoreSumsq epi{s.s2, ly.ld_out};
+  PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, planes_W(ly), epi,
+                           slots_b, &np, 0, w_d));
+  {
+    Launch k(c, KC_SMALL, s.st, 8.0 * (grid + np), 0);
+    finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
+  }
+  PD_CUDA(cudaMemcpyAsync(s.h_flag, &ly.sc->accepted, sizeof(int), cudaMemcpyDeviceToHost, s.st));
+  PD_CUDA(cudaEventRecord(s.ev_flag, s.st));
+  return PDADMM_OK;
+}
+// After the first trial of layer l was queued on the current lane: wait for its flag, run further trials while it
+// says no, then take the trial: p, codes <- trial, r <- r + W d.
+static int q_finish(pdadmm_ctx *c, int l, bool *hit_cap) {
+  Layer &ly = c->layers[l];
+  Scratch &s = *c->cur;
+  const size_t n4r = (size_t)c->N * ly.ld_out / 4;
   const int max_trials = 30;
   for (int trial = 0;; ++trial) {
-    const int grid = ew_grid(n4p);
-    uint32_t *w_d = nullptr;               // max|d| of this trial
-    if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_d = amax_take(c); }
-    {
-      Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
-      quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
-                                                       s.codes_new, c->code_bytes == 2, n4p, s.slots,
-                                                       c->use_tc ? ly.amax_p : nullptr, w_d);
-    }
-    int np = 0;
-    double *slots_b = s.slots + s.n_slots / 2;
-    EpiStoreSumsq epi{s.s2, ly.ld_out};
-    PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, planes_W(ly), epi,
-                             slots_b, &np, 0, w_d));
-    {
-      Launch k(c, KC_SMALL, s.st, 8.0 * (grid + np), 0);
-      finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
-    }
-    PD_CUDA(cudaMemcpyAsync(c->h_pinned, &ly.sc->accepted, sizeof(int), cudaMemcpyDeviceToHost, s.st));
-    PD_CUDA(cudaStreamSynchronize(s.st));
-    if (c->h_pinned[0] || trial + 1 >= max_trials) {
-      if (!c->h_pinned[0]) *hit_cap = true;
+    PD_CUDA(cudaEventSynchronize(s.ev_flag));
+    if (*s.h_flag || trial + 1 >= max_trials) {
+      if (!*s.h_flag) *hit_cap = true;
       break;
     }
+    PD_TRY(q_trial(c, l));
   }
   std::swap(ly.p, s.p_new);
   std::swap(ly.codes, s.codes_new);
   {
-    Launch k(c, KC_AXPY, s.st, 12.0 * N * ly.n_out, 0);
+    Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_out, 0);
     add_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, n4r, ly.amax_r);
   }
   return PDADMM_OK;
@@ -652,18 +667,36 @@ static int iterate_once(pdadmm_ctx *c, bool *hit_cap) {
   if (c->use_tc)
     for (int i = 0; i < S; ++i) { c->cur = &lane(c, i); PD_TRY(amax_reset(c, c->cur->st)); }
   // p-update of layers 2..L from the iterates of the previous iteration.  The quantised update reads an accept
-  // flag on the host after every trial, so it stays on the main stream.
+  // flag on the host after every trial: the host queues layer l's gradient and first trial on its lane, and only
+  // then waits for the flag of the layer that it queued on that lane before (layer l - S), so that the GPU always
+  // has the other lane's work while a flag travels.
+  std::vector<int> waiting(S, -1);                   // layer whose first trial is in flight on each lane
   for (int l = 1; l < c->L; ++l) {
-    c->cur = c->levels ? &c->scr : &lane_of(l);
-    PD_TRY(p_gradient_and_tau(c, l));
-    if (c->levels) PD_TRY(p_step_quantised(c, l, hit_cap));
-    else p_step_plain(c, l);
-    if (S > 1) PD_CUDA(cudaEventRecord(c->ev_p[l], c->cur->st));
+    c->cur = &lane_of(l);
+    if (c->levels) {
+      int &w = waiting[l % S];
+      if (w >= 0) {
+        PD_TRY(q_finish(c, w, hit_cap));
+        if (S > 1) PD_CUDA(cudaEventRecord(c->ev_p[w], c->cur->st));
+      }
+      PD_TRY(p_gradient_and_tau(c, l));
+      PD_TRY(q_trial(c, l));
+      w = l;
+    } else {
+      PD_TRY(p_gradient_and_tau(c, l));
+      p_step_plain(c, l);
+      if (S > 1) PD_CUDA(cudaEventRecord(c->ev_p[l], c->cur->st));
+    }
+  }
+  for (int i = 0; i < S && c->levels; ++i) {
+    if (waiting[i] < 0) continue;
+    c->cur = &lane(c, i);
+    PD_TRY(q_finish(c, waiting[i], hit_cap));
+    if (S > 1) PD_CUDA(cudaEventRecord(c->ev_p[waiting[i]], c->cur->st));
   }
   // W- and b-update of every layer with the new p
   for (int l = 0; l < c->L; ++l) {
     c->cur = &lane_of(l);
-    if (S > 1 && l >= 1 && c->levels && c->cur != &c->scr) PD_CUDA(cudaStreamWaitEvent(c->cur->st, c->ev_p[l], 0));
     PD_TRY(w_and_b_step(c, l));
   }
   // z-, q-, u-update (q_l and u_l need p_{l+1} of this iteration, which another lane may have written)
@@ -799,6 +832,17 @@ static int build_csr(pdadmm_ctx *c, const pdadmm_config *cfg) {
   return PDADMM_OK;
 }
 
+// buffers of a lane's quantised trials: trial p, d, codes (they trade places with a layer's p and codes when a
+// trial is taken, so all have one size), the pinned word and the event of the accept flag
+static int alloc_trial_buffers(pdadmm_ctx *c, Scratch &s, size_t n) {
+  PD_TRY(dev_alloc(c, &s.p_new, n));
+  PD_TRY(dev_alloc(c, &s.d, n));
+  PD_TRY(dev_alloc(c, &s.codes_new, n * c->code_bytes));
+  PD_CUDA(cudaMallocHost((void **)&s.h_flag, sizeof(int)));
+  PD_CUDA(cudaEventCreateWithFlags(&s.ev_flag, cudaEventDisableTiming));
+  return PDADMM_OK;
+}
+
 // transposed planes of r_l (up to max_out columns) and of p_l, l >= 2 (up to max_in columns) of one lane
 static int alloc_transposed(pdadmm_ctx *c, Scratch &s, int max_out, int max_in) {
   if (max_out > 0) {
@@ -898,11 +942,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   const size_t e_max = (size_t)N * std::max(max_in, max_out);
   PD_TRY(dev_alloc(c, &s.s1, e_max));
   PD_TRY(dev_alloc(c, &s.s2, (size_t)N * max_out));
-  if (c->levels) {
-    PD_TRY(dev_alloc(c, &s.p_new, (size_t)N * max_in));
-    PD_TRY(dev_alloc(c, &s.d, (size_t)N * max_in));
-    PD_TRY(dev_alloc(c, &s.codes_new, (size_t)N * max_in * c->code_bytes));
-  }
+  if (c->levels) PD_TRY(alloc_trial_buffers(c, s, (size_t)N * max_in));
   PD_TRY(dev_alloc(c, &s.part, max_part));
   s.n_slots = std::max<size_t>((size_t)c->n_sms * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
   s.n_slots *= 2;                       // two halves: consecutive reductions of one layer use different halves
@@ -937,6 +977,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &x.s1, e_max));
     PD_TRY(dev_alloc(c, &x.s2, (size_t)N * max_out));
     PD_TRY(dev_alloc(c, &x.part, max_part));
+    if (c->levels) PD_TRY(alloc_trial_buffers(c, x, (size_t)N * max_in));
     x.n_slots = s.n_slots;
     PD_TRY(dev_alloc(c, &x.slots, x.n_slots));
     if (c->use_tc) {
@@ -1010,6 +1051,11 @@ static void destroy(pdadmm_ctx *c) {
   if (c->iter_graph) cudaGraphExecDestroy(c->iter_graph);
   for (auto e : c->ev_p) cudaEventDestroy(e);
   for (auto e : c->ev_lane) cudaEventDestroy(e);
+  for (int i = 0; i <= (int)c->more_lanes.size(); ++i) {
+    pd::Scratch &x = i == 0 ? c->scr : *c->more_lanes[i - 1];
+    if (x.h_flag) cudaFreeHost(x.h_flag);
+    if (x.ev_flag) cudaEventDestroy(x.ev_flag);
+  }
   for (auto &x : c->more_lanes) if (x->st) cudaStreamDestroy(x->st);
   if (c->scr.st) cudaStreamDestroy(c->scr.st);
   delete c;
