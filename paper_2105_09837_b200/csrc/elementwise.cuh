@@ -83,7 +83,22 @@ axpy_neg_kernel(float *__restrict__ y, const float *__restrict__ x, const float 
                 uint32_t *__restrict__ amax /* receives max|y| (see commit_amax); may be null */) {
   const float a = *inv;
   uint32_t m = 0u;
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
+  // four groups per pass: eight loads in flight per thread
+  for (; i + 3 * stride < n4; i += 4 * stride) {
+    float4 v[4], w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { v[k] = ld4(y, i + k * stride); w[k] = ld4(x, i + k * stride); }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      v[k].x = fmaf(-a, w[k].x, v[k].x); v[k].y = fmaf(-a, w[k].y, v[k].y);
+      v[k].z = fmaf(-a, w[k].z, v[k].z); v[k].w = fmaf(-a, w[k].w, v[k].w);
+      st4(y, i + k * stride, v[k]);
+      m = max(m, abs_bits(v[k]));
+    }
+  }
+  for (; i < n4; i += stride) {
     float4 v = ld4(y, i);
     const float4 w = ld4(x, i);
     v.x = fmaf(-a, w.x, v.x); v.y = fmaf(-a, w.y, v.y); v.z = fmaf(-a, w.z, v.z); v.w = fmaf(-a, w.w, v.w);
