@@ -246,8 +246,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++ti) {
         int m0, n0, k_begin, n_kb, z;
         tile_coords(tile, m0, n0, k_begin, n_kb, z);
-        // the correction tile of the previous output tile must have been read before it is overwritten
-        if (ti > 0 && n_kb > 0) ok = ptx::mbar_wait(corr_empty, (ti - 1) & 1, abort_flag);
         for (int kb = 0; kb < n_kb && ok; ++kb) {
           const bool first = kb % TC_FLUSH == 0, last = kb % TC_FLUSH == TC_FLUSH - 1 || kb == n_kb - 1;
           if (!seen_conv) ok = ptx::mbar_wait(&ready_bar[s], sp, abort_flag);
@@ -263,22 +261,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int b_next = b + 1 == TC_ACC_BUFS ? 0 : b + 1;
           const uint32_t bp_next = b + 1 == TC_ACC_BUFS ? bp ^ 1u : bp;
           const bool round_next = first_round && b + 1 != TC_ACC_BUFS;
-#pragma unroll
-          for (int kk = 0; kk < TC_KSTEPS; ++kk) {
+          // the MMAs of K step kk: the two correction terms and / or the main term
+          auto issue = [&](int kk, bool corr, bool main) {
             const uint32_t ah = ta + 8u * kk, al = ah + 32u;
             const uint64_t dbh = ptx::smem_desc(hi_b, lb + kk * step_b);
             const uint64_t dbl = ptx::smem_desc(hi_b, lb + (TC_PLANE_BYTES >> 4) + kk * step_b);
             if constexpr (PP) {
               const uint64_t dah = ptx::smem_desc(hi_b, la + kk * step_b);
               const uint64_t dal = ptx::smem_desc(hi_b, la + (TC_PLANE_BYTES >> 4) + kk * step_b);
-              ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
-              ptx::mma_f16(d_corr, dah, dbl, idesc, true);
-              ptx::mma_f16(d, dah, dbh, idesc, !first || kk > 0);
+              if (corr) {
+                ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
+                ptx::mma_f16(d_corr, dah, dbl, idesc, true);
+              }
+              if (main) ptx::mma_f16(d, dah, dbh, idesc, !first || kk > 0);
             } else {
-              ptx::mma_f16_ts(d_corr, al, dbh, idesc, kb > 0 || kk > 0);
-              ptx::mma_f16_ts(d_corr, ah, dbl, idesc, true);
-              ptx::mma_f16_ts(d, ah, dbh, idesc, !first || kk > 0);
+              if (corr) {
+                ptx::mma_f16_ts(d_corr, al, dbh, idesc, kb > 0 || kk > 0);
+                ptx::mma_f16_ts(d_corr, ah, dbl, idesc, true);
+              }
+              if (main) ptx::mma_f16_ts(d, ah, dbh, idesc, !first || kk > 0);
             }
+          };
+          const bool split_first = kb == 0 && ti > 0;
+          if (split_first) {
+            // The correction tile still holds the previous output tile until the accumulate warps have read it:
+            // the main-term MMAs of this block, which do not touch it, go first and keep the tensor pipe busy
+            // while that read finishes.
+#pragma unroll
+            for (int kk = 0; kk < TC_KSTEPS; ++kk) issue(kk, false, true);
+            ok = ptx::mbar_wait(corr_empty, (ti - 1) & 1, abort_flag);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+          }
+#pragma unroll
+          for (int kk = 0; kk < TC_KSTEPS; ++kk) {
+            issue(kk, true, !split_first);
             if (kk == TC_KSTEPS - 2) {
               // probe the coming block's barriers while the tensor pipe still has work queued
               seen_conv = ptx::mbar_test_wait(&ready_bar[s_next], sp_next);
