@@ -375,7 +375,10 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
   int n_units = n_tiles;
   const int tail = n_tiles % c->n_sms, n_kb = (int)ceil_div(K, TC_BK);
   if (tail > 0 && c->cur->tail_ws != nullptr) {
-    const int split = std::min(std::min(c->n_sms / tail, n_kb / 2), 8);     // at least 2 K blocks per slice
+    // at least 8 K blocks per slice: parking and merging the slices of a tile costs about as much as four K blocks,
+    // and with two lanes the other layer's kernels fill the SMs that a short last round leaves idle (workload c2,
+    // 8 K blocks per tile: 281 iterations/s with 4 slices of 2 blocks, 289 without)
+    const int split = std::min(std::min(c->n_sms / tail, n_kb / 8), 8);
     if (split > 1) {
       prm.tail_begin = n_tiles - tail; prm.tail_split = split;
       prm.tail_ws = c->cur->tail_ws; prm.tail_count = c->cur->tail_count;
