@@ -203,6 +203,29 @@ def test_get_set_round_trip_and_size_checks():
     ctx.destroy()
 
 
+@pytest.mark.parametrize("levels", [0, 16])
+def test_lanes_and_graph_replay_do_not_change_a_bit(levels):
+    """The layers' kernels run on two concurrent lanes and, for pdADMM-G, from a captured graph.  Every reduction
+    has a fixed order and every lane its own scratch, so the iterates must be bit-identical to those of a run that
+    queues everything on one stream and launches directly: a difference would mean a race between lanes."""
+    inp = synth.make_inputs(synth.small("c2", 3000, feat_dim=40, hidden=150, n_layers=5, quant_levels=levels))
+    ref = None
+    for flags in (B.FLAG_ONE_LANE | B.FLAG_NO_GRAPH, B.FLAG_ONE_LANE, B.FLAG_NO_GRAPH, 0):
+        ctx = B.from_inputs(inp, flags=flags)
+        ctx.step(2)
+        ctx.step(3)                                   # the second call replays the graph where there is one
+        st = U.read_state(ctx)
+        obj = ctx.objective()
+        ctx.destroy()
+        if ref is None:
+            ref = (st, obj)
+            continue
+        for k in st:
+            for a, b in zip(st[k], ref[0][k]):
+                assert np.array_equal(a, b), (flags, k)
+        assert np.array_equal(obj, ref[1])
+
+
 def test_profile_counters_and_launch_count():
     inp = synth.make_inputs(synth.small("c2", 400, feat_dim=8, hidden=12, n_layers=3))
     ctx = B.from_inputs(inp)
