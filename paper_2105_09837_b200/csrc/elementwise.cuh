@@ -295,8 +295,8 @@ make_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, cons
 // contracts over the nodes (the W-gradient r^T p+), for layers where splitting them once here is cheaper than
 // splitting them once per output tile inside that product.  Scaling and split as in make_planes_kernel; the
 // exponent goes to *exp_out.
-// A warp handles 32 nodes x 16 columns: lane (q, g) loads the 4 x 4 block of nodes 4q..4q+3, columns 4g..4g+3
-// (four 16-byte loads, 64 contiguous bytes per row and warp), transposes it in registers and stores, per column,
+// A warp handles 32 nodes x 32 columns: lane (q, g) loads the 4 x 8 block of nodes 4q..4q+3, columns 8g..8g+7
+// (eight 16-byte loads, 128 contiguous bytes per row and warp), transposes it in registers and stores, per column,
 // the four nodes as 8 bytes of each plane (64 contiguous bytes per column and warp): whole sectors both ways, no
 // shared memory.  Tiles are numbered with the node index fastest.
 __global__ void __launch_bounds__(256)
@@ -306,19 +306,23 @@ transpose_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld,
   if (blockIdx.x == 0 && threadIdx.x == 0) *exp_out = e;
   const float scale = __uint_as_float((uint32_t)(e + 127) << 23);
   const int lane = threadIdx.x & 31, q = lane & 7, g = lane >> 3;
-  const long long row_tiles = (rows + 31) / 32, n_tiles = row_tiles * ((cols + 15) / 16);
+  const long long row_tiles = (rows + 31) / 32, n_tiles = row_tiles * ((cols + 31) / 32);
   for (long long wt = blockIdx.x * 8ll + (threadIdx.x >> 5); wt < n_tiles; wt += gridDim.x * 8ll) {
-    const int node0 = (int)(wt % row_tiles) * 32 + 4 * q, col = (int)(wt / row_tiles) * 16 + 4 * g;
+    const int node0 = (int)(wt % row_tiles) * 32 + 4 * q, col = (int)(wt / row_tiles) * 32 + 8 * g;
     if (node0 >= rows || col >= cols) continue;
-    float v[4][4];
+    float v[4][8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (node0 + i < rows) t = *reinterpret_cast<const float4 *>(x + (size_t)(node0 + i) * ld + col);   // col + 3 < ld
-      v[i][0] = t.x; v[i][1] = t.y; v[i][2] = t.z; v[i][3] = t.w;
+      float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f), t1 = t0;
+      if (node0 + i < rows) {                  // ld is a multiple of 4: a group of 4 columns is inside the row or not
+        t0 = *reinterpret_cast<const float4 *>(x + (size_t)(node0 + i) * ld + col);
+        if (col + 4 < ld) t1 = *reinterpret_cast<const float4 *>(x + (size_t)(node0 + i) * ld + col + 4);
+      }
+      v[i][0] = t0.x; v[i][1] = t0.y; v[i][2] = t0.z; v[i][3] = t0.w;
+      v[i][4] = t1.x; v[i][5] = t1.y; v[i][6] = t1.z; v[i][7] = t1.w;
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < 8; ++j) {
       if (col + j >= cols) break;
       float h[4], l[4];
 #pragma unroll

@@ -393,7 +393,7 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
 static void transpose_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, int rows, int cols, int ld,
                              const uint32_t *amax, __half *hiT, __half *loT, int ldT, int *exp_out) {
   Launch l(c, KC_PLANES, st, 8.0 * rows * cols, 0);
-  const int64_t warp_tiles = ceil_div(rows, 32) * ceil_div(cols, 16);
+  const int64_t warp_tiles = ceil_div(rows, 32) * ceil_div(cols, 32);
   const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(ceil_div(warp_tiles, 8), 148 * 16));
   transpose_planes_kernel<<<grid, 256, 0, st>>>(x, rows, cols, ld, amax, exp_out, hiT, loT, ldT);
 }
