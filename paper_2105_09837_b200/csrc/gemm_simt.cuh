@@ -40,6 +40,17 @@ struct EpiStoreSumsq {        // C = acc, accumulates sum(acc^2)
     return a;
   }
 };
+struct EpiNormOnly {          // nothing is stored: only sum(acc^2) is wanted (||W g||^2 of the quantised update, whose
+                              // step uses W d instead of W g)
+  static constexpr bool kDirect = true, kSumsq = true, kStore = false;
+  static constexpr int kInputs = 0;
+  float *C; int ldc;          // ldc = padded width of the output; C is written by the CUDA-core kernels only
+  __device__ __forceinline__ void prefetch(int, int) const {}
+  __device__ __forceinline__ float4 operator()(int, int, float4 a, double &ss) const {
+    ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
+    return a;
+  }
+};
 struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b - z)
   static constexpr bool kDirect = false, kSumsq = false;
   static constexpr int kInputs = 1;        // float4 loads per output group: load() fetches, apply() combines

@@ -22,6 +22,8 @@
 
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "gemm_simt.cuh"   // epilogue functors
 #include "tc_ptx.cuh"
@@ -66,6 +68,10 @@ __device__ __forceinline__ void tc_split8(const float (&x)[8], float scale, uint
   h = make_uint4(pack(hi[0], hi[1]), pack(hi[2], hi[3]), pack(hi[4], hi[5]), pack(hi[6], hi[7]));
   l = make_uint4(pack(lo[0], lo[1]), pack(lo[2], lo[3]), pack(lo[4], lo[5]), pack(lo[6], lo[7]));
 }
+
+// Epilogues store their result unless they say otherwise (kStore = false).
+template <class Epi, class = void> struct epi_stores { static constexpr bool value = true; };
+template <class Epi> struct epi_stores<Epi, std::enable_if_t<!Epi::kStore>> { static constexpr bool value = false; };
 
 struct TcParams {
   int M, N, K;            // output rows, output columns, contraction length
@@ -504,7 +510,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // time, lanes 8g..8g+7 take row 4 step + g, 4 consecutive columns per lane.  The loads of four or eight steps
       // are issued together (rows past the end are clamped, their results dropped).
       double ss = 0.0;
-      {
+      if constexpr (!epi_stores<Epi>::value) {
+        // only the squared norm: straight from the registers (rows and columns outside the matrix hold exact zeros)
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < 64; ++j) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
+        ss = ((double)s4[0] + (double)s4[1]) + ((double)s4[2] + (double)s4[3]);
+      } else {
         float *C = epi.C + (size_t)z * prm.c_split_stride;
         float ssf = 0.f;
         uint32_t mx = 0u;                  // largest magnitude stored by this thread

@@ -480,9 +480,16 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
                           epi, s.slots, &np, 4.0 * N * ly.n_in, ly.amax_r));
   int np2 = 0;
   double *slots_b = s.slots + s.n_slots / 2;          // second half of the slot buffer
-  EpiStoreSumsq epi2{s.s2, ly.ld_out};
-  PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
-                           epi2, slots_b, &np2, 0, w_g));
+  if (c->levels && c->use_tc) {
+    // the quantised update only needs ||W g||^2 (for the first tau); its residual update uses W d
+    EpiNormOnly epi2{s.s2, ly.ld_out};
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
+                             epi2, slots_b, &np2, 0, w_g));
+  } else {
+    EpiStoreSumsq epi2{s.s2, ly.ld_out};
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
+                             epi2, slots_b, &np2, 0, w_g));
+  }
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
     finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2,
