@@ -159,7 +159,9 @@ struct pdadmm_ctx {
   std::vector<cudaEvent_t> ev_pool;
   double prof_ms[pd::KC_COUNT] = {0}, prof_bytes[pd::KC_COUNT] = {0}, prof_flops[pd::KC_COUNT] = {0};
   int64_t prof_n[pd::KC_COUNT] = {0};
-  std::vector<void *> allocs;
+  std::vector<void *> allocs;       // driver allocations: chunks and large arrays
+  char *arena_base = nullptr;       // current chunk
+  size_t arena_cap = 0, arena_used = 0, arena_next = size_t(64) << 20;
   bool use_tc = true;               // dense products on the tensor cores
   cudaGraphExec_t iter_graph = nullptr;   // one captured pdADMM-G iteration (no host round trips in it)
   int64_t iter_graph_launches = 0;
@@ -175,16 +177,35 @@ struct pdadmm_ctx {
 namespace pd {
 
 // ---- allocation bookkeeping -------------------------------------------------------------------------
+// Device memory of a context.  Arrays of up to 64 MB are carved out of chunks (64 MB at first, doubling up to
+// 1 GB), 256-byte aligned: a context has some twenty arrays per layer, and one driver allocation each made
+// pdadmm_init spend most of its time in the allocator.  Larger arrays get an allocation of their own, so that
+// a chunk never wastes more than one small array at its end.  Everything is released by destroy().
+constexpr size_t ARENA_MAX_ARRAY = size_t(64) << 20, ARENA_MAX_CHUNK = size_t(1) << 30;   // first chunk: arena_next
 template <class T>
 static int dev_alloc(pdadmm_ctx *c, T **ptr, size_t count, bool zero = true) {
-  void *p = nullptr;
-  const size_t bytes = count * sizeof(T) + 256;     // slack: operand copies may read up to 31 floats past a matrix
-  cudaError_t e = cudaMalloc(&p, bytes);
-  if (e != cudaSuccess) {
-    cudaGetLastError();
-    return fail(PDADMM_ENOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+  // slack: operand copies may read up to 31 floats past a matrix
+  const size_t bytes = (count * sizeof(T) + 256 + 255) & ~size_t(255);
+  char *p = nullptr;
+  if (bytes <= ARENA_MAX_ARRAY && c->arena_used + bytes <= c->arena_cap) {
+    p = c->arena_base + c->arena_used;
+    c->arena_used += bytes;
+  } else {
+    const bool chunk = bytes <= ARENA_MAX_ARRAY;
+    const size_t want = chunk ? std::max(bytes, c->arena_next) : bytes;
+    void *q = nullptr;
+    const cudaError_t e = cudaMalloc(&q, want);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return fail(PDADMM_ENOMEM, "cudaMalloc of %zu bytes failed: %s", want, cudaGetErrorString(e));
+    }
+    c->allocs.push_back(q);
+    p = (char *)q;
+    if (chunk) {
+      c->arena_base = p; c->arena_cap = want; c->arena_used = bytes;
+      c->arena_next = std::min(ARENA_MAX_CHUNK, 2 * want);
+    }
   }
-  c->allocs.push_back(p);
   if (zero) PD_CUDA(cudaMemsetAsync(p, 0, bytes, c->scr.st));   // same stream as every kernel that uses it
   *ptr = (T *)p;
   return PDADMM_OK;
