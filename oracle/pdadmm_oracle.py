@@ -80,6 +80,7 @@ class Params:
     level_lo: float = 0.0                 # smallest level delta_0
     level_step: float = 0.0               # > 0: the same fixed step for every layer; 0: step from max(p) at the start
     slope: float = 0.0                    # 0: f_l = ReLU; in (0, 1): leaky ReLU with that slope for x <= 0
+    risk: str = "ce"                      # R: "ce" cross-entropy (the paper's experiments), "ls" least squares
 
 
 @dataclasses.dataclass
@@ -368,6 +369,28 @@ def risk(zL, y, mask) -> float:
     return float(np.sum(ce[np.asarray(mask, dtype=bool)]))
 
 
+def risk_least_squares(zL, y, mask) -> float:
+    """R(z_L; y) = (1/2) sum over labelled nodes of ||z_L[:, j] - e_{y_j}||^2: another risk that Problem 1 admits
+    (Sec. "Problem Formulation" only asks R to be convex and continuous)."""
+    E = np.zeros_like(zL)
+    E[np.asarray(y), np.arange(zL.shape[1])] = 1.0
+    d = (zL - E)[:, np.asarray(mask, dtype=bool)]
+    return float(0.5 * np.sum(d * d))
+
+
+def update_z_last_least_squares(a, y, mask, nu):
+    """Eq. (update zl) with the least-squares risk: argmin_z (1/2)||z - e_y||^2 + (nu/2)||z - a||^2 per labelled
+    node, i.e. z = (e_y + nu a) / (1 + nu) (the stationary point of a strictly convex quadratic); unlabelled nodes
+    take z = a."""
+    z = np.array(a, dtype=np.float64)
+    lab = np.flatnonzero(np.asarray(mask, dtype=bool))
+    if lab.size:
+        E = np.zeros((a.shape[0], lab.size))
+        E[np.asarray(y)[lab], np.arange(lab.size)] = 1.0
+        z[:, lab] = (E + nu * a[:, lab]) / (1.0 + nu)
+    return z
+
+
 def softmax_col(z_col):
     e = np.exp(z_col - np.max(z_col))
     return e / np.sum(e)
@@ -586,6 +609,8 @@ def iterate(s: State, prm: Params) -> State:
         a = n.W[l] @ n.p[l] + n.b[l][:, None]
         if l < L - 1:
             n.z[l] = update_z_hidden(a, s.q[l], s.z[l], prm.slope)
+        elif prm.risk == "ls":
+            n.z[l] = update_z_last_least_squares(a, s.y, s.mask, nu)
         else:
             n.z[l] = update_z_last(a, s.y, s.mask, nu)
     # q_l^{k+1}, then u_l^{k+1}
@@ -609,7 +634,7 @@ def objective(s: State, prm: Params) -> np.ndarray:
     """Components of the augmented Lagrangian L_rho and their sum:
     [R, (nu/2) sum||z - W p - b||^2, (nu/2) sum||q - f(z)||^2, sum<u, p+ - q>, (rho/2) sum||p+ - q||^2, L_rho]."""
     rho, nu, L = prm.rho, prm.nu, s.L
-    R = risk(s.z[L - 1], s.y, s.mask)
+    R = risk_least_squares(s.z[L - 1], s.y, s.mask) if prm.risk == "ls" else risk(s.z[L - 1], s.y, s.mask)
     lin = sum(float(np.sum((s.z[l] - s.W[l] @ s.p[l] - s.b[l][:, None]) ** 2)) for l in range(L))
     act = sum(float(np.sum((s.q[l] - relu(s.z[l], prm.slope)) ** 2)) for l in range(L - 1))
     dual = sum(float(np.sum(s.u[l] * (s.p[l + 1] - s.q[l]))) for l in range(L - 1))
