@@ -67,6 +67,9 @@ typedef enum {
 #define PDADMM_FLAG_QUANT_Q 2u       /* pdADMM-G-Q variant that keeps q_l on the level set of p_{l+1} as well   */
 #define PDADMM_FLAG_NO_GRAPH 4u      /* launch every kernel of an iteration directly instead of replaying a CUDA graph */
 #define PDADMM_FLAG_ONE_LANE 8u      /* queue all layers on one stream instead of spreading them over concurrent lanes */
+#define PDADMM_FLAG_LEAST_SQUARES 16u /* R(z_L; y) = 1/2 sum over labelled nodes ||z_L - e_y||^2 instead of the cross-entropy
+                                         (paper, "Problem Formulation": R is any convex, continuous risk); the z_L
+                                         update then is the closed form z = (e_y + nu a)/(1 + nu)          */
 
 /*
  * Problem statement (paper: Problem 2 / Problem 3, Algorithm 1 "Require", and the experimental

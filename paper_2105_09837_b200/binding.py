@@ -22,6 +22,7 @@ FLAG_SIMT_GEMM = 1
 FLAG_QUANT_Q = 2
 FLAG_NO_GRAPH = 4
 FLAG_ONE_LANE = 8
+FLAG_LEAST_SQUARES = 16
 
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 

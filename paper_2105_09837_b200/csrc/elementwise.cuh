@@ -482,13 +482,17 @@ constexpr int ZL_MAX_C = 64;
 __global__ void __launch_bounds__(128)
 zlast_kernel(float *__restrict__ r, float *__restrict__ z, const float *__restrict__ shift,
              const int *__restrict__ labels, const uint8_t *__restrict__ mask, int n_rows, int C, int ld,
-             double nu, int *__restrict__ not_converged, uint32_t *__restrict__ amax_r /* max|r|, may be null */) {
+             double nu, int *__restrict__ not_converged, uint32_t *__restrict__ amax_r /* max|r|, may be null */,
+             int least_squares /* R = 1/2 ||z - e_y||^2: z+ = (e_y + nu a)/(1 + nu) */) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n_rows) return;
   float *rj = r + (size_t)j * ld, *zj = z + (size_t)j * ld;
   double a[ZL_MAX_C], x[ZL_MAX_C], s[ZL_MAX_C], st[ZL_MAX_C];
   for (int c = 0; c < C; ++c) { a[c] = (double)((rj[c] - shift[c]) + zj[c]); x[c] = a[c]; }
-  if (mask[j]) {
+  if (mask[j] && least_squares) {
+    const int y = labels[j];
+    for (int c = 0; c < C; ++c) x[c] = ((c == y ? 1.0 : 0.0) + nu * a[c]) / (1.0 + nu);
+  } else if (mask[j]) {
     const int y = labels[j];
     auto fval = [&](const double *v) {
       double m = v[0];
@@ -609,15 +613,25 @@ objective_layer_kernel(const float *__restrict__ r, const float *__restrict__ z,
   t = block_sum<EW_THREADS>(s3, red); if (threadIdx.x == 0) slots[blockIdx.x * 4 + 3] = t;
 }
 
-// R(z_L; y): sum over masked nodes of -z_y + logsumexp(z).  One thread per node, one slot per block.
+// R(z_L; y): sum over masked nodes of -z_y + logsumexp(z), or of 1/2 ||z - e_y||^2 (least_squares).
+// One thread per node, one slot per block.
 __global__ void __launch_bounds__(EW_THREADS)
 risk_kernel(const float *__restrict__ z, const int *__restrict__ labels, const uint8_t *__restrict__ mask,
-            int n_rows, int C, int ld, double *__restrict__ slots) {
+            int n_rows, int C, int ld, double *__restrict__ slots, int least_squares) {
   __shared__ double red[EW_THREADS / 32];
   double acc = 0.0;
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n_rows; j += gridDim.x * blockDim.x) {
     if (!mask[j]) continue;
     const float *zj = z + (size_t)j * ld;
+    if (least_squares) {
+      double sq = 0.0;
+      for (int c = 0; c < C; ++c) {
+        const double d = (double)zj[c] - (c == labels[j] ? 1.0 : 0.0);
+        sq += d * d;
+      }
+      acc += 0.5 * sq;
+      continue;
+    }
     double m = zj[0];
     for (int c = 1; c < C; ++c) m = fmax(m, (double)zj[c]);
     double se = 0.0;

@@ -129,6 +129,7 @@ struct pdadmm_ctx {
   float fixed_step = 0.f;          // > 0: the same level spacing for every layer
   bool quant_q = false;            // q_l is kept on the level set of p_{l+1} as well
   float slope = 0.f;               // f_l: 0 = ReLU, (0, 1) = leaky ReLU with that slope for x <= 0
+  bool ls_risk = false;            // R = least squares instead of cross-entropy
   float rho = 0, nu = 0;
   uint32_t flags = 0;
   int64_t nnz = 0;
@@ -679,7 +680,7 @@ static void zqu_step(pdadmm_ctx *c, int l) {
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
     zlast_kernel<<<(int)ceil_div(N, 128), 128, 0, s.st>>>(ly.r, ly.z, ly.shift, c->labels, c->mask, N, ly.n_out,
-                                                          ly.ld_out, (double)c->nu, c->d_flag, ly.amax_r);
+                                                          ly.ld_out, (double)c->nu, c->d_flag, ly.amax_r, c->ls_risk ? 1 : 0);
   }
 }
 
@@ -897,6 +898,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->code_bytes = cfg->quant_levels > 256 ? 2 : 1;
   c->quant_q = (cfg->flags & PDADMM_FLAG_QUANT_Q) != 0;
   c->slope = cfg->leaky_slope;
+  c->ls_risk = (cfg->flags & PDADMM_FLAG_LEAST_SQUARES) != 0;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
   PD_CUDA(cudaSetDevice(cfg->device));
@@ -1252,7 +1254,8 @@ extern "C" int pdadmm_objective(pdadmm_ctx *c, double out[6]) {
   {
     Layer &ly = c->layers[c->L - 1];
     const int grid = (int)std::min<int64_t>(512, ceil_div(c->N, EW_THREADS));
-    risk_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, c->labels, c->mask, (int)c->N, ly.n_out, ly.ld_out, c->scr.slots);
+    risk_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, c->labels, c->mask, (int)c->N, ly.n_out, ly.ld_out, c->scr.slots,
+                                             c->ls_risk ? 1 : 0);
     PD_TRY(read_slots(c, grid, 1, 1, &R));
   }
   PD_CUDA(cudaGetLastError());

@@ -9,14 +9,15 @@ import oracle.pdadmm_oracle as o
 from paper_2105_09837_b200 import binding as B
 
 
-def oracle_problem(inp, rho=None, nu=None, quant_levels=None, quantize_q=False, neg_levels=0, step=0.0, slope=0.0):
+def oracle_problem(inp, rho=None, nu=None, quant_levels=None, quantize_q=False, neg_levels=0, step=0.0, slope=0.0,
+                   risk="ce"):
     """(Params, initial oracle State) for a synth.Inputs bundle.  neg_levels / step: a fixed level set
     {(c - neg_levels) step} as the C ABI's quant_neg_levels / quant_step describe it."""
     w = inp.workload
     lo = float(np.float32(-neg_levels) * np.float32(step))
     prm = o.Params(w.rho if rho is None else rho, w.nu if nu is None else nu,
                    w.quant_levels if quant_levels is None else quant_levels,
-                   quantize_q=quantize_q, level_lo=lo, level_step=step, slope=slope)
+                   quantize_q=quantize_q, level_lo=lo, level_step=step, slope=slope, risk=risk)
     A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
     X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
     s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels, inp.train_mask, prm)

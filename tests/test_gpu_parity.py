@@ -258,6 +258,23 @@ def test_teacher_forced_leaky_relu(case, slope, levels, neg, step):
     ctx.destroy()
 
 
+@pytest.mark.parametrize("case,levels", [("er-small", 0), ("ba-ragged", 0), ("c4-like", 64)])
+def test_teacher_forced_least_squares_risk(case, levels):
+    """R = least squares (PDADMM_FLAG_LEAST_SQUARES): the last layer's z-update is its closed form and the
+    objective's first component is that risk; everything else is unchanged."""
+    inp = _inputs(case, quant_levels=levels)
+    prm, s, _ = U.oracle_problem(inp, risk="ls")
+    ctx = B.from_inputs(inp, flags=B.FLAG_LEAST_SQUARES)
+    for k in range(4):
+        prev = U.round_state(s)
+        U.load_state(ctx, prev, levels > 0)
+        s = _compare_iteration(ctx, prev, prm, f"{case}/ls/k={k}")
+    got, want = ctx.objective(), o.objective(s, prm)
+    assert abs(got[0] - want[0]) <= 1e-4 * abs(want[0]) and abs(got[5] - want[5]) <= 1e-3 * abs(want[5])
+    assert abs(want[0] - o.risk(s.z[-1], s.y, s.mask)) > 1e-2 * abs(want[0])     # not the cross-entropy
+    ctx.destroy()
+
+
 def ctx_weights(ctx):
     L = ctx.n_layers
     return ([ctx.get_tensor(B.T_W, l).astype(np.float64) for l in range(1, L + 1)],
