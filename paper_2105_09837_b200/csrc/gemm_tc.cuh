@@ -12,11 +12,12 @@
 //
 // TMA brings fp32 tiles of the node-sized operand into shared memory; converter warps turn them into the two
 // fp16 planes, which they write to tensor memory; the small operand (a weight matrix) arrives as two precomputed
-// fp16 planes (K-major, 128-byte swizzle).  One thread issues tcgen05.mma; completion is tracked with mbarriers; eight more
-// warps read each K block's main term from tensor memory, add it to a register accumulator and finally apply
-// the scaling and the fused epilogue.
+// fp16 planes (K-major, 128-byte swizzle).  One thread issues tcgen05.mma; completion is tracked with mbarriers;
+// eight more warps read each K block's main term from tensor memory, add it to a register accumulator and finally
+// apply the scaling and the fused epilogue.
 //
-// Tile: 128 x 128 outputs per CTA, 64-deep K blocks, 3 stages of 64 KB, four accumulator tiles in tensor memory.
+// Tile: 128 x 128 outputs per CTA, 64-deep K blocks, 3 stages of 64 KB.  Tensor memory (512 columns): two
+// accumulator tiles for the main term, one for the correction terms, two slots for the planes of A.
 // Every wait is bounded; a wait that expires raises an error word in global memory and the CTA drains and exits.
 #pragma once
 
