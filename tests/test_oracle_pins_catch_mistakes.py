@@ -8,6 +8,8 @@ import pytest
 import oracle.pdadmm_oracle as o
 import test_oracle_graph as tg
 import test_oracle_iteration as ti
+import test_oracle_objective as tobj
+import test_oracle_quantised_q as tq
 import test_oracle_subproblems as ts
 
 
@@ -65,6 +67,55 @@ def _quantize_truncating(x, scale, m, lo=0.0):
     return c.astype(np.uint8 if m <= 256 else np.uint16), (np.float32(lo) + c * np.float32(scale)).astype(np.float64)
 
 
+
+def _objective_variant(rho_factor=1.0, dual_sign=1.0, lin_factor=1.0, act_factor=1.0, dual_factor=1.0):
+    """L_rho with one component scaled, dropped or sign-flipped."""
+    def wrong(s, prm):
+        rho, nu, L = prm.rho, prm.nu, s.L
+        R = o.risk_least_squares(s.z[L - 1], s.y, s.mask) if prm.risk == "ls" else o.risk(s.z[L - 1], s.y, s.mask)
+        lin = sum(float(np.sum((s.z[l] - s.W[l] @ s.p[l] - s.b[l][:, None]) ** 2)) for l in range(L))
+        act = sum(float(np.sum((s.q[l] - o.relu(s.z[l], prm.slope)) ** 2)) for l in range(L - 1))
+        dual = sum(float(np.sum(s.u[l] * (s.p[l + 1] - s.q[l]))) for l in range(L - 1))
+        pen = sum(float(np.sum((s.p[l + 1] - s.q[l]) ** 2)) for l in range(L - 1))
+        comps = [R, lin_factor * 0.5 * nu * lin, act_factor * 0.5 * nu * act, dual_sign * dual_factor * dual,
+                 rho_factor * 0.5 * rho * pen]
+        return np.array(comps + [sum(comps)])
+    return wrong
+
+
+def _residuals_without_the_square(s):
+    return np.array([float(np.sum(np.abs(s.p[l + 1] - s.q[l]))) for l in range(s.L - 1)])
+
+
+def _residuals_doubled(s):
+    return np.array([2.0 * float(np.sum((s.p[l + 1] - s.q[l]) ** 2)) for l in range(s.L - 1)])
+
+
+def _residuals_of_the_wrong_pair(s):
+    return np.array([float(np.sum((s.p[l] [:s.q[l].shape[0]] - s.q[l]) ** 2)) if s.p[l].shape[0] >= s.q[l].shape[0]
+                     else 0.0 for l in range(s.L - 1)])
+
+
+def _risk_as_a_mean(zL, y, mask):
+    m = np.max(zL, axis=0)
+    ce = m + np.log(np.sum(np.exp(zL - m[None, :]), axis=0)) - zL[y, np.arange(zL.shape[1])]
+    return float(np.mean(ce[np.asarray(mask, dtype=bool)]))
+
+
+def _nearest_level_rounding_down_at_ties(x, scale, m, lo=0.0):
+    x = np.asarray(x, dtype=np.float64)
+    lev = o.level_set(scale, m, lo)
+    c = np.clip(np.ceil((x - lo) / scale - 0.5), 0, m - 1).astype(np.int64)
+    return c.astype(np.uint8 if m <= 256 else np.uint16), lev[c]
+
+
+def _nearest_level_truncating(x, scale, m, lo=0.0):
+    x = np.asarray(x, dtype=np.float64)
+    lev = o.level_set(scale, m, lo)
+    c = np.clip(np.floor((x - lo) / scale), 0, m - 1).astype(np.int64)
+    return c.astype(np.uint8 if m <= 256 else np.uint16), lev[c]
+
+
 _GOOD_ADJACENCY = o.renormalized_adjacency
 
 
@@ -85,10 +136,21 @@ MISTAKES = [
     ("update_b", _update_b_mean_of_wrong_thing, [ts.test_b_update_is_the_minimiser_grid_and_gradient], ()),
     ("quantize", _quantize_truncating, [tg.test_quantize_ties_and_clamps], ()),
     ("renormalized_adjacency", _adjacency_without_self_loops, [tg.test_golden_path_graph], ()),
+    ("nearest_level", _nearest_level_rounding_down_at_ties, [tq.test_nearest_level_is_the_argmin_over_all_levels], (22, 1.0, -1.0)),
+    ("nearest_level", _nearest_level_truncating, [tq.test_nearest_level_is_the_argmin_over_all_levels], (16, 0.0173, -0.0371)),
+    ("objective", _objective_variant(rho_factor=2.0), [tobj.test_objective_components_equal_the_hand_worked_values], ()),
+    ("objective", _objective_variant(dual_sign=-1.0), [tobj.test_objective_components_equal_the_hand_worked_values], ()),
+    ("objective", _objective_variant(lin_factor=2.0), [tobj.test_objective_components_equal_the_hand_worked_values], ()),
+    ("objective", _objective_variant(act_factor=0.0), [tobj.test_objective_components_equal_the_hand_worked_values], ()),
+    ("objective", _objective_variant(dual_factor=0.0), [tobj.test_objective_components_equal_the_hand_worked_values], ()),
+    ("residuals_sq", _residuals_without_the_square, [tobj.test_residuals_equal_the_hand_worked_values], ()),
+    ("residuals_sq", _residuals_doubled, [tobj.test_residuals_equal_the_hand_worked_values], ()),
+    ("residuals_sq", _residuals_of_the_wrong_pair, [tobj.test_residuals_equal_the_hand_worked_values], ()),
+    ("risk", _risk_as_a_mean, [tobj.test_objective_components_equal_the_hand_worked_values], ()),
 ]
 
 
-@pytest.mark.parametrize("name,wrong,tests,extra", MISTAKES, ids=[f"{m[0]}:{m[1].__name__}" for m in MISTAKES])
+@pytest.mark.parametrize("name,wrong,tests,extra", MISTAKES, ids=[f"{i}-{m[0]}:{m[1].__name__}" for i, m in enumerate(MISTAKES)])
 def test_planted_mistake_is_caught(monkeypatch, name, wrong, tests, extra):
     for t in tests:                                    # the pins pass on the oracle as it stands ...
         args = extra if t.__code__.co_argcount else ()
