@@ -12,7 +12,7 @@ paper's order: p (l = 2..L), W, b, z, q, residual, u.  Where the paper leaves a
 choice open the reading is stated in the function's docstring.
 
 Parity status: every function below is pinned by the CPU tests (grid search,
-closed forms, invariants); nothing is "parity unpinned".
+closed forms, invariants, hand-worked values); nothing is "parity unpinned".
 """
 
 from __future__ import annotations
@@ -220,16 +220,34 @@ def level_set(scale: float, m: int, lo: float = 0.0) -> np.ndarray:
     return (np.float32(lo) + np.arange(m, dtype=np.float32) * np.float32(scale)).astype(np.float64)
 
 
-def quantize(x, scale: float, m: int, lo: float = 0.0):
-    """Nearest element of Delta, element by element: argmin_delta |delta - x|.
+def nearest_level(x, scale: float, m: int, lo: float = 0.0):
+    """Nearest element of Delta, element by element, by definition: argmin_{delta in Delta} |delta - x| in double
+    precision, Delta = level_set(scale, m, lo).
 
-    Since ||delta - x||^2 is separable the argmin of Eq. (update p quantized)
-    is taken per element.  For uniform levels it is a rounding:
-    code = clamp(floor((x - lo)/s + 1/2), 0, m-1) (ties at half-levels go up).
-    The rounding decision is taken in single precision, the precision of the
-    kernel that takes the same decision.  Returns (codes, p in Delta); codes are
-    uint8 for up to 256 levels and uint16 above (the 8- and 16-bit cases of Sec.
-    "Communication Overheads").
+    ||delta - x||^2 is separable, so the argmin of Eq. (update p quantized) is taken per element.  The levels are
+    (nearly) uniform, so the rounding floor((x - lo)/s + 1/2) gives a candidate; because the levels themselves are
+    rounded single-precision numbers the candidate and its two neighbours are then compared by their actual
+    distances.  An exact tie between two levels goes to the upper one (the paper does not say; both are minimisers).
+    Returns (codes, p in Delta); codes are uint8 for up to 256 levels and uint16 above (the 8- and 16-bit cases of
+    Sec. "Communication Overheads").
+    """
+    x = np.asarray(x, dtype=np.float64)
+    lev = level_set(scale, m, lo)
+    c = np.clip(np.floor((x - float(np.float32(lo))) / float(np.float32(scale)) + 0.5), 0, m - 1).astype(np.int64)
+    best, best_d = c, np.abs(lev[c] - x)
+    for cand in (np.clip(c - 1, 0, m - 1), np.clip(c + 1, 0, m - 1)):
+        d = np.abs(lev[cand] - x)
+        take = (d < best_d) | ((d == best_d) & (cand > best))
+        best, best_d = np.where(take, cand, best), np.where(take, d, best_d)
+    return best.astype(np.uint8 if m <= 256 else np.uint16), lev[best]
+
+
+def quantize(x, scale: float, m: int, lo: float = 0.0):
+    """The same projection as a single-precision program computes it: code = clamp(floor((x - lo)/s + 1/2), 0, m-1)
+    with x, the division, the sum and the floor all in float32 (ties at half-levels go up), value = fl32(lo + fl32(c s)).
+
+    Not used by ``iterate``: it serves the comparisons in which both sides are handed identical float32 inputs and
+    the result has to agree bit for bit.  Returns (codes, p in Delta) like ``nearest_level``.
     """
     x32 = np.asarray(x, dtype=np.float32)
     t = (x32 - np.float32(lo)) / np.float32(scale)
@@ -260,7 +278,7 @@ def update_p_quantized(p, W, b, z, nu, q_prev, u_prev, rho, scale, m, max_trials
     tau = tau_smallest_admissible(g, W, nu, rho)
     phi_old = phi(p, W, b, z, nu, q_prev, u_prev, rho)
     for trial in range(1, max_trials + 1):
-        codes, p_new = quantize(p - g / tau, scale, m, lo)
+        codes, p_new = nearest_level(p - g / tau, scale, m, lo)
         d = p_new - p
         dd = float(np.sum(d * d))
         lhs = phi(p_new, W, b, z, nu, q_prev, u_prev, rho)
@@ -539,7 +557,7 @@ def update_q_quantized(p_next, u, z, rho, nu, scale, m, lo=0.0, slope: float = 0
     """The variant with q_l in Delta as well: q_l^{k+1} = argmin_{delta in Delta}
     ||delta - (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)||, element by element
     (Sec. "Quantization Extension", last paragraph).  Delta is the level set of p_{l+1}, which q_l has to equal."""
-    return quantize(update_q(p_next, u, z, rho, nu, slope), scale, m, lo)[1]
+    return nearest_level(update_q(p_next, u, z, rho, nu, slope), scale, m, lo)[1]
 
 
 def update_u(u, p_next, q, rho):
@@ -574,7 +592,7 @@ def init_state(X, W0, y, mask, prm: Params) -> State:
             if prm.quant_levels:
                 scale[l + 1] = (float(np.float32(prm.level_step)) if prm.level_step > 0
                                 else quantization_scale(q[l], prm.quant_levels))
-                p.append(quantize(q[l], scale[l + 1], prm.quant_levels, prm.level_lo)[1])
+                p.append(nearest_level(q[l], scale[l + 1], prm.quant_levels, prm.level_lo)[1])
                 if prm.quantize_q:
                     q[l] = p[l + 1].copy()
             else:

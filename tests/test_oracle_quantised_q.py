@@ -45,6 +45,31 @@ def test_quantize_with_offset_is_nearest_level_brute_force(m, scale, lo):
     assert np.array_equal(codes[far], dist.argmin(axis=1)[far].astype(codes.dtype))
 
 
+@pytest.mark.parametrize("m,scale,lo", [(2, 0.5, 0.0), (22, 1.0, -1.0), (16, 0.0173, -0.0371), (256, 0.011, 0.25),
+                                        (1000, 0.003, -0.3)])
+def test_nearest_level_is_the_argmin_over_all_levels(m, scale, lo):
+    """The projection that the quantised updates use is exactly argmin_delta |delta - x| (no tolerance): brute force
+    over all m levels in double precision, exact ties resolved towards the upper level, ends clamped."""
+    rng = np.random.default_rng(7 * m)
+    scale, lo = float(np.float32(scale)), float(np.float32(lo))
+    levels = o.level_set(scale, m, lo)
+    x = rng.uniform(lo - 2 * scale, lo + (m + 1) * scale, size=6000)
+    x[:m - 1] = 0.5 * (levels[:-1] + levels[1:])              # exact midpoints of neighbouring levels
+    x[m:2 * m] = levels + rng.uniform(-1e-9, 1e-9, size=m)    # values within rounding of a level
+    codes, vals = o.nearest_level(x, scale, m, lo)
+    dist = np.abs(x[:, None] - levels[None, :])
+    # first minimum from the top = the upper of two tied levels
+    want = (m - 1 - np.argmin(dist[:, ::-1], axis=1))
+    assert np.array_equal(codes.astype(np.int64), want)
+    assert np.array_equal(vals, levels[want])
+    assert codes.dtype == (np.uint8 if m <= 256 else np.uint16)
+    # the single-precision rounding agrees with it away from the rounding boundaries
+    c32 = o.quantize(x, scale, m, lo)[0]
+    t = (x - lo) / scale
+    far = np.abs(np.abs(t - np.floor(t)) - 0.5) > 1e-3
+    assert np.array_equal(c32[far], codes[far])
+
+
 def test_quantised_q_minimises_the_q_subproblem_over_delta():
     """Brute force: per element, the level with the smallest value of the terms of L_rho that contain q_l,
     (nu/2)(q - f(z))^2 + u (p_next - q) + (rho/2)(p_next - q)^2, is the one update_q_quantized returns."""
