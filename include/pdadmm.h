@@ -214,6 +214,8 @@ int pdadmm_matmul(int device, int mode, int M, int N, int K, const float *A, con
  * not take the allocator lock or cause an implicit device synchronisation, or a layer that was given all of
  * its buffers up front.
  *  - dA, dB, dC: device pointers on `device`, 16-byte aligned; lda >= M, ldb >= N, both multiples of 4.
+ *    The operands are read in groups of four columns: columns M..lda-1 of dA and N..ldb-1 of dB must be readable
+ *    but may hold anything (NaN included); they reach neither the valid block nor the padding of C.
  *  - Limit: M * ldc <= 1048576 floats (one partial tile must fit the built-in array); larger outputs are
  *    rejected with PDADMM_EINVAL and a message that names both sizes.  Every GPU that loads the library holds
  *    the 4 MiB until the process exits.
@@ -227,6 +229,16 @@ int pdadmm_matmul(int device, int mode, int M, int N, int K, const float *A, con
  */
 int pdadmm_matmul_tn_static(int device, int M, int N, int K, const float *dA, int lda, const float *dB, int ldb,
                             float *dC, void *stream);
+
+/*
+ * pdadmm_selftest_bounded_wait -- exercises the error path of PDADMM_ETIMEOUT without any faulty input: one warp
+ * waits, with the wait routine of the tensor-core products, on a barrier that nothing arrives at; the wait gives up
+ * after about limit_cycles SM cycles (1 .. 1e8), the kernel raises the products' error word and returns by itself.
+ * Always returns PDADMM_ETIMEOUT when the device is usable (PDADMM_OK would mean the wait was satisfied, which cannot
+ * happen); *waited_cycles (may be null) receives the cycles the wait lasted.  The context of the process stays usable:
+ * a product launched afterwards runs normally.
+ */
+int pdadmm_selftest_bounded_wait(int device, long long limit_cycles, long long *waited_cycles);
 
 /*
  * Per-kernel timing.  pdadmm_profile(ctx, 1) makes every later kernel launch of pdadmm_step be

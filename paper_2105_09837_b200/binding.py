@@ -28,7 +28,8 @@ OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5,
 
 EXPORTS = [
     "pdadmm_init", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
-    "pdadmm_set_tensor", "pdadmm_predict", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_profile", "pdadmm_profile_classes",
+    "pdadmm_set_tensor", "pdadmm_predict", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_selftest_bounded_wait",
+    "pdadmm_profile", "pdadmm_profile_classes",
     "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_destroy", "pdadmm_last_error",
 ]
 
@@ -78,6 +79,7 @@ def lib() -> C.CDLL:
                                     C.POINTER(C.c_double), C.c_uint32]
         L.pdadmm_matmul_tn_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_int,
                                               C.c_void_p, C.c_void_p]
+        L.pdadmm_selftest_bounded_wait.argtypes = [C.c_int, C.c_longlong, C.POINTER(C.c_longlong)]
         L.pdadmm_profile.argtypes = [C.c_void_p, C.c_int]
         L.pdadmm_profile_name.argtypes = [C.c_int]
         L.pdadmm_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64),
@@ -295,3 +297,10 @@ def matmul_tn_static(dA: int, lda: int, dB: int, ldb: int, dC: int, M: int, N: i
     """
     _check(lib().pdadmm_matmul_tn_static(device, M, N, K, C.c_void_p(dA), lda, C.c_void_p(dB), ldb, C.c_void_p(dC),
                                          C.c_void_p(stream)))
+
+
+def selftest_bounded_wait(limit_cycles: int = 100000, device: int = 0):
+    """``pdadmm_selftest_bounded_wait``: returns (status code, cycles waited); the status is ETIMEOUT by design."""
+    waited = C.c_longlong(0)
+    rc = lib().pdadmm_selftest_bounded_wait(device, limit_cycles, C.byref(waited))
+    return rc, int(waited.value), lib().pdadmm_last_error().decode()

@@ -120,7 +120,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_blo,
                const TcParams prm, Epi epi, double *__restrict__ partials) {
   constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN;
-  if (*reinterpret_cast<volatile int *>(prm.error) != 0) return;   // an earlier block gave up: do not queue behind it
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *tr_base = smem + TC_STAGES * TC_STAGE_BYTES;
@@ -130,6 +129,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint64_t *corr_empty = acc_empty + TC_ACC_BUFS, *drain_bar = corr_empty + 1, *a_empty = drain_bar + 1;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(a_empty + TC_A_SLOTS);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  volatile int *skip_flag = abort_flag + 1;           // an earlier block gave up: this one does no work
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int ACC0 = 2 + TC_CONV_WARPS;              // first accumulate warp
@@ -153,6 +153,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::mbar_init(drain_bar, 1);
     for (int a = 0; a < TC_A_SLOTS; ++a) ptx::mbar_init(&a_empty[a], 1);
     *abort_flag = 0;
+    // One thread reads the error word for the whole block, so that all warps take the same path: every block still
+    // allocates and releases its tensor memory and passes both block-wide barriers.
+    *skip_flag = *reinterpret_cast<volatile int *>(prm.error) != 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&map_a);
     ptx::prefetch_tmap(&map_b);
@@ -193,7 +196,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   };
 
-  if (warp == 0) {
+  if (*skip_flag) {
+    // nothing: do not queue work behind a block whose bounded wait expired
+  } else if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (one lane)
     if (lane == 0) {
       int it = 0;

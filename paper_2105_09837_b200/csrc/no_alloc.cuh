@@ -22,15 +22,21 @@ static __device__ __align__(256) float g_static_scratch[STATIC_SCRATCH_FLOATS];
 constexpr int STATIC_MAX_DEVICES = 64;
 static float *g_static_scratch_ptr[STATIC_MAX_DEVICES];   // device address of the array, per device; null = not set up
 
-// sum of the partial tiles in slice order (no scaling, no norm)
+// sum of the partial tiles in slice order (no scaling, no norm).  Rows of C are ldc = 4 * ldc4 floats wide with N
+// valid columns: the padding columns are written as zero whatever the partial tiles hold there (the product reads
+// the operand in groups of four columns, so those entries are products with the caller's padding of B).
 __global__ void __launch_bounds__(EW_THREADS)
-sum_partial_tiles_kernel(const float *__restrict__ part, int n_split, size_t n4, float *__restrict__ C) {
+sum_partial_tiles_kernel(const float *__restrict__ part, int n_split, size_t n4, int ldc4, int N, float *__restrict__ C) {
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < n_split; ++s) {
       const float4 v = ld4(part + (size_t)s * n4 * 4, i);
       a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
     }
+    const int col = (int)(i % (size_t)ldc4) * 4;
+    if (col + 1 >= N) a.y = 0.f;
+    if (col + 2 >= N) a.z = 0.f;
+    if (col + 3 >= N) a.w = 0.f;
     st4(C, i, a);
   }
 }
@@ -73,7 +79,7 @@ extern "C" int pdadmm_matmul_tn_static(int device, int M, int N, int K, const fl
     gemm_tn_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, k_chunk, dA, lda, dB, ldb, part, ldc);
     const size_t n4 = tile_floats / 4;
     const int g = (int)std::max<size_t>(1, std::min<size_t>(ceil_div((int64_t)n4, EW_THREADS), 148 * 8));
-    sum_partial_tiles_kernel<<<g, EW_THREADS, 0, st>>>(part, n_split, n4, dC);
+    sum_partial_tiles_kernel<<<g, EW_THREADS, 0, st>>>(part, n_split, n4, ldc / 4, N, dC);
     PD_CUDA(cudaPeekAtLastError());
     return PDADMM_OK;
   };

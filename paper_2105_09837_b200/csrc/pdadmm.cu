@@ -302,10 +302,12 @@ static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, cons
                      const CUtensorMap &mbl, const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
   auto kern = gemm_tc_kernel<MODE, Epi>;
   const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
-  static bool configured = false;
-  if (!configured) {
+  // the attribute belongs to (kernel, device): one flag per device ordinal for this instantiation
+  static bool configured[64] = {false};
+  const int dev = c->device;
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(ma, mal, mb, mbl, prm, epi, partials);
   return PDADMM_OK;
@@ -1583,6 +1585,51 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
   };
   const int rc = body();
   destroy(c);
+  return rc;
+}
+
+// ---- self-test of the bounded waits ------------------------------------------------------------------------------
+namespace pd {
+// One warp waits, with the products' own wait routine, on an mbarrier that nothing ever arrives at.  The wait gives up
+// after `limit_cycles`, raises the block's abort flag, and the block reports through the same error word as the
+// products and returns by itself.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles, int *error, long long *waited) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  volatile int *abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const long long t0 = clock64();
+    const bool ok = ptx::mbar_wait(&bar, 0, abort_flag, limit_cycles);
+    *waited = clock64() - t0;
+    if (!ok) atomicExch(error, 1);
+  }
+}
+}  // namespace pd
+
+extern "C" int pdadmm_selftest_bounded_wait(int device, long long limit_cycles, long long *waited_cycles) {
+  if (limit_cycles < 1 || limit_cycles > 100000000ll) return fail(PDADMM_EINVAL, "limit_cycles must be in [1, 1e8]");
+  PD_CUDA(cudaSetDevice(device));
+  int *d_err = nullptr;
+  auto body = [&]() -> int {
+    PD_CUDA(cudaMalloc((void **)&d_err, 16));
+    PD_CUDA(cudaMemset(d_err, 0, 16));
+    bounded_wait_selftest_kernel<<<1, 32>>>(limit_cycles, d_err, reinterpret_cast<long long *>(d_err) + 1);
+    PD_CUDA(cudaGetLastError());
+    PD_CUDA(cudaDeviceSynchronize());
+    long long h[2] = {0, 0};
+    PD_CUDA(cudaMemcpy(h, d_err, 16, cudaMemcpyDeviceToHost));
+    if (waited_cycles) *waited_cycles = h[1];
+    if ((int)h[0] != 0) return fail(PDADMM_ETIMEOUT, "a bounded device-side wait expired after %lld cycles", h[1]);
+    return PDADMM_OK;
+  };
+  const int rc = body();
+  cudaFree(d_err);
   return rc;
 }
 

@@ -1,15 +1,18 @@
 """Small, self-contained invocations for kernel profilers (one kernel class each, a few launches).
 
-    python -m paper_2105_09837_b200.profile_case matmul MODE M N K [--simt]    # one dense product, run twice
-    python -m paper_2105_09837_b200.profile_case iterate WORKLOAD N_NODES ITERS [--no-graph]  # a (reduced) workload
+    python profile_case.py matmul MODE M N K [--simt]    # one dense product, run twice
+    python profile_case.py iterate WORKLOAD N_NODES ITERS [--no-graph]  # a (reduced) workload
 """
 
+import os
 import sys
 
 import numpy as np
 
-from . import binding as B
-from . import synth
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+
+from paper_2105_09837_b200 import binding as B      # noqa: E402
+from paper_2105_09837_b200 import synth             # noqa: E402
 
 
 def main(argv):

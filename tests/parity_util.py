@@ -110,7 +110,37 @@ def q_boundary_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=None
     v = o.update_q(nxt.p[l + 1], prev.u[l], nxt.z[l], prm.rho, prm.nu)
     # the value to project carries the single-precision error of z+ (a chain of products and sums, about
     # 1e-6 of the largest value), which with many levels exceeds the band of the storage roundings alone
-    tol = max(band(prm), 1e-6 * float(np.abs(v).max()) / prev.scale[l + 1]) if tol is None else tol
+    if tol is None:
+        tol = max(band(prm), 1e-6 * float(np.abs(v).max()) / prev.scale[l + 1])
     t = (v - prm.level_lo) / prev.scale[l + 1]
     frac = t - np.floor(t)
     return np.abs(frac - 0.5) <= tol
+
+
+def redo_after_p(s: o.State, n: o.State, prm: o.Params) -> o.State:
+    """The rest of one iteration of Algorithm 1 (W, b, z, q, u, in that order) for the new p held in `n`, by the
+    oracle's own update functions.  Used where the device and the oracle projected some entries of p, each within
+    rounding of a boundary between two levels, to different neighbours: the oracle then continues from the device's
+    choice, so that everything computed from p is compared on equal terms."""
+    rho, nu, L = prm.rho, prm.nu, s.L
+    for l in range(L):
+        n.W[l], n.theta[l] = o.update_W(n.p[l], s.W[l], s.b[l], s.z[l], nu)
+    for l in range(L):
+        n.b[l] = o.update_b(n.p[l], n.W[l], s.b[l], s.z[l], nu)
+    for l in range(L):
+        a = n.W[l] @ n.p[l] + n.b[l][:, None]
+        if l < L - 1:
+            n.z[l] = o.update_z_hidden(a, s.q[l], s.z[l], prm.slope)
+        elif prm.risk == "ls":
+            n.z[l] = o.update_z_last_least_squares(a, s.y, s.mask, nu)
+        else:
+            n.z[l] = o.update_z_last(a, s.y, s.mask, nu)
+    for l in range(L - 1):
+        if prm.quant_levels and prm.quantize_q:
+            n.q[l] = o.update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels,
+                                          prm.level_lo, prm.slope)
+        else:
+            n.q[l] = o.update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.slope)
+    for l in range(L - 1):
+        n.u[l] = o.update_u(s.u[l], n.p[l + 1], n.q[l], rho)
+    return n

@@ -257,3 +257,19 @@ def test_non_finite_state_is_reported_not_propagated_silently():
         ctx.step(1)
     assert e.value.code == B.ENUMERIC
     ctx.destroy()
+
+
+def test_bounded_wait_runs_out_and_the_device_stays_usable():
+    """A wait that nothing satisfies gives up after its cycle limit, the kernel returns by itself, the host reports
+    PDADMM_ETIMEOUT, and a tensor-core product launched afterwards in the same process is correct."""
+    rc, waited, text = B.selftest_bounded_wait(limit_cycles=100000)
+    assert rc == B.ETIMEOUT and "expired" in text
+    assert 100000 < waited < 50_000_000              # gave up soon after the limit (polled every 256 probes)
+    rng = np.random.default_rng(0)
+    a = rng.standard_normal((300, 200)).astype(np.float32)
+    b = rng.standard_normal((150, 200)).astype(np.float32)
+    c, _ = B.matmul(0, a, b)
+    want = a.astype(np.float64) @ b.astype(np.float64).T
+    assert U.rel_err(c.astype(np.float64), want) < 1e-6
+    with pytest.raises(B.PdadmmError):
+        B._check(B.lib().pdadmm_selftest_bounded_wait(0, 0, None))       # limit out of range: EINVAL, nothing launched

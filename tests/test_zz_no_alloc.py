@@ -41,3 +41,28 @@ def test_static_scratch_product_matches_the_allocating_entry_point_twice_in_a_ro
         # same tolerance as the other kernel tests: relative Frobenius error
         assert np.linalg.norm(got - want) <= 1e-5 * np.linalg.norm(want)
         assert np.linalg.norm(got - ref) <= 1e-5 * np.linalg.norm(ref)
+
+
+@pytest.mark.gpu
+def test_static_scratch_product_with_ragged_widths_and_dirty_padding():
+    """Widths that are no multiples of 4, leading dimensions larger than the widths, and NaN in every padding column
+    of the operands: the valid block equals the allocating entry point's, the padding columns of C come out as zero."""
+    import torch
+    rng = np.random.default_rng(7)
+    dev = torch.device("cuda", 0)
+    for (K, M, N, lda, ldb) in [(1031, 37, 53, 44, 60), (300, 5, 3, 8, 4)]:
+        A = rng.standard_normal((K, M)).astype(np.float32)
+        Bm = rng.standard_normal((K, N)).astype(np.float32)
+        want, _ = B.matmul(2, A, Bm, flags=B.FLAG_SIMT_GEMM)
+        Ap = np.full((K, lda), np.nan, np.float32)
+        Bp = np.full((K, ldb), np.nan, np.float32)
+        Ap[:, :M], Bp[:, :N] = A, Bm
+        ldc = (N + 3) // 4 * 4
+        dA, dB = torch.from_numpy(Ap).to(dev), torch.from_numpy(Bp).to(dev)
+        dC = torch.full((M, ldc), float("nan"), device=dev, dtype=torch.float32)
+        torch.cuda.synchronize()
+        B.matmul_tn_static(dA.data_ptr(), lda, dB.data_ptr(), ldb, dC.data_ptr(), M, N, K, stream=0, device=0)
+        torch.cuda.synchronize()
+        got = dC.cpu().numpy()
+        assert np.linalg.norm(got[:, :N] - want) <= 1e-5 * np.linalg.norm(want)
+        assert np.all(got[:, N:] == 0)
