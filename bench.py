@@ -1,12 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the pdADMM-G iteration: ADMM iterations per second over all layers.
 
-    python bench.py --gpus N --steps K --warmup W [--workload c2] [--impl reference]
+    python bench.py --gpus N --steps K --warmup W [--workload c1..c5|all] [--impl reference]
 
 One step is one iteration of Algorithm 1 over every layer (p, W, b, z, q, u updates).  With N > 1 the
 script runs under torchrun, one process per GPU; every rank runs an independent replica of the
 workload (the path has no cross-GPU exchange), the timed region is bracketed by barriers and the
-reported time is the maximum over ranks.  Rank 0 prints one JSON line.
+reported time is the maximum over ranks.  Rank 0 prints one JSON line: its top-level fields are the headline
+workload (c2), and on one GPU `workloads` holds one record for each of the five workloads.
 """
 
 from __future__ import annotations
@@ -114,65 +115,211 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------------------- oracle timing
 
-def oracle_layer_sample(inp, n_threads_hint=None):
-    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: after one untimed full
-    set-up (augmentation, feasible start), the per-layer updates of one iteration are run for layer 1,
-    one middle layer and layer L; the middle layers are identical in shape, so the time of a full
-    iteration is t_1 + (L-2) t_mid + t_L.  Returns (seconds per iteration, description, threads)."""
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_whole_iterations(inp, warmup, steps, budget_s):
+    """Times whole iterations of the fp64 oracle, as it stands, from the feasible start (untimed set-up:
+    adjacency, augmentation, start of Algorithm 1).  `warmup` untimed iterations, then up to `steps` timed ones,
+    stopping early once `budget_s` seconds of timed work are spent.  Returns (list of seconds, description)."""
     import oracle.pdadmm_oracle as o
     w = inp.workload
     prm = o.Params(w.rho, w.nu, w.quant_levels)
     A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
     X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
     s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels, inp.train_mask, prm)
-    L = s.L
-    mid = L // 2 if L >= 3 else None
-    picks = sorted(set([0, L - 1] + ([mid] if mid is not None else [])))
-    # make the start non-trivial: perturb z so that gradients are not identically zero
-    rng = np.random.default_rng(0)
-    for l in picks:
-        s.z[l] = s.z[l] + 0.01 * rng.standard_normal(s.z[l].shape)
-
-    def layer_pass(l):
+    times = []
+    for i in range(warmup + steps):
         t0 = time.perf_counter()
-        p = s.p[l]
-        if l >= 1:
-            if prm.quant_levels:
-                p = o.update_p_quantized(s.p[l], s.W[l], s.b[l], s.z[l], prm.nu, s.q[l - 1], s.u[l - 1], prm.rho,
-                                         s.scale[l], prm.quant_levels)[0]
-            else:
-                p = o.update_p(s.p[l], s.W[l], s.b[l], s.z[l], prm.nu, s.q[l - 1], s.u[l - 1], prm.rho)[0]
-        W, _ = o.update_W(p, s.W[l], s.b[l], s.z[l], prm.nu)
-        b = o.update_b(p, W, s.b[l], s.z[l], prm.nu)
-        a = W @ p + b[:, None]
-        if l < L - 1:
-            z = o.update_z_hidden(a, s.q[l], s.z[l])
-            q = o.update_q(s.p[l + 1], s.u[l], z, prm.rho, prm.nu)
-            o.update_u(s.u[l], s.p[l + 1], q, prm.rho)
-        else:
-            o.update_z_last(a, s.y, s.mask, prm.nu)
-        return time.perf_counter() - t0
+        s = o.iterate(s, prm)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+            if sum(times) > budget_s:
+                break
+    desc = (f"{len(times)} whole oracle iterations of workload {w.name} (all {w.n_layers} layers, every update of "
+            f"Algorithm 1) after {warmup} untimed ones")
+    return times, desc
 
-    t = {l: layer_pass(l) for l in picks}
-    total = t[0] + (t[L - 1] if L > 1 else 0.0) + (max(L - 2, 0) * t[mid] if mid is not None else 0.0)
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
-    except Exception:
-        threads = os.cpu_count() or 1
-    desc = (f"one oracle iteration of workload {w.name}: layers {[l + 1 for l in picks]} timed, "
-            f"the {max(L - 2, 0)} identical middle layers extrapolated from layer {(mid or 0) + 1}")
-    return total, desc, threads
+
+def oracle_node_sample(inp, n_sample):
+    """For workloads whose oracle iteration does not fit the time or the host memory: one whole oracle iteration on
+    the sub-problem of the first n_sample nodes (all layers at full width; every per-layer update is linear in the
+    node count), scaled by N / n_sample.  The sparse augmentation is done on the full graph and is not timed.
+    Returns (seconds per full-size iteration, description)."""
+    import oracle.pdadmm_oracle as o
+    w = inp.workload
+    prm = o.Params(w.rho, w.nu, w.quant_levels)
+    A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
+    X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)[:, :n_sample]
+    s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels[:n_sample], inp.train_mask[:n_sample], prm)
+    s = o.iterate(s, prm)                      # untimed: leaves the feasible start, where every gradient is zero
+    t0 = time.perf_counter()
+    o.iterate(s, prm)
+    dt = time.perf_counter() - t0
+    desc = (f"one whole oracle iteration of workload {w.name} on its first {n_sample} of {w.n_nodes} nodes "
+            f"(all {w.n_layers} layers at full width), time scaled by {w.n_nodes / n_sample:.1f}")
+    return dt * w.n_nodes / n_sample, desc
+
+
+def cpu_baseline_for(inp, budget_s=25.0):
+    """The oracle on the host cores for one workload, bounded to about `budget_s` seconds of timed work."""
+    w = inp.workload
+    flop = 8.0 * w.n_nodes * w.hidden * w.hidden * max(w.n_layers - 2, 0) + 4.0 * w.n_nodes * w.hidden * w.n0
+    if flop < 2e12:                                       # whole iterations fit: c1, c2, c3
+        times, desc = oracle_whole_iterations(inp, 1, 3, budget_s)
+        sec = sum(times) / len(times)
+    else:
+        n_sample = max(256, int(w.n_nodes * 3e11 / flop))
+        sec, desc = oracle_node_sample(inp, n_sample)
+    return {"value": 1.0 / sec, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": desc}
+
+
+# --------------------------------------------------------------------------------------- one workload on the device
+
+def describe(w, quant_q=False):
+    return (f"{w.name}: N={w.n_nodes} {w.graph.upper()} graph, d={w.feat_dim} x {w.n_blocks} hop blocks "
+            f"(n0={w.n0}), {w.n_layers} layers x {w.hidden}, {w.n_classes} classes, "
+            f"{'pdADMM-G' if not w.quant_levels else f'pdADMM-G-Q {w.quant_levels} levels'}"
+            f"{' (p and q quantised)' if quant_q else ''}, rho=nu={w.rho}")
+
+
+def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu, with_e2e=True):
+    """Times `steps` iterations of one workload (after `warmup`), a per-kernel pass, the end-to-end leg and the
+    oracle sample.  Returns the record of that workload."""
+    import torch
+    from paper_2105_09837_b200 import binding as B
+    from paper_2105_09837_b200 import replicas, synth
+    w = synth.get(name)
+    inp = synth.make_inputs(w)
+    pk = peaks()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    ctx = B.from_inputs(inp, device=device, flags=flags)
+    ctx.step(warmup)
+    launches0 = ctx.launches()
+    barrier()
+    with ClockSampler(device) as clk:
+        ctx.step(steps)
+        ms = ctx.last_step_ms()
+        barrier()
+    launches = ctx.launches() - launches0
+    ms = replicas.max_over_ranks(ms, dist, f"cuda:{device}")
+    value = replicas.job_throughput(world, steps, ms)
+    clocks = clk.summary()
+    obj = ctx.objective()
+    spmm = None
+    if w.n_blocks > 1:
+        hop_ms, hop_bytes = ctx.time_augmentation(20)
+        spmm = {"ms_per_hop": hop_ms, "gbs": hop_bytes / (hop_ms * 1e-3) / 1e9, "frac_of_hbm_peak": hop_bytes / (hop_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                "note": "algorithmic bytes nnz(8+4d)+8Nd; the gathered rows are served from L2 where the block fits"}
+
+    # per-kernel device times (second pass with an event pair around every launch, one lane)
+    ctx.profile(True)
+    n_prof = min(steps, 5)
+    ctx.step(n_prof)
+    prof = ctx.profile_read()
+    ctx.profile(False)
+    ctx.destroy()
+    # Denominators: the burst figure of the measured bf16 GEMM where the clocks stayed at their maximum, the sustained
+    # one where the power cap was active during the timed region (fp16 MMAs run at the bf16 rate)
+    capped = "sw_power_cap" in (clocks.get("reasons") or [])
+    tensor_peak = pk["bf16_tflops_sustained"] if capped else pk["bf16_tflops"]
+    tensor_peak_name = f"{pk['source']} bf16 GEMM, {'sustained (power cap active)' if capped else 'burst (clocks at maximum)'}"
+    if simt:
+        tensor_peak, tensor_peak_name = FP32_FMA_PEAK_TFLOPS, "148 SMs x 128 fp32 lanes x 2 flop x 1.965 GHz"
+    kernels, t_roof = {}, 0.0
+    for k, v in prof.items():
+        if v["launches"] == 0:
+            continue
+        sec = v["ms"] * 1e-3
+        # roofline time of the class: the larger of its algorithmic flop over the tensor peak and bytes over the copy peak
+        roof_s = max(v["flops"] / (tensor_peak * 1e12), v["bytes"] / (pk["hbm_gbs"] * 1e9))
+        t_roof += roof_s / n_prof
+        kernels[k] = {"ms_per_iter": v["ms"] / n_prof, "launches_per_iter": v["launches"] / n_prof,
+                      "gbs": v["bytes"] / sec / 1e9 if sec > 0 else None,
+                      "tflops": v["flops"] / sec / 1e12 if sec > 0 else None,
+                      "roof_ms_per_iter": roof_s * 1e3 / n_prof, "frac": roof_s / sec if sec > 0 else None}
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_iter"])
+    d = prof[dom]
+    if d["flops"] > 0:
+        achieved = d["flops"] / (d["ms"] * 1e-3) / 1e12
+        roof = {"bound": "alu" if simt else "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
+                "peak_source": tensor_peak_name}
+    else:
+        roof = {"bound": "hbm", "achieved": d["bytes"] / (d["ms"] * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
+                "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    if roof["bound"] == "tensor":
+        # every useful product is issued as three fp16 MMAs (hi*hi, hi*lo, lo*hi): the tensor pipe's own load
+        roof["frac_issued"] = 3.0 * roof["frac"]
+        roof["note"] = "achieved counts useful fp32-equivalent flop; the kernel issues three fp16 MMAs per product"
+    roof["kernel"] = dom
+    roof["traffic"] = measured_traffic(name, dom)
+
+    rec = {"workload": describe(w, bool(flags & B.FLAG_QUANT_Q)), "value": value, "unit": UNIT, "steps": steps, "warmup": warmup,
+           "ms_per_step": ms / steps, "clocks": clocks, "gpu_launches": launches, "roofline": roof,
+           "t_roof_ms": t_roof * 1e3, "frac_t_roof": t_roof * 1e3 / (ms / steps),
+           "t_roof_note": "sum over kernel classes of max(algorithmic flop / tensor peak, algorithmic bytes / copy peak), "
+                          "per iteration; frac_t_roof = t_roof / measured time per iteration",
+           "kernels": kernels, "spmm": spmm, "objective": float(obj[5])}
+
+    if with_e2e:
+        # end to end through the public API from host buffers: init (H2D of graph, features, weights), K iterations,
+        # objective and trained weights back to the host
+        h2d = (inp.edge_src.nbytes + inp.edge_dst.nbytes + inp.features.nbytes + inp.labels.nbytes + inp.train_mask.nbytes
+               + sum(x.nbytes for x in inp.init_W))
+
+        def pinned(a):      # page-locked host buffers of the large inputs, as a caller that cares about the copy keeps them
+            return torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
+        inp.features = pinned(inp.features)
+        inp.init_W = [pinned(x) for x in inp.init_W]
+        barrier()
+        t0 = time.perf_counter()
+        ctx2 = B.from_inputs(inp, device=device, flags=flags)
+        ctx2.step(steps)
+        ctx2.objective()
+        d2h = 48
+        for l in range(1, w.n_layers + 1):
+            Wl, bl = ctx2.get_tensor(B.T_W, l), ctx2.get_tensor(B.T_B, l)
+            d2h += Wl.nbytes + bl.nbytes
+        torch.cuda.synchronize(device)
+        e2e_s = time.perf_counter() - t0
+        ctx2.destroy()
+        e2e_s = replicas.max_over_ranks(e2e_s, dist, f"cuda:{device}")
+        rec["e2e"] = {"value": replicas.job_throughput(world, steps, e2e_s * 1e3), "unit": UNIT,
+                      "h2d_bytes_per_step": h2d / steps, "d2h_bytes_per_step": d2h / steps,
+                      "note": "pdadmm_init from host buffers (features and weights page-locked) + K iterations + objective "
+                              "and W,b read back; the one-off set-up is spread over only K iterations"}
+    if with_cpu:
+        rec["cpu_baseline"] = cpu_baseline_for(inp)
+    return rec
 
 
 # --------------------------------------------------------------------------------------- main
+
+ALL = ["c1", "c2", "c3", "c4", "c5"]
+HEADLINE = "c2"        # the configuration the metric is quoted on that fits one GPU with the oracle affordable beside it
+STEP_CAP = {"c4": 10, "c5": 6}      # iterations of the two large workloads (0.13 s and 0.47 s each)
+
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default=None,
+                    help="c1..c5: that workload alone; 'all' or nothing: the headline workload in the top-level fields "
+                         "and one record per workload under 'workloads' (single GPU)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--simt", action="store_true", help="run the dense products on CUDA cores")
     ap.add_argument("--one-lane", action="store_true", help="queue all layers on one stream (no concurrency across layers)")
@@ -185,13 +332,9 @@ def main():
 
     from paper_2105_09837_b200 import replicas, synth
     rank, world, local_rank = replicas.env_rank_world()
-
-    w = synth.get(args.workload)
-    config = {"workload": f"{w.name}: N={w.n_nodes} {w.graph.upper()} graph, d={w.feat_dim} x {w.n_blocks} hop blocks "
-                          f"(n0={w.n0}), {w.n_layers} layers x {w.hidden}, {w.n_classes} classes, "
-                          f"{'pdADMM-G' if not w.quant_levels else f'pdADMM-G-Q {w.quant_levels} levels'}"
-                          f"{' (p and q quantised)' if args.quant_q else ''}, rho=nu={w.rho}",
-              "replicas": args.gpus,
+    head = args.workload if args.workload in ALL else HEADLINE
+    w = synth.get(head)
+    config = {"workload": describe(w, args.quant_q), "replicas": args.gpus,
               "l2": "state (about %.1f GB per replica) is far larger than the 126 MB L2" %
                     (5 * 4e-9 * w.n_nodes * w.hidden * w.n_layers)}
 
@@ -199,20 +342,15 @@ def main():
         if rank != 0:
             return 0
         inp = synth.make_inputs(w)
-        times = []
-        desc, threads = "", 1
-        for i in range(args.warmup + args.steps):
-            t, desc, threads = oracle_layer_sample(inp)
-            if i >= args.warmup:
-                times.append(t)
-            if sum(times) > 240 and len(times) >= 1 and i >= args.warmup:
-                break                              # keep the whole run within a few minutes
+        # whole oracle iterations: W untimed, then up to K timed ones within about four minutes
+        times, desc = oracle_whole_iterations(inp, args.warmup, args.steps, 200.0)
         sec = sum(times) / len(times)
         value = 1.0 / sec
         line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-                "steps": len(times), "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
-                "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+                "steps": len(times), "steps_requested": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": config,
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": desc},
                 "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
         print(json.dumps(line))
         return 0
@@ -232,104 +370,32 @@ def main():
     flags = (B.FLAG_SIMT_GEMM if args.simt else 0) | (B.FLAG_QUANT_Q if args.quant_q else 0)
     flags |= B.FLAG_ONE_LANE if args.one_lane else 0
 
-    inp = synth.make_inputs(w)
-    ctx = B.from_inputs(inp, device=device, flags=flags)
-    ctx.step(args.warmup)
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize(device)
-
-    # timed region: exactly K iterations, device time from CUDA events on the library's stream
-    launches0 = ctx.launches()
-    barrier()
-    with ClockSampler(device) as clk:
-        t0 = time.perf_counter()
-        ctx.step(args.steps)
-        ms = ctx.last_step_ms()
-        barrier()
-        wall = time.perf_counter() - t0
-    launches = ctx.launches() - launches0
-    ms = replicas.max_over_ranks(ms, dist, f"cuda:{device}")
-    value = replicas.job_throughput(world, args.steps, ms)
-    obj = ctx.objective()
-
-    # per-kernel device times (second pass with an event pair around every launch)
-    ctx.profile(True)
-    n_prof = min(args.steps, 5)
-    ctx.step(n_prof)
-    prof = ctx.profile_read()
-    ctx.profile(False)
-    pk = peaks()
-    kernels = {}
-    for name, v in prof.items():
-        if v["launches"] == 0:
-            continue
-        sec = v["ms"] * 1e-3
-        kernels[name] = {"ms_per_iter": v["ms"] / n_prof, "launches_per_iter": v["launches"] / n_prof,
-                         "gbs": v["bytes"] / sec / 1e9 if sec > 0 else None,
-                         "tflops": v["flops"] / sec / 1e12 if sec > 0 else None}
-    dom = max(kernels, key=lambda k: kernels[k]["ms_per_iter"])
-    d = prof[dom]
-    if d["flops"] > 0:
-        achieved = d["flops"] / (d["ms"] * 1e-3) / 1e12
-        if args.simt:
-            roof = {"bound": "alu", "achieved": achieved, "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s",
-                    "peak_source": "148 SMs x 128 fp32 lanes x 2 flop x 1.965 GHz"}
-        else:
-            # the products run as fp16 MMAs with fp32 accumulation: same tensor rate as the measured bf16 GEMM
-            roof = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s", "peak_source": f"{pk['source']} bf16 GEMM, sustained (fp16 MMAs run at the bf16 rate)"}
-    else:
-        roof = {"bound": "hbm", "achieved": d["bytes"] / (d["ms"] * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
-                "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    if roof["bound"] == "tensor":
-        # every useful product is issued as three fp16 MMAs (hi*hi, hi*lo, lo*hi): the tensor pipe's own load
-        roof["frac_issued"] = 3.0 * roof["frac"]
-        roof["note"] = "achieved counts useful fp32-equivalent flop; the kernel issues three fp16 MMAs per product"
-    roof["kernel"] = dom
-    roof["traffic"] = measured_traffic(args.workload, dom)
-    ctx.destroy()
-
-    # end to end through the public API from host buffers: init (H2D of graph, features, weights), K iterations,
-    # objective and trained weights back to the host
-    h2d = (inp.edge_src.nbytes + inp.edge_dst.nbytes + inp.features.nbytes + inp.labels.nbytes + inp.train_mask.nbytes
-           + sum(x.nbytes for x in inp.init_W))
-    # the host buffers of the large inputs are page-locked, as a caller that cares about the copy would keep them
-    def pinned(a):
-        return torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
-    inp.features = pinned(inp.features)
-    inp.init_W = [pinned(x) for x in inp.init_W]
-    barrier()
-    t0 = time.perf_counter()
-    ctx2 = B.from_inputs(inp, device=device, flags=flags)
-    ctx2.step(args.steps)
-    out = [ctx2.objective()]
-    d2h = 48
-    for l in range(1, w.n_layers + 1):
-        Wl, bl = ctx2.get_tensor(B.T_W, l), ctx2.get_tensor(B.T_B, l)
-        d2h += Wl.nbytes + bl.nbytes
-    torch.cuda.synchronize(device)
-    e2e_s = time.perf_counter() - t0
-    ctx2.destroy()
-    e2e_s = replicas.max_over_ranks(e2e_s, dist, f"cuda:{device}")
-    e2e = {"value": replicas.job_throughput(world, args.steps, e2e_s * 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d / args.steps,
-           "d2h_bytes_per_step": d2h / args.steps,
-           "note": "pdadmm_init from host buffers (features and weights page-locked) + K iterations + objective and W,b read back"}
-
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sec, desc, threads = oracle_layer_sample(inp)
-        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+    with_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
+    t_start = time.perf_counter()
+    rec = run_workload(head, min(args.steps, STEP_CAP.get(head, args.steps)), args.warmup, flags, device, world, dist,
+                       args.simt, with_cpu)
+    workloads = {head: rec}
+    if args.workload in (None, "all") and world == 1:
+        # the metric is quoted per workload: the other four, each with its own clocks, roofline, end-to-end leg and oracle sample
+        for name in ALL:
+            if name == head:
+                continue
+            try:
+                q_flags = flags if synth.get(name).quant_levels else flags & ~B.FLAG_QUANT_Q
+                workloads[name] = run_workload(name, min(args.steps, STEP_CAP.get(name, args.steps)), args.warmup, q_flags,
+                                               device, world, dist, args.simt, with_cpu)
+            except Exception as e:                                  # a workload that fails must not hide the others
+                workloads[name] = {"error": f"{type(e).__name__}: {e}"}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        line = {"metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": world, "steps": rec["steps"],
+                "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-                "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roof,
-                "cpu_baseline": cpu, "kernels": kernels, "objective": float(obj[5]), "wall_s": wall}
+                "clocks": rec["clocks"], "e2e": rec.get("e2e"), "gpu_launches": rec["gpu_launches"], "roofline": rec["roofline"],
+                "cpu_baseline": rec.get("cpu_baseline"), "t_roof_ms": rec["t_roof_ms"], "frac_t_roof": rec["frac_t_roof"],
+                "kernels": rec["kernels"], "objective": rec["objective"],
+                "workloads": {k: v for k, v in sorted(workloads.items())},
+                "wall_s": time.perf_counter() - t_start}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

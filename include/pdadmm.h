@@ -254,6 +254,16 @@ const char *pdadmm_profile_name(int k);
 int pdadmm_profile_read(pdadmm_ctx *ctx, int k, double *ms, int64_t *launches, double *bytes, double *flops);
 int pdadmm_launches(pdadmm_ctx *ctx, int64_t *count);
 
+/*
+ * pdadmm_time_augmentation -- device time of one hop of the feature augmentation X_{k+1} = X_k A~ (paper, "Problem
+ * Formulation"; the sparse products run once inside pdadmm_init, where they cannot be timed apart from the copies):
+ * repeats the first hop `reps` times (1..1000) on the context's own CSR matrix and input block, writing the block of
+ * X it already holds (same kernel, same data, same bits), between CUDA events on the context's stream.
+ * *ms_per_hop receives the mean; *bytes_per_hop (may be null) the algorithmic bytes of a hop,
+ * nnz (8 + 4 d) + 8 N d.  EINVAL if the input has a single block.
+ */
+int pdadmm_time_augmentation(pdadmm_ctx *ctx, int reps, double *ms_per_hop, double *bytes_per_hop);
+
 /* Release the context and all of its device memory.  Null is accepted. */
 int pdadmm_destroy(pdadmm_ctx *ctx);
 

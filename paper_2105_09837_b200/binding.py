@@ -30,7 +30,7 @@ EXPORTS = [
     "pdadmm_init", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
     "pdadmm_set_tensor", "pdadmm_predict", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_selftest_bounded_wait",
     "pdadmm_profile", "pdadmm_profile_classes",
-    "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_destroy", "pdadmm_last_error",
+    "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_time_augmentation", "pdadmm_destroy", "pdadmm_last_error",
 ]
 
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.pdadmm_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64),
                                           C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.pdadmm_launches.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        L.pdadmm_time_augmentation.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.pdadmm_destroy.argtypes = [C.c_void_p]
         _lib = L
     return _lib
@@ -218,6 +219,12 @@ class Context:
             _check(lib().pdadmm_profile_read(self._h, k, C.byref(ms), C.byref(n), C.byref(by), C.byref(fl)))
             out[lib().pdadmm_profile_name(k).decode()] = dict(ms=ms.value, launches=n.value, bytes=by.value, flops=fl.value)
         return out
+
+    def time_augmentation(self, reps: int = 20):
+        """``pdadmm_time_augmentation``: (ms per hop, algorithmic bytes per hop)."""
+        ms, by = C.c_double(), C.c_double()
+        _check(lib().pdadmm_time_augmentation(self._h, reps, C.byref(ms), C.byref(by)))
+        return ms.value, by.value
 
     def launches(self) -> int:
         n = C.c_int64()

@@ -42,7 +42,7 @@ struct EpiStoreSumsq {        // C = acc, accumulates sum(acc^2)
 };
 struct EpiNormOnly {          // nothing is stored: only sum(acc^2) is wanted (||W g||^2 of the quantised update, whose
                               // step uses W d instead of W g)
-  static constexpr bool kDirect = true, kSumsq = true, kStore = false;
+  static constexpr bool kDirect = true, kSumsq = true, kStore = false, kCoarse = true;
   static constexpr int kInputs = 0;
   float *C; int ldc;          // ldc = padded width of the output; C is written by the CUDA-core kernels only
   __device__ __forceinline__ void prefetch(int, int) const {}

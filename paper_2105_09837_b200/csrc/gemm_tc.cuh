@@ -13,8 +13,10 @@
 // TMA brings fp32 tiles of the node-sized operand into shared memory; converter warps turn them into the two
 // fp16 planes, which they write to tensor memory; the small operand (a weight matrix) arrives as two precomputed
 // fp16 planes (K-major, 128-byte swizzle).  One thread issues tcgen05.mma; completion is tracked with mbarriers;
-// eight more warps read each K block's main term from tensor memory, add it to a register accumulator and finally
-// apply the scaling and the fused epilogue.
+// two sets of four accumulate warps take the output tiles of a block in turn: a set reads each K block's main term
+// from tensor memory, adds it to a register accumulator and finally applies the scaling and the fused epilogue --
+// while it is in that epilogue the other set already accumulates the next tile, so the tensor pipe never waits for
+// a store phase.
 //
 // Tile: 128 x 128 outputs per CTA, 64-deep K blocks, 3 stages of 64 KB.  Tensor memory (512 columns): two
 // accumulator tiles for the main term, one for the correction terms, two slots for the planes of A.
@@ -36,12 +38,21 @@ constexpr int TC_KSTEPS = TC_BK / 16;                          // MMAs (K = 16) 
 constexpr int TC_FLUSH = 1;                                    // K blocks per read-out of the main accumulator
 constexpr int TC_PLANE_BYTES = 128 * TC_BK * 2;                // 16 KB: one 128 x 64 fp16 operand plane
 constexpr int TC_STAGE_BYTES = 4 * TC_PLANE_BYTES;             // A_hi, A_lo, B_hi, B_lo (= two fp32 tiles of 128 x 64)
-// warp 0: TMA, warp 1: MMA, then 8 converter warps, then 8 accumulate + epilogue warps (two warps per 32-lane
-// quarter of tensor memory, 64 columns each)
-constexpr int TC_CONV_WARPS = 8;
-constexpr int TC_THREADS = 32 * (2 + TC_CONV_WARPS + 8);      // 576
-constexpr int TC_ACC_THREADS = 256;
+// Four warpgroups (register budgets are set per warpgroup): 0 = TMA warp, MMA warp and two idle warps; 1 = four
+// converter warps (one 32-lane quarter of tensor memory each); 2, 3 = the two accumulate sets, four warps each (a
+// warp owns one quarter of the tile's rows and all 128 columns: 128 accumulators per thread).
+// Registers: the block is launched with 512 x 128 = 65536; warpgroup 0 keeps 40 per thread, the converters 112, the
+// accumulate sets take 168 (the compiler spills least there): 128 (40 + 112 + 2 x 168) = 62464 <= 65536, so every increase is satisfiable.
+constexpr int TC_CONV_WARPS = 4;
+constexpr int TC_CONV0 = 4, TC_ACC0 = 8;                      // first converter warp, first accumulate warp
+constexpr int TC_THREADS = 512;
+constexpr int TC_ACC_THREADS = 128;                            // threads of one accumulate set
+constexpr int TC_REGS_LAUNCH = 128, TC_REGS_CTRL = 40, TC_REGS_CONV = 112, TC_REGS_ACC = 168;
+static_assert(TC_THREADS * TC_REGS_LAUNCH <= 65536, "register file");
+static_assert(128 * (TC_REGS_CTRL + TC_REGS_CONV + 2 * TC_REGS_ACC) <= TC_THREADS * TC_REGS_LAUNCH,
+              "the warpgroups' register shares exceed what the block is launched with: an increase would wait for ever");
 constexpr int TC_ACC_BUFS = 2;                                 // main-term accumulator tiles in tensor memory
+static_assert(TC_ACC_BUFS == 2, "the accumulate warps keep one phase counter per buffer");
 constexpr int TC_A_SLOTS = 2;                                  // K blocks of A planes in tensor memory
 constexpr int TC_TMEM_COLS = 512;                              // 2 main tiles, 1 correction tile, 2 x (A_hi, A_lo)
 constexpr uint32_t TC_COL_CORR = TC_ACC_BUFS * TC_BN;          // first column of the correction tile
@@ -73,6 +84,12 @@ __device__ __forceinline__ void tc_split8(const float (&x)[8], float scale, uint
 // Epilogues store their result unless they say otherwise (kStore = false).
 template <class Epi, class = void> struct epi_stores { static constexpr bool value = true; };
 template <class Epi> struct epi_stores<Epi, std::enable_if_t<!Epi::kStore>> { static constexpr bool value = false; };
+// An epilogue that wants nothing but the sum of squares of the product may say kCoarse = true: the product is then
+// issued as the main term A_hi B_hi alone (one MMA instead of three).  Each term then carries an independent relative
+// rounding of 2^-11 instead of 2^-22; over the 1e6..1e9 squares of the sum these average out to far below the
+// single-precision accuracy of the sum itself.
+template <class Epi, class = void> struct epi_coarse { static constexpr bool value = false; };
+template <class Epi> struct epi_coarse<Epi, std::enable_if_t<Epi::kCoarse>> { static constexpr bool value = true; };
 
 struct TcParams {
   int M, N, K;            // output rows, output columns, contraction length
@@ -89,8 +106,8 @@ struct TcParams {
   // A slice leaves its accumulators in tail_ws; the warp that finds itself last (tail_count) adds the slices
   // in slice order and runs the epilogue.  tail_split <= 1 switches this off.
   int tail_begin, tail_split;
-  float *tail_ws;         // [tiles from tail_begin][tail_split][8 warps][64][32] floats
-  int *tail_count;        // [tiles from tail_begin][8 warps], zero before and after every launch
+  float *tail_ws;         // [tiles from tail_begin][tail_split][4 row quarters][128][32] floats
+  int *tail_count;        // [tiles from tail_begin][4 row quarters], zero before and after every launch
 };
 
 // MODE TC_RAW_K:  A is [M][K] fp32, contiguous along K (a node-major matrix, rows = nodes), converted in the kernel;
@@ -119,20 +136,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_alo,
                const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_blo,
                const TcParams prm, Epi epi, double *__restrict__ partials) {
-  constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN;
+  constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN, COARSE = epi_coarse<Epi>::value;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *tr_base = smem + TC_STAGES * TC_STAGE_BYTES;
   uint64_t *bars = reinterpret_cast<uint64_t *>(tr_base + TC_TR_BYTES);
   uint64_t *full_bar = bars, *conv_bar = bars + TC_STAGES, *empty_bar = bars + 2 * TC_STAGES;
-  uint64_t *acc_full = bars + 3 * TC_STAGES, *acc_empty = acc_full + TC_ACC_BUFS;
+  uint64_t *acc_full = bars + 3 * TC_STAGES, *acc_empty = acc_full + 2 * TC_ACC_BUFS;     // acc_full: [set][buffer]
   uint64_t *corr_empty = acc_empty + TC_ACC_BUFS, *drain_bar = corr_empty + 1, *a_empty = drain_bar + 1;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(a_empty + TC_A_SLOTS);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   volatile int *skip_flag = abort_flag + 1;           // an earlier block gave up: this one does no work
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int ACC0 = 2 + TC_CONV_WARPS;              // first accumulate warp
+  constexpr int ACC0 = TC_ACC0;                        // first accumulate warp
   const int tiles_n = (prm.N + TC_BN - 1) / TC_BN, tiles_m = (prm.M + TC_BM - 1) / TC_BM;
   const int n_out_tiles = tiles_n * tiles_m * prm.n_split;
   const bool tail_on = prm.tail_split > 1;
@@ -147,6 +164,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     for (int b = 0; b < TC_ACC_BUFS; ++b) {
       ptx::mbar_init(&acc_full[b], 1);
+      ptx::mbar_init(&acc_full[TC_ACC_BUFS + b], 1);
       ptx::mbar_init(&acc_empty[b], TC_ACC_THREADS);
     }
     ptx::mbar_init(corr_empty, TC_ACC_THREADS);
@@ -196,9 +214,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   };
 
-  if (*skip_flag) {
+  // Register budgets per warpgroup (every warp of a warpgroup executes the same instruction; the choice is
+  // block-uniform, so a block that skips its work leaves the budgets alone).
+  const bool skip = *skip_flag != 0;
+  if (skip) {
     // nothing: do not queue work behind a block whose bounded wait expired
-  } else if (warp == 0) {
+  } else if (warp < TC_CONV0) {
+   ptx::setmaxnreg_dec<TC_REGS_CTRL>();
+   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (one lane)
     if (lane == 0) {
       int it = 0;
@@ -237,7 +260,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           ptx::mbar_wait(&full_bar[j % TC_STAGES], (j / TC_STAGES) & 1, abort_flag, 200000000ll, false);
       }
     }
-  } else if (warp == 1) {
+   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (one lane)
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::idesc_f16(TC_BM, TC_BN);
@@ -294,7 +317,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               if (main) ptx::mma_f16_ts(d, ah, dbh, idesc, !first || kk > 0);
             }
           };
-          const bool split_first = kb == 0 && ti > 0;
+          const bool split_first = !COARSE && kb == 0 && ti > 0;
           if (split_first) {
             // The correction tile still holds the previous output tile until the accumulate warps have read it:
             // the main-term MMAs of this block, which do not touch it, go first and keep the tensor pipe busy
@@ -307,7 +330,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
 #pragma unroll
           for (int kk = 0; kk < TC_KSTEPS; ++kk) {
-            issue(kk, true, !split_first);
+            issue(kk, !COARSE, !split_first);
             if (kk == TC_KSTEPS - 2) {
               // probe the coming block's barriers while the tensor pipe still has work queued
               seen_conv = ptx::mbar_test_wait(&ready_bar[s_next], sp_next);
@@ -320,7 +343,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             aslot ^= 1u;
           }
           if (last) {
-            ptx::mma_commit(&acc_full[b]);         // this group's partial product is complete
+            // this group's partial product is complete.  Each accumulate set has its own pair of barriers: a set
+            // is idle during the other set's tiles, and a waiter that lags by more than one phase of a barrier
+            // would take an earlier completion of the same parity for its own.
+            ptx::mma_commit(&acc_full[(ti & 1) * TC_ACC_BUFS + b]);
             if (b + 1 == TC_ACC_BUFS) first_round = false;
             b = b_next; bp = bp_next;
           }
@@ -333,25 +359,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ptx::mbar_wait(drain_bar, 0, abort_flag, 200000000ll, false);
       }
     }
+   }   // warps 2 and 3 of warpgroup 0 are spare
   } else if (warp < ACC0) {
-    // ---------------------------------------------------------------- converters (256 threads; idle with TC_PLANES)
+    ptx::setmaxnreg_dec<TC_REGS_CONV>();
+    // ---------------------------------------------------------------- converters (128 threads; idle with TC_PLANES)
     // The planes of A go to tensor memory, where the MMA reads them without touching shared memory: row i of the
-    // tile lives in lane i, and a warp can only write the 32 lanes of its own quarter (warp index mod 4).  So two
-    // warps share a quarter: thread (row t = 32 (warp mod 4) + lane, half h) converts the 32 values h*32 .. h*32+31
-    // of the K block of row t and writes 16 + 16 columns.
+    // tile lives in lane i, and a warp can only write the 32 lanes of its own quarter (warp index mod 4).  Thread
+    // t = 32 (warp mod 4) + lane converts row t of the K block, 32 values at a time (16 + 16 columns per half).
     // TC_RAW_K:  the values come from the swizzled [128][64] fp32 tile (row t, 16-byte chunks).
     // TC_RAW_MN: the tile is [64][128] (contraction index first), so the thread reads a column; and B is converted
-    //             too, in place in shared memory: thread (output index tb, half hb) reads its 32 values, all 256
-    //             threads wait until everyone has read (the planes overwrite the fp32 tile), then the thread writes
-    //             four 16-byte chunks of row tb of the hi and of the lo plane, chunk j at position j ^ (tb mod 8)
+    //             too, in place in shared memory: thread tb reads the 64 values of output index tb, all 128 threads
+    //             wait until everyone has read (the planes overwrite the fp32 tile), then the thread writes eight
+    //             16-byte chunks of row tb of the hi and of the lo plane, chunk j at position j ^ (tb mod 8)
     //             (the 128-byte swizzle).
     if constexpr (!PP) {
-      const int cw = warp - 2;                               // 0 .. 7
-      const int quarter = warp & 3, half = cw >> 2;
+      const int quarter = warp & 3;
       const int t = quarter * 32 + lane;
-      const int ct = threadIdx.x - 64, tb = ct & 127, hb = ct >> 7;
       const float scale_a = tc_pow2(exp_a), scale_b = tc_pow2(exp_b);
-      const uint32_t sw = (uint32_t)((MN ? tb : t) & 7);
+      const uint32_t sw = (uint32_t)(t & 7);
       bool ok = true;
       int it = 0;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -366,53 +391,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           ok = __all_sync(0xffffffffu, ok);                  // the tensor-memory stores below are warp-wide
           if (ok) {
             ptx::tc_fence_after_sync();
-            float v[32];
-            if (MN) {
-              const float *raw = reinterpret_cast<const float *>(stage);     // [64][128]
 #pragma unroll
-              for (int k = 0; k < 32; ++k) v[k] = raw[(32 * half + k) * 128 + t];
-            } else {
+            for (int half = 0; half < 2; ++half) {
+              float v[32];
+              if (MN) {
+                const float *raw = reinterpret_cast<const float *>(stage);     // [64][128]
 #pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                const float4 q = *reinterpret_cast<const float4 *>(stage + half * TC_PLANE_BYTES + t * 128 +
-                                                                   (((uint32_t)c ^ sw) << 4));
-                v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
+                for (int k = 0; k < 32; ++k) v[k] = raw[(32 * half + k) * 128 + t];
+              } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                  const float4 q = *reinterpret_cast<const float4 *>(stage + half * TC_PLANE_BYTES + t * 128 +
+                                                                     (((uint32_t)c ^ sw) << 4));
+                  v[4 * c] = q.x; v[4 * c + 1] = q.y; v[4 * c + 2] = q.z; v[4 * c + 3] = q.w;
+                }
               }
-            }
-            uint32_t hreg[16], lreg[16];
+              uint32_t hreg[16], lreg[16];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              float x[8];
+              for (int j = 0; j < 4; ++j) {
+                float x[8];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
-              uint4 h, l;
-              tc_split8(x, scale_a, h, l);
-              hreg[4 * j] = h.x; hreg[4 * j + 1] = h.y; hreg[4 * j + 2] = h.z; hreg[4 * j + 3] = h.w;
-              lreg[4 * j] = l.x; lreg[4 * j + 1] = l.y; lreg[4 * j + 2] = l.z; lreg[4 * j + 3] = l.w;
+                for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
+                uint4 h, l;
+                tc_split8(x, scale_a, h, l);
+                hreg[4 * j] = h.x; hreg[4 * j + 1] = h.y; hreg[4 * j + 2] = h.z; hreg[4 * j + 3] = h.w;
+                lreg[4 * j] = l.x; lreg[4 * j + 1] = l.y; lreg[4 * j + 2] = l.z; lreg[4 * j + 3] = l.w;
+              }
+              const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + TC_COL_A + (uint32_t)aslot * 64u +
+                                   16u * (uint32_t)half;
+              ptx::tmem_st16(col, hreg);
+              ptx::tmem_st16(col + 32u, lreg);
             }
-            const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + TC_COL_A + (uint32_t)aslot * 64u +
-                                 16u * (uint32_t)half;
-            ptx::tmem_st16(col, hreg);
-            ptx::tmem_st16(col + 32u, lreg);
           }
           if constexpr (MN) {
             uint8_t *region = stage + 2 * TC_PLANE_BYTES;
             const float *raw = reinterpret_cast<const float *>(region);      // [64][128]
-            float v[32];
+            float v[64];
             if (ok) {
 #pragma unroll
-              for (int k = 0; k < 32; ++k) v[k] = raw[(32 * hb + k) * 128 + tb];
+              for (int k = 0; k < 64; ++k) v[k] = raw[k * 128 + t];
             }
             // everyone has read its values of B (or someone gave up: then all stop here)
-            if (ptx::named_barrier_or(1, 256, !ok)) { ok = false; break; }
+            if (ptx::named_barrier_or(1, 32 * TC_CONV_WARPS, !ok)) { ok = false; break; }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < 8; ++j) {
               float x[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i) x[i] = v[8 * j + i];
               uint4 h, l;
               tc_split8(x, scale_b, h, l);
-              const uint32_t off = (uint32_t)tb * 128u + (((uint32_t)(4 * hb + j) ^ sw) << 4);
+              const uint32_t off = (uint32_t)t * 128u + (((uint32_t)j ^ sw) << 4);
               *reinterpret_cast<uint4 *>(region + off) = h;
               *reinterpret_cast<uint4 *>(region + TC_PLANE_BYTES + off) = l;
             }
@@ -427,47 +455,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ---------------------------------------------------------------- accumulate, then epilogue (256 threads)
-    // warp w owns tensor-memory lanes 32 (w mod 4) .. +31 = output rows m0 + that range, and the column half
-    // (w - 6) / 4 of the tile (64 columns)
-    const int lane_base = (warp & 3) * 32;
-    const int chalf = (warp - ACC0) >> 2;
-    float4 *tr = reinterpret_cast<float4 *>(tr_base) + (size_t)(warp - ACC0) * 32 * 8;    // 32 rows x 8 float4 per warp
+    ptx::setmaxnreg_inc<TC_REGS_ACC>();
+    // ---------------------------------------------------------------- accumulate, then epilogue (2 sets x 128 threads)
+    // The block's output tiles go to the two sets in turn.  Warp w of a set owns tensor-memory lanes 32 (w mod 4) ..
+    // +31 = output rows m0 + that range, and all 128 columns of the tile.  Both sets count every K block, so that the
+    // accumulator buffers and their barrier phases stay in step.
+    const int aw = warp - ACC0, set = aw >> 2, quarter = warp & 3;
+    const int lane_base = quarter * 32;
+    float4 *tr = reinterpret_cast<float4 *>(tr_base) + (size_t)aw * 32 * 8;    // 32 rows x 8 float4 per warp
     // columns up to the leading dimension are written: those from N on come out as exact zeros (zero-filled
     // operand rows, zero padding of the epilogue inputs), which keeps the padding of every matrix zero
     const int n_pad = epi.ldc;
     bool ok = true;
-    int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    int it = 0, ti = 0;
+    uint32_t uses0 = 0u, uses1 = 0u;                   // completions of this set's two acc_full barriers seen so far
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++ti) {
       int m0, n0, k_begin, n_kb, z;
       tile_coords(tile, m0, n0, k_begin, n_kb, z);
+      if ((ti & 1) != set) { it += n_kb; continue; }     // the other set's tile
       if (m0 + lane_base + lane < prm.M) {          // this thread's row of the epilogue inputs, on its way to L2
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int col = n0 + chalf * 64 + h * 32;
+        for (int h = 0; h < 4; ++h) {
+          const int col = n0 + h * 32;
           if (col < n_pad) epi.prefetch(m0 + lane_base + lane, col);
         }
       }
-      float acc[64];
+      float acc[128];
 #pragma unroll
-      for (int j = 0; j < 64; ++j) acc[j] = 0.f;
+      for (int j = 0; j < 128; ++j) acc[j] = 0.f;
       auto add_tile = [&](uint32_t col_base, float w) {       // acc += w * tile (w = 1: plain add)
-        const uint32_t src = tmem_base + ((uint32_t)lane_base << 16) + col_base + (uint32_t)(chalf * 64);
-        // 576 threads leave about 100 registers per thread: 16 columns at a time
+        const uint32_t src = tmem_base + ((uint32_t)lane_base << 16) + col_base;
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
-          uint32_t v[16];
-          ptx::tmem_ld16(src + 16u * h, v);
+          uint32_t v[32];
+          ptx::tmem_ld32(src + 32u * h, v);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) acc[16 * h + j] = fmaf(w, __uint_as_float(v[j]), acc[16 * h + j]);
+          for (int j = 0; j < 32; ++j) acc[32 * h + j] = fmaf(w, __uint_as_float(v[j]), acc[32 * h + j]);
         }
       };
-      const int n_grp = (n_kb + TC_FLUSH - 1) / TC_FLUSH;
-      for (int g = 0; g < n_grp && ok; ++g, ++it) {
-        const int b = it % TC_ACC_BUFS, buse = it / TC_ACC_BUFS;
-        ok = ptx::mbar_wait(&acc_full[b], buse & 1, abort_flag);
+      for (int g = 0; g < n_kb && ok; ++g, ++it) {
+        const int b = it % TC_ACC_BUFS;
+        ok = ptx::mbar_wait(&acc_full[set * TC_ACC_BUFS + b], (b ? uses1 : uses0) & 1u, abort_flag);
         if (!ok) break;
+        if (b) ++uses1; else ++uses0;
         ptx::tc_fence_after_sync();
         add_tile((uint32_t)(b * TC_BN), 1.0f);
         ptx::tc_fence_before_sync();
@@ -475,41 +506,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       if (!ok) break;
       if (n_kb > 0) {
-        // correction terms: complete once the last block's commit has arrived (it covers every earlier MMA)
-        add_tile(TC_COL_CORR, 1.0f / 2048.0f);
-        ptx::tc_fence_before_sync();
-        ptx::mbar_arrive(corr_empty);
+        if constexpr (!COARSE) {
+          // correction terms: complete once the last block's commit has arrived (it covers every earlier MMA)
+          add_tile(TC_COL_CORR, 1.0f / 2048.0f);
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(corr_empty);
+        }
         // undo the operand scalings (two exact factors, so that neither leaves the range on its own)
         const int e1 = (exp_a + exp_b) / 2, e2 = exp_a + exp_b - e1;
         const float u1 = tc_pow2(-e1), u2 = tc_pow2(-e2);
 #pragma unroll
-        for (int j = 0; j < 64; ++j) acc[j] = (acc[j] * u1) * u2;
+        for (int j = 0; j < 128; ++j) acc[j] = (acc[j] * u1) * u2;
       }
       int out_tile = tile;
       if (tile >= tail_begin) {
         // contraction slice of a tail tile: park the accumulators; the last warp to arrive sums the slices
         const int u = tile - tail_begin, t_idx = u / prm.tail_split;
         out_tile = tail_begin + t_idx;
-        float *mine = prm.tail_ws + ((size_t)u * 8 + (warp - ACC0)) * 2048;
+        float *mine = prm.tail_ws + ((size_t)u * 4 + quarter) * 4096;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) mine[j * 32 + lane] = acc[j];
+        for (int j = 0; j < 128; ++j) mine[j * 32 + lane] = acc[j];
         __threadfence();
         __syncwarp();
         int prev = 0;
-        if (lane == 0) prev = atomicAdd(prm.tail_count + t_idx * 8 + (warp - ACC0), 1);
+        if (lane == 0) prev = atomicAdd(prm.tail_count + t_idx * 4 + quarter, 1);
         prev = __shfl_sync(0xffffffffu, prev, 0);
         if (prev != prm.tail_split - 1) continue;
         __threadfence();
-        if (lane == 0) prm.tail_count[t_idx * 8 + (warp - ACC0)] = 0;
+        if (lane == 0) prm.tail_count[t_idx * 4 + quarter] = 0;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) acc[j] = 0.f;
+        for (int j = 0; j < 128; ++j) acc[j] = 0.f;
         for (int sl = 0; sl < prm.tail_split; ++sl) {
-          const float *part = prm.tail_ws + ((size_t)(t_idx * prm.tail_split + sl) * 8 + (warp - ACC0)) * 2048;
+          const float *part = prm.tail_ws + ((size_t)(t_idx * prm.tail_split + sl) * 4 + quarter) * 4096;
 #pragma unroll
-          for (int j = 0; j < 64; ++j) acc[j] += __ldcg(part + j * 32 + lane);
+          for (int j = 0; j < 128; ++j) acc[j] += __ldcg(part + j * 32 + lane);
         }
       }
-      // Epilogue.  Thread i of the warp holds row (lane_base + i), 64 columns.  The warp's piece goes through shared
+      // Epilogue.  Thread i of the warp holds row (lane_base + i), 128 columns.  The warp's piece goes through shared
       // memory 32 columns at a time: thread i writes its 8 float4 groups with the group index XOR-ed by (i mod 8)
       // (conflict-free 128-bit stores), then the warp reads the piece back transposed, so that the output is written,
       // and the inputs of the epilogue are read, in a coalesced pattern: the warp walks over its rows four at a
@@ -520,14 +553,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // only the squared norm: straight from the registers (rows and columns outside the matrix hold exact zeros)
         float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < 64; ++j) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
+        for (int j = 0; j < 128; ++j) s4[j & 3] = fmaf(acc[j], acc[j], s4[j & 3]);
         ss = ((double)s4[0] + (double)s4[1]) + ((double)s4[2] + (double)s4[3]);
       } else {
         float *C = epi.C + (size_t)z * prm.c_split_stride;
         float ssf = 0.f;
         uint32_t mx = 0u;                  // largest magnitude stored by this thread
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < 4; ++h) {
           __syncwarp();
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -535,7 +568,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tr[lane * 8 + (j ^ (lane & 7))] = make_float4(acc[4 * jj], acc[4 * jj + 1], acc[4 * jj + 2], acc[4 * jj + 3]);
           }
           __syncwarp();
-          const int col = n0 + chalf * 64 + h * 32 + 4 * (lane & 7);
+          const int col = n0 + h * 32 + 4 * (lane & 7);
           if (col < n_pad) {
             constexpr int BATCH = Epi::kInputs <= 1 ? 8 : 4;       // row steps whose loads are in flight together
 #pragma unroll
@@ -566,9 +599,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (epi.amax != nullptr) commit_amax(mx, epi.amax);      // the output is an operand of a later product
         }
       }
-      if (partials != nullptr) {          // one slot per tile and warp; the host adds the slots in index order
+      if (partials != nullptr) {          // one slot per tile and row quarter; a single block adds the slots in index order
         ss = warp_sum(ss);
-        if (lane == 0) partials[(size_t)out_tile * 8 + (warp - ACC0)] = ss;
+        if (lane == 0) partials[(size_t)out_tile * 4 + quarter] = ss;
       }
     }
   }

@@ -306,6 +306,14 @@ static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, cons
   static bool configured[64] = {false};
   const int dev = c->device;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
+    // The kernel's warpgroups re-divide the registers the block is launched with; their shares were added up
+    // against TC_REGS_LAUNCH per thread.  A build that launches with fewer would make an increase wait for ever:
+    // refuse to launch it.
+    cudaFuncAttributes attr;
+    PD_CUDA(cudaFuncGetAttributes(&attr, kern));
+    if (attr.numRegs != TC_REGS_LAUNCH)
+      return fail(PDADMM_ECUDA, "tensor-core product kernel was built with %d registers per thread, %d expected",
+                  attr.numRegs, TC_REGS_LAUNCH);
     PD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -384,7 +392,7 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     return PDADMM_OK;
   }
   const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM));
-  if (n_partials) *n_partials = 8 * n_tiles;        // one slot per tile and epilogue warp
+  if (n_partials) *n_partials = 4 * n_tiles;        // one slot per tile and row quarter
   if (amax_a == nullptr) {
     PD_TRY(amax_reserve(c, st, 1));
     amax_a = amax_of(c, st, A, (size_t)M * lda / 4);
@@ -1651,6 +1659,26 @@ extern "C" int pdadmm_profile_read(pdadmm_ctx *c, int k, double *ms, int64_t *la
   if (launches) *launches = c->prof_n[k];
   if (bytes) *bytes = c->prof_bytes[k];
   if (flops) *flops = c->prof_flops[k];
+  return PDADMM_OK;
+}
+extern "C" int pdadmm_time_augmentation(pdadmm_ctx *c, int reps, double *ms_per_hop, double *bytes_per_hop) {
+  if (!c || reps < 1 || reps > 1000 || !ms_per_hop) return fail(PDADMM_EINVAL, "bad argument");
+  if (c->n_blocks < 2) return fail(PDADMM_EINVAL, "the input has a single block: no sparse product to time");
+  PD_CUDA(cudaSetDevice(c->device));
+  Layer &l0 = c->layers[0];
+  cudaStream_t st = c->scr.st;
+  // the first hop again, block 0 -> block 1 of X: the same kernel on the same data writes the same bits
+  launch_spmm(st, c->row_ptr, c->col_idx, c->csr_val, (int)c->N, l0.p, l0.p + c->d, c->d, l0.ld_in);
+  PD_CUDA(cudaEventRecord(c->ev_begin, st));
+  for (int i = 0; i < reps; ++i)
+    launch_spmm(st, c->row_ptr, c->col_idx, c->csr_val, (int)c->N, l0.p, l0.p + c->d, c->d, l0.ld_in);
+  PD_CUDA(cudaEventRecord(c->ev_end, st));
+  PD_CUDA(cudaStreamSynchronize(st));
+  PD_CUDA(cudaGetLastError());
+  float ms = 0.f;
+  PD_CUDA(cudaEventElapsedTime(&ms, c->ev_begin, c->ev_end));
+  *ms_per_hop = ms / reps;
+  if (bytes_per_hop) *bytes_per_hop = (double)c->nnz * (8.0 + 4.0 * c->d) + 8.0 * (double)c->N * c->d;
   return PDADMM_OK;
 }
 extern "C" int pdadmm_last_step_ms(pdadmm_ctx *c, double *ms) {

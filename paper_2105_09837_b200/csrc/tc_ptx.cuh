@@ -141,6 +141,10 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- register budget of a warpgroup (four consecutive warps, all of which must execute the instruction) -----------
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // ---- descriptors -------------------------------------------------------------------------------------------
 // Shared-memory matrix descriptor (the tile base must be aligned to the swizzle period).
 // K-major operand  (rows = output index, k_row_bytes = 64 or 128 bytes of K per row): swizzle of the row width

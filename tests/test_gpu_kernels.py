@@ -65,7 +65,8 @@ def test_spmm_against_sparse_library(width):
 
 @pytest.mark.parametrize("mode,M,N,K", [(0, 300, 200, 100), (1, 300, 200, 100), (2, 300, 200, 1000), (0, 1000, 500, 500),
                                         (1, 1000, 500, 500), (2, 500, 500, 5000), (0, 129, 7, 65), (1, 5, 131, 3),
-                                        (2, 7, 100, 129), (2, 1000, 600, 333), (0, 2500, 120, 1100), (1, 1300, 250, 2100)])
+                                        (2, 7, 100, 129), (2, 1000, 600, 333), (0, 2500, 120, 1100), (1, 1300, 250, 2100),
+                                        (0, 30000, 300, 200), (1, 26000, 200, 330), (2, 1500, 1400, 3000)])
 @pytest.mark.parametrize("kind", ["normal", "positive", "tiny", "huge", "mixed"])
 def test_dense_products_keep_single_precision_accuracy_at_any_scale(mode, M, N, K, kind):
     """The tensor-core products split each operand into two half-precision planes after scaling it by a power of two
@@ -75,7 +76,9 @@ def test_dense_products_keep_single_precision_accuracy_at_any_scale(mode, M, N, 
     tiles and with contraction lengths that are not a multiple of the K block.  The last shape has enough output
     tiles (40) for the contraction over rows to take its operands as planes split beforehand; the smaller ones
     split them inside the product.  The last two have a partly filled last round of the persistent grid and a long
-    contraction, so their tiles are cut into 2 and 4 contraction slices that one warp per tile adds up."""
+    contraction, so their tiles are cut into 2 and 4 contraction slices that one warp per tile adds up.  The last three
+    have several output tiles per block of the persistent grid (705, 408 and 132 x 8 slices on 148 blocks), so the two
+    accumulate sets of a block alternate many times."""
     rng = np.random.default_rng(1000 * mode + M + N + K)
     a = rng.standard_normal((K, M) if mode == 2 else (M, K))
     b = rng.standard_normal((N, K) if mode == 0 else (K, N))
