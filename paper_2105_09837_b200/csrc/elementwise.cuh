@@ -290,6 +290,36 @@ make_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, cons
   }
 }
 
+// ---- fp16 planes of a node-major matrix, same orientation -------------------------------------------
+// x [rows][ld] fp32 -> hi, lo [rows][ld] halves (the padding columns, zero in x, come out as zero): the streamed
+// operand of a product whose output is several column tiles wide, split once here instead of once per column tile
+// inside the product.  Scaling and split as in make_planes_kernel; the exponent goes to *exp_out.  A thread converts
+// eight consecutive values (two 16-byte loads, one 16-byte store per plane).
+__global__ void __launch_bounds__(256)
+rows_planes_kernel(const float *__restrict__ x, size_t n8, const uint32_t *__restrict__ amax, int *__restrict__ exp_out,
+                   __half *__restrict__ hi, __half *__restrict__ lo) {
+  const int e = tc_scale_exp(*amax);
+  if (blockIdx.x == 0 && threadIdx.x == 0) *exp_out = e;
+  const float scale = __uint_as_float((uint32_t)(e + 127) << 23);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 a = reinterpret_cast<const float4 *>(x)[2 * i], b = reinterpret_cast<const float4 *>(x)[2 * i + 1];
+    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    float h[8], l[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float xs = v[k] * scale;
+      h[k] = __uint_as_float((__float_as_uint(xs) + 0x1000u) & 0xFFFFE000u);
+      l[k] = (xs - h[k]) * 2048.0f;
+    }
+    auto pack = [](float p, float q) {
+      const __half2 t = __floats2half2_rn(p, q);
+      return *reinterpret_cast<const uint32_t *>(&t);
+    };
+    reinterpret_cast<uint4 *>(hi)[i] = make_uint4(pack(h[0], h[1]), pack(h[2], h[3]), pack(h[4], h[5]), pack(h[6], h[7]));
+    reinterpret_cast<uint4 *>(lo)[i] = make_uint4(pack(l[0], l[1]), pack(l[2], l[3]), pack(l[4], l[5]), pack(l[6], l[7]));
+  }
+}
+
 // ---- fp16 planes of a node-major matrix, transposed -------------------------------------------------
 // x [rows = nodes][ld] fp32 -> hiT, loT [cols][ldT] with the node index contiguous: operands of the product that
 // contracts over the nodes (the W-gradient r^T p+), for layers where splitting them once here is cheaper than

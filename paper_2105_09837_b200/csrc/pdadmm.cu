@@ -83,6 +83,8 @@ struct Layer {
   Planes Gp;                // fp16 planes of grad_W: [n_out][ldh_in]
   __half *xT_hi = nullptr, *xT_lo = nullptr;   // layer 1 only: transposed planes of p_1 = X, which never changes
   int *xT_exp = nullptr;
+  __half *x_hi = nullptr, *x_lo = nullptr;     // layer 1 only: planes of X in its own orientation [N][ld_in]
+  int *x_exp = nullptr;
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in] codes of 1 byte (up to 256 levels) or 2 bytes, quantised mode, l >= 2
   float scale = 1.0f;       // level spacing s_l of p_l
@@ -112,6 +114,10 @@ struct Scratch {
   // transposed fp16 planes ([width][ldT], node index contiguous) of r_l and p_l for the product over the nodes
   __half *rT_hi = nullptr, *rT_lo = nullptr, *pT_hi = nullptr, *pT_lo = nullptr;
   int *rT_exp = nullptr, *pT_exp = nullptr;
+  // planes [N][ld] of the streamed operand of a product over several column tiles (split once per product)
+  __half *a_hi = nullptr, *a_lo = nullptr;
+  size_t a_cap = 0;                // elements each of the two holds
+  int *a_exp = nullptr;
   int *h_flag = nullptr;           // pinned word that receives the accept flag of the lane's quantised trial
   cudaEvent_t ev_flag = nullptr;   // recorded after the copy of that flag
 };
@@ -161,6 +167,7 @@ struct pdadmm_ctx {
   double prof_ms[pd::KC_COUNT] = {0}, prof_bytes[pd::KC_COUNT] = {0}, prof_flops[pd::KC_COUNT] = {0};
   int64_t prof_n[pd::KC_COUNT] = {0};
   std::vector<void *> allocs;       // driver allocations: chunks and large arrays
+  size_t bytes_handed_out = 0;      // device bytes handed out by dev_alloc so far
   char *arena_base = nullptr;       // current chunk
   size_t arena_cap = 0, arena_used = 0, arena_next = size_t(64) << 20;
   bool use_tc = true;               // dense products on the tensor cores
@@ -208,6 +215,7 @@ static int dev_alloc(pdadmm_ctx *c, T **ptr, size_t count, bool zero = true) {
     }
   }
   if (zero) PD_CUDA(cudaMemsetAsync(p, 0, bytes, c->scr.st));   // same stream as every kernel that uses it
+  c->bytes_handed_out += bytes;
   *ptr = (T *)p;
   return PDADMM_OK;
 }
@@ -379,10 +387,19 @@ static int alloc_planes(pdadmm_ctx *c, int rows, int cols, bool transposed_too, 
 // C[M][N] = A[M][K] * op(B), fused epilogue; per-block sums of squares go to `partials` (or nullptr).
 // B is given by its fp32 matrix (CUDA-core path; B_NMAJOR tells its orientation) and by its two fp16 planes
 // [N][K] (tensor-core path).  `amax_a`: the largest magnitude of A if the caller has it, else it is computed here.
+// The streamed operand A is split into its planes tile by tile inside the product, or once beforehand
+// (rows_planes_kernel into the lane's scratch, or planes the caller keeps: `Ap`).  Inside, every column tile of the
+// output converts the same rows of A again and the converters' tensor-memory stores slow the MMAs down (measured:
+// 2640 cycles per 64-deep K block against 1610 with both operands as planes); beforehand costs one pass of
+// 8 bytes per element at HBM speed.  Measured per product (split pass included): 4 column tiles 69 against 58 us,
+// 8 tiles 1.18 against 1.21 ms, 16 tiles 2.42 against 2.29 ms -- beforehand wins from 16 column tiles on, and
+// always where the planes are kept (X).
+constexpr int PLANES_FROM_COL_TILES = 16;
 template <bool B_NMAJOR, class Epi>
 static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
                       const float *B, int ldb, const PlaneRef &Bp, const Epi &epi, double *partials,
-                      int *n_partials, double extra_bytes, const uint32_t *amax_a = nullptr) {
+                      int *n_partials, double extra_bytes, const uint32_t *amax_a = nullptr,
+                      const PlaneRef *Ap = nullptr) {
   const double bytes = 4.0 * ((double)M * K + (double)N * K + (double)M * N) + extra_bytes;
   if (!c->use_tc) {
     dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM));
@@ -397,11 +414,29 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     PD_TRY(amax_reserve(c, st, 1));
     amax_a = amax_of(c, st, A, (size_t)M * lda / 4);
   }
-  CUtensorMap ma, mb, mbl;
-  PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TM_RAW_K, &ma));
+  PlaneRef a_planes{nullptr, nullptr, 0, nullptr};
+  if (Ap != nullptr && Ap->hi != nullptr) {
+    a_planes = *Ap;
+  } else if (c->cur->a_hi != nullptr && lda % 8 == 0 && (size_t)M * lda <= c->cur->a_cap &&
+             ceil_div(N, TC_BN) >= PLANES_FROM_COL_TILES) {
+    Scratch &sc = *c->cur;
+    const size_t n8 = (size_t)M * lda / 8;
+    Launch l(c, KC_PLANES, st, 8.0 * M * K, 0);
+    rows_planes_kernel<<<ew_grid(n8), 256, 0, st>>>(A, n8, amax_a, sc.a_exp, sc.a_hi, sc.a_lo);
+    a_planes = PlaneRef{sc.a_hi, sc.a_lo, lda, sc.a_exp};
+  }
+  const bool pp = a_planes.hi != nullptr;
+  CUtensorMap ma, mal, mb, mbl;
+  if (pp) {
+    PD_TRY(get_tmap(c, a_planes.hi, (uint64_t)K, (uint64_t)M, (uint64_t)a_planes.ld, TM_PLANE, &ma));
+    PD_TRY(get_tmap(c, a_planes.lo, (uint64_t)K, (uint64_t)M, (uint64_t)a_planes.ld, TM_PLANE, &mal));
+  } else {
+    PD_TRY(get_tmap(c, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, TM_RAW_K, &ma));
+    mal = ma;
+  }
   PD_TRY(get_tmap(c, Bp.hi, (uint64_t)K, (uint64_t)N, (uint64_t)Bp.ld, TM_PLANE, &mb));
   PD_TRY(get_tmap(c, Bp.lo, (uint64_t)K, (uint64_t)N, (uint64_t)Bp.ld, TM_PLANE, &mbl));
-  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1, amax_a, nullptr, nullptr, Bp.exp};
+  TcParams prm{M, N, K, round_up(K, TC_BK), 1, 0, c->d_flag + 1, pp ? nullptr : amax_a, nullptr, pp ? a_planes.exp : nullptr, Bp.exp};
   // The persistent grid works through the tiles in rounds of n_sms; a last round that fills only part of the
   // SMs costs as much as a full one, so its tiles are cut along the contraction into as many slices as fit.
   int n_units = n_tiles;
@@ -418,6 +453,7 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     }
   }
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
+  if (pp) return launch_tc<TC_PLANES, Epi>(c, st, ma, mal, mb, mbl, prm, epi, partials, n_units);
   return launch_tc<TC_RAW_K, Epi>(c, st, ma, ma, mb, mbl, prm, epi, partials, n_units);
 }
 
@@ -484,12 +520,16 @@ static PlaneRef planes_W(const Layer &ly) { return PlaneRef{ly.Wp.hi, ly.Wp.lo, 
 static PlaneRef planes_WT(const Layer &ly) { return PlaneRef{ly.Wp.hiT, ly.Wp.loT, ly.Wp.ldhT, ly.Wp.exp}; }
 static PlaneRef planes_G(const Layer &ly) { return PlaneRef{ly.Gp.hi, ly.Gp.lo, ly.Gp.ldh, ly.Gp.exp}; }
 
+// planes of p_1 = X, which never changes, in its own orientation (null planes if the layer does not keep them)
+static PlaneRef planes_X(const Layer &ly) { return PlaneRef{ly.x_hi, ly.x_lo, ly.ld_in, ly.x_exp}; }
+
 // r_l = P_l W_l^T + b_l - z_l from scratch (only when the cached residual is not valid).
 static int refresh_residual(pdadmm_ctx *c, Layer &ly, cudaStream_t st) {
   PD_CUDA(cudaMemsetAsync(ly.amax_r, 0, sizeof(uint32_t), st));
   EpiLinearResidual epi{ly.r, ly.ld_out, ly.b, ly.z, ly.amax_r};
+  const PlaneRef xp = planes_X(ly);
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)c->N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in,
-                           planes_W(ly), epi, nullptr, nullptr, 4.0 * c->N * ly.n_out, ly.amax_p));
+                           planes_W(ly), epi, nullptr, nullptr, 4.0 * c->N * ly.n_out, ly.amax_p, &xp));
   if (!c->use_tc) {       // the CUDA-core product does not track the maximum of what it stores
     Launch l(c, KC_AMAX, st, 4.0 * c->N * ly.ld_out, 0);
     absmax_kernel<<<ew_grid((size_t)c->N * ly.ld_out / 4), EW_THREADS, 0, st>>>(ly.r, (size_t)c->N * ly.ld_out / 4, ly.amax_r);
@@ -641,8 +681,9 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
   int np = 0;
   double *slots_b = s.slots + s.n_slots / 2;
   EpiStoreSumsq epi{s.s1, ly.ld_out};
+  const PlaneRef xp = planes_X(ly);
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.ld_in, planes_G(ly),
-                           epi, slots_b, &np, 0, ly.amax_p));
+                           epi, slots_b, &np, 0, ly.amax_p, &xp));
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (gw + np), 0);
     finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2, ly.amax_r);
@@ -886,6 +927,15 @@ static int alloc_trial_buffers(pdadmm_ctx *c, Scratch &s, size_t n) {
 }
 
 // transposed planes of r_l (up to max_out columns) and of p_l, l >= 2 (up to max_in columns) of one lane
+// planes of the streamed operand of a product, once per lane: as wide as the widest matrix the lane's s1 holds
+static int alloc_row_planes(pdadmm_ctx *c, Scratch &s, size_t n) {
+  PD_TRY(dev_alloc(c, &s.a_hi, n, false));
+  PD_TRY(dev_alloc(c, &s.a_lo, n, false));
+  PD_TRY(dev_alloc(c, &s.a_exp, 1));
+  s.a_cap = n;
+  return PDADMM_OK;
+}
+
 static int alloc_transposed(pdadmm_ctx *c, Scratch &s, int max_out, int max_in) {
   if (max_out > 0) {
     PD_TRY(dev_alloc(c, &s.rT_hi, (size_t)max_out * c->ldT));
@@ -982,6 +1032,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   // scratch
   Scratch &s = c->scr;
   int tr_out = 0, tr_in = 0;
+  const size_t bytes_before_scratch = c->bytes_handed_out;
   const size_t e_max = (size_t)N * std::max(max_in, max_out);
   PD_TRY(dev_alloc(c, &s.s1, e_max));
   PD_TRY(dev_alloc(c, &s.s2, (size_t)N * max_out));
@@ -1003,7 +1054,17 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
       if (l > 0) tr_in = std::max(tr_in, ly.n_in);
     }
     PD_TRY(alloc_transposed(c, s, tr_out, tr_in));
+    // planes of streamed operands: needed if some layer's products are at least PLANES_FROM_COL_TILES column tiles wide
+    bool want_row_planes = false;
+    for (int l = 0; l < c->L; ++l)
+      want_row_planes |= std::max(ceil_div(c->layers[l].n_out, TC_BN), l > 0 ? ceil_div(c->layers[l].n_in, TC_BN) : 0) >= PLANES_FROM_COL_TILES;
+    if (want_row_planes) PD_TRY(alloc_row_planes(c, s, e_max));
     Layer &l0 = c->layers[0];
+    if (ceil_div(l0.n_out, TC_BN) >= 2) {      // X is split once for ever: worth it from two column tiles on
+      PD_TRY(dev_alloc(c, &l0.x_hi, (size_t)N * l0.ld_in, false));
+      PD_TRY(dev_alloc(c, &l0.x_lo, (size_t)N * l0.ld_in, false));
+      PD_TRY(dev_alloc(c, &l0.x_exp, 1));
+    }
     if (planes_beforehand(l0.n_out, l0.n_in, true)) {
       PD_TRY(dev_alloc(c, &l0.xT_hi, (size_t)l0.n_in * c->ldT));
       PD_TRY(dev_alloc(c, &l0.xT_lo, (size_t)l0.n_in * c->ldT));
@@ -1011,8 +1072,14 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     PD_TRY(dev_alloc(c, &l0.xT_exp, 1));
   }
 
-  // further lanes for the concurrency across layers: own stream, product outputs, partial tiles, slots
-  const int n_lanes = (cfg->flags & PDADMM_FLAG_ONE_LANE) ? 1 : std::min(c->L, PDADMM_N_LANES);
+  // further lanes for the concurrency across layers: own stream, product outputs, partial tiles, slots.
+  // Small problems are bound by the latency of their chain of launches, which only more concurrent chains shorten
+  // (workload c1, 10 layers: 2 lanes 0.40 ms per iteration); large ones gain little beyond two (c2: 2 lanes 273,
+  // 4 lanes 278 iterations/s) and their scratch is gigabytes per lane.  So: as many lanes as 2 GB of scratch pay for,
+  // at least PDADMM_N_LANES, at most one per layer.
+  const size_t lane_bytes = std::max<size_t>(c->bytes_handed_out - bytes_before_scratch, 1);
+  const int affordable = (int)std::min<size_t>(64, (size_t(2) << 30) / lane_bytes);
+  const int n_lanes = (cfg->flags & PDADMM_FLAG_ONE_LANE) ? 1 : std::min(c->L, std::max(PDADMM_N_LANES, affordable));
   for (int i = 1; i < n_lanes; ++i) {
     c->more_lanes.emplace_back(new Scratch());
     Scratch &x = *c->more_lanes.back();
@@ -1028,6 +1095,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
       PD_TRY(dev_alloc(c, &x.tail_count, (size_t)c->n_sms * 8));
       PD_TRY(dev_alloc(c, &x.amax_pool, (size_t)AMAX_POOL));
       PD_TRY(alloc_transposed(c, x, tr_out, tr_in));
+      if (s.a_hi != nullptr) PD_TRY(alloc_row_planes(c, x, e_max));
     }
   }
   c->ev_p.resize(c->L);
@@ -1048,8 +1116,13 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     EpiStore epi{ly.z, ly.ld_out};
     PD_TRY(split_planes(c, st, ly.W, ly.n_out, ly.n_in, ly.ld_in, ly.Wp));
     absmax_kernel<<<ew_grid((size_t)N * ly.ld_in / 4), EW_THREADS, 0, st>>>(ly.p, (size_t)N * ly.ld_in / 4, ly.amax_p);
+    if (l == 0 && ly.x_hi != nullptr) {
+      const size_t n8 = (size_t)N * ly.ld_in / 8;
+      rows_planes_kernel<<<ew_grid(n8), 256, 0, st>>>(ly.p, n8, ly.amax_p, ly.x_exp, ly.x_hi, ly.x_lo);
+    }
+    const PlaneRef xp = planes_X(ly);
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
-                             epi, nullptr, nullptr, 0, ly.amax_p));
+                             epi, nullptr, nullptr, 0, ly.amax_p, &xp));
     if (l + 1 == c->L) break;
     Layer &nx = c->layers[l + 1];
     const size_t n4 = (size_t)N * ly.ld_out / 4;
@@ -1077,6 +1150,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->r_valid = true;                        // z = W p + b exactly by construction, r = 0 (allocated as zero)
   c->w_planes_valid = true;
   c->amax_p_valid = true;
+  c->xT_valid = false;            // the transposed planes of X are made by the first step
   c->launches = 0;
   return PDADMM_OK;
 }
@@ -1155,9 +1229,15 @@ static int ensure_residual(pdadmm_ctx *c) {
     }
     c->amax_p_valid = true;
   }
-  if (!c->xT_valid && c->use_tc && planes_beforehand(c->layers[0].n_out, c->layers[0].n_in, true)) {
+  if (!c->xT_valid && c->use_tc) {          // both kinds of planes of X follow the stored X
     Layer &l0 = c->layers[0];
-    transpose_planes(c, c->scr.st, l0.p, (int)c->N, l0.n_in, l0.ld_in, l0.amax_p, l0.xT_hi, l0.xT_lo, c->ldT, l0.xT_exp);
+    if (planes_beforehand(l0.n_out, l0.n_in, true))
+      transpose_planes(c, c->scr.st, l0.p, (int)c->N, l0.n_in, l0.ld_in, l0.amax_p, l0.xT_hi, l0.xT_lo, c->ldT, l0.xT_exp);
+    if (l0.x_hi != nullptr) {
+      const size_t n8 = (size_t)c->N * l0.ld_in / 8;
+      Launch k(c, KC_PLANES, c->scr.st, 8.0 * c->N * l0.n_in, 0);
+      rows_planes_kernel<<<ew_grid(n8), 256, 0, c->scr.st>>>(l0.p, n8, l0.amax_p, l0.x_exp, l0.x_hi, l0.x_lo);
+    }
     c->xT_valid = true;
   }
   if (!c->t_valid) {
@@ -1298,8 +1378,10 @@ extern "C" int pdadmm_predict(pdadmm_ctx *c, float *logits_out, int32_t *pred_ou
     uint32_t *w_out = nullptr;
     if (c->use_tc) w_out = amax_take(c);
     EpiBiasAct epi{out, ly.ld_out, ly.b, l + 1 < c->L ? 1 : 0, c->slope, w_out};
+    // the first layer's input is X: its planes are kept by the context while they match the stored X
+    const PlaneRef xp = (l == 0 && c->xT_valid) ? planes_X(ly) : PlaneRef{nullptr, nullptr, 0, nullptr};
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, N, ly.n_out, ly.n_in, in, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
-                             epi, nullptr, nullptr, 0, w_in));
+                             epi, nullptr, nullptr, 0, w_in, &xp));
     w_in = w_out;
     in = out;
   }
@@ -1519,7 +1601,7 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
     // operand shapes as stored: rows x cols
     const int a_rows = mode == 2 ? K : M, a_cols = mode == 2 ? M : K;
     const int b_rows = mode == 0 ? N : K, b_cols = mode == 0 ? K : N;
-    const int lda = round_up(a_cols, 4), ldb = round_up(b_cols, 4), ldc = round_up(N, 4);
+    const int lda = round_up(a_cols, mode == 2 ? 4 : 8), ldb = round_up(b_cols, 4), ldc = round_up(N, 4);
     float *dA, *dB, *dC, *part = nullptr;
     double *slots;
     Planes Bp;
@@ -1535,6 +1617,7 @@ extern "C" int pdadmm_matmul(int device, int mode, int M, int N, int K, const fl
       // planes of B as [N][K]: B itself in mode 0, its transpose in mode 1
       if (mode != 2) PD_TRY(alloc_planes(c, b_rows, b_cols, mode == 1, mode == 0, &Bp));
       if (mode != 2) PD_TRY(split_planes(c, st, dB, b_rows, b_cols, ldb, Bp));
+      if (mode != 2) PD_TRY(alloc_row_planes(c, c->scr, (size_t)a_rows * lda));     // used from four column tiles on
     }
     int np = 0;
     if (mode == 0) {
