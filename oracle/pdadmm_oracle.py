@@ -666,6 +666,129 @@ def lagrangian(s: State, prm: Params) -> float:
 
 
 # ----------------------------------------------------------------------------
+# The same iteration on node shards
+# ----------------------------------------------------------------------------
+
+def split_nodes(n_nodes: int, n_parts: int):
+    """Contiguous, balanced node ranges: part r holds nodes [r N // R, (r+1) N // R)."""
+    return [slice(r * n_nodes // n_parts, (r + 1) * n_nodes // n_parts) for r in range(n_parts)]
+
+
+def shard_state(s: State, parts) -> List[State]:
+    """The columns (nodes) of p, z, q, u, y, mask of each part; W, b and the level spacings are replicated."""
+    out = []
+    for sl in parts:
+        out.append(State([a[:, sl].copy() for a in s.p], [w.copy() for w in s.W], [b.copy() for b in s.b],
+                         [a[:, sl].copy() for a in s.z], [a[:, sl].copy() for a in s.q], [a[:, sl].copy() for a in s.u],
+                         s.y[sl].copy(), s.mask[sl].copy(), list(s.scale), list(s.tau), list(s.theta), list(s.trials)))
+    return out
+
+
+def merge_shards(shards: List[State]) -> State:
+    """Inverse of shard_state (W, b, scalars from the first shard: they are identical on all)."""
+    f = shards[0]
+    cat = lambda name, l: np.concatenate([getattr(x, name)[l] for x in shards], axis=1)
+    return State([cat("p", l) for l in range(f.L)], [w.copy() for w in f.W], [b.copy() for b in f.b],
+                 [cat("z", l) for l in range(f.L)], [cat("q", l) for l in range(f.L - 1)],
+                 [cat("u", l) for l in range(f.L - 1)], np.concatenate([x.y for x in shards]),
+                 np.concatenate([x.mask for x in shards]), list(f.scale), list(f.tau), list(f.theta), list(f.trials))
+
+
+def _local_sum(values):
+    """Sum of the partial results of this process's shards, in shard order."""
+    total = values[0]
+    for v in values[1:]:
+        total = total + v
+    return total
+
+
+def iterate_sharded(shards: List[State], prm: Params, allreduce=None) -> List[State]:
+    """One pass of Algorithm 1 with the nodes divided among shards (the multi-device form that the augmented MLP
+    admits: once X is built, p_l, z_l, q_l, u_l are one column per node and W_l, b_l are shared).
+
+    Every update acts on each node's column by itself except for the sums over nodes inside the step parameters
+    and the shared variables: ||g||^2 and ||W g||^2 (tau, Eq. update p), the sums of the acceptance test of the
+    quantised update, nabla_W phi = nu sum_j (W p + b - z)_j p_j^T and ||G p||^2 (theta, Eq. update W), and
+    nabla_b phi = nu sum_j (W p + b - z)_j (Eq. update b).  Each shard forms its part of these sums; `allreduce`
+    receives this process's part (its shards added in shard order) and returns the sum over all processes.  With
+    allreduce=None the given shards are all there is.  The result equals `iterate` on the merged state up to the
+    order of those additions.
+    """
+    rho, nu, L = prm.rho, prm.nu, shards[0].L
+    total = (lambda parts: _local_sum(parts)) if allreduce is None else (lambda parts: allreduce(_local_sum(parts)))
+    new = [s.copy() for s in shards]
+    n_total = int(total([np.array(float(s.p[0].shape[1])) for s in shards]))
+    # p_l^{k+1}, l = 2..L
+    for l in range(1, L):
+        g = [grad_p_phi(s.p[l], s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho) for s in shards]
+        sums = total([np.array([float(np.sum(gi * gi)), float(np.sum((s.W[l] @ gi) ** 2))]) for s, gi in zip(shards, g)])
+        gg, wg = float(sums[0]), float(sums[1])
+        tau = float(rho) if gg == 0.0 else float(rho + nu * wg / gg)
+        trials = 0
+        if prm.quant_levels:
+            phi_old = [phi(s.p[l], s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho) for s in shards]
+            for trial in range(1, prm.max_trials + 1):
+                p_new = [nearest_level(s.p[l] - gi / tau, s.scale[l], prm.quant_levels, prm.level_lo)[1]
+                         for s, gi in zip(shards, g)]
+                parts = []
+                for s, gi, pn, po in zip(shards, g, p_new, phi_old):
+                    d = pn - s.p[l]
+                    parts.append(np.array([phi(pn, s.W[l], s.b[l], s.z[l], nu, s.q[l - 1], s.u[l - 1], rho), po,
+                                           float(np.sum(gi * d)), float(np.sum(d * d))]))
+                lhs, po, gd, dd = (float(x) for x in total(parts))
+                trials = trial
+                if lhs <= po + gd + 0.5 * tau * dd + 0.5 * prm.accept_slack * tau * dd:
+                    break
+                tau *= 2.0
+            else:
+                trials = -1
+        else:
+            p_new = [s.p[l] - gi / tau for s, gi in zip(shards, g)]
+        for n, pn in zip(new, p_new):
+            n.p[l], n.tau[l], n.trials[l] = pn, tau, trials
+    # W_l^{k+1}: the gradient is a sum over nodes, theta needs ||G p||^2
+    for l in range(L):
+        G = total([grad_W_phi(n.p[l], s.W[l], s.b[l], s.z[l], nu) for s, n in zip(shards, new)])
+        GG = float(np.sum(G * G))
+        Gp2 = float(total([np.array(float(np.sum((G @ n.p[l]) ** 2))) for n in new]))
+        theta = 0.0 if GG == 0.0 else float(nu * Gp2 / GG)
+        for s, n in zip(shards, new):
+            n.W[l] = s.W[l].copy() if theta == 0.0 else s.W[l] - G / theta
+            n.theta[l] = theta
+    # b_l^{k+1}: the gradient is a sum over nodes, the step is 1 / (nu |V|) with |V| the total node count
+    for l in range(L):
+        gb = total([grad_b_phi(n.p[l], n.W[l], s.b[l], s.z[l], nu) for s, n in zip(shards, new)])
+        for s, n in zip(shards, new):
+            n.b[l] = s.b[l] - gb / (nu * n_total)
+    # z, q, u: node by node
+    for s, n in zip(shards, new):
+        for l in range(L):
+            a = n.W[l] @ n.p[l] + n.b[l][:, None]
+            if l < L - 1:
+                n.z[l] = update_z_hidden(a, s.q[l], s.z[l], prm.slope)
+            elif prm.risk == "ls":
+                n.z[l] = update_z_last_least_squares(a, s.y, s.mask, nu)
+            else:
+                n.z[l] = update_z_last(a, s.y, s.mask, nu)
+        for l in range(L - 1):
+            if prm.quant_levels and prm.quantize_q:
+                n.q[l] = update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels,
+                                            prm.level_lo, prm.slope)
+            else:
+                n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.slope)
+        for l in range(L - 1):
+            n.u[l] = update_u(s.u[l], n.p[l + 1], n.q[l], rho)
+    return new
+
+
+def objective_sharded(shards: List[State], prm: Params, allreduce=None) -> np.ndarray:
+    """The components of L_rho of the merged state: every component is a sum over nodes."""
+    parts = [objective(s, prm)[:5] for s in shards]
+    comps = _local_sum(parts) if allreduce is None else allreduce(_local_sum(parts))
+    return np.concatenate([comps, [np.sum(comps)]])
+
+
+# ----------------------------------------------------------------------------
 # The trained model: forward pass, prediction, accuracy
 # ----------------------------------------------------------------------------
 
