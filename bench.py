@@ -4,9 +4,10 @@
     python bench.py --gpus N --steps K --warmup W [--workload c1..c5|all] [--impl reference]
 
 One step is one iteration of Algorithm 1 over every layer (p, W, b, z, q, u updates).  With N > 1 the
-script runs under torchrun, one process per GPU; every rank runs an independent replica of the
-workload (the path has no cross-GPU exchange), the timed region is bracketed by barriers and the
-reported time is the maximum over ranks.  Rank 0 prints one JSON line: its top-level fields are the headline
+script runs under torchrun, one process per GPU; the nodes of the workload are divided among the
+ranks (W and b replicated, the sums over nodes all-reduced by NCCL), or with --replicas every rank
+runs an independent copy; the timed region is bracketed by barriers and the reported time is the
+maximum over ranks.  Rank 0 prints one JSON line: its top-level fields are the headline
 workload (c2), and on one GPU `workloads` holds one record for each of the five workloads.
 """
 
@@ -189,7 +190,7 @@ def describe(w, quant_q=False):
             f"{' (p and q quantised)' if quant_q else ''}, rho=nu={w.rho}")
 
 
-def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu, with_e2e=True):
+def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu, with_e2e=True, shard_nodes=False):
     """Times `steps` iterations of one workload (after `warmup`), a per-kernel pass, the end-to-end leg and the
     oracle sample.  Returns the record of that workload."""
     import torch
@@ -204,7 +205,17 @@ def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu
             dist.barrier()
         torch.cuda.synchronize(device)
 
-    ctx = B.from_inputs(inp, device=device, flags=flags)
+    # several GPUs: the nodes are divided among the ranks (every rank keeps p, z, q, u of its nodes and a copy of W, b;
+    # the sums over nodes go through NCCL), so the job is ONE problem and more GPUs make it faster (strong scaling);
+    # with --replicas every rank runs the whole problem on its own (weak scaling)
+    shard, reducer = None, None
+    if shard_nodes and world > 1:
+        from paper_2105_09837_b200 import sharded
+        reducer = sharded.TorchAllReduce(device)
+        lo, cnt = sharded.node_range(dist.get_rank(), world, w.n_nodes)
+        shard = (lo, cnt, reducer.fn)
+    jobs = 1 if shard is not None else world
+    ctx = B.from_inputs(inp, device=device, flags=flags, shard=shard)
     ctx.step(warmup)
     launches0 = ctx.launches()
     barrier()
@@ -214,11 +225,12 @@ def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu
         barrier()
     launches = ctx.launches() - launches0
     ms = replicas.max_over_ranks(ms, dist, f"cuda:{device}")
-    value = replicas.job_throughput(world, steps, ms)
+    value = replicas.job_throughput(jobs, steps, ms)
     clocks = clk.summary()
+    comm = ctx.comm_bytes() if shard is not None else 0
     obj = ctx.objective()
     spmm = None
-    if w.n_blocks > 1:
+    if w.n_blocks > 1 and shard is None:
         hop_ms, hop_bytes = ctx.time_augmentation(20)
         spmm = {"ms_per_hop": hop_ms, "gbs": hop_bytes / (hop_ms * 1e-3) / 1e9, "frac_of_hbm_peak": hop_bytes / (hop_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
                 "note": "algorithmic bytes nnz(8+4d)+8Nd; the gathered rows are served from L2 where the block fits"}
@@ -272,6 +284,8 @@ def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu
            "t_roof_note": "sum over kernel classes of max(algorithmic flop / tensor peak, algorithmic bytes / copy peak), "
                           "per iteration; frac_t_roof = t_roof / measured time per iteration",
            "kernels": kernels, "spmm": spmm, "objective": float(obj[5])}
+    if shard is not None:
+        rec["allreduce_bytes_per_step"] = comm / (warmup + steps)
 
     if with_e2e:
         # end to end through the public API from host buffers: init (H2D of graph, features, weights), K iterations,
@@ -285,7 +299,7 @@ def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu
         inp.init_W = [pinned(x) for x in inp.init_W]
         barrier()
         t0 = time.perf_counter()
-        ctx2 = B.from_inputs(inp, device=device, flags=flags)
+        ctx2 = B.from_inputs(inp, device=device, flags=flags, shard=shard)
         ctx2.step(steps)
         ctx2.objective()
         d2h = 48
@@ -296,7 +310,7 @@ def run_workload(name, steps, warmup, flags, device, world, dist, simt, with_cpu
         e2e_s = time.perf_counter() - t0
         ctx2.destroy()
         e2e_s = replicas.max_over_ranks(e2e_s, dist, f"cuda:{device}")
-        rec["e2e"] = {"value": replicas.job_throughput(world, steps, e2e_s * 1e3), "unit": UNIT,
+        rec["e2e"] = {"value": replicas.job_throughput(jobs, steps, e2e_s * 1e3), "unit": UNIT,
                       "h2d_bytes_per_step": h2d / steps, "d2h_bytes_per_step": d2h / steps,
                       "note": "pdadmm_init from host buffers (features and weights page-locked) + K iterations + objective "
                               "and W,b read back; the one-off set-up is spread over only K iterations"}
@@ -326,6 +340,9 @@ def main():
     ap.add_argument("--quant-q", action="store_true",
                     help="pdADMM-G-Q workloads: keep q on the level set as well (variant of Sec. Quantization Extension)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--replicas", action="store_true",
+                    help="several GPUs: one independent copy of the workload per GPU instead of one problem with its nodes "
+                         "divided among the GPUs")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -334,7 +351,10 @@ def main():
     rank, world, local_rank = replicas.env_rank_world()
     head = args.workload if args.workload in ALL else HEADLINE
     w = synth.get(head)
-    config = {"workload": describe(w, args.quant_q), "replicas": args.gpus,
+    sharded_run = args.gpus > 1 and not args.replicas
+    config = {"workload": describe(w, args.quant_q),
+              "parallelism": (f"nodes divided among {args.gpus} GPUs, W and b replicated, sums over nodes by NCCL all-reduce"
+                              if sharded_run else f"{args.gpus} independent replica(s)"),
               "l2": "state (about %.1f GB per replica) is far larger than the 126 MB L2" %
                     (5 * 4e-9 * w.n_nodes * w.hidden * w.n_layers)}
 
@@ -373,7 +393,7 @@ def main():
     with_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     t_start = time.perf_counter()
     rec = run_workload(head, min(args.steps, STEP_CAP.get(head, args.steps)), args.warmup, flags, device, world, dist,
-                       args.simt, with_cpu)
+                       args.simt, with_cpu, shard_nodes=sharded_run)
     workloads = {head: rec}
     if args.workload in (None, "all") and world == 1:
         # the metric is quoted per workload: the other four, each with its own clocks, roofline, end-to-end leg and oracle sample
@@ -389,7 +409,8 @@ def main():
 
     if rank == 0:
         line = {"metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": world, "steps": rec["steps"],
-                "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True,
+                "scaling": "strong" if sharded_run else "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
                 "clocks": rec["clocks"], "e2e": rec.get("e2e"), "gpu_launches": rec["gpu_launches"], "roofline": rec["roofline"],
                 "cpu_baseline": rec.get("cpu_baseline"), "t_roof_ms": rec["t_roof_ms"], "frac_t_roof": rec["frac_t_roof"],

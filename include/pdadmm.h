@@ -115,6 +115,40 @@ typedef struct {
 int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out);
 
 /*
+ * Node sharding (multi-GPU): after the augmentation every update of Algorithm 1 acts on one node's column at a time,
+ * except for sums over nodes inside tau (Eq. "update p"), theta and nabla_W phi (Eq. "update W"), nabla_b phi (Eq.
+ * "update b") and the acceptance test of Eq. "update p quantized".  A context may therefore own the nodes
+ * [node_begin, node_begin + node_count) only -- p, z, q, u of those nodes, and full copies of W and b -- and hand every
+ * such sum to the caller, who adds it over the contexts of all shards (one per GPU).  The paper distributes layers
+ * over clients instead (Sec. "The pdADMM-G Algorithm"); sharding by nodes exchanges O(L h^2) bytes per iteration
+ * instead of O(|V| h).
+ *
+ * pdadmm_allreduce_fn: reduce `count` elements (dtype 0: float, 1: double) at the DEVICE pointer `buf`, in place,
+ * over all shards with op 0 (sum) or 1 (max), ordered after the work already queued on `stream` (a cudaStream_t of
+ * the context) and before work queued on it later; return 0, anything else aborts the call with PDADMM_ECUDA.  The
+ * buffer belongs to the context and lies in its own GPU's memory.  Every shard's context issues the same sequence of
+ * calls, so a collective library can be called directly.  `user` is passed through.
+ *
+ * pdadmm_init_sharded: like pdadmm_init; cfg describes the WHOLE graph (all nodes, features, labels, mask: the graph
+ * operator needs the neighbours of the shard's nodes) and the context keeps the shard.  Every shard must pass the same
+ * cfg and init_W.  shard == NULL, or a null allreduce with the full node range, is pdadmm_init.  In a sharded context
+ * tensors of node-sized kinds (X, P, Z, Q, U, CODES) are the shard's rows; pdadmm_objective and pdadmm_residuals
+ * return the totals over all shards (they reduce, so all shards must call them together); pdadmm_predict counts the
+ * shard's nodes.
+ */
+typedef int (*pdadmm_allreduce_fn)(void *user, void *buf, size_t count, int dtype, int op, void *stream);
+typedef struct {
+  int64_t node_begin;            /* first node of the shard                              */
+  int64_t node_count;            /* >= 1, node_begin + node_count <= cfg->n_nodes       */
+  pdadmm_allreduce_fn allreduce; /* adds over all shards; required unless the shard is the whole graph */
+  void *user;
+} pdadmm_shard;
+int pdadmm_init_sharded(const pdadmm_config *cfg, const pdadmm_shard *shard, pdadmm_ctx **out);
+
+/* Bytes handed to the reduction callback by pdadmm_step so far (the volume entering the all-reduces). */
+int pdadmm_comm_bytes(pdadmm_ctx *ctx, int64_t *bytes);
+
+/*
  * pdadmm_step -- run n_iters iterations of Algorithm 1: for every layer the p-update (Eq. "update
  * p"; pdADMM-G-Q: Eq. "update p quantized"), W-update (Eq. "update W"), b-update (Eq. "update b"),
  * z-update (Eq. "update z" with the ReLU closed form, Eq. "update zl" for the last layer), q-update

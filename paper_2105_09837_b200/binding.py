@@ -27,7 +27,7 @@ FLAG_LEAST_SQUARES = 16
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 
 EXPORTS = [
-    "pdadmm_init", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
+    "pdadmm_init", "pdadmm_init_sharded", "pdadmm_comm_bytes", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
     "pdadmm_set_tensor", "pdadmm_predict", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_selftest_bounded_wait",
     "pdadmm_profile", "pdadmm_profile_classes",
     "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_time_augmentation", "pdadmm_destroy", "pdadmm_last_error",
@@ -55,6 +55,13 @@ class _Config(C.Structure):
     ]
 
 
+ALLREDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_void_p)
+
+
+class _Shard(C.Structure):
+    _fields_ = [("node_begin", C.c_int64), ("node_count", C.c_int64), ("allreduce", ALLREDUCE_FN), ("user", C.c_void_p)]
+
+
 def lib() -> C.CDLL:
     """Load the shared library (once)."""
     global _lib
@@ -65,6 +72,8 @@ def lib() -> C.CDLL:
         L.pdadmm_last_error.restype = C.c_char_p
         L.pdadmm_profile_name.restype = C.c_char_p
         L.pdadmm_init.argtypes = [C.POINTER(_Config), C.POINTER(C.c_void_p)]
+        L.pdadmm_init_sharded.argtypes = [C.POINTER(_Config), C.POINTER(_Shard), C.POINTER(C.c_void_p)]
+        L.pdadmm_comm_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         L.pdadmm_step.argtypes = [C.c_void_p, C.c_int]
         L.pdadmm_last_step_ms.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
         L.pdadmm_objective.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
@@ -106,7 +115,9 @@ class Context:
     def __init__(self, n_nodes: int, edge_src, edge_dst, features, n_hops: int, n_classes: int, labels, train_mask,
                  layer_widths: Sequence[int], rho: float, nu: float, quant_levels: int, init_W: List[np.ndarray],
                  device: int = 0, flags: int = 0, quant_neg_levels: int = 0, quant_step: float = 0.0,
-                 leaky_slope: float = 0.0):
+                 leaky_slope: float = 0.0, shard=None):
+        """shard: None, or (node_begin, node_count, allreduce) with allreduce an ``ALLREDUCE_FN`` object (kept alive
+        here): the context then owns those nodes only (``pdadmm_init_sharded``)."""
         self._h = C.c_void_p()
         src = np.ascontiguousarray(edge_src, dtype=np.int32)
         dst = np.ascontiguousarray(edge_dst, dtype=np.int32)
@@ -132,10 +143,18 @@ class Context:
                       len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, quant_neg_levels, quant_step, leaky_slope, wp,
                       device, flags)
         self.n_nodes, self.n_layers = int(n_nodes), len(widths)
+        self.n_nodes_total = int(n_nodes)
         self.n0 = (n_hops + 1) * feat.shape[1]
         self.widths = [int(x) for x in widths]
         self.quant_levels = int(quant_levels)
-        _check(lib().pdadmm_init(C.byref(cfg), C.byref(self._h)))
+        if shard is None:
+            _check(lib().pdadmm_init(C.byref(cfg), C.byref(self._h)))
+        else:
+            begin, count, fn = shard
+            self._allreduce = fn                      # the library keeps the pointer: the object must outlive the context
+            sh = _Shard(int(begin), int(count), fn, None)
+            self.n_nodes = int(count)
+            _check(lib().pdadmm_init_sharded(C.byref(cfg), C.byref(sh), C.byref(self._h)))
 
     # ---- same names as the C ABI
     def step(self, n_iters: int = 1):
@@ -189,7 +208,7 @@ class Context:
         if kind == T_TRIALS:
             return (1,), np.int32
         if kind == T_CSR_ROWPTR:
-            return (N + 1,), np.int32
+            return (self.n_nodes_total + 1,), np.int32
         raise ValueError(kind)
 
     def get_tensor(self, kind: int, layer: int = 1) -> np.ndarray:
@@ -226,6 +245,11 @@ class Context:
         _check(lib().pdadmm_time_augmentation(self._h, reps, C.byref(ms), C.byref(by)))
         return ms.value, by.value
 
+    def comm_bytes(self) -> int:
+        n = C.c_int64()
+        _check(lib().pdadmm_comm_bytes(self._h, C.byref(n)))
+        return n.value
+
     def launches(self) -> int:
         n = C.c_int64()
         _check(lib().pdadmm_launches(self._h, C.byref(n)))
@@ -245,13 +269,13 @@ class Context:
 
 def from_inputs(inp, device: int = 0, flags: int = 0, rho: Optional[float] = None, nu: Optional[float] = None,
                 quant_levels: Optional[int] = None, quant_neg_levels: int = 0, quant_step: float = 0.0,
-                leaky_slope: float = 0.0) -> Context:
+                leaky_slope: float = 0.0, shard=None) -> Context:
     """Context for a ``synth.Inputs`` bundle."""
     w = inp.workload
     return Context(w.n_nodes, inp.edge_src, inp.edge_dst, inp.features, w.n_hops, w.n_classes, inp.labels,
                    inp.train_mask, w.widths, w.rho if rho is None else rho, w.nu if nu is None else nu,
                    w.quant_levels if quant_levels is None else quant_levels, inp.init_W, device, flags,
-                   quant_neg_levels, quant_step, leaky_slope)
+                   quant_neg_levels, quant_step, leaky_slope, shard)
 
 
 def quantize(x, scale: float, levels: int, device: int = 0, lo: float = 0.0):

@@ -435,6 +435,40 @@ resid_colsum_kernel(float *__restrict__ r, const float *__restrict__ gp, const L
   }
 }
 
+// out[c] = sum over the blocks' slots of column c (the first half of finalize_bias_kernel, for a context that owns only
+// part of the nodes: the totals are then added over the shards before the mean is taken).  Same thread layout.
+__global__ void __launch_bounds__(256)
+colsum_total_kernel(const double *__restrict__ slots, int n_slots, int ld, double *__restrict__ out) {
+  __shared__ double sh[8][33];
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  double s = 0.0;
+  if (c < ld)
+    for (int i = threadIdx.y; i < n_slots; i += 8) s += slots[(size_t)i * ld + c];
+  sh[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && c < ld) {
+    double t = 0.0;
+    for (int k = 0; k < 8; ++k) t += sh[k][threadIdx.x];
+    out[c] = t;
+  }
+}
+
+// sum of squares (one slot per block) and largest magnitude of a weight-sized matrix
+__global__ void __launch_bounds__(EW_THREADS)
+sumsq_amax_kernel(const float *__restrict__ G, size_t n4, uint32_t *__restrict__ amax, double *__restrict__ slots) {
+  __shared__ double red[EW_THREADS / 32];
+  double ss = 0.0;
+  uint32_t m = 0u;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 a = ld4(G, i);
+    ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
+    m = max(m, abs_bits(a));
+  }
+  if (amax != nullptr) commit_amax(m, amax);
+  const double tot = block_sum<EW_THREADS>(ss, red);
+  if (threadIdx.x == 0) slots[blockIdx.x] = tot;
+}
+
 // b+ = b - mean_j r[j][:]  (Eq. "update b" with the step 1/(nu N), i.e. the exact minimiser);
 // shift[c] = that mean, which the z-update subtracts from r.  blockDim = (32 columns, 8 slot groups): group g adds
 // the slots g, g+8, ... of its column, the 8 group sums are then added in group order.

@@ -107,6 +107,7 @@ struct Scratch {
   float *part = nullptr;    // partial tiles of grad_W
   double *slots = nullptr;  // per-block partial sums
   size_t n_slots = 0;
+  double *red = nullptr;    // sums on their way through the reduction over shards (widest layer + 8 values)
   float *tail_ws = nullptr; // accumulators of the contraction slices of tail tiles (one tile per SM at most)
   int *tail_count = nullptr;
   uint32_t *amax_pool = nullptr;   // words for the largest magnitudes of product operands, handed out in stream order
@@ -128,7 +129,11 @@ struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
 
 struct pdadmm_ctx {
   int device = 0;
-  int64_t N = 0;
+  int64_t N = 0;                   // nodes this context owns
+  int64_t N_total = 0, node_begin = 0;   // the whole graph; first owned node
+  pdadmm_allreduce_fn reduce = nullptr;  // adds over the shards' contexts (null: this context holds every node)
+  void *reduce_user = nullptr;
+  int64_t comm_bytes = 0;
   int L = 0, d = 0, n_blocks = 0, n0 = 0, ld0 = 0, C = 0, levels = 0;
   int code_bytes = 1;              // 1 for up to 256 levels, else 2
   int neg_levels = 0;              // levels below zero
@@ -222,6 +227,21 @@ static int dev_alloc(pdadmm_ctx *c, T **ptr, size_t count, bool zero = true) {
 
 static inline int ew_grid(size_t n_items) {
   return (int)std::max<size_t>(1, std::min<size_t>(ceil_div((int64_t)n_items, EW_THREADS), 148 * 8));
+}
+
+// ---- sums over the shards' contexts ---------------------------------------------------------------------------
+static int shard_sum(pdadmm_ctx *c, cudaStream_t st, void *buf, size_t count, int is_double, int op = 0) {
+  if (c->reduce == nullptr) return PDADMM_OK;
+  c->comm_bytes += (int64_t)(count * (is_double ? 8 : 4));
+  const int rc = c->reduce(c->reduce_user, buf, count, is_double, op, (void *)st);
+  if (rc != 0) return fail(PDADMM_ECUDA, "the reduction callback returned %d", rc);
+  return PDADMM_OK;
+}
+// fixed-order totals of up to two slot arrays into red[0], red[1], then their sum over the shards
+static int shard_sum_slots(pdadmm_ctx *c, cudaStream_t st, double *red, const double *a, int na, const double *b, int nb) {
+  reduce_slots_kernel<<<1, 256, 0, st>>>(a, na, 1, 1, red);
+  if (b != nullptr) reduce_slots_kernel<<<1, 256, 0, st>>>(b, nb, 1, 1, red + 1);
+  return shard_sum(c, st, red, b != nullptr ? 2 : 1, 1);
 }
 
 // ---- profiling hooks ----------------------------------------------------------------------------------
@@ -562,6 +582,13 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
                              epi2, slots_b, &np2, 0, w_g));
   }
+  if (c->reduce != nullptr) {
+    // ||g||^2 and ||W g||^2 are sums over nodes: this shard's totals, added over the shards, then tau
+    PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, np, slots_b, np2));
+    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.red, 1, s.red + 1, 1, c->d_flag + 2,
+                                             ly.amax_p);
+    return PDADMM_OK;
+  }
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
     finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2,
@@ -609,7 +636,10 @@ static int q_trial(pdadmm_ctx *c, int l) {
   EpiStoreSumsq epi{s.s2, ly.ld_out};
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, planes_W(ly), epi,
                            slots_b, &np, 0, w_d));
-  {
+  if (c->reduce != nullptr) {
+    PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, grid, slots_b, np));
+    finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.red, 1, s.red + 1, 1);
+  } else {
     Launch k(c, KC_SMALL, s.st, 8.0 * (grid + np), 0);
     finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
   }
@@ -676,6 +706,12 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
     uint32_t *w = nullptr;
     if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w = amax_take(c); }
     reduce_gradW_kernel<<<gw, EW_THREADS, 0, s.st>>>(s.part, ly.n_split, n4w, c->nu, ly.gradW, w, s.slots);
+    if (c->reduce != nullptr) {
+      // nabla_W phi is a sum over nodes: add the shards' parts, then take the norm and the largest magnitude of the total
+      PD_TRY(shard_sum(c, s.st, ly.gradW, n4w * 4, 0));
+      if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w = amax_take(c); }
+      sumsq_amax_kernel<<<gw, EW_THREADS, 0, s.st>>>(ly.gradW, n4w, w, s.slots);
+    }
     if (c->use_tc) make_planes(c, s.st, ly.gradW, ly.n_out, ly.n_in, ly.ld_in, w, ly.Gp);
   }
   int np = 0;
@@ -684,7 +720,11 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
   const PlaneRef xp = planes_X(ly);
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.ld_in, planes_G(ly),
                            epi, slots_b, &np, 0, ly.amax_p, &xp));
-  {
+  if (c->reduce != nullptr) {
+    // ||G p+||^2 is a sum over nodes (||G||^2 is the same on every shard already)
+    PD_TRY(shard_sum_slots(c, s.st, s.red, slots_b, np, nullptr, 0));
+    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, s.red, 1, c->d_flag + 2, ly.amax_r);
+  } else {
     Launch k(c, KC_SMALL, s.st, 8.0 * (gw + np), 0);
     finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2, ly.amax_r);
   }
@@ -705,7 +745,13 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
     Launch k(c, KC_COLSUM, s.st, 12.0 * N * ly.n_out, 0);
     resid_colsum_kernel<<<used_blocks, EW_THREADS, sh, s.st>>>(ly.r, s.s1, ly.sc, N, ly.ld_out, rows_per_block, s.slots);
   }
-  {
+  if (c->reduce != nullptr) {
+    // the column sums run over all nodes: this shard's sums, added over the shards, then the mean over |V|
+    colsum_total_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, s.red);
+    PD_TRY(shard_sum(c, s.st, s.red, (size_t)ly.ld_out, 1));
+    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.red, 1, ly.ld_out, ly.n_out,
+                                                                                1.0 / (double)c->N_total, ly.b, ly.shift);
+  } else {
     Launch k(c, KC_SMALL, s.st, 8.0 * used_blocks * ly.ld_out, 0);
     finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
                                                                                 1.0 / (double)N, ly.b, ly.shift);
@@ -950,9 +996,15 @@ static int alloc_transposed(pdadmm_ctx *c, Scratch &s, int max_out, int max_in) 
   return PDADMM_OK;
 }
 
-static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
-  const int64_t N = cfg->n_nodes;
-  c->device = cfg->device; c->N = N; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
+static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *shard) {
+  const int64_t Ntot = cfg->n_nodes;
+  const bool sharded = shard != nullptr && shard->allreduce != nullptr;
+  const int64_t N = sharded ? shard->node_count : Ntot;
+  const int64_t node0 = sharded ? shard->node_begin : 0;
+  c->N_total = Ntot; c->node_begin = node0;
+  if (sharded) { c->reduce = shard->allreduce; c->reduce_user = shard->user; }
+  // the graph stage works on all nodes: c->N is the whole graph until X is built
+  c->device = cfg->device; c->N = Ntot; c->L = cfg->n_layers; c->d = cfg->feat_dim; c->n_blocks = cfg->n_hops + 1;
   c->n0 = c->n_blocks * c->d; c->ld0 = round_up(c->n0, LD_ALIGN); c->C = cfg->n_classes; c->levels = cfg->quant_levels;
   c->neg_levels = cfg->quant_neg_levels; c->fixed_step = cfg->quant_step;
   c->code_bytes = cfg->quant_levels > 256 ? 2 : 1;
@@ -972,12 +1024,27 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
 
   // graph: CSR pattern, values and sparse products all on the device
   PD_TRY(build_csr(c, cfg));
-  adjacency_values_kernel<<<(int)ceil_div(N * 32, 256), 256, 0, st>>>(c->row_ptr, c->col_idx, (int)N, c->csr_val);
+  adjacency_values_kernel<<<(int)ceil_div(Ntot * 32, 256), 256, 0, st>>>(c->row_ptr, c->col_idx, (int)Ntot, c->csr_val);
   PD_TRY(dev_alloc(c, &c->labels, (size_t)N, false));
   PD_TRY(dev_alloc(c, &c->mask, (size_t)N, false));
-  PD_CUDA(cudaMemcpyAsync(c->labels, cfg->labels, (size_t)N * 4, cudaMemcpyHostToDevice, st));
-  PD_CUDA(cudaMemcpyAsync(c->mask, cfg->train_mask, (size_t)N, cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaMemcpyAsync(c->labels, cfg->labels + node0, (size_t)N * 4, cudaMemcpyHostToDevice, st));
+  PD_CUDA(cudaMemcpyAsync(c->mask, cfg->train_mask + node0, (size_t)N, cudaMemcpyHostToDevice, st));
   PD_CUDA(cudaStreamSynchronize(st));
+  // X = [H, A~ H, A~^2 H, ...] for all nodes (a shard needs its neighbours' features, and theirs, ...); a shard then
+  // keeps the rows of its own nodes
+  float *x_full = nullptr;
+  void *x_full_alloc = nullptr;
+  if (sharded) {
+    const size_t bytes = (size_t)Ntot * c->ld0 * 4 + 256;
+    if (cudaMalloc(&x_full_alloc, bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(PDADMM_ENOMEM, "cudaMalloc of %zu bytes failed", bytes);
+    }
+    x_full = (float *)x_full_alloc;
+    PD_CUDA(cudaMemsetAsync(x_full, 0, bytes, st));
+  }
+  struct FreeLater { void *p; ~FreeLater() { if (p) cudaFree(p); } } free_x{x_full_alloc};
+  c->N = N;                                  // from here on: the nodes this context owns
 
   // layers
   c->layers.resize(c->L);
@@ -1041,6 +1108,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   s.n_slots = std::max<size_t>((size_t)c->n_sms * 4 * max_out, 8 * (size_t)ceil_div(N, SG_BM) * ceil_div(std::max(max_in, max_out), SG_BN) + 148 * 8 * 4);
   s.n_slots *= 2;                       // two halves: consecutive reductions of one layer use different halves
   PD_TRY(dev_alloc(c, &s.slots, s.n_slots));
+  PD_TRY(dev_alloc(c, &s.red, (size_t)max_out + 8));
   if (c->use_tc) {
     PD_TRY(dev_alloc(c, &s.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
     PD_TRY(dev_alloc(c, &s.tail_count, (size_t)c->n_sms * 8));
@@ -1090,6 +1158,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
     if (c->levels) PD_TRY(alloc_trial_buffers(c, x, (size_t)N * max_in));
     x.n_slots = s.n_slots;
     PD_TRY(dev_alloc(c, &x.slots, x.n_slots));
+    PD_TRY(dev_alloc(c, &x.red, (size_t)max_out + 8));
     if (c->use_tc) {
       PD_TRY(dev_alloc(c, &x.tail_ws, (size_t)c->n_sms * TC_BM * TC_BN, false));
       PD_TRY(dev_alloc(c, &x.tail_count, (size_t)c->n_sms * 8));
@@ -1105,10 +1174,15 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
 
   // X = [H, A~ H, A~^2 H, ...] in the column blocks of p_1
   Layer &l0 = c->layers[0];
-  PD_TRY(upload_rows(st, l0.p, l0.ld_in, cfg->features, c->d, N));
-  for (int k = 1; k < c->n_blocks; ++k)
-    launch_spmm(st, c->row_ptr, c->col_idx, c->csr_val, (int)N, l0.p + (size_t)(k - 1) * c->d, l0.p + (size_t)k * c->d,
-                c->d, l0.ld_in);
+  {
+    float *xb = sharded ? x_full : l0.p;
+    PD_TRY(upload_rows(st, xb, l0.ld_in, cfg->features, c->d, Ntot));
+    for (int k = 1; k < c->n_blocks; ++k)
+      launch_spmm(st, c->row_ptr, c->col_idx, c->csr_val, (int)Ntot, xb + (size_t)(k - 1) * c->d, xb + (size_t)k * c->d,
+                  c->d, l0.ld_in);
+    if (sharded)
+      PD_CUDA(cudaMemcpyAsync(l0.p, x_full + (size_t)node0 * l0.ld_in, (size_t)N * l0.ld_in * 4, cudaMemcpyDeviceToDevice, st));
+  }
 
   // start of Algorithm 1: b = 0, z_l = W_l p_l, q_l = ReLU(z_l), p_{l+1} = q_l (projected in -Q mode), u = 0
   for (int l = 0; l < c->L; ++l) {
@@ -1135,6 +1209,12 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
       PD_CUDA(cudaStreamSynchronize(st));
       float mx = 0.f;
       for (float v : hm) mx = std::max(mx, v);
+      if (c->reduce != nullptr) {            // the level spacing comes from the largest entry over all nodes
+        PD_CUDA(cudaMemcpyAsync(s.red, &mx, 4, cudaMemcpyHostToDevice, st));
+        PD_TRY(shard_sum(c, st, s.red, 1, 0, 1));
+        PD_CUDA(cudaMemcpyAsync(&mx, s.red, 4, cudaMemcpyDeviceToHost, st));
+        PD_CUDA(cudaStreamSynchronize(st));
+      }
       nx.scale = c->fixed_step > 0.f ? c->fixed_step : (mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f);
       nx.lo = -(float)c->neg_levels * nx.scale;
       quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes,
@@ -1152,6 +1232,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg) {
   c->amax_p_valid = true;
   c->xT_valid = false;            // the transposed planes of X are made by the first step
   c->launches = 0;
+  c->comm_bytes = 0;
   return PDADMM_OK;
 }
 
@@ -1187,10 +1268,25 @@ using namespace pd;
 
 extern "C" const char *pdadmm_last_error(void) { return err_text().c_str(); }
 
-extern "C" int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out) {
+extern "C" int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out) { return pdadmm_init_sharded(cfg, nullptr, out); }
+
+extern "C" int pdadmm_comm_bytes(pdadmm_ctx *c, int64_t *bytes) {
+  if (!c || !bytes) return fail(PDADMM_EINVAL, "null argument");
+  *bytes = c->comm_bytes;
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_init_sharded(const pdadmm_config *cfg, const pdadmm_shard *shard, pdadmm_ctx **out) {
   if (!out) return fail(PDADMM_EINVAL, "out is null");
   *out = nullptr;
   PD_TRY(check_config(cfg));
+  if (shard != nullptr) {
+    if (shard->node_begin < 0 || shard->node_count < 1 || shard->node_begin + shard->node_count > cfg->n_nodes)
+      return fail(PDADMM_EINVAL, "shard [%lld, +%lld) is not inside the %lld nodes", (long long)shard->node_begin,
+                  (long long)shard->node_count, (long long)cfg->n_nodes);
+    if (shard->allreduce == nullptr && (shard->node_begin != 0 || shard->node_count != cfg->n_nodes))
+      return fail(PDADMM_EINVAL, "a shard that is not the whole graph needs an allreduce callback");
+  }
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
     cudaGetLastError();
@@ -1201,7 +1297,7 @@ extern "C" int pdadmm_init(const pdadmm_config *cfg, pdadmm_ctx **out) {
   if (!c) return fail(PDADMM_ENOMEM, "out of host memory");
   int rc;
   try {
-    rc = build(c, cfg);
+    rc = build(c, cfg, shard);
   } catch (const std::bad_alloc &) {
     rc = fail(PDADMM_ENOMEM, "out of host memory");
   }
@@ -1268,7 +1364,9 @@ extern "C" int pdadmm_step(pdadmm_ctx *c, int n_iters) {
   // is captured once into a CUDA graph and replayed; pointers and tensor maps never change in that mode.
   // pdADMM-G-Q reads the accept flag of every tau trial on the host, and per-kernel timing needs its events:
   // both stay eager.
-  const bool may_graph = c->levels == 0 && !c->profiling && !c->graph_failed && !(c->flags & PDADMM_FLAG_NO_GRAPH);
+  // A sharded context calls back for its sums over shards in the middle of an iteration: eager as well.
+  const bool may_graph = c->levels == 0 && !c->profiling && !c->graph_failed && !(c->flags & PDADMM_FLAG_NO_GRAPH) &&
+                         c->reduce == nullptr;
   int k = 0;
   if (may_graph && c->iter_graph == nullptr && n_iters > 1) {
     PD_TRY(iterate_once(c, &hit_cap));
@@ -1349,6 +1447,14 @@ extern "C" int pdadmm_objective(pdadmm_ctx *c, double out[6]) {
     PD_TRY(read_slots(c, grid, 1, 1, &R));
   }
   PD_CUDA(cudaGetLastError());
+  if (c->reduce != nullptr) {                 // every component is a sum over nodes
+    double h[5] = {R, lin, act, dual, pen};
+    PD_CUDA(cudaMemcpyAsync(c->scr.red, h, sizeof h, cudaMemcpyHostToDevice, st));
+    PD_TRY(shard_sum(c, st, c->scr.red, 5, 1));
+    PD_CUDA(cudaMemcpyAsync(h, c->scr.red, sizeof h, cudaMemcpyDeviceToHost, st));
+    PD_CUDA(cudaStreamSynchronize(st));
+    R = h[0]; lin = h[1]; act = h[2]; dual = h[3]; pen = h[4];
+  }
   out[0] = R; out[1] = 0.5 * c->nu * lin; out[2] = 0.5 * c->nu * act; out[3] = dual; out[4] = 0.5 * c->rho * pen;
   out[5] = out[0] + out[1] + out[2] + out[3] + out[4];
   return PDADMM_OK;
@@ -1423,6 +1529,13 @@ extern "C" int pdadmm_residuals(pdadmm_ctx *c, double *per_layer_sq, int n) {
     per_layer_sq[l] = h[3];
   }
   PD_CUDA(cudaGetLastError());
+  if (c->reduce != nullptr && n > 0) {
+    if ((size_t)n > 8 + (size_t)c->layers[0].ld_out) return fail(PDADMM_EINVAL, "too many layers for the reduction buffer");
+    PD_CUDA(cudaMemcpyAsync(c->scr.red, per_layer_sq, (size_t)n * 8, cudaMemcpyHostToDevice, c->scr.st));
+    PD_TRY(shard_sum(c, c->scr.st, c->scr.red, (size_t)n, 1));
+    PD_CUDA(cudaMemcpyAsync(per_layer_sq, c->scr.red, (size_t)n * 8, cudaMemcpyDeviceToHost, c->scr.st));
+    PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  }
   return PDADMM_OK;
 }
 
@@ -1452,7 +1565,7 @@ static int locate(pdadmm_ctx *c, int kind, int layer, TensorRef *t) {
     case PDADMM_T_TAU: { PD_TRY(need(2, L)); *t = {&c->layers[layer - 1].sc->tau, 1, 1, 1, 8, false}; return PDADMM_OK; }
     case PDADMM_T_THETA: { PD_TRY(need(1, L)); *t = {&c->layers[layer - 1].sc->theta, 1, 1, 1, 8, false}; return PDADMM_OK; }
     case PDADMM_T_TRIALS: { PD_TRY(need(2, L)); *t = {&c->layers[layer - 1].sc->trials, 1, 1, 1, 4, false}; return PDADMM_OK; }
-    case PDADMM_T_CSR_ROWPTR: *t = {c->row_ptr, 1, N + 1, N + 1, 4, false}; return PDADMM_OK;
+    case PDADMM_T_CSR_ROWPTR: *t = {c->row_ptr, 1, (size_t)c->N_total + 1, (size_t)c->N_total + 1, 4, false}; return PDADMM_OK;
     case PDADMM_T_CSR_COLIDX: *t = {c->col_idx, 1, (size_t)c->nnz, (size_t)c->nnz, 4, false}; return PDADMM_OK;
     case PDADMM_T_CSR_VAL: *t = {c->csr_val, 1, (size_t)c->nnz, (size_t)c->nnz, 4, false}; return PDADMM_OK;
     default: return fail(PDADMM_EINVAL, "unknown tensor kind %d", kind);
@@ -1747,6 +1860,7 @@ extern "C" int pdadmm_profile_read(pdadmm_ctx *c, int k, double *ms, int64_t *la
 extern "C" int pdadmm_time_augmentation(pdadmm_ctx *c, int reps, double *ms_per_hop, double *bytes_per_hop) {
   if (!c || reps < 1 || reps > 1000 || !ms_per_hop) return fail(PDADMM_EINVAL, "bad argument");
   if (c->n_blocks < 2) return fail(PDADMM_EINVAL, "the input has a single block: no sparse product to time");
+  if (c->N != c->N_total) return fail(PDADMM_EINVAL, "a sharded context keeps only its own rows of X");
   PD_CUDA(cudaSetDevice(c->device));
   Layer &l0 = c->layers[0];
   cudaStream_t st = c->scr.st;
