@@ -666,6 +666,65 @@ def lagrangian(s: State, prm: Params) -> float:
 
 
 # ----------------------------------------------------------------------------
+# Greedy layer-wise training: growing a trained shallow model
+# ----------------------------------------------------------------------------
+
+def start_layers_from(s: State, prm: Params, first: int) -> State:
+    """The start of Algorithm 1 for layers first..L (1-based) from the current p_first: b_l = 0, z_l = W_l p_l,
+    q_l = f_l(z_l), p_{l+1} = q_l (pdADMM-G-Q: the nearest level, with the spacing taken from max(q_l) like at the very
+    start), u_l = 0.  Layers below `first` are left as they are."""
+    n = s.copy()
+    L = n.L
+    for l in range(first - 1, L):
+        n.b[l] = np.zeros_like(n.b[l])
+        n.z[l] = n.W[l] @ n.p[l]
+        if l < L - 1:
+            n.q[l] = relu(n.z[l], prm.slope)
+            n.u[l] = np.zeros_like(n.q[l])
+            if prm.quant_levels:
+                n.scale[l + 1] = (float(np.float32(prm.level_step)) if prm.level_step > 0
+                                  else quantization_scale(n.q[l], prm.quant_levels))
+                n.p[l + 1] = nearest_level(n.q[l], n.scale[l + 1], prm.quant_levels, prm.level_lo)[1]
+                if prm.quantize_q:
+                    n.q[l] = n.p[l + 1].copy()
+            else:
+                n.p[l + 1] = n.q[l].copy()
+    return n
+
+
+def grow(s: State, prm: Params, W_new: List[np.ndarray]) -> State:
+    """Greedy layer-wise training (end of Sec. "The pdADMM-G Algorithm"; Sec. "Performance": 2, then 5, then 10
+    layers): a trained model with L layers becomes one with L - 1 + len(W_new) layers.
+
+    The paper says that layers are added and trained, not how they start.  Reading: the hidden layers 1..L-1 keep
+    everything they have (p_l, W_l, b_l, z_l, q_l, u_l, the level spacing of p_l); the old output layer, whose width
+    is the number of classes, cannot serve as a hidden layer and is dropped; the layers L.., the last of which is the
+    new output layer, take the weights `W_new` (drawn by the caller like the initial ones) and start from the forward
+    pass of the model trained so far, i.e. the start of Algorithm 1 from the kept p_L (``start_layers_from``): the
+    constraints p_{l+1} = q_l hold for them and their duals are zero.
+    """
+    L_old = s.L
+    keep = L_old - 1
+    L_new = keep + len(W_new)
+    W = [w.copy() for w in s.W[:keep]] + [np.asarray(w, dtype=np.float64).copy() for w in W_new]
+    n_nodes = s.p[0].shape[1]
+    b = [x.copy() for x in s.b[:keep]] + [np.zeros(w.shape[0]) for w in W_new]
+    p = [x.copy() for x in s.p[:keep + 1]] + [None] * (L_new - keep - 1)
+    z = [x.copy() for x in s.z[:keep]] + [None] * (L_new - keep)
+    q = [x.copy() for x in s.q[:keep]] + [None] * (L_new - 1 - keep)
+    u = [x.copy() for x in s.u[:keep]] + [None] * (L_new - 1 - keep)
+    for l in range(keep, L_new):           # placeholders of the right shape; start_layers_from fills them
+        z[l] = np.zeros((W[l].shape[0], n_nodes))
+        if l < L_new - 1:
+            q[l - 0] = np.zeros((W[l].shape[0], n_nodes))
+            u[l - 0] = np.zeros((W[l].shape[0], n_nodes))
+            p[l + 1] = np.zeros((W[l].shape[0], n_nodes))
+    scale = list(s.scale[:keep + 1]) + [1.0] * (L_new - keep - 1)
+    grown = State(p, W, b, z, q, u, s.y.copy(), s.mask.copy(), scale, [0.0] * L_new, [0.0] * L_new, [0] * L_new)
+    return start_layers_from(grown, prm, keep + 1)
+
+
+# ----------------------------------------------------------------------------
 # The same iteration on node shards
 # ----------------------------------------------------------------------------
 
