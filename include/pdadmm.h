@@ -204,6 +204,16 @@ int pdadmm_get_tensor(pdadmm_ctx *ctx, int kind, int layer, void *host_dst, size
 int pdadmm_set_tensor(pdadmm_ctx *ctx, int kind, int layer, const void *host_src, size_t bytes);
 
 /*
+ * pdadmm_start_layers_from -- the start of Algorithm 1 for layers first_layer..L from the current p_{first_layer}:
+ * b_l = 0, z_l = W_l p_l, q_l = f_l(z_l), p_{l+1} = q_l (pdADMM-G-Q: its nearest level, the spacing taken from max(q_l)),
+ * u_l = 0; the layers below keep their state.  It is the building block of the greedy layer-wise strategy (paper, end
+ * of Section "The pdADMM-G Algorithm"; "Performance": two layers first, then five, then all ten): a deeper context is
+ * created, the trained layers' tensors are copied in with pdadmm_set_tensor, and the added layers are started here from
+ * the forward pass of the model trained so far.  first_layer = 1 restores the initial state for the current W.
+ */
+int pdadmm_start_layers_from(pdadmm_ctx *ctx, int first_layer);
+
+/*
  * pdadmm_quantize -- the projection used by Eq. "update p quantized" on its own: for n host floats x,
  * code = clamp(floor((x - lo)/scale + 1/2), 0, levels-1) as uint8 and p = lo + code * scale (one rounded
  * single-precision multiply, one rounded add), computed by the same device function as inside

@@ -27,7 +27,7 @@ FLAG_LEAST_SQUARES = 16
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 
 EXPORTS = [
-    "pdadmm_init", "pdadmm_init_sharded", "pdadmm_comm_bytes", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
+    "pdadmm_init", "pdadmm_init_sharded", "pdadmm_comm_bytes", "pdadmm_start_layers_from", "pdadmm_step", "pdadmm_last_step_ms", "pdadmm_objective", "pdadmm_residuals", "pdadmm_get_tensor",
     "pdadmm_set_tensor", "pdadmm_predict", "pdadmm_quantize", "pdadmm_spmm", "pdadmm_matmul", "pdadmm_matmul_tn_static", "pdadmm_selftest_bounded_wait",
     "pdadmm_profile", "pdadmm_profile_classes",
     "pdadmm_profile_name", "pdadmm_profile_read", "pdadmm_launches", "pdadmm_time_augmentation", "pdadmm_destroy", "pdadmm_last_error",
@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         L.pdadmm_init.argtypes = [C.POINTER(_Config), C.POINTER(C.c_void_p)]
         L.pdadmm_init_sharded.argtypes = [C.POINTER(_Config), C.POINTER(_Shard), C.POINTER(C.c_void_p)]
         L.pdadmm_comm_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        L.pdadmm_start_layers_from.argtypes = [C.c_void_p, C.c_int]
         L.pdadmm_step.argtypes = [C.c_void_p, C.c_int]
         L.pdadmm_last_step_ms.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
         L.pdadmm_objective.argtypes = [C.c_void_p, C.POINTER(C.c_double)]
@@ -159,6 +160,9 @@ class Context:
     # ---- same names as the C ABI
     def step(self, n_iters: int = 1):
         _check(lib().pdadmm_step(self._h, int(n_iters)))
+
+    def start_layers_from(self, first_layer: int):
+        _check(lib().pdadmm_start_layers_from(self._h, int(first_layer)))
 
     def last_step_ms(self) -> float:
         ms = C.c_double()

@@ -996,6 +996,61 @@ static int alloc_transposed(pdadmm_ctx *c, Scratch &s, int max_out, int max_in) 
   return PDADMM_OK;
 }
 
+// Start of Algorithm 1 for layers first..L-1 (0-based) from the current p_first: b = 0, z_l = W_l p_l, q_l = f(z_l),
+// p_{l+1} = q_l (projected in -Q mode, with the level spacing from max(q_l)), u = 0, r = 0.
+static int feasible_start(pdadmm_ctx *c, int first) {
+  const int64_t N = c->N;
+  cudaStream_t st = c->scr.st;
+  Scratch &s = c->scr;
+  for (int l = first; l < c->L; ++l) {
+    Layer &ly = c->layers[l];
+    EpiStore epi{ly.z, ly.ld_out};
+    PD_TRY(split_planes(c, st, ly.W, ly.n_out, ly.n_in, ly.ld_in, ly.Wp));
+    PD_CUDA(cudaMemsetAsync(ly.amax_p, 0, sizeof(uint32_t), st));
+    absmax_kernel<<<ew_grid((size_t)N * ly.ld_in / 4), EW_THREADS, 0, st>>>(ly.p, (size_t)N * ly.ld_in / 4, ly.amax_p);
+    if (l == 0 && ly.x_hi != nullptr) {
+      const size_t n8 = (size_t)N * ly.ld_in / 8;
+      rows_planes_kernel<<<ew_grid(n8), 256, 0, st>>>(ly.p, n8, ly.amax_p, ly.x_exp, ly.x_hi, ly.x_lo);
+    }
+    const PlaneRef xp = planes_X(ly);
+    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
+                             epi, nullptr, nullptr, 0, ly.amax_p, &xp));
+    PD_CUDA(cudaMemsetAsync(ly.b, 0, (size_t)ly.ld_out * 4, st));
+    PD_CUDA(cudaMemsetAsync(ly.shift, 0, (size_t)ly.ld_out * 4, st));
+    PD_CUDA(cudaMemsetAsync(ly.r, 0, (size_t)N * ly.ld_out * 4, st));
+    PD_CUDA(cudaMemsetAsync(ly.amax_r, 0, sizeof(uint32_t), st));
+    if (l + 1 == c->L) break;
+    PD_CUDA(cudaMemsetAsync(ly.u, 0, (size_t)N * ly.ld_out * 4, st));
+    Layer &nx = c->layers[l + 1];
+    const size_t n4 = (size_t)N * ly.ld_out / 4;
+    const int grid = ew_grid(n4);
+    float *bm = reinterpret_cast<float *>(s.slots);
+    relu_max_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, ly.q, n4, c->slope, bm);
+    if (c->levels) {
+      std::vector<float> hm(grid);
+      PD_CUDA(cudaMemcpyAsync(hm.data(), bm, grid * sizeof(float), cudaMemcpyDeviceToHost, st));
+      PD_CUDA(cudaStreamSynchronize(st));
+      float mx = 0.f;
+      for (float v : hm) mx = std::max(mx, v);
+      if (c->reduce != nullptr) {            // the level spacing comes from the largest entry over all nodes
+        PD_CUDA(cudaMemcpyAsync(s.red, &mx, 4, cudaMemcpyHostToDevice, st));
+        PD_TRY(shard_sum(c, st, s.red, 1, 0, 1));
+        PD_CUDA(cudaMemcpyAsync(&mx, s.red, 4, cudaMemcpyDeviceToHost, st));
+        PD_CUDA(cudaStreamSynchronize(st));
+      }
+      nx.scale = c->fixed_step > 0.f ? c->fixed_step : (mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f);
+      nx.lo = -(float)c->neg_levels * nx.scale;
+      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes,
+                                                              c->code_bytes == 2);
+      if (c->quant_q)      // start inside the level set: q_l = p_{l+1}
+        PD_CUDA(cudaMemcpyAsync(ly.q, nx.p, n4 * 16, cudaMemcpyDeviceToDevice, st));
+    } else {
+      PD_CUDA(cudaMemcpyAsync(nx.p, ly.q, n4 * 16, cudaMemcpyDeviceToDevice, st));
+    }
+  }
+  return PDADMM_OK;
+}
+
 static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *shard) {
   const int64_t Ntot = cfg->n_nodes;
   const bool sharded = shard != nullptr && shard->allreduce != nullptr;
@@ -1184,47 +1239,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
       PD_CUDA(cudaMemcpyAsync(l0.p, x_full + (size_t)node0 * l0.ld_in, (size_t)N * l0.ld_in * 4, cudaMemcpyDeviceToDevice, st));
   }
 
-  // start of Algorithm 1: b = 0, z_l = W_l p_l, q_l = ReLU(z_l), p_{l+1} = q_l (projected in -Q mode), u = 0
-  for (int l = 0; l < c->L; ++l) {
-    Layer &ly = c->layers[l];
-    EpiStore epi{ly.z, ly.ld_out};
-    PD_TRY(split_planes(c, st, ly.W, ly.n_out, ly.n_in, ly.ld_in, ly.Wp));
-    absmax_kernel<<<ew_grid((size_t)N * ly.ld_in / 4), EW_THREADS, 0, st>>>(ly.p, (size_t)N * ly.ld_in / 4, ly.amax_p);
-    if (l == 0 && ly.x_hi != nullptr) {
-      const size_t n8 = (size_t)N * ly.ld_in / 8;
-      rows_planes_kernel<<<ew_grid(n8), 256, 0, st>>>(ly.p, n8, ly.amax_p, ly.x_exp, ly.x_hi, ly.x_lo);
-    }
-    const PlaneRef xp = planes_X(ly);
-    PD_TRY(gemm_nodes<false>(c, KC_GEMM_RESID, st, (int)N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
-                             epi, nullptr, nullptr, 0, ly.amax_p, &xp));
-    if (l + 1 == c->L) break;
-    Layer &nx = c->layers[l + 1];
-    const size_t n4 = (size_t)N * ly.ld_out / 4;
-    const int grid = ew_grid(n4);
-    float *bm = reinterpret_cast<float *>(s.slots);
-    relu_max_kernel<<<grid, EW_THREADS, 0, st>>>(ly.z, ly.q, n4, c->slope, bm);
-    if (c->levels) {
-      std::vector<float> hm(grid);
-      PD_CUDA(cudaMemcpyAsync(hm.data(), bm, grid * sizeof(float), cudaMemcpyDeviceToHost, st));
-      PD_CUDA(cudaStreamSynchronize(st));
-      float mx = 0.f;
-      for (float v : hm) mx = std::max(mx, v);
-      if (c->reduce != nullptr) {            // the level spacing comes from the largest entry over all nodes
-        PD_CUDA(cudaMemcpyAsync(s.red, &mx, 4, cudaMemcpyHostToDevice, st));
-        PD_TRY(shard_sum(c, st, s.red, 1, 0, 1));
-        PD_CUDA(cudaMemcpyAsync(&mx, s.red, 4, cudaMemcpyDeviceToHost, st));
-        PD_CUDA(cudaStreamSynchronize(st));
-      }
-      nx.scale = c->fixed_step > 0.f ? c->fixed_step : (mx > 0.f ? mx / (float)(c->levels - 1) : 1.0f);
-      nx.lo = -(float)c->neg_levels * nx.scale;
-      quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes,
-                                                              c->code_bytes == 2);
-      if (c->quant_q)      // start inside the level set: q_l = p_{l+1}
-        PD_CUDA(cudaMemcpyAsync(ly.q, nx.p, n4 * 16, cudaMemcpyDeviceToDevice, st));
-    } else {
-      PD_CUDA(cudaMemcpyAsync(nx.p, ly.q, n4 * 16, cudaMemcpyDeviceToDevice, st));
-    }
-  }
+  PD_TRY(feasible_start(c, 0));
   PD_CUDA(cudaStreamSynchronize(st));
   PD_CUDA(cudaGetLastError());
   c->r_valid = true;                        // z = W p + b exactly by construction, r = 0 (allocated as zero)
@@ -1303,6 +1318,19 @@ extern "C" int pdadmm_init_sharded(const pdadmm_config *cfg, const pdadmm_shard 
   }
   if (rc != PDADMM_OK) { destroy(c); return rc; }
   *out = c;
+  return PDADMM_OK;
+}
+
+extern "C" int pdadmm_start_layers_from(pdadmm_ctx *c, int first_layer) {
+  if (!c) return fail(PDADMM_EINVAL, "context is null");
+  if (first_layer < 1 || first_layer > c->L) return fail(PDADMM_EINVAL, "first_layer must be in [1, %d]", c->L);
+  PD_CUDA(cudaSetDevice(c->device));
+  PD_TRY(feasible_start(c, first_layer - 1));
+  PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  PD_CUDA(cudaGetLastError());
+  // the linear residual of the restarted layers is zero by construction; everything derived from the other tensors
+  // (the residual of the kept layers, t, planes, largest magnitudes) is rebuilt by the next call that needs it
+  c->r_valid = false; c->t_valid = false; c->w_planes_valid = false; c->amax_p_valid = false;
   return PDADMM_OK;
 }
 
