@@ -81,6 +81,17 @@ class Params:
     level_step: float = 0.0               # > 0: the same fixed step for every layer; 0: step from max(p) at the start
     slope: float = 0.0                    # 0: f_l = ReLU; in (0, 1): leaky ReLU with that slope for x <= 0
     risk: str = "ce"                      # R: "ce" cross-entropy (the paper's experiments), "ls" least squares
+    activation: str = "relu"              # f_l: "relu" (with `slope`: leaky), or the smooth "tanh" / "sigmoid", whose
+    table_lo: float = -4.0                #   z-update searches a lookup table of table_size equally spaced candidates
+    table_hi: float = 4.0                 #   on [table_lo, table_hi] (remark after Eq. "update z")
+    table_size: int = 257
+
+    @property
+    def f(self):
+        """What the functions below take as their `slope` argument: the leaky slope, or the smooth activation itself."""
+        if self.activation == "relu":
+            return self.slope
+        return {"tanh": np.tanh, "sigmoid": lambda x: 1.0 / (1.0 + np.exp(-x))}[self.activation]
 
 
 @dataclasses.dataclass
@@ -106,9 +117,12 @@ class State:
         return copy.deepcopy(self)
 
 
-def relu(x, slope: float = 0.0):
+def relu(x, slope=0.0):
     """f_l: ReLU, or, with 0 < slope < 1, the leaky ReLU f(x) = x (x > 0), slope x (x <= 0), which the paper
-    names beside ReLU as an activation its assumptions cover (Sec. "Convergence Analysis")."""
+    names beside ReLU as an activation its assumptions cover (Sec. "Convergence Analysis").  A callable in place of
+    the slope is a smooth activation (tanh, sigmoid: ``Params.f``) and is simply applied."""
+    if callable(slope):
+        return slope(x)
     return np.maximum(x, 0.0) if slope == 0.0 else np.where(x > 0, x, slope * x)
 
 
@@ -372,6 +386,28 @@ def update_z_hidden(a, q, z_old, slope: float = 0.0):
     return np.where(f_pos < f_neg, z_pos, z_neg)
 
 
+def table_points(lo: float, hi: float, size: int) -> np.ndarray:
+    """The candidates of the lookup table: z_i = fl32(lo + fl32(i h)), h = fl32((hi - lo) / (size - 1)), i = 0..size-1
+    (single-precision numbers, so that a z taken from the table is exactly representable in the fp32 state)."""
+    h = np.float32((np.float32(hi) - np.float32(lo)) / np.float32(size - 1))
+    return (np.float32(lo) + np.arange(size, dtype=np.float32) * h).astype(np.float64)
+
+
+def update_z_hidden_table(a, q, z_old, f, points):
+    """Eq. (update z) for a smooth activation f (tanh, sigmoid), for which the paper recommends a lookup table (remark
+    after Eq. "update z") instead of a closed form: the minimiser of (z - a)^2 + (q - f(z))^2 + (z - z^k)^2 over the
+    table's candidate values, element by element; the first candidate wins a tie.  The result is the best point of the
+    table, within half a table step of a minimiser of the continuous problem in objective value (second order)."""
+    best = np.full(np.shape(a), np.inf)
+    arg = np.zeros(np.shape(a))
+    for zi in points:
+        h = (zi - a) ** 2 + (q - f(zi)) ** 2 + (zi - z_old) ** 2
+        take = h < best
+        best = np.where(take, h, best)
+        arg = np.where(take, zi, arg)
+    return arg
+
+
 def cross_entropy(z_col, y: int) -> float:
     """CE(z; y) = -z_y + log sum_c exp(z_c) for one node."""
     m = np.max(z_col)
@@ -548,12 +584,12 @@ def update_z_last(a, y, mask, nu):
 # q-update (Eq. update q), dual update (Eq. update u)
 # ----------------------------------------------------------------------------
 
-def update_q(p_next, u, z, rho, nu, slope: float = 0.0):
+def update_q(p_next, u, z, rho, nu, slope=0.0):
     """q_l^{k+1} = (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)."""
     return (rho * p_next + u + nu * relu(z, slope)) / (rho + nu)
 
 
-def update_q_quantized(p_next, u, z, rho, nu, scale, m, lo=0.0, slope: float = 0.0):
+def update_q_quantized(p_next, u, z, rho, nu, scale, m, lo=0.0, slope=0.0):
     """The variant with q_l in Delta as well: q_l^{k+1} = argmin_{delta in Delta}
     ||delta - (rho p_{l+1}^{k+1} + u_l^k + nu f_l(z_l^{k+1})) / (rho + nu)||, element by element
     (Sec. "Quantization Extension", last paragraph).  Delta is the level set of p_{l+1}, which q_l has to equal."""
@@ -587,7 +623,7 @@ def init_state(X, W0, y, mask, prm: Params) -> State:
     for l in range(L):
         z.append(W[l] @ p[l])
         if l < L - 1:
-            q.append(relu(z[l], prm.slope))
+            q.append(relu(z[l], prm.f))
             u.append(np.zeros_like(q[l]))
             if prm.quant_levels:
                 scale[l + 1] = (float(np.float32(prm.level_step)) if prm.level_step > 0
@@ -599,6 +635,13 @@ def init_state(X, W0, y, mask, prm: Params) -> State:
                 p.append(q[l].copy())
     return State(p, W, b, z, q, u, np.asarray(y), np.asarray(mask, dtype=bool), scale,
                  [0.0] * L, [0.0] * L, [0] * L)
+
+
+def _update_z_hidden_for(prm: Params, a, q, z_old):
+    """The z-update of a hidden layer for the activation in `prm`: closed form for (leaky) ReLU, table search else."""
+    if prm.activation == "relu":
+        return update_z_hidden(a, q, z_old, prm.slope)
+    return update_z_hidden_table(a, q, z_old, prm.f, table_points(prm.table_lo, prm.table_hi, prm.table_size))
 
 
 def iterate(s: State, prm: Params) -> State:
@@ -626,7 +669,7 @@ def iterate(s: State, prm: Params) -> State:
     for l in range(L):
         a = n.W[l] @ n.p[l] + n.b[l][:, None]
         if l < L - 1:
-            n.z[l] = update_z_hidden(a, s.q[l], s.z[l], prm.slope)
+            n.z[l] = _update_z_hidden_for(prm, a, s.q[l], s.z[l])
         elif prm.risk == "ls":
             n.z[l] = update_z_last_least_squares(a, s.y, s.mask, nu)
         else:
@@ -635,9 +678,9 @@ def iterate(s: State, prm: Params) -> State:
     for l in range(L - 1):
         if prm.quant_levels and prm.quantize_q:
             n.q[l] = update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels,
-                                        prm.level_lo, prm.slope)
+                                        prm.level_lo, prm.f)
         else:
-            n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.slope)
+            n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.f)
     for l in range(L - 1):
         n.u[l] = update_u(s.u[l], n.p[l + 1], n.q[l], rho)
     return n
@@ -654,7 +697,7 @@ def objective(s: State, prm: Params) -> np.ndarray:
     rho, nu, L = prm.rho, prm.nu, s.L
     R = risk_least_squares(s.z[L - 1], s.y, s.mask) if prm.risk == "ls" else risk(s.z[L - 1], s.y, s.mask)
     lin = sum(float(np.sum((s.z[l] - s.W[l] @ s.p[l] - s.b[l][:, None]) ** 2)) for l in range(L))
-    act = sum(float(np.sum((s.q[l] - relu(s.z[l], prm.slope)) ** 2)) for l in range(L - 1))
+    act = sum(float(np.sum((s.q[l] - relu(s.z[l], prm.f)) ** 2)) for l in range(L - 1))
     dual = sum(float(np.sum(s.u[l] * (s.p[l + 1] - s.q[l]))) for l in range(L - 1))
     pen = float(np.sum(residuals_sq(s)))
     comps = [R, 0.5 * nu * lin, 0.5 * nu * act, dual, 0.5 * rho * pen]
@@ -679,7 +722,7 @@ def start_layers_from(s: State, prm: Params, first: int) -> State:
         n.b[l] = np.zeros_like(n.b[l])
         n.z[l] = n.W[l] @ n.p[l]
         if l < L - 1:
-            n.q[l] = relu(n.z[l], prm.slope)
+            n.q[l] = relu(n.z[l], prm.f)
             n.u[l] = np.zeros_like(n.q[l])
             if prm.quant_levels:
                 n.scale[l + 1] = (float(np.float32(prm.level_step)) if prm.level_step > 0
@@ -824,7 +867,7 @@ def iterate_sharded(shards: List[State], prm: Params, allreduce=None) -> List[St
         for l in range(L):
             a = n.W[l] @ n.p[l] + n.b[l][:, None]
             if l < L - 1:
-                n.z[l] = update_z_hidden(a, s.q[l], s.z[l], prm.slope)
+                n.z[l] = _update_z_hidden_for(prm, a, s.q[l], s.z[l])
             elif prm.risk == "ls":
                 n.z[l] = update_z_last_least_squares(a, s.y, s.mask, nu)
             else:
@@ -832,9 +875,9 @@ def iterate_sharded(shards: List[State], prm: Params, allreduce=None) -> List[St
         for l in range(L - 1):
             if prm.quant_levels and prm.quantize_q:
                 n.q[l] = update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels,
-                                            prm.level_lo, prm.slope)
+                                            prm.level_lo, prm.f)
             else:
-                n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.slope)
+                n.q[l] = update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.f)
         for l in range(L - 1):
             n.u[l] = update_u(s.u[l], n.p[l + 1], n.q[l], rho)
     return new
@@ -851,7 +894,7 @@ def objective_sharded(shards: List[State], prm: Params, allreduce=None) -> np.nd
 # The trained model: forward pass, prediction, accuracy
 # ----------------------------------------------------------------------------
 
-def forward(X, W, b, slope: float = 0.0) -> np.ndarray:
+def forward(X, W, b, slope=0.0) -> np.ndarray:
     """z_L of the GA-MLP of Problem 1 with the constraints enforced: p_1 = X,
     z_l = W_l p_l + b_l, p_{l+1} = f_l(z_l) = relu(z_l) (l < L).  Returns z_L (n_L x |V|)."""
     p = np.asarray(X, dtype=np.float64)
@@ -861,7 +904,7 @@ def forward(X, W, b, slope: float = 0.0) -> np.ndarray:
     return z
 
 
-def predict(X, W, b, slope: float = 0.0) -> np.ndarray:
+def predict(X, W, b, slope=0.0) -> np.ndarray:
     """Class of every node: the largest entry of z_L (the class the cross-entropy risk R(z_L; y) rewards);
     the first one if several are equal."""
     return np.argmax(forward(X, W, b, slope), axis=0)
