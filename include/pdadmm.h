@@ -97,6 +97,13 @@ typedef struct {
   float quant_step;              /* > 0: the same level spacing s for every layer; 0: s_l = max(p_l^0)/(m-1)  */
   float leaky_slope;             /* f_l of the hidden layers: 0 = ReLU; in (0, 1) = leaky ReLU, f(x) = slope x
                                     for x <= 0 (paper, "Convergence Analysis": both satisfy its assumptions) */
+  int32_t activation;            /* f_l of the hidden layers: 0 = ReLU / leaky ReLU (leaky_slope); 1 = tanh; 2 = logistic
+                                    sigmoid.  The smooth ones have no closed-form z-update: following the paper's remark
+                                    after Eq. "update z" it is taken from a lookup table, the best of table_size candidates
+                                    z_i = table_lo + i (table_hi - table_lo)/(table_size - 1) (single precision), i.e. z is
+                                    resolved to the table step                                            */
+  int32_t table_size;            /* 2..4096 candidates (activation 1, 2 only)                              */
+  float table_lo, table_hi;      /* range of the candidates: should cover the values z takes              */
   const float *const *init_W;    /* [L] pointers: W_l^0 as [n_l][n_{l-1}] (required; the caller draws them) */
   int32_t device;                /* CUDA device ordinal                                                 */
   uint32_t flags;                /* PDADMM_FLAG_*                                                       */

@@ -23,6 +23,7 @@ FLAG_QUANT_Q = 2
 FLAG_NO_GRAPH = 4
 FLAG_ONE_LANE = 8
 FLAG_LEAST_SQUARES = 16
+ACT_RELU, ACT_TANH, ACT_SIGMOID = 0, 1, 2
 
 OK, EINVAL, ENOMEM, ECUDA, ETIMEOUT, ENUMERIC, ENOTCONV = 0, -1, -2, -3, -4, -5, -6
 
@@ -50,6 +51,7 @@ class _Config(C.Structure):
         ("n_layers", C.c_int32), ("layer_widths", C.POINTER(C.c_int32)),
         ("rho", C.c_float), ("nu", C.c_float), ("quant_levels", C.c_int32),
         ("quant_neg_levels", C.c_int32), ("quant_step", C.c_float), ("leaky_slope", C.c_float),
+        ("activation", C.c_int32), ("table_size", C.c_int32), ("table_lo", C.c_float), ("table_hi", C.c_float),
         ("init_W", C.POINTER(C.POINTER(C.c_float))),
         ("device", C.c_int32), ("flags", C.c_uint32),
     ]
@@ -116,7 +118,7 @@ class Context:
     def __init__(self, n_nodes: int, edge_src, edge_dst, features, n_hops: int, n_classes: int, labels, train_mask,
                  layer_widths: Sequence[int], rho: float, nu: float, quant_levels: int, init_W: List[np.ndarray],
                  device: int = 0, flags: int = 0, quant_neg_levels: int = 0, quant_step: float = 0.0,
-                 leaky_slope: float = 0.0, shard=None):
+                 leaky_slope: float = 0.0, shard=None, activation: int = 0, table=(0, 0.0, 0.0)):
         """shard: None, or (node_begin, node_count, allreduce) with allreduce an ``ALLREDUCE_FN`` object (kept alive
         here): the context then owns those nodes only (``pdadmm_init_sharded``)."""
         self._h = C.c_void_p()
@@ -141,8 +143,8 @@ class Context:
         wp = (C.POINTER(C.c_float) * len(Ws))(*[_ptr(w, C.c_float) for w in Ws])
         cfg = _Config(n_nodes, src.size, _ptr(src, C.c_int32), _ptr(dst, C.c_int32), feat.shape[1],
                       _ptr(feat, C.c_float), n_hops, n_classes, _ptr(lab, C.c_int32), _ptr(msk, C.c_uint8),
-                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, quant_neg_levels, quant_step, leaky_slope, wp,
-                      device, flags)
+                      len(widths), _ptr(widths, C.c_int32), rho, nu, quant_levels, quant_neg_levels, quant_step, leaky_slope,
+                      int(activation), int(table[0]), float(table[1]), float(table[2]), wp, device, flags)
         self.n_nodes, self.n_layers = int(n_nodes), len(widths)
         self.n_nodes_total = int(n_nodes)
         self.n0 = (n_hops + 1) * feat.shape[1]
@@ -273,13 +275,13 @@ class Context:
 
 def from_inputs(inp, device: int = 0, flags: int = 0, rho: Optional[float] = None, nu: Optional[float] = None,
                 quant_levels: Optional[int] = None, quant_neg_levels: int = 0, quant_step: float = 0.0,
-                leaky_slope: float = 0.0, shard=None) -> Context:
+                leaky_slope: float = 0.0, shard=None, activation: int = 0, table=(0, 0.0, 0.0)) -> Context:
     """Context for a ``synth.Inputs`` bundle."""
     w = inp.workload
     return Context(w.n_nodes, inp.edge_src, inp.edge_dst, inp.features, w.n_hops, w.n_classes, inp.labels,
                    inp.train_mask, w.widths, w.rho if rho is None else rho, w.nu if nu is None else nu,
                    w.quant_levels if quant_levels is None else quant_levels, inp.init_W, device, flags,
-                   quant_neg_levels, quant_step, leaky_slope, shard)
+                   quant_neg_levels, quant_step, leaky_slope, shard, activation, table)
 
 
 def quantize(x, scale: float, levels: int, device: int = 0, lo: float = 0.0):

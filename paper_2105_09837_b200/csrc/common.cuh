@@ -68,6 +68,16 @@ __device__ __forceinline__ void commit_amax(uint32_t m, uint32_t *__restrict__ w
   m = __reduce_max_sync(active, m);
   if ((int)(threadIdx.x & 31) == __ffs(active) - 1 && m != 0u) atomicMax(word, m);
 }
+// ---- f_l ----------------------------------------------------------------------------------------------------
+// The activation travels through the kernels as one float: a value in [0, 1) is ReLU (0) or leaky ReLU with that slope
+// for x <= 0; 2 is tanh, 3 the logistic sigmoid (the smooth activations, whose z-update searches a lookup table).
+constexpr float ACT_TANH = 2.0f, ACT_SIGMOID = 3.0f;
+__device__ __forceinline__ float act_eval(float x, float sel) {
+  if (sel < 1.0f) return x > 0.f ? x : sel * x;
+  if (sel == ACT_TANH) return tanhf(x);
+  return 1.0f / (1.0f + expf(-x));
+}
+
 // ---- device reductions -------------------------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -537,6 +537,64 @@ zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, 
   if (threadIdx.x == 0) slots[blockIdx.x] = tot;
 }
 
+// ---- the same for a smooth activation: z-update by lookup table ---------------------------------------------
+// f = tanh or sigmoid has no closed-form z-update; the paper recommends a lookup table (remark after Eq. "update z").
+// The table holds T equally spaced candidates z_i = lo + i h with f(z_i); z+ is the candidate with the smallest
+// (z - a)^2 + (q - f(z))^2 + (z - z^k)^2 (the first one if equal), element by element.  q, u, r, t as in zqu_kernel.
+// Dynamic shared memory: 2 T floats.
+__global__ void __launch_bounds__(EW_THREADS)
+zqu_table_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
+                 const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
+                 float rho, float nu, float act, float t_lo, float t_step, int T, float q_scale, float q_lo, float q_top,
+                 float *__restrict__ t_next, double *__restrict__ slots, uint32_t *__restrict__ amax_r) {
+  extern __shared__ float table_sh[];              // z_i, then f(z_i)
+  __shared__ double red[EW_THREADS / 32];
+  for (int i = threadIdx.x; i < T; i += blockDim.x) {
+    const float zi = __fadd_rn(t_lo, __fmul_rn((float)i, t_step));
+    table_sh[i] = zi;
+    table_sh[T + i] = act_eval(zi, act);
+  }
+  __syncthreads();
+  const float inv_rn = 1.0f / (rho + nu);
+  double ss = 0.0;
+  uint32_t mr = 0u;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 sh = ld4(shift, i % ld4cols);
+    const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i), pv = ld4(p_next, i);
+    const float a[4] = {(rv.x - sh.x) + zv.x, (rv.y - sh.y) + zv.y, (rv.z - sh.z) + zv.z, (rv.w - sh.w) + zv.w};
+    const float zo[4] = {zv.x, zv.y, zv.z, zv.w}, qo[4] = {qv.x, qv.y, qv.z, qv.w};
+    float best[4] = {3.0e38f, 3.0e38f, 3.0e38f, 3.0e38f}, zb[4] = {0.f, 0.f, 0.f, 0.f}, fb[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k = 0; k < T; ++k) {
+      const float zi = table_sh[k], fi = table_sh[T + k];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float d0 = zi - a[e], d1 = qo[e] - fi, d2 = zi - zo[e];
+        const float h = fmaf(d0, d0, fmaf(d1, d1, d2 * d2));
+        if (h < best[e]) { best[e] = h; zb[e] = zi; fb[e] = fi; }
+      }
+    }
+    const float pn[4] = {pv.x, pv.y, pv.z, pv.w}, uo[4] = {uv.x, uv.y, uv.z, uv.w};
+    float zn[4], qn[4], un[4], rn[4], tn[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float qq = (rho * pn[e] + uo[e] + nu * fb[e]) * inv_rn;
+      if (q_top >= 0.0f) { unsigned code; qq = quantize_one(qq, q_scale, q_lo, q_top, code); }
+      const float res = pn[e] - qq;
+      zn[e] = zb[e]; qn[e] = qq; un[e] = fmaf(rho, res, uo[e]); rn[e] = a[e] - zb[e];
+      tn[e] = fmaf(rho, res, un[e]);
+      ss += (double)res * res;
+    }
+    st4(z, i, make_float4(zn[0], zn[1], zn[2], zn[3])); st4(q, i, make_float4(qn[0], qn[1], qn[2], qn[3]));
+    st4(u, i, make_float4(un[0], un[1], un[2], un[3]));
+    const float4 r4 = make_float4(rn[0], rn[1], rn[2], rn[3]);
+    st4(r, i, r4); st4(t_next, i, make_float4(tn[0], tn[1], tn[2], tn[3]));
+    mr = max(mr, abs_bits(r4));
+  }
+  if (amax_r != nullptr) commit_amax(mr, amax_r);
+  const double tot = block_sum<EW_THREADS>(ss, red);
+  if (threadIdx.x == 0) slots[blockIdx.x] = tot;
+}
+
 // ---- z-update of the last layer -------------------------------------------------------------------
 // One thread per node.  a = (r - shift) + z.  Labelled node: z+ = argmin CE(z; y) + (nu/2)||z - a||^2
 // (Eq. "update zl"), the unique root of softmax(z) - e_y + nu (z - a) = 0, by damped Newton with the
@@ -637,8 +695,7 @@ relu_max_kernel(const float *__restrict__ z, float *__restrict__ q, size_t n4, f
   float m = 0.0f;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = ld4(z, i);
-    v.x = v.x > 0.f ? v.x : slope * v.x; v.y = v.y > 0.f ? v.y : slope * v.y;
-    v.z = v.z > 0.f ? v.z : slope * v.z; v.w = v.w > 0.f ? v.w : slope * v.w;
+    v.x = act_eval(v.x, slope); v.y = act_eval(v.y, slope); v.z = act_eval(v.z, slope); v.w = act_eval(v.w, slope);
     m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
     st4(q, i, v);
   }
@@ -664,7 +721,7 @@ objective_layer_kernel(const float *__restrict__ r, const float *__restrict__ z,
     s0 += rv * rv;
     if (q != nullptr) {
       const float zv = z[i];
-      const double qv = q[i], act = zv > 0.0f ? zv : slope * zv, res = (double)p_next[i] - qv;
+      const double qv = q[i], act = act_eval(zv, slope), res = (double)p_next[i] - qv;
       s1 += (qv - act) * (qv - act);
       s2 += (double)u[i] * res;
       s3 += res * res;

@@ -69,11 +69,11 @@ struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b
     return make_float4(a.x + b.x - z.x, a.y + b.y - z.y, a.z + b.z - z.z, a.w + b.w - z.w);
   }
 };
-struct EpiBiasAct {           // C = acc + b[col], then f (ReLU, leaky with `slope`) if relu != 0   (z = W p + b, p' = f(z))
+struct EpiBiasAct {           // C = acc + b[col], then f (selected by `slope`, see act_eval) if relu != 0   (z = W p + b, p' = f(z))
   static constexpr bool kDirect = false, kSumsq = false;
   static constexpr int kInputs = 0;
   float *C; int ldc; const float *bias; int relu; float slope; uint32_t *amax;
-  __device__ __forceinline__ float f(float x) const { return x > 0.f ? x : slope * x; }
+  __device__ __forceinline__ float f(float x) const { return act_eval(x, slope); }
   __device__ __forceinline__ void prefetch(int, int) const {}
   __device__ __forceinline__ void load(int, int, float4 *) const {}
   __device__ __forceinline__ float4 apply(int col, float4 a, const float4 *) const {

@@ -139,7 +139,9 @@ struct pdadmm_ctx {
   int neg_levels = 0;              // levels below zero
   float fixed_step = 0.f;          // > 0: the same level spacing for every layer
   bool quant_q = false;            // q_l is kept on the level set of p_{l+1} as well
-  float slope = 0.f;               // f_l: 0 = ReLU, (0, 1) = leaky ReLU with that slope for x <= 0
+  float slope = 0.f;               // f_l (see act_eval): [0, 1) = (leaky) ReLU with that slope for x <= 0, 2 = tanh, 3 = sigmoid
+  float table_lo = 0.f, table_step = 0.f;   // lookup table of the z-update of a smooth activation: z_i = lo + i step
+  int table_size = 0;
   bool ls_risk = false;            // R = least squares instead of cross-entropy
   float rho = 0, nu = 0;
   uint32_t flags = 0;
@@ -767,7 +769,13 @@ static void zqu_step(pdadmm_ctx *c, int l) {
   if (l + 1 < c->L) {
     const size_t n4 = (size_t)N * ly.ld_out / 4;
     const int grid = ew_grid(n4);
-    {
+    if (c->table_size > 0) {
+      Launch k(c, KC_ZQU, s.st, 40.0 * N * ly.n_out, 0);
+      const Layer &nx = c->layers[l + 1];
+      zqu_table_kernel<<<grid, EW_THREADS, 2 * c->table_size * sizeof(float), s.st>>>(
+          ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu, c->slope, c->table_lo, c->table_step,
+          c->table_size, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, nx.t, s.slots, ly.amax_r);
+    } else {
       Launch k(c, KC_ZQU, s.st, 40.0 * N * ly.n_out, 0);
       const Layer &nx = c->layers[l + 1];
       zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu,
@@ -875,6 +883,12 @@ static int check_config(const pdadmm_config *cfg) {
     return fail(PDADMM_EINVAL, "quant_step must be >= 0, and > 0 when quant_neg_levels > 0");
   if (!(cfg->leaky_slope >= 0.f && cfg->leaky_slope < 1.f))
     return fail(PDADMM_EINVAL, "leaky_slope must be in [0, 1)");
+  if (cfg->activation < 0 || cfg->activation > 2) return fail(PDADMM_EINVAL, "activation must be 0, 1 or 2");
+  if (cfg->activation != 0) {
+    if (cfg->leaky_slope != 0.f) return fail(PDADMM_EINVAL, "leaky_slope belongs to activation 0");
+    if (cfg->table_size < 2 || cfg->table_size > 4096 || !(cfg->table_hi > cfg->table_lo))
+      return fail(PDADMM_EINVAL, "a smooth activation needs table_size in [2, 4096] and table_lo < table_hi");
+  }
   if ((cfg->flags & PDADMM_FLAG_QUANT_Q) && cfg->quant_levels == 0)
     return fail(PDADMM_EINVAL, "PDADMM_FLAG_QUANT_Q needs quant_levels >= 2");
   for (int64_t j = 0; j < cfg->n_nodes; ++j)
@@ -1064,7 +1078,12 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
   c->neg_levels = cfg->quant_neg_levels; c->fixed_step = cfg->quant_step;
   c->code_bytes = cfg->quant_levels > 256 ? 2 : 1;
   c->quant_q = (cfg->flags & PDADMM_FLAG_QUANT_Q) != 0;
-  c->slope = cfg->leaky_slope;
+  c->slope = cfg->activation == 1 ? ACT_TANH : (cfg->activation == 2 ? ACT_SIGMOID : cfg->leaky_slope);
+  if (cfg->activation != 0) {
+    c->table_size = cfg->table_size;
+    c->table_lo = cfg->table_lo;
+    c->table_step = (cfg->table_hi - cfg->table_lo) / (float)(cfg->table_size - 1);      // single precision, like the candidates
+  }
   c->ls_risk = (cfg->flags & PDADMM_FLAG_LEAST_SQUARES) != 0;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;

@@ -10,14 +10,15 @@ from paper_2105_09837_b200 import binding as B
 
 
 def oracle_problem(inp, rho=None, nu=None, quant_levels=None, quantize_q=False, neg_levels=0, step=0.0, slope=0.0,
-                   risk="ce"):
+                   risk="ce", activation="relu", table=(257, -4.0, 4.0)):
     """(Params, initial oracle State) for a synth.Inputs bundle.  neg_levels / step: a fixed level set
     {(c - neg_levels) step} as the C ABI's quant_neg_levels / quant_step describe it."""
     w = inp.workload
     lo = float(np.float32(-neg_levels) * np.float32(step))
     prm = o.Params(w.rho if rho is None else rho, w.nu if nu is None else nu,
                    w.quant_levels if quant_levels is None else quant_levels,
-                   quantize_q=quantize_q, level_lo=lo, level_step=step, slope=slope, risk=risk)
+                   quantize_q=quantize_q, level_lo=lo, level_step=step, slope=slope, risk=risk, activation=activation,
+                   table_size=table[0], table_lo=table[1], table_hi=table[2])
     A = o.renormalized_adjacency(w.n_nodes, inp.edge_src, inp.edge_dst)
     X = o.augment(inp.features.T.astype(np.float64), A, w.n_blocks)
     s = o.init_state(X, [x.astype(np.float64) for x in inp.init_W], inp.labels, inp.train_mask, prm)
@@ -130,7 +131,7 @@ def redo_after_p(s: o.State, n: o.State, prm: o.Params) -> o.State:
     for l in range(L):
         a = n.W[l] @ n.p[l] + n.b[l][:, None]
         if l < L - 1:
-            n.z[l] = o.update_z_hidden(a, s.q[l], s.z[l], prm.slope)
+            n.z[l] = o._update_z_hidden_for(prm, a, s.q[l], s.z[l])
         elif prm.risk == "ls":
             n.z[l] = o.update_z_last_least_squares(a, s.y, s.mask, nu)
         else:
@@ -138,9 +139,23 @@ def redo_after_p(s: o.State, n: o.State, prm: o.Params) -> o.State:
     for l in range(L - 1):
         if prm.quant_levels and prm.quantize_q:
             n.q[l] = o.update_q_quantized(n.p[l + 1], s.u[l], n.z[l], rho, nu, s.scale[l + 1], prm.quant_levels,
-                                          prm.level_lo, prm.slope)
+                                          prm.level_lo, prm.f)
         else:
-            n.q[l] = o.update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.slope)
+            n.q[l] = o.update_q(n.p[l + 1], s.u[l], n.z[l], rho, nu, prm.f)
     for l in range(L - 1):
         n.u[l] = o.update_u(s.u[l], n.p[l + 1], n.q[l], rho)
     return n
+
+
+def z_table_tie_mask(prev: o.State, nxt: o.State, prm: o.Params, l: int, tol=1e-5):
+    """Lookup-table z-update of hidden layer l (0-based): elements where a neighbouring candidate of the table is
+    (nearly) as good as the chosen one, so that single and double precision may pick different candidates."""
+    a = nxt.W[l] @ nxt.p[l] + nxt.b[l][:, None]
+    pts = o.table_points(prm.table_lo, prm.table_hi, prm.table_size)
+    step = pts[1] - pts[0]
+    f = prm.f
+    h = lambda z: (z - a) ** 2 + (prev.q[l] - f(z)) ** 2 + (z - prev.z[l]) ** 2
+    best = h(nxt.z[l])
+    other = np.minimum(h(np.clip(nxt.z[l] - step, pts[0], pts[-1])), h(np.clip(nxt.z[l] + step, pts[0], pts[-1])))
+    edge = (nxt.z[l] <= pts[0]) | (nxt.z[l] >= pts[-1])
+    return ((other - best) <= tol * (np.abs(best) + 1e-30)) & ~edge
