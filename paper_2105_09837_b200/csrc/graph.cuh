@@ -164,6 +164,10 @@ __global__ void adjacency_values_kernel(const int *__restrict__ row_ptr, const i
 // Y[i][0:width] = sum_e val[e] * X[col[e]][0:width], one warp per row, entries in CSR order.
 // X and Y are addressed with the same row stride ld (they are column blocks of one matrix).
 // VEC = 4, 2 or 1 floats per lane and access, chosen by the alignment of the blocks.
+// The gathered rows are what costs: the lanes first fetch up to 32 (column, value) pairs of the row together and hand
+// them round by shuffle, and every lane keeps SPMM_CH column groups in flight per neighbour (independent loads), so a
+// warp has 4 x 32 x VEC floats of a neighbour's row on their way at a time instead of 32 x VEC.
+constexpr int SPMM_CH = 4;
 template <int VEC>
 __global__ void __launch_bounds__(256)
 spmm_kernel(const int *__restrict__ row_ptr, const int *__restrict__ col_idx, const float *__restrict__ val,
@@ -171,28 +175,61 @@ spmm_kernel(const int *__restrict__ row_ptr, const int *__restrict__ col_idx, co
   const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (row >= n_rows) return;
   const int b = row_ptr[row], e = row_ptr[row + 1];
-  for (int c0 = lane * VEC; c0 < width; c0 += 32 * VEC) {
-    float acc[VEC];
+  for (int base = 0; base < width; base += 32 * VEC * SPMM_CH) {
+    float acc[SPMM_CH][VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
-    for (int k = b; k < e; ++k) {
-      const float a = __ldg(val + k);
-      const float *xr = X + (size_t)__ldg(col_idx + k) * ld + c0;
-      if (VEC == 4) {
-        const float4 x = *reinterpret_cast<const float4 *>(xr);
-        acc[0] = fmaf(a, x.x, acc[0]); acc[1] = fmaf(a, x.y, acc[1]);
-        acc[2 % VEC] = fmaf(a, x.z, acc[2 % VEC]); acc[3 % VEC] = fmaf(a, x.w, acc[3 % VEC]);
-      } else if (VEC == 2) {
-        const float2 x = *reinterpret_cast<const float2 *>(xr);
-        acc[0] = fmaf(a, x.x, acc[0]); acc[1 % VEC] = fmaf(a, x.y, acc[1 % VEC]);
-      } else {
-        acc[0] = fmaf(a, *xr, acc[0]);
+    for (int ch = 0; ch < SPMM_CH; ++ch)
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) acc[ch][v] = 0.f;
+    for (int k0 = b; k0 < e; k0 += 32) {
+      const int n = min(32, e - k0);
+      const int my_col = lane < n ? __ldg(col_idx + k0 + lane) : 0;
+      const float my_val = lane < n ? __ldg(val + k0 + lane) : 0.f;
+      // four neighbours at a time: their loads are independent (an entry past the end of the row repeats the first
+      // of the four with the value 0, so it reads nothing that the row does not read anyway)
+      for (int j = 0; j < n; j += 4) {
+        float a[4];
+        const float *xr[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          a[t] = __shfl_sync(0xffffffffu, my_val, (j + t) & 31);
+          xr[t] = X + (size_t)__shfl_sync(0xffffffffu, my_col, (j + t) & 31) * ld;
+          if (j + t >= n) { a[t] = 0.f; xr[t] = xr[0]; }
+        }
+#pragma unroll
+        for (int ch = 0; ch < SPMM_CH; ++ch) {
+          const int c0 = base + (ch * 32 + lane) * VEC;
+          if (c0 >= width) continue;
+          float x[4][VEC];
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            if (VEC == 4) {
+              const float4 q = *reinterpret_cast<const float4 *>(xr[t] + c0);
+              x[t][0] = q.x; x[t][1 % VEC] = q.y; x[t][2 % VEC] = q.z; x[t][3 % VEC] = q.w;
+            } else if (VEC == 2) {
+              const float2 q = *reinterpret_cast<const float2 *>(xr[t] + c0);
+              x[t][0] = q.x; x[t][1 % VEC] = q.y;
+            } else {
+              x[t][0] = xr[t][c0];
+            }
+          }
+          // added in entry order, like a loop over single entries
+#pragma unroll
+          for (int t = 0; t < 4; ++t)
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[ch][v] = fmaf(a[t], x[t][v], acc[ch][v]);
+        }
       }
     }
-    float *yr = Y + (size_t)row * ld + c0;
-    if (VEC == 4) *reinterpret_cast<float4 *>(yr) = make_float4(acc[0], acc[1 % VEC], acc[2 % VEC], acc[3 % VEC]);
-    else if (VEC == 2) *reinterpret_cast<float2 *>(yr) = make_float2(acc[0], acc[1 % VEC]);
-    else *yr = acc[0];
+#pragma unroll
+    for (int ch = 0; ch < SPMM_CH; ++ch) {
+      const int c0 = base + (ch * 32 + lane) * VEC;
+      if (c0 >= width) continue;
+      float *yr = Y + (size_t)row * ld + c0;
+      if (VEC == 4) *reinterpret_cast<float4 *>(yr) = make_float4(acc[ch][0], acc[ch][1 % VEC], acc[ch][2 % VEC], acc[ch][3 % VEC]);
+      else if (VEC == 2) *reinterpret_cast<float2 *>(yr) = make_float2(acc[ch][0], acc[ch][1 % VEC]);
+      else *yr = acc[ch][0];
+    }
   }
 }
 

@@ -527,7 +527,7 @@ static int gemm_over_nodes_raw(pdadmm_ctx *c, int cls, cudaStream_t st, int M, i
 // never changes and keeps its planes.
 static bool planes_beforehand(int M, int N, bool second_operand_cached) {
   const int64_t tiles = ceil_div(M, TC_BM) * ceil_div(N, TC_BN);
-  return tiles >= 32 || (second_operand_cached && tiles >= 8);
+  return tiles >= 16 || (second_operand_cached && tiles >= 8);
 }
 
 }  // namespace pd
