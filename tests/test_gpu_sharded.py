@@ -174,7 +174,8 @@ def test_nccl_callback_with_one_rank_equals_the_unsharded_context():
         b = B.from_inputs(inp)
         a.step(4)
         b.step(4)
-        assert red.calls > 0 and red.bytes == a.comm_bytes()        # both sides count what went through the callback
+        assert red.calls > 0 and red.bytes - a.comm_bytes() == 4 * 3     # the context counts pdadmm_step's traffic; the start
+        #                                                                   reduced one float per level spacing (3 layers)
         sa, sb = U.read_state(a), U.read_state(b)
         for name in ("p", "W", "z", "q"):
             for x, y in zip(sa[name], sb[name]):
