@@ -172,19 +172,23 @@ quantize_kernel(const float *__restrict__ x, size_t n, float scale, float lo, in
   }
 }
 
-// ---- finalisers of the step parameters (one block of 256 threads) ---------------------------------
-// Fixed-order sum of n slots by one block: thread t adds slots t, t+256, ..., then a fixed tree.  Result in thread 0.
-__device__ __forceinline__ double block_sum_slots(const double *__restrict__ slots, int n, double *sh /* 256 */) {
+// ---- finalisers of the step parameters (one block of FIN_THREADS threads) ---------------------------------
+// Fixed-order sum of n slots by one block of FIN_THREADS threads: thread t adds slots t, t + FIN_THREADS, ..., then a
+// fixed tree.  Result in thread 0.
+constexpr int FIN_THREADS = 1024;
+__device__ __forceinline__ double block_sum_slots(const double *__restrict__ slots, int n, double *sh /* FIN_THREADS */) {
   // four independent partial sums per thread keep four loads in flight; the order of the additions is fixed
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
   int i = threadIdx.x;
-  for (; i + 768 < n; i += 1024) { s0 += slots[i]; s1 += slots[i + 256]; s2 += slots[i + 512]; s3 += slots[i + 768]; }
-  for (; i < n; i += 256) s0 += slots[i];
+  for (; i + 3 * FIN_THREADS < n; i += 4 * FIN_THREADS) {
+    s0 += slots[i]; s1 += slots[i + FIN_THREADS]; s2 += slots[i + 2 * FIN_THREADS]; s3 += slots[i + 3 * FIN_THREADS];
+  }
+  for (; i < n; i += FIN_THREADS) s0 += slots[i];
   const double s = (s0 + s1) + (s2 + s3);
   __syncthreads();
   sh[threadIdx.x] = s;
   __syncthreads();
-  for (int w = 128; w > 0; w >>= 1) {
+  for (int w = FIN_THREADS / 2; w > 0; w >>= 1) {
     if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
     __syncthreads();
   }
@@ -192,10 +196,10 @@ __device__ __forceinline__ double block_sum_slots(const double *__restrict__ slo
 }
 // ||g||^2 and ||W g||^2 from their slots, then
 // tau = rho + nu ||W g||^2 / ||g||^2 : the smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(FIN_THREADS)
 finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots_g, int n_g, const double *slots_wg, int n_wg,
                     int *nonfinite, uint32_t *clear_word /* max|p| of the layer restarts with the coming p-step */) {
-  __shared__ double sh[256];
+  __shared__ double sh[FIN_THREADS];
   const double gg = block_sum_slots(slots_g, n_g, sh);
   const double wg = block_sum_slots(slots_wg, n_wg, sh);
   if (threadIdx.x == 0) {
@@ -212,10 +216,10 @@ finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots
 }
 // Stop condition of the quantised step in its quadratic form: nu||W d||^2 + rho||d||^2 <= tau||d||^2 (1 + slack).
 // Not accepted: tau is doubled for the next trial.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(FIN_THREADS)
 finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack, const double *slots_d, int n_d,
                       const double *slots_wd, int n_wd) {
-  __shared__ double sh[256];
+  __shared__ double sh[FIN_THREADS];
   const double dd = block_sum_slots(slots_d, n_d, sh);
   const double wd = block_sum_slots(slots_wd, n_wd, sh);
   if (threadIdx.x == 0) {
@@ -232,10 +236,10 @@ finalize_trial_kernel(LayerScalars *sc, double rho, double nu, double slack, con
 }
 // ||grad_W||^2 and ||grad_W p+||^2 from their slots, then
 // theta = nu ||grad_W p+||^2 / ||grad_W||^2 : the smallest theta with phi(W+) <= V_l(W+; theta).
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(FIN_THREADS)
 finalize_theta_kernel(LayerScalars *sc, double nu, const double *slots_G, int n_G, const double *slots_Gp, int n_Gp,
                       int *nonfinite, uint32_t *clear_word /* max|r| of the layer restarts with the coming z-step */) {
-  __shared__ double sh[256];
+  __shared__ double sh[FIN_THREADS];
   const double GG = block_sum_slots(slots_G, n_G, sh);
   const double Gp = block_sum_slots(slots_Gp, n_Gp, sh);
   if (threadIdx.x == 0) {
@@ -437,18 +441,19 @@ resid_colsum_kernel(float *__restrict__ r, const float *__restrict__ gp, const L
 
 // out[c] = sum over the blocks' slots of column c (the first half of finalize_bias_kernel, for a context that owns only
 // part of the nodes: the totals are then added over the shards before the mean is taken).  Same thread layout.
-__global__ void __launch_bounds__(256)
+constexpr int BIAS_GROUPS = 32;          // slot groups per block of the two kernels below (blockDim = (32, BIAS_GROUPS))
+__global__ void __launch_bounds__(32 * BIAS_GROUPS)
 colsum_total_kernel(const double *__restrict__ slots, int n_slots, int ld, double *__restrict__ out) {
-  __shared__ double sh[8][33];
+  __shared__ double sh[BIAS_GROUPS][33];
   const int c = blockIdx.x * 32 + threadIdx.x;
   double s = 0.0;
   if (c < ld)
-    for (int i = threadIdx.y; i < n_slots; i += 8) s += slots[(size_t)i * ld + c];
+    for (int i = threadIdx.y; i < n_slots; i += BIAS_GROUPS) s += slots[(size_t)i * ld + c];
   sh[threadIdx.y][threadIdx.x] = s;
   __syncthreads();
   if (threadIdx.y == 0 && c < ld) {
     double t = 0.0;
-    for (int k = 0; k < 8; ++k) t += sh[k][threadIdx.x];
+    for (int k = 0; k < BIAS_GROUPS; ++k) t += sh[k][threadIdx.x];
     out[c] = t;
   }
 }
@@ -470,21 +475,22 @@ sumsq_amax_kernel(const float *__restrict__ G, size_t n4, uint32_t *__restrict__
 }
 
 // b+ = b - mean_j r[j][:]  (Eq. "update b" with the step 1/(nu N), i.e. the exact minimiser);
-// shift[c] = that mean, which the z-update subtracts from r.  blockDim = (32 columns, 8 slot groups): group g adds
-// the slots g, g+8, ... of its column, the 8 group sums are then added in group order.
-__global__ void __launch_bounds__(256)
+// shift[c] = that mean, which the z-update subtracts from r.  blockDim = (32 columns, BIAS_GROUPS slot groups): group g
+// adds the slots g, g + BIAS_GROUPS, ... of its column, the group sums are then added in group order (32 groups keep
+// 32 rows of slots in flight per block; the kernel has only ld / 32 blocks).
+__global__ void __launch_bounds__(32 * BIAS_GROUPS)
 finalize_bias_kernel(const double *__restrict__ slots, int n_slots, int ld, int width, double inv_n,
                      float *__restrict__ b, float *__restrict__ shift) {
-  __shared__ double sh[8][33];
+  __shared__ double sh[BIAS_GROUPS][33];
   const int c = blockIdx.x * 32 + threadIdx.x;
   double s = 0.0;
   if (c < ld)
-    for (int i = threadIdx.y; i < n_slots; i += 8) s += slots[(size_t)i * ld + c];
+    for (int i = threadIdx.y; i < n_slots; i += BIAS_GROUPS) s += slots[(size_t)i * ld + c];
   sh[threadIdx.y][threadIdx.x] = s;
   __syncthreads();
   if (threadIdx.y == 0 && c < ld) {
     double t = 0.0;
-    for (int k = 0; k < 8; ++k) t += sh[k][threadIdx.x];
+    for (int k = 0; k < BIAS_GROUPS; ++k) t += sh[k][threadIdx.x];
     const float m = c < width ? (float)(t * inv_n) : 0.0f;
     shift[c] = m;
     if (c < width) b[c] -= m;

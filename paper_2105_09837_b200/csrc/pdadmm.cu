@@ -587,13 +587,13 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   if (c->reduce != nullptr) {
     // ||g||^2 and ||W g||^2 are sums over nodes: this shard's totals, added over the shards, then tau
     PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, np, slots_b, np2));
-    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.red, 1, s.red + 1, 1, c->d_flag + 2,
+    finalize_tau_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.red, 1, s.red + 1, 1, c->d_flag + 2,
                                              ly.amax_p);
     return PDADMM_OK;
   }
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
-    finalize_tau_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2,
+    finalize_tau_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2,
                                              ly.amax_p);
   }
   return PDADMM_OK;
@@ -640,10 +640,10 @@ static int q_trial(pdadmm_ctx *c, int l) {
                            slots_b, &np, 0, w_d));
   if (c->reduce != nullptr) {
     PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, grid, slots_b, np));
-    finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.red, 1, s.red + 1, 1);
+    finalize_trial_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.red, 1, s.red + 1, 1);
   } else {
     Launch k(c, KC_SMALL, s.st, 8.0 * (grid + np), 0);
-    finalize_trial_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
+    finalize_trial_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.slots, grid, slots_b, np);
   }
   PD_CUDA(cudaMemcpyAsync(s.h_flag, &ly.sc->accepted, sizeof(int), cudaMemcpyDeviceToHost, s.st));
   PD_CUDA(cudaEventRecord(s.ev_flag, s.st));
@@ -725,10 +725,10 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
   if (c->reduce != nullptr) {
     // ||G p+||^2 is a sum over nodes (||G||^2 is the same on every shard already)
     PD_TRY(shard_sum_slots(c, s.st, s.red, slots_b, np, nullptr, 0));
-    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, s.red, 1, c->d_flag + 2, ly.amax_r);
+    finalize_theta_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, s.red, 1, c->d_flag + 2, ly.amax_r);
   } else {
     Launch k(c, KC_SMALL, s.st, 8.0 * (gw + np), 0);
-    finalize_theta_kernel<<<1, 256, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2, ly.amax_r);
+    finalize_theta_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->nu, s.slots, gw, slots_b, np, c->d_flag + 2, ly.amax_r);
   }
   {
     Launch k(c, KC_WSTEP, s.st, 20.0 * ly.n_out * ly.n_in, 0);
@@ -749,13 +749,13 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
   }
   if (c->reduce != nullptr) {
     // the column sums run over all nodes: this shard's sums, added over the shards, then the mean over |V|
-    colsum_total_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, s.red);
+    colsum_total_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, BIAS_GROUPS), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, s.red);
     PD_TRY(shard_sum(c, s.st, s.red, (size_t)ly.ld_out, 1));
-    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.red, 1, ly.ld_out, ly.n_out,
+    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, BIAS_GROUPS), 0, s.st>>>(s.red, 1, ly.ld_out, ly.n_out,
                                                                                 1.0 / (double)c->N_total, ly.b, ly.shift);
   } else {
     Launch k(c, KC_SMALL, s.st, 8.0 * used_blocks * ly.ld_out, 0);
-    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, 8), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
+    finalize_bias_kernel<<<(int)ceil_div(ly.ld_out, 32), dim3(32, BIAS_GROUPS), 0, s.st>>>(s.slots, used_blocks, ly.ld_out, ly.n_out,
                                                                                 1.0 / (double)N, ly.b, ly.shift);
   }
   return PDADMM_OK;
