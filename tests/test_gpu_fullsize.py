@@ -97,6 +97,73 @@ def test_c4_c5_full_size_parts_and_invariants(name):
     ctx.destroy()
 
 
+def _rows(ctx, kind, layer, nodes):
+    """Rows `nodes` of a node-major tensor as the oracle's columns (float64)."""
+    return ctx.get_tensor(kind, layer)[nodes].T.astype(np.float64)
+
+
+@pytest.mark.parametrize("name", ["c4", "c5"])
+def test_c4_c5_full_size_node_wise_updates_on_sampled_nodes(name):
+    """At full size the oracle cannot afford an iteration, but every update except the sums over nodes acts on one
+    node's column at a time.  So for 48 sampled nodes the p-, z-, q- and u-updates of one device iteration are
+    recomputed by the oracle's own update functions from the device's state before the iteration and the quantities
+    that are sums over all nodes as the device has them afterwards (tau, W+, b+, which the reduced-size tests compare
+    with the oracle).  Launch configuration: exactly what bench.py times."""
+    w = synth.get(name)
+    inp = synth.make_inputs(w)
+    ctx = B.from_inputs(inp)
+    ctx.step(2)                                      # leave the feasible start
+    rng = np.random.default_rng(5)
+    nodes = np.sort(rng.choice(w.n_nodes, size=48, replace=False))
+    L, m, rho, nu = w.n_layers, w.quant_levels, w.rho, w.nu
+    layers = sorted(set([1, 2, L // 2, L - 1, L]))
+    before = {}
+    for l in layers:
+        before[l] = dict(p=_rows(ctx, B.T_P, l, nodes), z=_rows(ctx, B.T_Z, l, nodes),
+                         W=ctx.get_tensor(B.T_W, l).astype(np.float64), b=ctx.get_tensor(B.T_B, l).astype(np.float64))
+        if l < L:
+            before[l].update(q=_rows(ctx, B.T_Q, l, nodes), u=_rows(ctx, B.T_U, l, nodes))
+        if l >= 2:
+            before[l].update(q_prev=_rows(ctx, B.T_Q, l - 1, nodes), u_prev=_rows(ctx, B.T_U, l - 1, nodes))
+    ctx.step(1)
+    y, mask = inp.labels[nodes], inp.train_mask[nodes].astype(bool)
+    for l in layers:
+        s0 = before[l]
+        p_new = _rows(ctx, B.T_P, l, nodes)
+        if l >= 2:
+            tau = float(ctx.get_tensor(B.T_TAU, l)[0])
+            scale = float(ctx.get_tensor(B.T_QSCALE, l)[0])
+            g = o.grad_p_phi(s0["p"], s0["W"], s0["b"], s0["z"], nu, s0["q_prev"], s0["u_prev"], rho)
+            x = s0["p"] - g / tau
+            codes, want_p = o.nearest_level(x, scale, m)
+            t = x / scale
+            clear = np.abs(t - np.floor(t) - 0.5) > 2e-3          # away from a rounding boundary (x carries fp32 rounding)
+            assert np.array_equal(p_new[clear], want_p[clear]), (name, l)
+            assert np.max(np.abs(p_new - want_p)) <= scale * (1 + 1e-6) and clear.mean() > 0.99
+        else:
+            assert np.array_equal(p_new, s0["p"])                # p_1 = X never moves
+        W1, b1 = ctx.get_tensor(B.T_W, l).astype(np.float64), ctx.get_tensor(B.T_B, l).astype(np.float64)
+        a = W1 @ p_new + b1[:, None]
+        z_new = _rows(ctx, B.T_Z, l, nodes)
+        if l < L:
+            want_z = o.update_z_hidden(a, s0["q"], s0["z"])
+            zn = np.minimum((a + s0["z"]) / 2, 0.0)
+            zp = np.maximum((a + s0["q"] + s0["z"]) / 3, 0.0)
+            fn, fp = o.z_objective_hidden(zn, a, s0["q"], s0["z"]), o.z_objective_hidden(zp, a, s0["q"], s0["z"])
+            tie = (np.abs(fp - fn) <= 1e-5 * (np.abs(fp) + np.abs(fn) + 1e-30)) & (zp != zn)
+            assert U.rel_err(z_new, want_z, tie) < 1e-4, (name, l)
+            p_next = _rows(ctx, B.T_P, l + 1, nodes)
+            q_new, u_new = _rows(ctx, B.T_Q, l, nodes), _rows(ctx, B.T_U, l, nodes)
+            want_q = o.update_q(p_next, s0["u"], z_new, rho, nu)
+            assert U.rel_err(q_new, want_q) < 1e-5, (name, l)
+            want_u = o.update_u(s0["u"], p_next, q_new, rho)
+            assert np.linalg.norm(u_new - want_u) <= 1e-5 * max(np.linalg.norm(want_u), rho * np.linalg.norm(p_next) * 1e-2), (name, l)
+        else:
+            want_z = o.update_z_last(a, y, mask, nu)
+            assert U.rel_err(z_new, want_z) < 1e-4, (name, l)
+    ctx.destroy()
+
+
 def test_c4_full_size_level_set_variant_and_prediction():
     """Workload c4 with the paper's level set {-1..20} for p and q: after two iterations both are on the set bit
     for bit, and the forward pass of the trained model agrees with the oracle on sampled nodes."""
