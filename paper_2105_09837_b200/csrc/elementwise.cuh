@@ -128,7 +128,10 @@ __global__ void __launch_bounds__(EW_THREADS)
 quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, const LayerScalars *__restrict__ sc,
                    float scale, float lo, int levels, float *__restrict__ p_new, float *__restrict__ d,
                    void *__restrict__ codes, int wide_codes, size_t n4, double *__restrict__ slots,
-                   uint32_t *__restrict__ amax_p /* max|p_new|, may be null */, uint32_t *__restrict__ amax_d /* max|d| */) {
+                   uint32_t *__restrict__ amax_p /* max|p_new|, may be null */, uint32_t *__restrict__ amax_d /* max|d| */,
+                   const void *__restrict__ codes_old /* codes of p; with the two planes below, else null */,
+                   __half *__restrict__ pn_plane /* the new codes as fp16 integers (operand plane of p_new = code * scale) */,
+                   __half *__restrict__ d_plane /* new code - old code as fp16 integers (operand plane of d) */) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_tau = sc->inv_tau, top = (float)(levels - 1);
   double ss = 0.0;
@@ -150,6 +153,22 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
       reinterpret_cast<ushort4 *>(codes)[i] = make_ushort4((unsigned short)c0, (unsigned short)c1, (unsigned short)c2, (unsigned short)c3);
     else
       reinterpret_cast<uchar4 *>(codes)[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
+    if (pn_plane != nullptr) {
+      // integers below 2048 are exact in fp16: the planes hold the codes themselves and their change
+      int o0, o1, o2, o3;
+      if (wide_codes) {
+        const ushort4 o = reinterpret_cast<const ushort4 *>(codes_old)[i];
+        o0 = o.x; o1 = o.y; o2 = o.z; o3 = o.w;
+      } else {
+        const uchar4 o = reinterpret_cast<const uchar4 *>(codes_old)[i];
+        o0 = o.x; o1 = o.y; o2 = o.z; o3 = o.w;
+      }
+      const __half2 a = __floats2half2_rn((float)c0, (float)c1), b = __floats2half2_rn((float)c2, (float)c3);
+      const __half2 e = __floats2half2_rn((float)((int)c0 - o0), (float)((int)c1 - o1));
+      const __half2 f = __floats2half2_rn((float)((int)c2 - o2), (float)((int)c3 - o3));
+      reinterpret_cast<uint2 *>(pn_plane)[i] = make_uint2(*reinterpret_cast<const uint32_t *>(&a), *reinterpret_cast<const uint32_t *>(&b));
+      reinterpret_cast<uint2 *>(d_plane)[i] = make_uint2(*reinterpret_cast<const uint32_t *>(&e), *reinterpret_cast<const uint32_t *>(&f));
+    }
   }
   if (amax_p != nullptr) { commit_amax(mp, amax_p); commit_amax(md, amax_d); }
   const double tot = block_sum<EW_THREADS>(ss, red);
@@ -169,6 +188,49 @@ quantize_kernel(const float *__restrict__ x, size_t n, float scale, float lo, in
       if (wide_codes) reinterpret_cast<uint16_t *>(codes_out)[i] = (uint16_t)c;
       else reinterpret_cast<uint8_t *>(codes_out)[i] = (uint8_t)c;
     }
+  }
+}
+
+// ---- operand planes of a quantised p from its codes ------------------------------------------------------------
+// p = code * s with code < 2048: the fp16 plane of the integer codes is the whole operand (the products multiply by s).
+// Same orientation [N][ld] ...
+__global__ void __launch_bounds__(EW_THREADS)
+codes_to_plane_kernel(const void *__restrict__ codes, int wide_codes, size_t n4, __half *__restrict__ plane) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float c0, c1, c2, c3;
+    if (wide_codes) {
+      const ushort4 o = reinterpret_cast<const ushort4 *>(codes)[i];
+      c0 = o.x; c1 = o.y; c2 = o.z; c3 = o.w;
+    } else {
+      const uchar4 o = reinterpret_cast<const uchar4 *>(codes)[i];
+      c0 = o.x; c1 = o.y; c2 = o.z; c3 = o.w;
+    }
+    const __half2 a = __floats2half2_rn(c0, c1), b = __floats2half2_rn(c2, c3);
+    reinterpret_cast<uint2 *>(plane)[i] = make_uint2(*reinterpret_cast<const uint32_t *>(&a), *reinterpret_cast<const uint32_t *>(&b));
+  }
+}
+// ... and transposed [cols][ldT] (node index contiguous), for the product that contracts over the nodes.  One block of
+// 32 x 8 threads per tile of 32 nodes x 32 columns, through shared memory.
+__global__ void __launch_bounds__(256)
+transpose_codes_kernel(const void *__restrict__ codes, int wide_codes, int rows, int cols, int ld,
+                       __half *__restrict__ planeT, int ldT) {
+  __shared__ __half sh[32][33];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + threadIdx.y + 8 * i, c = c0 + threadIdx.x;
+    float v = 0.f;
+    if (r < rows && c < cols) {
+      const size_t o = (size_t)r * ld + c;
+      v = wide_codes ? (float)reinterpret_cast<const uint16_t *>(codes)[o] : (float)reinterpret_cast<const uint8_t *>(codes)[o];
+    }
+    sh[threadIdx.y + 8 * i][threadIdx.x] = __float2half_rn(v);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = c0 + threadIdx.y + 8 * i, r = r0 + threadIdx.x;
+    if (c < cols && r < rows) planeT[(size_t)c * ldT + r] = sh[threadIdx.x][threadIdx.y + 8 * i];
   }
 }
 

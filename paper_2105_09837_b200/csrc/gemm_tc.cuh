@@ -108,6 +108,7 @@ struct TcParams {
   int tail_begin, tail_split;
   float *tail_ws;         // [tiles from tail_begin][tail_split][4 row quarters][128][32] floats
   int *tail_count;        // [tiles from tail_begin][4 row quarters], zero before and after every launch
+  float mul = 1.0f;       // factor applied to the result after the power-of-two scalings (integer operands, see ZERO)
 };
 
 // MODE TC_RAW_K:  A is [M][K] fp32, contiguous along K (a node-major matrix, rows = nodes), converted in the kernel;
@@ -130,13 +131,22 @@ struct TcParams {
 // warps read it out and add it to a register accumulator with round-to-nearest, while the MMAs of the next
 // block fill the other buffer.  The two correction terms are 2^-11 of the main term, so they are summed over
 // the whole contraction in a fourth tensor-memory tile and added once at the end.
+//
+// ZERO (TC_PLANES only): bit 0 = the lo plane of A is identically zero, bit 1 = the lo plane of B is.  An operand of
+// pdADMM-G-Q that lies on a level set {c s} (the quantised p, or the difference of two of them) is the spacing s times
+// a small integer, and integers up to 2048 are exact in one fp16 plane: its plane holds the integers, there is no lo
+// plane to load and no MMA for it (two MMAs per product instead of three), and prm.mul = s restores the values.
 enum : int { TC_RAW_K = 0, TC_RAW_MN = 1, TC_PLANES = 2 };
-template <int MODE, class Epi>
+template <int MODE, class Epi, int ZERO = 0>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_alo,
                const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_blo,
                const TcParams prm, Epi epi, double *__restrict__ partials) {
-  constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN, COARSE = epi_coarse<Epi>::value;
+  constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN, COARSE = epi_coarse<Epi>::value || ZERO == 3;
+  constexpr bool A_LO = !(ZERO & 1), B_LO = !(ZERO & 2);      // which lo planes exist
+  static_assert(ZERO == 0 || MODE == TC_PLANES, "operands without a lo plane come as planes");
+  constexpr uint32_t STAGE_TX = MODE == TC_PLANES ? (uint32_t)(2 + (A_LO ? 1 : 0) + (B_LO ? 1 : 0)) * TC_PLANE_BYTES
+                                                   : (uint32_t)TC_STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *tr_base = smem + TC_STAGES * TC_STAGE_BYTES;
@@ -178,7 +188,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::prefetch_tmap(&map_a);
     ptx::prefetch_tmap(&map_b);
     ptx::prefetch_tmap(&map_blo);
-    if (PP) ptx::prefetch_tmap(&map_alo);
+    if (PP && A_LO) ptx::prefetch_tmap(&map_alo);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, TC_TMEM_COLS);
@@ -234,7 +244,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (use > 0 && !ptx::mbar_wait(&empty_bar[s], (use - 1) & 1, abort_flag)) { ok = false; break; }
           uint8_t *st = smem + s * TC_STAGE_BYTES;
           const int k0 = k_begin + kb * TC_BK;
-          ptx::mbar_expect_tx(&full_bar[s], TC_STAGE_BYTES);
+          ptx::mbar_expect_tx(&full_bar[s], STAGE_TX);
           if (MN) {
             // fp32 [64 contraction rows][128 output indices], 512-byte rows, no swizzle (only the converters read it)
             ptx::tma_load_2d(st, &map_a, m0, k0, &full_bar[s]);
@@ -242,7 +252,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else {
             if (PP) {
               ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
-              ptx::tma_load_2d(st + TC_PLANE_BYTES, &map_alo, k0, m0, &full_bar[s]);
+              if (A_LO) ptx::tma_load_2d(st + TC_PLANE_BYTES, &map_alo, k0, m0, &full_bar[s]);
             } else {
               // fp32 [128 rows][64 floats] as two 128-byte-swizzled boxes of 32 floats
               ptx::tma_load_2d(st, &map_a, k0, m0, &full_bar[s]);
@@ -250,7 +260,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             // fp16 planes of B as the MMA reads them
             ptx::tma_load_2d(st + 2 * TC_PLANE_BYTES, &map_b, k0, n0, &full_bar[s]);
-            ptx::tma_load_2d(st + 3 * TC_PLANE_BYTES, &map_blo, k0, n0, &full_bar[s]);
+            if (B_LO) ptx::tma_load_2d(st + 3 * TC_PLANE_BYTES, &map_blo, k0, n0, &full_bar[s]);
           }
         }
       }
@@ -305,8 +315,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const uint64_t dah = ptx::smem_desc(hi_b, la + kk * step_b);
               const uint64_t dal = ptx::smem_desc(hi_b, la + (TC_PLANE_BYTES >> 4) + kk * step_b);
               if (corr) {
-                ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
-                ptx::mma_f16(d_corr, dah, dbl, idesc, true);
+                // the first correction MMA of a tile overwrites the tile, every later one accumulates
+                if (A_LO) ptx::mma_f16(d_corr, dal, dbh, idesc, kb > 0 || kk > 0);
+                if (B_LO) ptx::mma_f16(d_corr, dah, dbl, idesc, A_LO || kb > 0 || kk > 0);
               }
               if (main) ptx::mma_f16(d, dah, dbh, idesc, !first || kk > 0);
             } else {
@@ -517,6 +528,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const float u1 = tc_pow2(-e1), u2 = tc_pow2(-e2);
 #pragma unroll
         for (int j = 0; j < 128; ++j) acc[j] = (acc[j] * u1) * u2;
+        if constexpr (ZERO != 0) {
+          const float mul = prm.mul;
+#pragma unroll
+          for (int j = 0; j < 128; ++j) acc[j] *= mul;
+        }
       }
       int out_tile = tile;
       if (tile >= tail_begin) {

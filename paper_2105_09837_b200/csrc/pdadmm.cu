@@ -61,6 +61,9 @@ struct Planes {
 };
 // one operand of a tensor-core product as two fp16 planes [n][ld], contiguous along the contraction index
 struct PlaneRef { const __half *hi, *lo; int ld; const int *exp; };
+// an operand that is `mul` times small integers (a quantised p = code * s, or the difference of two): one fp16 plane
+// of the integers [n][ld], no lo plane
+struct IntPlane { const __half *plane; int ld; float mul; };
 
 // Rows of every node-major matrix start on a 128-byte boundary (leading dimensions are multiples of 32 floats):
 // tile copies and the coalesced stores of the epilogues then move whole 32-byte sectors.
@@ -87,6 +90,7 @@ struct Layer {
   int *x_exp = nullptr;
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in] codes of 1 byte (up to 256 levels) or 2 bytes, quantised mode, l >= 2
+  __half *p_plane = nullptr; // [N][ld_in] the codes as fp16 integers: operand plane of p_l = code * scale (see int_operands)
   float scale = 1.0f;       // level spacing s_l of p_l
   float lo = 0.0f;          // smallest level of p_l: -(levels below zero) * s_l
   LayerScalars *sc = nullptr;
@@ -104,6 +108,7 @@ struct Scratch {
   float *p_new = nullptr;   // quantised trial
   float *d = nullptr;       // quantised trial
   uint8_t *codes_new = nullptr;
+  __half *pn_plane = nullptr, *d_plane = nullptr;   // planes of the trial's codes and of their change (see int_operands)
   float *part = nullptr;    // partial tiles of grad_W
   double *slots = nullptr;  // per-block partial sums
   size_t n_slots = 0;
@@ -178,6 +183,10 @@ struct pdadmm_ctx {
   char *arena_base = nullptr;       // current chunk
   size_t arena_cap = 0, arena_used = 0, arena_next = size_t(64) << 20;
   bool use_tc = true;               // dense products on the tensor cores
+  // pdADMM-G-Q with at most 2048 levels starting at zero: p_l = code * s_l exactly, and the codes are exact in fp16, so
+  // the products whose operand is p_l (or d = p+ - p) take one plane of integers instead of a hi and a lo plane of
+  // the values: two MMAs per product instead of three, a quarter of the operand bytes, no split pass
+  bool int_operands = false;
   cudaGraphExec_t iter_graph = nullptr;   // one captured pdADMM-G iteration (no host round trips in it)
   int64_t iter_graph_launches = 0;
   bool graph_failed = false;
@@ -327,10 +336,10 @@ static int get_tmap(pdadmm_ctx *c, const void *base, uint64_t inner, uint64_t ou
   return PDADMM_OK;
 }
 
-template <int MODE, class Epi>
+template <int MODE, class Epi, int ZERO = 0>
 static int launch_tc(pdadmm_ctx *c, cudaStream_t st, const CUtensorMap &ma, const CUtensorMap &mal, const CUtensorMap &mb,
                      const CUtensorMap &mbl, const TcParams &prm, const Epi &epi, double *partials, int n_tiles) {
-  auto kern = gemm_tc_kernel<MODE, Epi>;
+  auto kern = gemm_tc_kernel<MODE, Epi, ZERO>;
   const dim3 grid((unsigned)std::min(n_tiles, c->n_sms));
   // the attribute belongs to (kernel, device): one flag per device ordinal for this instantiation
   static bool configured[64] = {false};
@@ -421,7 +430,7 @@ template <bool B_NMAJOR, class Epi>
 static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
                       const float *B, int ldb, const PlaneRef &Bp, const Epi &epi, double *partials,
                       int *n_partials, double extra_bytes, const uint32_t *amax_a = nullptr,
-                      const PlaneRef *Ap = nullptr) {
+                      const PlaneRef *Ap = nullptr, const IntPlane *Ai = nullptr) {
   const double bytes = 4.0 * ((double)M * K + (double)N * K + (double)M * N) + extra_bytes;
   if (!c->use_tc) {
     dim3 grid((unsigned)ceil_div(N, SG_BN), (unsigned)ceil_div(M, SG_BM));
@@ -432,12 +441,15 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
   }
   const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM));
   if (n_partials) *n_partials = 4 * n_tiles;        // one slot per tile and row quarter
-  if (amax_a == nullptr) {
+  const bool a_int = Ai != nullptr && Ai->plane != nullptr;
+  if (amax_a == nullptr && !a_int) {
     PD_TRY(amax_reserve(c, st, 1));
     amax_a = amax_of(c, st, A, (size_t)M * lda / 4);
   }
   PlaneRef a_planes{nullptr, nullptr, 0, nullptr};
-  if (Ap != nullptr && Ap->hi != nullptr) {
+  if (a_int) {
+    a_planes = PlaneRef{Ai->plane, Ai->plane, Ai->ld, nullptr};
+  } else if (Ap != nullptr && Ap->hi != nullptr) {
     a_planes = *Ap;
   } else if (c->cur->a_hi != nullptr && lda % 8 == 0 && (size_t)M * lda <= c->cur->a_cap &&
              ceil_div(N, TC_BN) >= PLANES_FROM_COL_TILES) {
@@ -475,6 +487,12 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     }
   }
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
+  if constexpr (std::is_same<Epi, EpiStoreSumsq>::value) {
+    if (a_int) {
+      prm.mul = Ai->mul;
+      return launch_tc<TC_PLANES, Epi, 1>(c, st, ma, ma, mb, mbl, prm, epi, partials, n_units);
+    }
+  }
   if (pp) return launch_tc<TC_PLANES, Epi>(c, st, ma, mal, mb, mbl, prm, epi, partials, n_units);
   return launch_tc<TC_RAW_K, Epi>(c, st, ma, ma, mb, mbl, prm, epi, partials, n_units);
 }
@@ -490,17 +508,23 @@ static void transpose_planes(pdadmm_ctx *c, cudaStream_t st, const float *x, int
 
 // C parts [n_split][M][ldc] = A^T B over node slices, both operands given by their transposed planes:
 // A^T = [M][K nodes], B^T = [N][K nodes]
+// b_mul > 0: B^T is one plane of integers (Bt.hi; the transposed codes of a quantised p) times b_mul
 static int gemm_over_nodes_tc(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const PlaneRef &At,
-                              const PlaneRef &Bt, float *part, int ldc, int k_chunk, int n_split) {
+                              const PlaneRef &Bt, float *part, int ldc, int k_chunk, int n_split, float b_mul = 0.f) {
   const int n_tiles = (int)(ceil_div(N, TC_BN) * ceil_div(M, TC_BM)) * n_split;
   CUtensorMap ma, mal, mb, mbl;
   PD_TRY(get_tmap(c, At.hi, (uint64_t)K, (uint64_t)M, (uint64_t)At.ld, TM_PLANE, &ma));
   PD_TRY(get_tmap(c, At.lo, (uint64_t)K, (uint64_t)M, (uint64_t)At.ld, TM_PLANE, &mal));
   PD_TRY(get_tmap(c, Bt.hi, (uint64_t)K, (uint64_t)N, (uint64_t)Bt.ld, TM_PLANE, &mb));
-  PD_TRY(get_tmap(c, Bt.lo, (uint64_t)K, (uint64_t)N, (uint64_t)Bt.ld, TM_PLANE, &mbl));
-  TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1, nullptr, nullptr, At.exp, Bt.exp};
+  if (b_mul > 0.f) mbl = mb;
+  else PD_TRY(get_tmap(c, Bt.lo, (uint64_t)K, (uint64_t)N, (uint64_t)Bt.ld, TM_PLANE, &mbl));
+  TcParams prm{M, N, K, k_chunk, n_split, (size_t)M * ldc, c->d_flag + 1, nullptr, nullptr, At.exp, b_mul > 0.f ? nullptr : Bt.exp};
   EpiStore epi{part, ldc};
   Launch k(c, cls, st, 4.0 * ((double)K * N + (double)K * M), 2.0 * K * N * M);
+  if (b_mul > 0.f) {
+    prm.mul = b_mul;
+    return launch_tc<TC_PLANES, EpiStore, 2>(c, st, ma, mal, mb, mb, prm, epi, nullptr, n_tiles);
+  }
   return launch_tc<TC_PLANES, EpiStore>(c, st, ma, mal, mb, mbl, prm, epi, nullptr, n_tiles);
 }
 
@@ -631,13 +655,15 @@ static int q_trial(pdadmm_ctx *c, int l) {
     Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
     quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
                                                      s.codes_new, c->code_bytes == 2, n4p, s.slots,
-                                                     c->use_tc ? ly.amax_p : nullptr, w_d);
+                                                     c->use_tc ? ly.amax_p : nullptr, w_d,
+                                                     c->int_operands ? ly.codes : nullptr, s.pn_plane, s.d_plane);
   }
   int np = 0;
   double *slots_b = s.slots + s.n_slots / 2;
   EpiStoreSumsq epi{s.s2, ly.ld_out};
+  const IntPlane di{c->int_operands ? s.d_plane : nullptr, ly.ld_in, ly.scale};      // d = (new code - old code) s
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, planes_W(ly), epi,
-                           slots_b, &np, 0, w_d));
+                           slots_b, &np, 0, w_d, nullptr, &di));
   if (c->reduce != nullptr) {
     PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, grid, slots_b, np));
     finalize_trial_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.red, 1, s.red + 1, 1);
@@ -666,6 +692,7 @@ static int q_finish(pdadmm_ctx *c, int l, bool *hit_cap) {
   }
   std::swap(ly.p, s.p_new);
   std::swap(ly.codes, s.codes_new);
+  std::swap(ly.p_plane, s.pn_plane);
   {
     Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_out, 0);
     add_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, n4r, ly.amax_r);
@@ -690,12 +717,20 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
     if (planes_beforehand(ly.n_out, ly.n_in, l == 0)) {
       transpose_planes(c, s.st, ly.r, N, ly.n_out, ly.ld_out, ly.amax_r, s.rT_hi, s.rT_lo, c->ldT, s.rT_exp);
       PlaneRef Bt{s.pT_hi, s.pT_lo, c->ldT, s.pT_exp};
-      if (l == 0)          // p_1 = X never changes: its planes are kept (made before the first iteration)
+      float b_mul = 0.f;
+      if (l == 0) {        // p_1 = X never changes: its planes are kept (made before the first iteration)
         Bt = PlaneRef{ly.xT_hi, ly.xT_lo, c->ldT, ly.xT_exp};
-      else
+      } else if (c->int_operands) {
+        // p+ = code * s: the transposed codes are the whole operand (1 byte read, 2 written per element instead of 4 + 4)
+        Launch k(c, KC_PLANES, s.st, 3.0 * N * ly.n_in, 0);
+        const dim3 grid((unsigned)ceil_div(ly.n_in, 32), (unsigned)ceil_div(N, 32));
+        transpose_codes_kernel<<<grid, dim3(32, 8), 0, s.st>>>(ly.codes, c->code_bytes == 2, N, ly.n_in, ly.ld_in, s.pT_hi, c->ldT);
+        b_mul = ly.scale;
+      } else {
         transpose_planes(c, s.st, ly.p, N, ly.n_in, ly.ld_in, ly.amax_p, s.pT_hi, s.pT_lo, c->ldT, s.pT_exp);
+      }
       PD_TRY(gemm_over_nodes_tc(c, KC_GEMM_GRADW, s.st, ly.n_out, ly.n_in, N,
-                                PlaneRef{s.rT_hi, s.rT_lo, c->ldT, s.rT_exp}, Bt, s.part, ly.ld_in, ly.k_chunk, ly.n_split));
+                                PlaneRef{s.rT_hi, s.rT_lo, c->ldT, s.rT_exp}, Bt, s.part, ly.ld_in, ly.k_chunk, ly.n_split, b_mul));
     } else {
       PD_TRY(gemm_over_nodes_raw(c, KC_GEMM_GRADW, s.st, ly.n_out, ly.n_in, N, ly.r, ly.ld_out, ly.p, ly.ld_in, s.part,
                                  ly.ld_in, ly.k_chunk, ly.n_split, ly.amax_r, ly.amax_p));
@@ -720,8 +755,9 @@ static int w_and_b_step(pdadmm_ctx *c, int l) {
   double *slots_b = s.slots + s.n_slots / 2;
   EpiStoreSumsq epi{s.s1, ly.ld_out};
   const PlaneRef xp = planes_X(ly);
+  const IntPlane pi{(c->int_operands && l > 0) ? ly.p_plane : nullptr, ly.ld_in, ly.scale};          // p+ = code * s
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_GP, s.st, N, ly.n_out, ly.n_in, ly.p, ly.ld_in, ly.gradW, ly.ld_in, planes_G(ly),
-                           epi, slots_b, &np, 0, ly.amax_p, &xp));
+                           epi, slots_b, &np, 0, ly.amax_p, &xp, &pi));
   if (c->reduce != nullptr) {
     // ||G p+||^2 is a sum over nodes (||G||^2 is the same on every shard already)
     PD_TRY(shard_sum_slots(c, s.st, s.red, slots_b, np, nullptr, 0));
@@ -981,6 +1017,10 @@ static int alloc_trial_buffers(pdadmm_ctx *c, Scratch &s, size_t n) {
   PD_TRY(dev_alloc(c, &s.p_new, n));
   PD_TRY(dev_alloc(c, &s.d, n));
   PD_TRY(dev_alloc(c, &s.codes_new, n * c->code_bytes));
+  if (c->int_operands) {
+    PD_TRY(dev_alloc(c, &s.pn_plane, n));
+    PD_TRY(dev_alloc(c, &s.d_plane, n));
+  }
   PD_CUDA(cudaMallocHost((void **)&s.h_flag, sizeof(int)));
   PD_CUDA(cudaEventCreateWithFlags(&s.ev_flag, cudaEventDisableTiming));
   return PDADMM_OK;
@@ -1056,6 +1096,7 @@ static int feasible_start(pdadmm_ctx *c, int first) {
       nx.lo = -(float)c->neg_levels * nx.scale;
       quantize_kernel<<<ew_grid(n4 * 4), EW_THREADS, 0, st>>>(ly.q, n4 * 4, nx.scale, nx.lo, c->levels, nx.p, nx.codes,
                                                               c->code_bytes == 2);
+      if (c->int_operands) codes_to_plane_kernel<<<ew_grid(n4), EW_THREADS, 0, st>>>(nx.codes, c->code_bytes == 2, n4, nx.p_plane);
       if (c->quant_q)      // start inside the level set: q_l = p_{l+1}
         PD_CUDA(cudaMemcpyAsync(ly.q, nx.p, n4 * 16, cudaMemcpyDeviceToDevice, st));
     } else {
@@ -1087,6 +1128,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
   c->ls_risk = (cfg->flags & PDADMM_FLAG_LEAST_SQUARES) != 0;
   c->rho = cfg->rho; c->nu = cfg->nu; c->flags = cfg->flags;
   c->use_tc = (cfg->flags & PDADMM_FLAG_SIMT_GEMM) == 0;
+  c->int_operands = c->use_tc && c->levels >= 2 && c->levels <= 2048 && c->neg_levels == 0;
   PD_CUDA(cudaSetDevice(cfg->device));
   PD_CUDA(cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, cfg->device));
   PD_CUDA(cudaStreamCreateWithFlags(&c->scr.st, cudaStreamNonBlocking));
@@ -1147,6 +1189,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
     PD_TRY(dev_alloc(c, &ly.r, e_out));
     if (l + 1 < c->L) { PD_TRY(dev_alloc(c, &ly.q, e_out)); PD_TRY(dev_alloc(c, &ly.u, e_out)); }
     if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in * c->code_bytes));
+    if (c->int_operands && l > 0) PD_TRY(dev_alloc(c, &ly.p_plane, e_in));
     if (l > 0) PD_TRY(dev_alloc(c, &ly.t, (size_t)N * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.sc, 1));
     PD_TRY(dev_alloc(c, &ly.amax_p, 1));
@@ -1670,6 +1713,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
     const size_t n = (size_t)c->N * y.ld_in;
     quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, y.lo, c->levels, nullptr, y.codes,
                                                               c->code_bytes == 2);
+    if (c->int_operands) codes_to_plane_kernel<<<ew_grid(n / 4), EW_THREADS, 0, c->scr.st>>>(y.codes, c->code_bytes == 2, n / 4, y.p_plane);
     PD_CUDA(cudaStreamSynchronize(c->scr.st));
   }
   return PDADMM_OK;
