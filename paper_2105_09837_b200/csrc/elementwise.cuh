@@ -382,7 +382,8 @@ rows_planes_kernel(const float *__restrict__ x, size_t n8, const uint32_t *__res
       return *reinterpret_cast<const uint32_t *>(&t);
     };
     reinterpret_cast<uint4 *>(hi)[i] = make_uint4(pack(h[0], h[1]), pack(h[2], h[3]), pack(h[4], h[5]), pack(h[6], h[7]));
-    reinterpret_cast<uint4 *>(lo)[i] = make_uint4(pack(l[0], l[1]), pack(l[2], l[3]), pack(l[4], l[5]), pack(l[6], l[7]));
+    if (lo != nullptr)        // a product that only wants its squared norm uses the hi plane alone
+      reinterpret_cast<uint4 *>(lo)[i] = make_uint4(pack(l[0], l[1]), pack(l[2], l[3]), pack(l[4], l[5]), pack(l[6], l[7]));
   }
 }
 

@@ -143,10 +143,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_blo,
                const TcParams prm, Epi epi, double *__restrict__ partials) {
   constexpr bool PP = MODE == TC_PLANES, MN = MODE == TC_RAW_MN, COARSE = epi_coarse<Epi>::value || ZERO == 3;
-  constexpr bool A_LO = !(ZERO & 1), B_LO = !(ZERO & 2);      // which lo planes exist
+  // which lo planes are loaded and used (a product that only wants its squared norm uses neither, and lets the main
+  // term accumulate in tensor memory over the whole contraction: the truncation of that accumulation, 1e-5 relative,
+  // does not matter to a norm that only starts a search)
+  constexpr bool A_LO = !(ZERO & 1) && !COARSE, B_LO = !(ZERO & 2) && !COARSE;
+  constexpr int FLUSH = COARSE ? (1 << 30) : TC_FLUSH;        // K blocks per read-out of the main accumulator
   static_assert(ZERO == 0 || MODE == TC_PLANES, "operands without a lo plane come as planes");
   constexpr uint32_t STAGE_TX = MODE == TC_PLANES ? (uint32_t)(2 + (A_LO ? 1 : 0) + (B_LO ? 1 : 0)) * TC_PLANE_BYTES
-                                                   : (uint32_t)TC_STAGE_BYTES;
+                              : MODE == TC_RAW_K  ? (uint32_t)(3 + (B_LO ? 1 : 0)) * TC_PLANE_BYTES
+                                                  : (uint32_t)TC_STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *tr_base = smem + TC_STAGES * TC_STAGE_BYTES;
@@ -292,7 +297,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int m0, n0, k_begin, n_kb, z;
         tile_coords(tile, m0, n0, k_begin, n_kb, z);
         for (int kb = 0; kb < n_kb && ok; ++kb) {
-          const bool first = kb % TC_FLUSH == 0, last = kb % TC_FLUSH == TC_FLUSH - 1 || kb == n_kb - 1;
+          const bool first = kb % FLUSH == 0, last = kb % FLUSH == FLUSH - 1 || kb == n_kb - 1;
           if (!seen_conv) ok = ptx::mbar_wait(&ready_bar[s], sp, abort_flag);
           if (ok && first && !first_round && !seen_acc) ok = ptx::mbar_wait(&acc_empty[b], bp, abort_flag);
           if (!ok) break;
@@ -431,7 +436,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const uint32_t col = tmem_base + ((uint32_t)(quarter * 32) << 16) + TC_COL_A + (uint32_t)aslot * 64u +
                                    16u * (uint32_t)half;
               ptx::tmem_st16(col, hreg);
-              ptx::tmem_st16(col + 32u, lreg);
+              if constexpr (!COARSE) ptx::tmem_st16(col + 32u, lreg);
             }
           }
           if constexpr (MN) {
@@ -483,7 +488,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++ti) {
       int m0, n0, k_begin, n_kb, z;
       tile_coords(tile, m0, n0, k_begin, n_kb, z);
-      if ((ti & 1) != set) { it += n_kb; continue; }     // the other set's tile
+      const int n_grp = COARSE ? (n_kb > 0 ? 1 : 0) : n_kb;   // read-outs of the main accumulator for this tile
+      if ((ti & 1) != set) { it += n_grp; continue; }    // the other set's tile
       if (m0 + lane_base + lane < prm.M) {          // this thread's row of the epilogue inputs, on its way to L2
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
@@ -505,7 +511,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int j = 0; j < 32; ++j) acc[32 * h + j] = fmaf(w, __uint_as_float(v[j]), acc[32 * h + j]);
         }
       };
-      for (int g = 0; g < n_kb && ok; ++g, ++it) {
+      for (int g = 0; g < n_grp && ok; ++g, ++it) {
         const int b = it % TC_ACC_BUFS;
         ok = ptx::mbar_wait(&acc_full[set * TC_ACC_BUFS + b], (b ? uses1 : uses0) & 1u, abort_flag);
         if (!ok) break;

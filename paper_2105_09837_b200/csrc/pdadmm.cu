@@ -455,8 +455,9 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
              ceil_div(N, TC_BN) >= PLANES_FROM_COL_TILES) {
     Scratch &sc = *c->cur;
     const size_t n8 = (size_t)M * lda / 8;
-    Launch l(c, KC_PLANES, st, 8.0 * M * K, 0);
-    rows_planes_kernel<<<ew_grid(n8), 256, 0, st>>>(A, n8, amax_a, sc.a_exp, sc.a_hi, sc.a_lo);
+    constexpr bool coarse = epi_coarse<Epi>::value;
+    Launch l(c, KC_PLANES, st, (coarse ? 6.0 : 8.0) * M * K, 0);
+    rows_planes_kernel<<<ew_grid(n8), 256, 0, st>>>(A, n8, amax_a, sc.a_exp, sc.a_hi, coarse ? nullptr : sc.a_lo);
     a_planes = PlaneRef{sc.a_hi, sc.a_lo, lda, sc.a_exp};
   }
   const bool pp = a_planes.hi != nullptr;
