@@ -424,7 +424,8 @@ static int alloc_planes(pdadmm_ctx *c, int rows, int cols, bool transposed_too, 
 // 2640 cycles per 64-deep K block against 1610 with both operands as planes); beforehand costs one pass of
 // 8 bytes per element at HBM speed.  Measured per product (split pass included): 4 column tiles 69 against 58 us,
 // 8 tiles 1.18 against 1.21 ms, 16 tiles 2.42 against 2.29 ms -- beforehand wins from 16 column tiles on, and
-// always where the planes are kept (X).
+// always where the planes are kept (X).  The norm-only product needs the hi plane alone (6 bytes per element) and
+// wins from 8 column tiles on (workload c4: 9.42 -> 9.74 iterations/s).
 constexpr int PLANES_FROM_COL_TILES = 16;
 template <bool B_NMAJOR, class Epi>
 static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int K, const float *A, int lda,
@@ -452,7 +453,7 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
   } else if (Ap != nullptr && Ap->hi != nullptr) {
     a_planes = *Ap;
   } else if (c->cur->a_hi != nullptr && lda % 8 == 0 && (size_t)M * lda <= c->cur->a_cap &&
-             ceil_div(N, TC_BN) >= PLANES_FROM_COL_TILES) {
+             (ceil_div(N, TC_BN) >= PLANES_FROM_COL_TILES || (epi_coarse<Epi>::value && ceil_div(N, TC_BN) >= PLANES_FROM_COL_TILES / 2))) {
     Scratch &sc = *c->cur;
     const size_t n8 = (size_t)M * lda / 8;
     constexpr bool coarse = epi_coarse<Epi>::value;
@@ -1244,6 +1245,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
     bool want_row_planes = false;
     for (int l = 0; l < c->L; ++l)
       want_row_planes |= std::max(ceil_div(c->layers[l].n_out, TC_BN), l > 0 ? ceil_div(c->layers[l].n_in, TC_BN) : 0) >= PLANES_FROM_COL_TILES;
+    want_row_planes |= c->levels > 0;       // the norm-only product of the quantised update always takes a hi plane
     if (want_row_planes) PD_TRY(alloc_row_planes(c, s, e_max));
     Layer &l0 = c->layers[0];
     if (ceil_div(l0.n_out, TC_BN) >= 2) {      // X is split once for ever: worth it from two column tiles on
