@@ -200,6 +200,7 @@ def _compare_iteration(ctx, prev, prm, label, tensor_cores=True, report=None, si
 @pytest.mark.parametrize("case,levels,flags", [
     ("er-small", 0, 0), ("ba-ragged", 0, 0), ("ba-wide", 0, 0), ("c4-like", 0, 0),
     ("er-small", 16, 0), ("ba-ragged", 256, 0), ("c4-like", 256, 0),
+    ("ba-wide", 1024, 0),          # 16-bit codes that are still exact in one fp16 plane (integer operands)
     ("ba-ragged", 0, B.FLAG_SIMT_GEMM), ("ba-ragged", 256, B.FLAG_SIMT_GEMM),
 ])
 def test_teacher_forced_iterations(case, levels, flags):
