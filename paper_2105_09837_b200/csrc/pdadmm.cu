@@ -654,7 +654,8 @@ static int q_trial(pdadmm_ctx *c, int l) {
   uint32_t *w_d = nullptr;               // max|d| of this trial
   if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_d = amax_take(c); }
   {
-    Launch k(c, KC_QUANT, s.st, 17.0 * N * ly.n_in, 0);
+    // reads p, g (and the old code); writes p+, d, the code (and the two integer planes)
+    Launch k(c, KC_QUANT, s.st, (c->int_operands ? 22.0 : 17.0) * N * ly.n_in, 0);
     quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
                                                      s.codes_new, c->code_bytes == 2, n4p, s.slots,
                                                      c->use_tc ? ly.amax_p : nullptr, w_d,
