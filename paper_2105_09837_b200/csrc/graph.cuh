@@ -183,10 +183,11 @@ spmm_kernel(const int *__restrict__ row_ptr, const int *__restrict__ col_idx, co
       for (int v = 0; v < VEC; ++v) acc[ch][v] = 0.f;
     for (int k0 = b; k0 < e; k0 += 32) {
       const int n = min(32, e - k0);
-      const int my_col = lane < n ? __ldg(col_idx + k0 + lane) : 0;
+      // lanes past the end of the row repeat the chunk's first entry with the value 0: nothing is read that the row
+      // does not read anyway
+      const int my_col = __ldg(col_idx + k0 + (lane < n ? lane : 0));
       const float my_val = lane < n ? __ldg(val + k0 + lane) : 0.f;
-      // four neighbours at a time: their loads are independent (an entry past the end of the row repeats the first
-      // of the four with the value 0, so it reads nothing that the row does not read anyway)
+      // four neighbours at a time: their loads are independent
       for (int j = 0; j < n; j += 4) {
         float a[4];
         const float *xr[4];
@@ -194,7 +195,6 @@ spmm_kernel(const int *__restrict__ row_ptr, const int *__restrict__ col_idx, co
         for (int t = 0; t < 4; ++t) {
           a[t] = __shfl_sync(0xffffffffu, my_val, (j + t) & 31);
           xr[t] = X + (size_t)__shfl_sync(0xffffffffu, my_col, (j + t) & 31) * ld;
-          if (j + t >= n) { a[t] = 0.f; xr[t] = xr[0]; }
         }
 #pragma unroll
         for (int ch = 0; ch < SPMM_CH; ++ch) {
