@@ -205,7 +205,10 @@ int pdadmm_predict(pdadmm_ctx *ctx, float *logits_out, int32_t *pred_out, int64_
  * exactly `bytes` bytes (dense, without the device's row padding).  Together they are the
  * checkpoint / resume interface.  Setting P, W, B or Z invalidates the cached linear residual
  * W p + b - z, which the next step recomputes.  Setting P in pdADMM-G-Q mode expects values on the
- * level set; CODES are recomputed from them.  EINVAL for a bad kind/layer/size or a get-only kind.
+ * level set: CODES are recomputed from them and P becomes the levels of those codes (the same bits for
+ * values on the level set; the kernels read p_l through its codes).  Setting QSCALE of a layer moves its
+ * p_l to the new level set in the same way, so set QSCALE before P.  EINVAL for a bad kind/layer/size or a
+ * get-only kind.
  */
 int pdadmm_get_tensor(pdadmm_ctx *ctx, int kind, int layer, void *host_dst, size_t bytes);
 int pdadmm_set_tensor(pdadmm_ctx *ctx, int kind, int layer, const void *host_src, size_t bytes);

@@ -75,6 +75,21 @@ __device__ __forceinline__ float quantize_one(float x, float s, float lo, float 
   return __fadd_rn(lo, __fmul_rn(c, s));
 }
 
+// Four consecutive values of a quantised matrix from its codes: lo + code * s, rounded as quantize_one rounds them,
+// i.e. bit for bit the stored values (1 or 2 bytes read per value instead of 4).
+__device__ __forceinline__ float4 levels_of4(const void *__restrict__ codes, int wide_codes, size_t i, float s, float lo) {
+  float c0, c1, c2, c3;
+  if (wide_codes) {
+    const ushort4 o = reinterpret_cast<const ushort4 *>(codes)[i];
+    c0 = o.x; c1 = o.y; c2 = o.z; c3 = o.w;
+  } else {
+    const uchar4 o = reinterpret_cast<const uchar4 *>(codes)[i];
+    c0 = o.x; c1 = o.y; c2 = o.z; c3 = o.w;
+  }
+  return make_float4(__fadd_rn(lo, __fmul_rn(c0, s)), __fadd_rn(lo, __fmul_rn(c1, s)), __fadd_rn(lo, __fmul_rn(c2, s)),
+                     __fadd_rn(lo, __fmul_rn(c3, s)));
+}
+
 // ---- y -= x * (*inv) ----------------------------------------------------------------------------
 // p-update  p+ = p - g/tau  (Eq. "update p") and the matching update of the linear residual,
 // r <- r - (W g)/tau, and r <- r - (grad_W p+)/theta after the W-update (Eq. "update W").
@@ -124,12 +139,14 @@ add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4, uint32
 
 // ---- quantised trial step ------------------------------------------------------------------------
 // x = p - g/tau; p_new = nearest level; d = p_new - p; codes; per-block sum of d^2.
+// p lies on the level set, p = lo + code * scale bit for bit (quantize_one), so it is read as its 1- or 2-byte codes
+// instead of as 4-byte values.
 __global__ void __launch_bounds__(EW_THREADS)
-quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, const LayerScalars *__restrict__ sc,
-                   float scale, float lo, int levels, float *__restrict__ p_new, float *__restrict__ d,
+quant_trial_kernel(const float *__restrict__ g, const LayerScalars *__restrict__ sc,
+                   float scale, float lo, int levels, float *__restrict__ p_new, float *__restrict__ d /* may be null */,
                    void *__restrict__ codes, int wide_codes, size_t n4, double *__restrict__ slots,
                    uint32_t *__restrict__ amax_p /* max|p_new|, may be null */, uint32_t *__restrict__ amax_d /* max|d| */,
-                   const void *__restrict__ codes_old /* codes of p; with the two planes below, else null */,
+                   const void *__restrict__ codes_old /* codes of p */,
                    __half *__restrict__ pn_plane /* the new codes as fp16 integers (operand plane of p_new = code * scale) */,
                    __half *__restrict__ d_plane /* new code - old code as fp16 integers (operand plane of d) */) {
   __shared__ double red[EW_THREADS / 32];
@@ -137,7 +154,17 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
   double ss = 0.0;
   uint32_t mp = 0u, md = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
-    const float4 pv = ld4(p, i), gv = ld4(g, i);
+    const float4 gv = ld4(g, i);
+    int o0, o1, o2, o3;
+    if (wide_codes) {
+      const ushort4 o = reinterpret_cast<const ushort4 *>(codes_old)[i];
+      o0 = o.x; o1 = o.y; o2 = o.z; o3 = o.w;
+    } else {
+      const uchar4 o = reinterpret_cast<const uchar4 *>(codes_old)[i];
+      o0 = o.x; o1 = o.y; o2 = o.z; o3 = o.w;
+    }
+    const float4 pv = make_float4(__fadd_rn(lo, __fmul_rn((float)o0, scale)), __fadd_rn(lo, __fmul_rn((float)o1, scale)),
+                                  __fadd_rn(lo, __fmul_rn((float)o2, scale)), __fadd_rn(lo, __fmul_rn((float)o3, scale)));
     unsigned c0, c1, c2, c3;
     float4 nv, dv;
     nv.x = quantize_one(fmaf(-inv_tau, gv.x, pv.x), scale, lo, top, c0);
@@ -147,7 +174,7 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
     dv.x = nv.x - pv.x; dv.y = nv.y - pv.y; dv.z = nv.z - pv.z; dv.w = nv.w - pv.w;
     ss += (double)dv.x * dv.x + (double)dv.y * dv.y + (double)dv.z * dv.z + (double)dv.w * dv.w;
     st4(p_new, i, nv);
-    st4(d, i, dv);
+    if (d != nullptr) st4(d, i, dv);     // with the integer planes below the product W d reads d_plane instead
     mp = max(mp, abs_bits(nv)); md = max(md, abs_bits(dv));
     if (wide_codes)      // more than 256 levels: 16-bit codes
       reinterpret_cast<ushort4 *>(codes)[i] = make_ushort4((unsigned short)c0, (unsigned short)c1, (unsigned short)c2, (unsigned short)c3);
@@ -155,14 +182,6 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
       reinterpret_cast<uchar4 *>(codes)[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
     if (pn_plane != nullptr) {
       // integers below 2048 are exact in fp16: the planes hold the codes themselves and their change
-      int o0, o1, o2, o3;
-      if (wide_codes) {
-        const ushort4 o = reinterpret_cast<const ushort4 *>(codes_old)[i];
-        o0 = o.x; o1 = o.y; o2 = o.z; o3 = o.w;
-      } else {
-        const uchar4 o = reinterpret_cast<const uchar4 *>(codes_old)[i];
-        o0 = o.x; o1 = o.y; o2 = o.z; o3 = o.w;
-      }
       const __half2 a = __floats2half2_rn((float)c0, (float)c1), b = __floats2half2_rn((float)c2, (float)c3);
       const __half2 e = __floats2half2_rn((float)((int)c0 - o0), (float)((int)c1 - o1));
       const __half2 f = __floats2half2_rn((float)((int)c2 - o2), (float)((int)c3 - o3));
@@ -177,7 +196,7 @@ quant_trial_kernel(const float *__restrict__ p, const float *__restrict__ g, con
 
 // Plain projection of an array (initial forward pass, pdadmm_quantize, pdadmm_set_tensor).
 __global__ void __launch_bounds__(EW_THREADS)
-quantize_kernel(const float *__restrict__ x, size_t n, float scale, float lo, int levels, float *__restrict__ p_out,
+quantize_kernel(const float *x, size_t n, float scale, float lo, int levels, float *p_out /* may be x itself */,
                 void *__restrict__ codes_out, int wide_codes) {
   const float top = (float)(levels - 1);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -571,14 +590,16 @@ __global__ void __launch_bounds__(EW_THREADS)
 zqu_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
            const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
            float rho, float nu, float slope, float q_scale, float q_lo, float q_top, float *__restrict__ t_next,
-           double *__restrict__ slots, uint32_t *__restrict__ amax_r /* max|r| (see commit_amax); may be null */) {
+           double *__restrict__ slots, uint32_t *__restrict__ amax_r /* max|r| (see commit_amax); may be null */,
+           const void *__restrict__ codes_next = nullptr /* pdADMM-G-Q: codes of p_next, read instead of it */, int wide_codes = 0) {
   __shared__ double red[EW_THREADS / 32];
   const float inv_rn = 1.0f / (rho + nu), inv_neg = 1.0f / (2.0f + slope * slope);
   double ss = 0.0;
   uint32_t mr = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 sh = ld4(shift, i % ld4cols);
-    const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i), pv = ld4(p_next, i);
+    const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i);
+    const float4 pv = codes_next != nullptr ? levels_of4(codes_next, wide_codes, i, q_scale, q_lo) : ld4(p_next, i);
     float4 zn, qn, un, rn, tn;
 #define PD_ZQU(f)                                                                   \
     {                                                                               \
@@ -615,7 +636,8 @@ __global__ void __launch_bounds__(EW_THREADS)
 zqu_table_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict__ q, float *__restrict__ u,
                  const float *__restrict__ p_next, const float *__restrict__ shift, int ld4cols, size_t n4,
                  float rho, float nu, float act, float t_lo, float t_step, int T, float q_scale, float q_lo, float q_top,
-                 float *__restrict__ t_next, double *__restrict__ slots, uint32_t *__restrict__ amax_r) {
+                 float *__restrict__ t_next, double *__restrict__ slots, uint32_t *__restrict__ amax_r,
+                 const void *__restrict__ codes_next = nullptr, int wide_codes = 0) {
   extern __shared__ float table_sh[];              // z_i, then f(z_i)
   __shared__ double red[EW_THREADS / 32];
   for (int i = threadIdx.x; i < T; i += blockDim.x) {
@@ -629,7 +651,8 @@ zqu_table_kernel(float *__restrict__ r, float *__restrict__ z, float *__restrict
   uint32_t mr = 0u;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float4 sh = ld4(shift, i % ld4cols);
-    const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i), pv = ld4(p_next, i);
+    const float4 rv = ld4(r, i), zv = ld4(z, i), qv = ld4(q, i), uv = ld4(u, i);
+    const float4 pv = codes_next != nullptr ? levels_of4(codes_next, wide_codes, i, q_scale, q_lo) : ld4(p_next, i);
     const float a[4] = {(rv.x - sh.x) + zv.x, (rv.y - sh.y) + zv.y, (rv.z - sh.z) + zv.z, (rv.w - sh.w) + zv.w};
     const float zo[4] = {zv.x, zv.y, zv.z, zv.w}, qo[4] = {qv.x, qv.y, qv.z, qv.w};
     float best[4] = {3.0e38f, 3.0e38f, 3.0e38f, 3.0e38f}, zb[4] = {0.f, 0.f, 0.f, 0.f}, fb[4] = {0.f, 0.f, 0.f, 0.f};

@@ -654,12 +654,14 @@ static int q_trial(pdadmm_ctx *c, int l) {
   uint32_t *w_d = nullptr;               // max|d| of this trial
   if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_d = amax_take(c); }
   {
-    // reads p, g (and the old code); writes p+, d, the code (and the two integer planes)
-    Launch k(c, KC_QUANT, s.st, (c->int_operands ? 22.0 : 17.0) * N * ly.n_in, 0);
-    quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.p, s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new, s.d,
+    // reads g and the codes of p; writes p+, the new codes and d -- as fp32, or, with integer operands, as the two
+    // fp16 planes of integers: 14 bytes per element with one-byte codes either way
+    Launch k(c, KC_QUANT, s.st, 14.0 * N * ly.n_in, 0);
+    quant_trial_kernel<<<grid, EW_THREADS, 0, s.st>>>(s.s1, ly.sc, ly.scale, ly.lo, c->levels, s.p_new,
+                                                     c->int_operands ? nullptr : s.d,
                                                      s.codes_new, c->code_bytes == 2, n4p, s.slots,
                                                      c->use_tc ? ly.amax_p : nullptr, w_d,
-                                                     c->int_operands ? ly.codes : nullptr, s.pn_plane, s.d_plane);
+                                                     ly.codes, s.pn_plane, s.d_plane);
   }
   int np = 0;
   double *slots_b = s.slots + s.n_slots / 2;
@@ -809,17 +811,18 @@ static void zqu_step(pdadmm_ctx *c, int l) {
     const size_t n4 = (size_t)N * ly.ld_out / 4;
     const int grid = ew_grid(n4);
     if (c->table_size > 0) {
-      Launch k(c, KC_ZQU, s.st, 40.0 * N * ly.n_out, 0);
+      Launch k(c, KC_ZQU, s.st, (c->levels ? 37.0 : 40.0) * N * ly.n_out, 0);
       const Layer &nx = c->layers[l + 1];
       zqu_table_kernel<<<grid, EW_THREADS, 2 * c->table_size * sizeof(float), s.st>>>(
           ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu, c->slope, c->table_lo, c->table_step,
-          c->table_size, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, nx.t, s.slots, ly.amax_r);
+          c->table_size, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, nx.t, s.slots, ly.amax_r,
+          c->levels ? nx.codes : nullptr, c->code_bytes == 2);
     } else {
-      Launch k(c, KC_ZQU, s.st, 40.0 * N * ly.n_out, 0);
+      Launch k(c, KC_ZQU, s.st, (c->levels ? 37.0 : 40.0) * N * ly.n_out, 0);      // p_{l+1} as one-byte codes
       const Layer &nx = c->layers[l + 1];
       zqu_kernel<<<grid, EW_THREADS, 0, s.st>>>(ly.r, ly.z, ly.q, ly.u, nx.p, ly.shift, ly.ld_out / 4, n4, c->rho, c->nu,
                                                c->slope, nx.scale, nx.lo, c->quant_q ? (float)(c->levels - 1) : -1.0f, nx.t,
-                                               s.slots, ly.amax_r);
+                                               s.slots, ly.amax_r, c->levels ? nx.codes : nullptr, c->code_bytes == 2);
     }
   } else {
     Launch k(c, KC_ZLAST, s.st, 16.0 * N * ly.n_out, 0);
@@ -1018,7 +1021,7 @@ static int build_csr(pdadmm_ctx *c, const pdadmm_config *cfg) {
 // trial is taken, so all have one size), the pinned word and the event of the accept flag
 static int alloc_trial_buffers(pdadmm_ctx *c, Scratch &s, size_t n) {
   PD_TRY(dev_alloc(c, &s.p_new, n));
-  PD_TRY(dev_alloc(c, &s.d, n));
+  if (!c->int_operands) PD_TRY(dev_alloc(c, &s.d, n));       // with integer operands d exists as d_plane only
   PD_TRY(dev_alloc(c, &s.codes_new, n * c->code_bytes));
   if (c->int_operands) {
     PD_TRY(dev_alloc(c, &s.pn_plane, n));
@@ -1685,6 +1688,21 @@ extern "C" int pdadmm_get_tensor(pdadmm_ctx *c, int kind, int layer, void *host_
   return PDADMM_OK;
 }
 
+// pdADMM-G-Q: the kernels read p_l (l >= 2, paper numbering) as its codes, so the two must always agree: the codes
+// are taken from p_l and p_l becomes the levels of those codes (the same bits if it was on the level set already).
+static int project_p_on_its_levels(pdadmm_ctx *c, int layer) {
+  Layer &y = c->layers[layer - 1];
+  const size_t n = (size_t)c->N * y.ld_in;
+  quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, y.lo, c->levels, y.p, y.codes, c->code_bytes == 2);
+  if (c->int_operands) codes_to_plane_kernel<<<ew_grid(n / 4), EW_THREADS, 0, c->scr.st>>>(y.codes, c->code_bytes == 2, n / 4, y.p_plane);
+  PD_CUDA(cudaGetLastError());
+  PD_CUDA(cudaStreamSynchronize(c->scr.st));
+  c->r_valid = false;
+  c->amax_p_valid = false;
+  c->t_valid = false;
+  return PDADMM_OK;
+}
+
 extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void *host_src, size_t bytes) {
   if (!c || !host_src) return fail(PDADMM_EINVAL, "null argument");
   PD_CUDA(cudaSetDevice(c->device));
@@ -1695,6 +1713,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
     if (!(v > 0.f)) return fail(PDADMM_EINVAL, "QSCALE must be positive");
     c->layers[layer - 1].scale = v;
     c->layers[layer - 1].lo = -(float)c->neg_levels * v;
+    if (c->levels) PD_TRY(project_p_on_its_levels(c, layer));       // p_l moves to the new level set
     return PDADMM_OK;
   }
   TensorRef t;
@@ -1712,14 +1731,7 @@ extern "C" int pdadmm_set_tensor(pdadmm_ctx *c, int kind, int layer, const void 
   if (kind == PDADMM_T_X || kind == PDADMM_T_P) c->amax_p_valid = false;
   if (kind == PDADMM_T_X || (kind == PDADMM_T_P && layer == 1)) c->xT_valid = false;
   if (kind == PDADMM_T_P || kind == PDADMM_T_Q || kind == PDADMM_T_U) c->t_valid = false;
-  if (kind == PDADMM_T_P && c->levels && layer >= 2) {
-    Layer &y = c->layers[layer - 1];
-    const size_t n = (size_t)c->N * y.ld_in;
-    quantize_kernel<<<ew_grid(n), EW_THREADS, 0, c->scr.st>>>(y.p, n, y.scale, y.lo, c->levels, nullptr, y.codes,
-                                                              c->code_bytes == 2);
-    if (c->int_operands) codes_to_plane_kernel<<<ew_grid(n / 4), EW_THREADS, 0, c->scr.st>>>(y.codes, c->code_bytes == 2, n / 4, y.p_plane);
-    PD_CUDA(cudaStreamSynchronize(c->scr.st));
-  }
+  if (kind == PDADMM_T_P && c->levels && layer >= 2) PD_TRY(project_p_on_its_levels(c, layer));
   return PDADMM_OK;
 }
 
