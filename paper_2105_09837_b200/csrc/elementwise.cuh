@@ -123,20 +123,6 @@ axpy_neg_kernel(float *__restrict__ y, const float *__restrict__ x, const float 
   if (amax != nullptr) commit_amax(m, amax);
 }
 
-// y += x   (r <- r + W d after an accepted quantised step)
-__global__ void __launch_bounds__(EW_THREADS)
-add_kernel(float *__restrict__ y, const float *__restrict__ x, size_t n4, uint32_t *__restrict__ amax) {
-  uint32_t m = 0u;
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
-    float4 v = ld4(y, i);
-    const float4 w = ld4(x, i);
-    v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
-    st4(y, i, v);
-    m = max(m, abs_bits(v));
-  }
-  if (amax != nullptr) commit_amax(m, amax);
-}
-
 // ---- quantised trial step ------------------------------------------------------------------------
 // x = p - g/tau; p_new = nearest level; d = p_new - p; codes; per-block sum of d^2.
 // p lies on the level set, p = lo + code * scale bit for bit (quantize_one), so it is read as its 1- or 2-byte codes

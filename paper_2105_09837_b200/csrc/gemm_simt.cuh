@@ -69,6 +69,24 @@ struct EpiLinearResidual {    // C = acc + b[col] - Z[row][col]     (r = W p + b
     return make_float4(a.x + b.x - z.x, a.y + b.y - z.y, a.z + b.z - z.z, a.w + b.w - z.w);
   }
 };
+struct EpiAddSumsq {          // C = acc + R, accumulates sum(acc^2)     (the quantised step: r + W d beside ||W d||^2)
+  static constexpr bool kDirect = false, kSumsq = true, kSumsqOfAcc = true;
+  static constexpr int kInputs = 1;
+  float *C; int ldc; const float *R; uint32_t *amax;
+  __device__ __forceinline__ void prefetch(int row, int col) const { prefetch_l2(R + (size_t)row * ldc + col); }
+  __device__ __forceinline__ void load(int row, int col, float4 *in) const {
+    in[0] = *reinterpret_cast<const float4 *>(R + (size_t)row * ldc + col);
+  }
+  __device__ __forceinline__ float4 apply(int, float4 a, const float4 *in) const {
+    return make_float4(a.x + in[0].x, a.y + in[0].y, a.z + in[0].z, a.w + in[0].w);
+  }
+  __device__ __forceinline__ float4 operator()(int row, int col, float4 a, double &ss) const {
+    float4 in;
+    load(row, col, &in);
+    ss += (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
+    return apply(col, a, &in);
+  }
+};
 struct EpiBiasAct {           // C = acc + b[col], then f (selected by `slope`, see act_eval) if relu != 0   (z = W p + b, p' = f(z))
   static constexpr bool kDirect = false, kSumsq = false;
   static constexpr int kInputs = 0;

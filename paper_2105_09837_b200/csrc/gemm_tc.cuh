@@ -88,6 +88,9 @@ template <class Epi> struct epi_stores<Epi, std::enable_if_t<!Epi::kStore>> { st
 // issued as the main term A_hi B_hi alone (one MMA instead of three).  Each term then carries an independent relative
 // rounding of 2^-11 instead of 2^-22; over the 1e6..1e9 squares of the sum these average out to far below the
 // single-precision accuracy of the sum itself.
+// An epilogue whose sum of squares is that of the product itself, not of what it stores, says kSumsqOfAcc = true.
+template <class Epi, class = void> struct epi_sumsq_acc { static constexpr bool value = false; };
+template <class Epi> struct epi_sumsq_acc<Epi, std::enable_if_t<Epi::kSumsqOfAcc>> { static constexpr bool value = true; };
 template <class Epi, class = void> struct epi_coarse { static constexpr bool value = false; };
 template <class Epi> struct epi_coarse<Epi, std::enable_if_t<Epi::kCoarse>> { static constexpr bool value = true; };
 
@@ -606,9 +609,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int r = 4 * (s0 + i) + (lane >> 3);
                 const int row = m0 + lane_base + r;
                 float4 o = tr[r * 8 + ((lane & 7) ^ (r & 7))];
+                if constexpr (epi_sumsq_acc<Epi>::value) {
+                  if (row < prm.M) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
+                }
                 if constexpr (!Epi::kDirect) o = epi.apply(col, o, in[i]);
                 if (row < prm.M) {
-                  if (Epi::kSumsq) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
+                  if (Epi::kSumsq && !epi_sumsq_acc<Epi>::value) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
                   *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
                   if constexpr (!Epi::kDirect) mx = max(mx, abs_bits(o));
                 }

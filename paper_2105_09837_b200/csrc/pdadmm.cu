@@ -489,11 +489,13 @@ static int gemm_nodes(pdadmm_ctx *c, int cls, cudaStream_t st, int M, int N, int
     }
   }
   Launch l(c, cls, st, bytes, 2.0 * M * N * K);
-  if constexpr (std::is_same<Epi, EpiStoreSumsq>::value) {
+  if constexpr (std::is_same<Epi, EpiStoreSumsq>::value || std::is_same<Epi, EpiAddSumsq>::value) {
     if (a_int) {
       prm.mul = Ai->mul;
       return launch_tc<TC_PLANES, Epi, 1>(c, st, ma, ma, mb, mbl, prm, epi, partials, n_units);
     }
+  } else {
+    if (a_int) return fail(PDADMM_EINVAL, "no integer-operand form of this product is built");
   }
   if (pp) return launch_tc<TC_PLANES, Epi>(c, st, ma, mal, mb, mbl, prm, epi, partials, n_units);
   return launch_tc<TC_RAW_K, Epi>(c, st, ma, ma, mb, mbl, prm, epi, partials, n_units);
@@ -665,10 +667,12 @@ static int q_trial(pdadmm_ctx *c, int l) {
   }
   int np = 0;
   double *slots_b = s.slots + s.n_slots / 2;
-  EpiStoreSumsq epi{s.s2, ly.ld_out};
+  // the trial's residual r + W d is written beside r (the two trade places when the trial is taken), with ||W d||^2;
+  // max|r| takes the trial's values too, which keeps it an upper bound whether or not the trial is taken
+  EpiAddSumsq epi{s.s2, ly.ld_out, ly.r, c->use_tc ? ly.amax_r : nullptr};
   const IntPlane di{c->int_operands ? s.d_plane : nullptr, ly.ld_in, ly.scale};      // d = (new code - old code) s
   PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.d, ly.ld_in, ly.W, ly.ld_in, planes_W(ly), epi,
-                           slots_b, &np, 0, w_d, nullptr, &di));
+                           slots_b, &np, 4.0 * N * ly.n_out, w_d, nullptr, &di));
   if (c->reduce != nullptr) {
     PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, grid, slots_b, np));
     finalize_trial_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, 1e-6, s.red, 1, s.red + 1, 1);
@@ -685,7 +689,6 @@ static int q_trial(pdadmm_ctx *c, int l) {
 static int q_finish(pdadmm_ctx *c, int l, bool *hit_cap) {
   Layer &ly = c->layers[l];
   Scratch &s = *c->cur;
-  const size_t n4r = (size_t)c->N * ly.ld_out / 4;
   const int max_trials = 30;
   for (int trial = 0;; ++trial) {
     PD_CUDA(cudaEventSynchronize(s.ev_flag));
@@ -698,10 +701,7 @@ static int q_finish(pdadmm_ctx *c, int l, bool *hit_cap) {
   std::swap(ly.p, s.p_new);
   std::swap(ly.codes, s.codes_new);
   std::swap(ly.p_plane, s.pn_plane);
-  {
-    Launch k(c, KC_AXPY, s.st, 12.0 * c->N * ly.n_out, 0);
-    add_kernel<<<ew_grid(n4r), EW_THREADS, 0, s.st>>>(ly.r, s.s2, n4r, ly.amax_r);
-  }
+  std::swap(ly.r, s.s2);                // r <- r + W d, written by the trial's product
   return PDADMM_OK;
 }
 
@@ -1173,6 +1173,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
   int max_in = 0, max_out = 0;
   size_t max_part = 0;
   for (int l = 1; l < c->L; ++l) max_in = std::max(max_in, round_up(cfg->layer_widths[l - 1], LD_ALIGN));
+  for (int l = 0; l < c->L; ++l) max_out = std::max(max_out, round_up(cfg->layer_widths[l], LD_ALIGN));
   for (int l = 0; l < c->L; ++l) {
     Layer &ly = c->layers[l];
     ly.n_in = l == 0 ? c->n0 : cfg->layer_widths[l - 1];
@@ -1192,7 +1193,8 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
     PD_TRY(dev_alloc(c, &ly.b, (size_t)ly.ld_out));
     PD_TRY(dev_alloc(c, &ly.shift, (size_t)ly.ld_out));
     PD_TRY(dev_alloc(c, &ly.z, e_out));
-    PD_TRY(dev_alloc(c, &ly.r, e_out));
+    // quantised mode: r_l (l >= 2) trades places with the lane's buffer for the trial's r + W d, so all have one size
+    PD_TRY(dev_alloc(c, &ly.r, (c->levels && l > 0) ? (size_t)N * max_out : e_out));
     if (l + 1 < c->L) { PD_TRY(dev_alloc(c, &ly.q, e_out)); PD_TRY(dev_alloc(c, &ly.u, e_out)); }
     if (c->levels && l > 0) PD_TRY(dev_alloc(c, &ly.codes, e_in * c->code_bytes));
     if (c->int_operands && l > 0) PD_TRY(dev_alloc(c, &ly.p_plane, e_in));
