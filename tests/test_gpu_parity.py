@@ -80,6 +80,33 @@ def test_init_quantised_start():
     ctx.destroy()
 
 
+def test_setting_p_or_its_spacing_keeps_p_equal_to_the_levels_of_its_codes():
+    """The kernels of pdADMM-G-Q read p_l through its codes, so whatever a caller stores must end up as a pair
+    (codes, p = levels of those codes): values off the level set are projected (Eq. "update p quantized": nearest level),
+    and a new spacing moves p_l to the new level set."""
+    inp = _inputs("ba-ragged", quant_levels=16)
+    ctx = B.from_inputs(inp)
+    rng = np.random.default_rng(5)
+    for l in (2, 3):
+        s = np.float32(ctx.get_tensor(B.T_QSCALE, l)[0])
+        p = ctx.get_tensor(B.T_P, l)
+        noisy = (p + np.float32(0.3) * s * rng.uniform(-1, 1, p.shape).astype(np.float32)).astype(np.float32)
+        ctx.set_tensor(B.T_P, l, noisy)
+        want_codes, want_p = o.quantize(noisy, float(s), 16)           # both sides get the same fp32 input: bit for bit
+        assert np.array_equal(ctx.get_tensor(B.T_CODES, l), want_codes)
+        assert np.array_equal(ctx.get_tensor(B.T_P, l), want_p.astype(np.float32))
+        s2 = np.float32(1.5) * s
+        ctx.set_tensor(B.T_QSCALE, l, np.array([s2], dtype=np.float32))
+        want_codes, want_p = o.quantize(want_p.astype(np.float32), float(s2), 16)
+        assert np.array_equal(ctx.get_tensor(B.T_CODES, l), want_codes)
+        assert np.array_equal(ctx.get_tensor(B.T_P, l), want_p.astype(np.float32))
+    ctx.step(2)                                                        # and the iteration keeps the pair together
+    for l in (2, 3):
+        s = np.float32(ctx.get_tensor(B.T_QSCALE, l)[0])
+        assert np.array_equal(ctx.get_tensor(B.T_P, l), ctx.get_tensor(B.T_CODES, l).astype(np.float32) * s)
+    ctx.destroy()
+
+
 # ----------------------------------------------------------------------------- one teacher-forced iteration
 
 def _compare_iteration(ctx, prev, prm, label, tensor_cores=True, report=None, single_bounds=False):
