@@ -54,6 +54,22 @@ __host__ __device__ __forceinline__ int tc_scale_exp(uint32_t amax_bits) {
   const int e = 14 - (E - 127);
   return e < -100 ? -100 : (e > 100 ? 100 : e);
 }
+// An fp16 copy of a matrix written before its largest magnitude is known takes its exponent from the maximum of the
+// previous iteration, two binary orders lower (room for a fourfold growth); TC_NO_PREDICTION if that maximum is no
+// normal number.  The copy is usable if the true maximum, scaled, lies in [2^4, 2^15): no overflow and at least 11
+// significant bits above the fp16 subnormals for the largest entries (it is used as a hi plane alone).
+constexpr int TC_NO_PREDICTION = -1000;
+__host__ __device__ __forceinline__ int tc_predict_exp(uint32_t amax_bits) {
+  const int E = (int)((amax_bits >> 23) & 0xFFu);
+  if (E == 0 || E == 255) return TC_NO_PREDICTION;
+  return tc_scale_exp(amax_bits) - 2;
+}
+__host__ __device__ __forceinline__ bool tc_prediction_usable(uint32_t amax_bits, int predicted) {
+  const int E = (int)((amax_bits >> 23) & 0xFFu);
+  if (E == 0 || E == 255 || predicted < -100 || predicted > 100) return false;
+  const int e = 14 - (E - 127);          // unclamped exponent of the exact scaling
+  return predicted <= e && predicted >= e - 10;
+}
 // ---- largest magnitude of an array, as a bit pattern ---------------------------------------------
 // The tensor-core products scale each operand by a power of two chosen from max|x|.  The maximum is kept as the
 // bit pattern of |x| in an unsigned word (for non-negative floats the integer order is the float order, a NaN

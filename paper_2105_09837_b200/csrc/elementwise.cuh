@@ -265,7 +265,8 @@ __device__ __forceinline__ double block_sum_slots(const double *__restrict__ slo
 // tau = rho + nu ||W g||^2 / ||g||^2 : the smallest tau with phi(p - g/tau) <= U_l(p - g/tau; tau).
 __global__ void __launch_bounds__(FIN_THREADS)
 finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots_g, int n_g, const double *slots_wg, int n_wg,
-                    int *nonfinite, uint32_t *clear_word /* max|p| of the layer restarts with the coming p-step */) {
+                    int *nonfinite, uint32_t *clear_word /* max|p| of the layer restarts with the coming p-step */,
+                    const uint32_t *amax_g = nullptr, int *next_g_exp = nullptr /* scaling of the next iteration's fp16 copy of g */) {
   __shared__ double sh[FIN_THREADS];
   const double gg = block_sum_slots(slots_g, n_g, sh);
   const double wg = block_sum_slots(slots_wg, n_wg, sh);
@@ -279,6 +280,7 @@ finalize_tau_kernel(LayerScalars *sc, double rho, double nu, const double *slots
     sc->accepted = 0;
     sc->trials = 0;
     if (clear_word != nullptr) *clear_word = 0u;
+    if (next_g_exp != nullptr) *next_g_exp = tc_predict_exp(*amax_g);
   }
 }
 // Stop condition of the quantised step in its quadratic form: nu||W d||^2 + rho||d||^2 <= tau||d||^2 (1 + slack).
@@ -366,9 +368,18 @@ make_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, cons
 // operand of a product whose output is several column tiles wide, split once here instead of once per column tile
 // inside the product.  Scaling and split as in make_planes_kernel; the exponent goes to *exp_out.  A thread converts
 // eight consecutive values (two 16-byte loads, one 16-byte store per plane).
+// `predicted` (may be null): the hi plane was already written by the kernel that produced x, scaled by 2^(*predicted),
+// an exponent chosen before max|x| was known (from the previous iteration's maximum, see tc_predict_exp).  If that
+// scaling turned out usable -- no overflow, at least 11 bits left: max|x| 2^e in [2^4, 2^15) -- nothing is left to do
+// but to publish the exponent; otherwise the plane is written again here with the exponent from the true maximum.
+// Only for hi-plane-only operands (lo == nullptr): 11 bits are all such a product wants.
 __global__ void __launch_bounds__(256)
 rows_planes_kernel(const float *__restrict__ x, size_t n8, const uint32_t *__restrict__ amax, int *__restrict__ exp_out,
-                   __half *__restrict__ hi, __half *__restrict__ lo) {
+                   __half *__restrict__ hi, __half *__restrict__ lo, const int *__restrict__ predicted = nullptr) {
+  if (predicted != nullptr && tc_prediction_usable(*amax, *predicted)) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) *exp_out = *predicted;
+    return;
+  }
   const int e = tc_scale_exp(*amax);
   if (blockIdx.x == 0 && threadIdx.x == 0) *exp_out = e;
   const float scale = __uint_as_float((uint32_t)(e + 127) << 23);

@@ -122,6 +122,12 @@ struct EpiGradT {             // C = nu*acc + T, accumulates sum(C^2); T = u_{l-
     return g;
   }
 };
+struct EpiGradTCopy : EpiGradT {   // the same, and (tensor-core kernel only) the result once more as an fp16 plane H [rows][ldc],
+                                   // scaled by 2^(*h_exp) and rounded to 11 bits like the hi plane of an operand
+                                   // (rows_planes_kernel says what it is for)
+  static constexpr bool kHalfCopy = true;
+  __half *H; const int *h_exp;
+};
 
 // ---- NT kernel -----------------------------------------------------------------------------------
 // Thread (tx, ty) of a 16x16 block owns rows {ty*4+i, 64+ty*4+i} and columns {tx*4+j, 64+tx*4+j}.

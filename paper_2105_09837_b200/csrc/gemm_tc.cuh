@@ -91,6 +91,9 @@ template <class Epi> struct epi_stores<Epi, std::enable_if_t<!Epi::kStore>> { st
 // An epilogue whose sum of squares is that of the product itself, not of what it stores, says kSumsqOfAcc = true.
 template <class Epi, class = void> struct epi_sumsq_acc { static constexpr bool value = false; };
 template <class Epi> struct epi_sumsq_acc<Epi, std::enable_if_t<Epi::kSumsqOfAcc>> { static constexpr bool value = true; };
+// An epilogue that can also leave an fp16 copy of its result (see EpiGradT) says kHalfCopy = true.
+template <class Epi, class = void> struct epi_half_copy { static constexpr bool value = false; };
+template <class Epi> struct epi_half_copy<Epi, std::enable_if_t<Epi::kHalfCopy>> { static constexpr bool value = true; };
 template <class Epi, class = void> struct epi_coarse { static constexpr bool value = false; };
 template <class Epi> struct epi_coarse<Epi, std::enable_if_t<Epi::kCoarse>> { static constexpr bool value = true; };
 
@@ -584,6 +587,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         float *C = epi.C + (size_t)z * prm.c_split_stride;
         float ssf = 0.f;
         uint32_t mx = 0u;                  // largest magnitude stored by this thread
+        float h_scale = 0.f;               // scaling of the fp16 copy, if one is wanted
+        if constexpr (epi_half_copy<Epi>::value) {
+          if (epi.H != nullptr) h_scale = tc_pow2(max(-100, min(100, *epi.h_exp)));
+        }
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
           __syncwarp();
@@ -616,6 +623,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (row < prm.M) {
                   if (Epi::kSumsq && !epi_sumsq_acc<Epi>::value) ssf = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssf))));
                   *reinterpret_cast<float4 *>(C + (size_t)row * epi.ldc + col) = o;
+                  if constexpr (epi_half_copy<Epi>::value) {
+                    if (epi.H != nullptr) {
+                      float h0, h1, h2, h3, lo_unused;
+                      tc_split(o.x, h_scale, h0, lo_unused); tc_split(o.y, h_scale, h1, lo_unused);
+                      tc_split(o.z, h_scale, h2, lo_unused); tc_split(o.w, h_scale, h3, lo_unused);
+                      const __half2 a = __floats2half2_rn(h0, h1), b = __floats2half2_rn(h2, h3);
+                      *reinterpret_cast<uint2 *>(epi.H + (size_t)row * epi.ldc + col) =
+                          make_uint2(*reinterpret_cast<const uint32_t *>(&a), *reinterpret_cast<const uint32_t *>(&b));
+                    }
+                  }
                   if constexpr (!Epi::kDirect) mx = max(mx, abs_bits(o));
                 }
               }

@@ -88,6 +88,7 @@ struct Layer {
   int *xT_exp = nullptr;
   __half *x_hi = nullptr, *x_lo = nullptr;     // layer 1 only: planes of X in its own orientation [N][ld_in]
   int *x_exp = nullptr;
+  int *g_exp = nullptr;     // l >= 2: exponent predicted for the scaling of the next fp16 copy of g_l (tc_predict_exp)
   float *shift = nullptr;   // [ld_out] column means removed by the b-update
   uint8_t *codes = nullptr; // [N][ld_in] codes of 1 byte (up to 256 levels) or 2 bytes, quantised mode, l >= 2
   __half *p_plane = nullptr; // [N][ld_in] the codes as fp16 integers: operand plane of p_l = code * scale (see int_operands)
@@ -124,6 +125,10 @@ struct Scratch {
   __half *a_hi = nullptr, *a_lo = nullptr;
   size_t a_cap = 0;                // elements each of the two holds
   int *a_exp = nullptr;
+  // quantised mode: fp16 copy [N][ld] of g, written by the epilogue of the p-gradient's product with a predicted
+  // scaling, for the norm-only product W g that follows (rows_planes_kernel)
+  __half *g_hi = nullptr;
+  int *g_hi_exp = nullptr;
   int *h_flag = nullptr;           // pinned word that receives the accept flag of the lane's quantised trial
   cudaEvent_t ev_flag = nullptr;   // recorded after the copy of that flag
 };
@@ -597,16 +602,35 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
   (void)prev;
   uint32_t *w_g = nullptr;                 // max|g|, kept by the epilogue that writes g
   if (c->use_tc) { PD_TRY(amax_reserve(c, s.st, 1)); w_g = amax_take(c); }
-  EpiGradT epi{s.s1, ly.ld_in, ly.t, c->nu, w_g};
-  PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.ld_in, planes_WT(ly),
-                          epi, s.slots, &np, 4.0 * N * ly.n_in, ly.amax_r));
+  // Quantised update, wide layers: the norm-only product W g takes g as one fp16 plane.  The epilogue that writes g
+  // writes that plane too, scaled by an exponent predicted from the previous iteration's max|g| (the true one is known
+  // only when the product has finished); rows_planes_kernel then confirms the prediction or, if max|g| moved by more
+  // than the plane can take, splits g again (6 bytes per element, the cost of every iteration before this).
+  const bool copy_g = c->levels && c->use_tc && s.g_hi != nullptr && (size_t)N * ly.ld_in <= s.a_cap &&
+                      ceil_div(ly.n_out, TC_BN) >= PLANES_FROM_COL_TILES / 2;
+  if (copy_g) {
+    EpiGradTCopy epi{{s.s1, ly.ld_in, ly.t, c->nu, w_g}, s.g_hi, ly.g_exp};
+    PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.ld_in, planes_WT(ly),
+                            epi, s.slots, &np, 6.0 * N * ly.n_in, ly.amax_r));
+  } else {
+    EpiGradT epi{s.s1, ly.ld_in, ly.t, c->nu, w_g};
+    PD_TRY(gemm_nodes<true>(c, KC_GEMM_GRADP, s.st, N, ly.n_in, ly.n_out, ly.r, ly.ld_out, ly.W, ly.ld_in, planes_WT(ly),
+                            epi, s.slots, &np, 4.0 * N * ly.n_in, ly.amax_r));
+  }
   int np2 = 0;
   double *slots_b = s.slots + s.n_slots / 2;          // second half of the slot buffer
   if (c->levels && c->use_tc) {
     // the quantised update only needs ||W g||^2 (for the first tau); its residual update uses W d
     EpiNormOnly epi2{s.s2, ly.ld_out};
+    PlaneRef gp{nullptr, nullptr, 0, nullptr};
+    if (copy_g) {
+      const size_t n8 = (size_t)N * ly.ld_in / 8;
+      Launch k(c, KC_PLANES, s.st, 0.0, 0);          // normally only publishes the exponent
+      rows_planes_kernel<<<ew_grid(n8), 256, 0, s.st>>>(s.s1, n8, w_g, s.g_hi_exp, s.g_hi, nullptr, ly.g_exp);
+      gp = PlaneRef{s.g_hi, s.g_hi, ly.ld_in, s.g_hi_exp};
+    }
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
-                             epi2, slots_b, &np2, 0, w_g));
+                             epi2, slots_b, &np2, 0, w_g, &gp));
   } else {
     EpiStoreSumsq epi2{s.s2, ly.ld_out};
     PD_TRY(gemm_nodes<false>(c, KC_GEMM_WG, s.st, N, ly.n_out, ly.n_in, s.s1, ly.ld_in, ly.W, ly.ld_in, planes_W(ly),
@@ -616,13 +640,13 @@ static int p_gradient_and_tau(pdadmm_ctx *c, int l /*0-based, >= 1*/) {
     // ||g||^2 and ||W g||^2 are sums over nodes: this shard's totals, added over the shards, then tau
     PD_TRY(shard_sum_slots(c, s.st, s.red, s.slots, np, slots_b, np2));
     finalize_tau_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.red, 1, s.red + 1, 1, c->d_flag + 2,
-                                             ly.amax_p);
+                                             ly.amax_p, w_g, copy_g ? ly.g_exp : nullptr);
     return PDADMM_OK;
   }
   {
     Launch k(c, KC_SMALL, s.st, 8.0 * (np + np2), 0);
     finalize_tau_kernel<<<1, FIN_THREADS, 0, s.st>>>(ly.sc, (double)c->rho, (double)c->nu, s.slots, np, slots_b, np2, c->d_flag + 2,
-                                             ly.amax_p);
+                                             ly.amax_p, w_g, copy_g ? ly.g_exp : nullptr);
   }
   return PDADMM_OK;
 }
@@ -1039,6 +1063,10 @@ static int alloc_row_planes(pdadmm_ctx *c, Scratch &s, size_t n) {
   PD_TRY(dev_alloc(c, &s.a_lo, n, false));
   PD_TRY(dev_alloc(c, &s.a_exp, 1));
   s.a_cap = n;
+  if (c->levels) {
+    PD_TRY(dev_alloc(c, &s.g_hi, n, false));
+    PD_TRY(dev_alloc(c, &s.g_hi_exp, 1));
+  }
   return PDADMM_OK;
 }
 
@@ -1200,6 +1228,7 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
     if (c->int_operands && l > 0) PD_TRY(dev_alloc(c, &ly.p_plane, e_in));
     if (l > 0) PD_TRY(dev_alloc(c, &ly.t, (size_t)N * ly.ld_in));
     PD_TRY(dev_alloc(c, &ly.sc, 1));
+    if (l > 0) PD_TRY(dev_alloc(c, &ly.g_exp, 1));
     PD_TRY(dev_alloc(c, &ly.amax_p, 1));
     PD_TRY(dev_alloc(c, &ly.amax_r, 1));
     PD_TRY(upload_rows(st, ly.W, ly.ld_in, cfg->init_W[l], ly.n_in, ly.n_out));
