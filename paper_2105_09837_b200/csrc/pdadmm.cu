@@ -1298,10 +1298,11 @@ static int build(pdadmm_ctx *c, const pdadmm_config *cfg, const pdadmm_shard *sh
   // further lanes for the concurrency across layers: own stream, product outputs, partial tiles, slots.
   // Small problems are bound by the latency of their chain of launches, which only more concurrent chains shorten
   // (workload c1, 10 layers: 2 lanes 0.40 ms per iteration); large ones gain little beyond two (c2: 2 lanes 273,
-  // 4 lanes 278 iterations/s) and their scratch is gigabytes per lane.  So: as many lanes as 2 GB of scratch pay for,
-  // at least PDADMM_N_LANES, at most one per layer.
+  // 4 lanes 278 iterations/s) and their scratch is gigabytes per lane.  So: as many lanes as 4 GB of scratch pay for,
+  // at least PDADMM_N_LANES, at most one per layer (c3, 0.4 GB per lane: 6 lanes 280, 10 lanes 301 iterations/s;
+  // c4, 5.5 GB per lane: 2 lanes 9.95, 4 lanes 9.99).
   const size_t lane_bytes = std::max<size_t>(c->bytes_handed_out - bytes_before_scratch, 1);
-  const int affordable = (int)std::min<size_t>(64, (size_t(2) << 30) / lane_bytes);
+  const int affordable = (int)std::min<size_t>(64, (size_t(4) << 30) / lane_bytes);
   const int n_lanes = (cfg->flags & PDADMM_FLAG_ONE_LANE) ? 1 : std::min(c->L, std::max(PDADMM_N_LANES, affordable));
   for (int i = 1; i < n_lanes; ++i) {
     c->more_lanes.emplace_back(new Scratch());
