@@ -42,6 +42,34 @@ def test_teacher_forced_iterations_at_the_shapes_of_the_large_workloads(name, n_
     ctx.destroy()
 
 
+def test_a_jump_in_the_size_of_the_gradient_between_iterations_is_handled():
+    """Wide quantised layers: the epilogue that writes g also writes its fp16 plane for the norm-only product W g, scaled
+    by an exponent predicted from the previous iteration's max|g|; a kernel then checks the prediction and redoes the
+    plane if it does not fit.  Here the dual variable is scaled by 1e4 and back between teacher-forced iterations, so
+    that max|g| jumps by four orders of magnitude each way (too large: the predicted scaling would overflow fp16; too
+    small: it would leave no significant bits).  That product only decides the tau at which the search of Eq. "update p
+    quantized" starts, tau = rho + nu ||W g||^2 / ||g||^2: it must agree with the oracle's in every one of these
+    iterations (the scaled states are far from anything the method produces, so nothing else is compared here)."""
+    import dataclasses
+    w = synth.small("c4", 2400, quant_levels=256)          # 1000-wide layers: 8 column tiles, the copy is in use
+    inp = synth.make_inputs(w)
+    prm, s, _ = U.oracle_problem(inp)
+    ctx = B.from_inputs(inp)
+    for k, factor in enumerate([1.0, 1.0, 1e4, 1e-4, 1.0]):
+        scaled = dataclasses.replace(s, u=[x * factor for x in s.u])
+        prev = U.round_state(scaled)
+        U.load_state(ctx, prev, True)
+        nxt = o.iterate(prev, prm)
+        ctx.step(1)
+        for l in range(1, prev.L):
+            tau_dev = float(ctx.get_tensor(B.T_TAU, l + 1)[0])
+            trials_dev = int(ctx.get_tensor(B.T_TRIALS, l + 1)[0])
+            start_dev, start_want = tau_dev / 2.0 ** (trials_dev - 1), nxt.tau[l] / 2.0 ** (nxt.trials[l] - 1)
+            assert abs(start_dev - start_want) <= 1e-5 * start_want, (k, factor, l + 1, start_dev, start_want)
+        s = nxt
+    ctx.destroy()
+
+
 @pytest.mark.parametrize("flags", [0, B.FLAG_SIMT_GEMM])
 def test_cached_linear_residual_does_not_drift_over_200_free_iterations(flags):
     """The library carries r = W p + b - z from step to step instead of recomputing it.  After 200 free iterations the
