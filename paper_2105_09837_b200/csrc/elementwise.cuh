@@ -376,7 +376,7 @@ make_planes_kernel(const float *__restrict__ x, int rows, int cols, int ld, cons
 __global__ void __launch_bounds__(256)
 rows_planes_kernel(const float *__restrict__ x, size_t n8, const uint32_t *__restrict__ amax, int *__restrict__ exp_out,
                    __half *__restrict__ hi, __half *__restrict__ lo, const int *__restrict__ predicted = nullptr) {
-  if (predicted != nullptr && tc_prediction_usable(*amax, *predicted)) {
+  if (predicted != nullptr && lo == nullptr && tc_prediction_usable(*amax, *predicted)) {
     if (blockIdx.x == 0 && threadIdx.x == 0) *exp_out = *predicted;
     return;
   }
